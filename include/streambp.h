@@ -1,0 +1,194 @@
+/*
+ * streambp.h -- C ABI of the B200 (sm_100a) streamed backward pass.
+ *
+ * The library computes the exact gradient of a decoder-only transformer by the
+ * sequence-partitioned accumulation of the paper's Eq. (1):
+ *     dL/dW = sum_i (dZ_out^(i)/dW)^T dL/dZ_out^(i)
+ * over chunks i of `chunk` consecutive token rows (the paper's "partition size";
+ * the last chunk may be shorter, and chunk >= T means a single chunk, i.e. the
+ * ordinary un-partitioned backward, Sec. 4.3 "partition will not be performed if
+ * it is larger than the sequence length").
+ *
+ * Conventions for every entry point
+ *   - All tensor pointers are DEVICE pointers owned by the caller, row-major,
+ *     16-byte aligned; `workspace` is device memory, 256-byte aligned.  Config and
+ *     weight/grad pointer structs are HOST memory, read during the call only.
+ *   - Matrices are stored [out_features, in_features] (y = x W^T).
+ *   - `dtype` selects the storage type of activations and weights (X, dY, dX, H,
+ *     dH, every weight): float or bf16.  Weight gradients, the loss and all
+ *     accumulators are always float (fp32).  bf16 runs multiply bf16 operands and
+ *     accumulate in fp32.
+ *   - The library allocates no device memory and keeps no state between calls;
+ *     it writes only to the outputs and the workspace.  Work is enqueued on
+ *     `cuda_stream` (a cudaStream_t passed as void*, NULL = default stream) and
+ *     the call returns without synchronising.
+ *   - Return value: STREAMBP_OK (0) or a negative streambp_status.  Errors found
+ *     on the host are returned before anything is enqueued.  Conditions only the
+ *     device can see (a label outside [0, vocab), no unmasked label, an expired
+ *     bounded wait inside a kernel) are recorded in the workspace header and read
+ *     back with streambp_last_device_status().  Nothing aborts, traps or throws.
+ *   - `accumulate` = 0 overwrites the weight-gradient outputs ("initialised from
+ *     zero", text after Eq. (3)); 1 adds to what they hold.
+ */
+#ifndef STREAMBP_H_
+#define STREAMBP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    STREAMBP_OK = 0,
+    STREAMBP_E_NULL = -1,            /* a required pointer is NULL */
+    STREAMBP_E_SHAPE = -2,           /* unsupported or inconsistent sizes */
+    STREAMBP_E_ALIGN = -3,           /* pointer alignment */
+    STREAMBP_E_WORKSPACE = -4,       /* workspace_bytes smaller than *_workspace_bytes() */
+    STREAMBP_E_DTYPE = -5,           /* unknown dtype */
+    STREAMBP_E_CUDA = -6,            /* a CUDA runtime / driver call failed */
+    STREAMBP_E_BAD_LABEL = -7,       /* device: label not in [0, vocab) and != ignore_index */
+    STREAMBP_E_NO_VALID_LABELS = -8, /* device: every label ignored; loss and grads are 0 */
+    STREAMBP_E_DEVICE_TIMEOUT = -9   /* device: a bounded wait inside a kernel ran out */
+} streambp_status;
+
+typedef enum { STREAMBP_F32 = 0, STREAMBP_BF16 = 1 } streambp_dtype;
+
+/* One pre-norm decoder layer: RMSNorm -> GQA causal attention with rotate-half RoPE
+ * -> residual -> RMSNorm -> SwiGLU MLP -> residual (the attention / MLP transformation
+ * of Sec. 3.2.2 with the normalisation, heads and residuals it leaves out restored). */
+typedef struct {
+    int32_t d_model;
+    int32_t n_q_heads;
+    int32_t n_kv_heads;   /* divides n_q_heads */
+    int32_t head_dim;     /* 64 or 128 */
+    int32_t d_ff;         /* SwiGLU intermediate width */
+    int32_t qkv_bias;     /* 1: bq, bk, bv present */
+    float rope_theta;
+    float rms_eps;
+    int32_t dtype;        /* streambp_dtype */
+} streambp_layer_cfg;
+
+/* Weights in storage dtype. g1,g2: [d_model]; wq: [Hq*dh, d]; wk,wv: [Hkv*dh, d];
+ * wo: [d, Hq*dh]; w_gate,w_up: [d_ff, d]; w_down: [d, d_ff]; bq: [Hq*dh]; bk,bv: [Hkv*dh]
+ * (biases NULL unless qkv_bias). */
+typedef struct {
+    const void *g1, *wq, *bq, *wk, *bk, *wv, *bv, *wo, *g2, *w_gate, *w_up, *w_down;
+} streambp_layer_weights;
+
+/* fp32 gradients, same shapes as the weights. */
+typedef struct {
+    float *g1, *wq, *bq, *wk, *bk, *wv, *bv, *wo, *g2, *w_gate, *w_up, *w_down;
+} streambp_layer_grads;
+
+/* Bytes of workspace streambp_layer_backward needs; 0 if the arguments are invalid. */
+size_t streambp_layer_workspace_bytes(const streambp_layer_cfg *cfg, int64_t T, int64_t chunk);
+
+/*
+ * Streamed backward of one decoder layer (Sec. 3.2.2, partitioned attention / MLP
+ * equations and the accumulation after them).
+ *
+ * Given the checkpointed layer input X [T, d_model], the upstream gradient dY [T, d_model]
+ * and the weights, computes dX [T, d_model] and every weight gradient.  K and V (after
+ * RoPE) are computed once for all T rows and cached in the workspace; then for each chunk
+ * the library re-forwards that chunk (norm, Q, attention of the chunk's queries against
+ * keys/values 0 .. chunk end only, output projection, norm, gate/up) and back-propagates
+ * it, adding into the fp32 weight gradients and into fp32 dK/dV accumulators for the key
+ * prefix.  `pos0` is the RoPE position of row 0.  The down-projection forward is never
+ * computed: dY is given.  dX may not alias X or dY.
+ */
+int streambp_layer_backward(const streambp_layer_cfg *cfg, const streambp_layer_weights *w,
+                            const void *X, const void *dY, int64_t T, int64_t chunk, int64_t pos0,
+                            int accumulate, const streambp_layer_grads *grads, void *dX,
+                            void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+typedef struct {
+    int32_t d_model;
+    int64_t vocab;
+    float rms_eps;
+    int64_t ignore_index;
+    int32_t dtype;        /* streambp_dtype */
+} streambp_head_cfg;
+
+size_t streambp_lmhead_workspace_bytes(const streambp_head_cfg *cfg, int64_t T, int64_t chunk);
+
+/*
+ * Streamed final-RMSNorm + LM head + cross-entropy backward (Sec. 3.2.1, SFT objective
+ * Eq. (2) and the accumulation Eq. (3)), normalised to the MEAN over unmasked tokens.
+ *
+ * H [T, d] are the last layer's hidden states, w_vocab [vocab, d], g_final [d],
+ * labels [T] (int64, already aligned to the logit rows; ignore_index marks masked rows).
+ * The number N of unmasked labels is counted first; then per chunk the fp32 logits
+ * [chunk, vocab] are formed, reduced to their log-sum-exp, turned into
+ * dlogits = (softmax - onehot)/N (zero rows where ignored) and consumed by the two
+ * gradient products, so that [T, vocab] never exists.
+ * Outputs: *loss (device float), *n_valid (device int64), dH [T, d] storage dtype,
+ * d_w_vocab [vocab, d] fp32, d_g_final [d] fp32.  `accumulate` applies to d_w_vocab and
+ * d_g_final.  If N == 0 the loss and all gradients are written as 0 and the device
+ * status becomes STREAMBP_E_NO_VALID_LABELS.
+ */
+int streambp_lmhead_ce_backward(const streambp_head_cfg *cfg, const void *g_final, const void *w_vocab,
+                                const void *H, const int64_t *labels, int64_t T, int64_t chunk,
+                                int accumulate, float *loss, int64_t *n_valid, void *dH,
+                                float *d_w_vocab, float *d_g_final,
+                                void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+typedef struct {
+    int32_t n_layers;
+    streambp_layer_cfg layer;
+    streambp_head_cfg head;
+} streambp_model_cfg;
+
+/* Includes the [n_layers][T, d] layer-input checkpoints (storage dtype). */
+size_t streambp_model_workspace_bytes(const streambp_model_cfg *cfg, int64_t T,
+                                      int64_t chunk_layer, int64_t chunk_head);
+
+/*
+ * Whole-model backward with layer-input checkpoints only (Sec. 2 / Sec. 3.1: the
+ * substrate the streamed backward sits on): embedding lookup (or X0 given), a chunked
+ * forward that stores each layer's input, the streamed head backward, then the streamed
+ * layer backward for l = L..1 with dY := dX of the layer above, and the embedding
+ * scatter-add.  `layers` and `layer_grads` are host arrays of n_layers structs.
+ * ids [T] int64 index `embed` [vocab, d]; if ids is NULL, X0 [T, d] is the first layer's
+ * input (then embed / d_embed may be NULL).  dX0 [T, d] (storage dtype) may be NULL.
+ */
+int streambp_model_backward(const streambp_model_cfg *cfg, const void *embed,
+                            const streambp_layer_weights *layers, const void *g_final, const void *w_vocab,
+                            const int64_t *ids, const void *X0, const int64_t *labels, int64_t T,
+                            int64_t chunk_layer, int64_t chunk_head, int accumulate,
+                            float *loss, float *d_embed, const streambp_layer_grads *layer_grads,
+                            float *d_g_final, float *d_w_vocab, void *dX0,
+                            void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Synchronises `cuda_stream` and returns the status the kernels of the last call using
+ * this workspace recorded (STREAMBP_OK, E_BAD_LABEL, E_NO_VALID_LABELS, E_DEVICE_TIMEOUT),
+ * or STREAMBP_E_CUDA if the stream reports an error. */
+int streambp_last_device_status(void *workspace, void *cuda_stream);
+
+const char *streambp_status_string(int status);
+
+/* The last CUDA error code (cudaError_t / CUresult as int) behind a STREAMBP_E_CUDA
+ * returned on the calling thread; 0 if none. */
+int streambp_last_cuda_error(void);
+
+/* Number of kernel launches the last call on the calling thread enqueued. */
+int64_t streambp_last_launch_count(void);
+
+/*
+ * Building block exposed for tests and profiling: C = A * B (+ bias) with the operand
+ * layouts the three gradient products of Eq. (1) need.  op: 0 = "NT" C[M,N] = A[M,K] B[N,K]^T
+ * (forward y = x W^T), 1 = "NN" C[M,N] = A[M,K] B[K,N] (input gradient dY W),
+ * 2 = "TN" C[M,N] = A[K,M]^T B[K,N] (weight gradient dY^T X).  A and B have `in_dtype`
+ * (row-major, leading dimensions lda/ldb in elements), C has `out_dtype`, leading dimension
+ * ldc; accumulate = 1 adds to C (fp32 C only).  engine: 0 = automatic, 1 = fp32 CUDA-core
+ * kernel, 2 = tcgen05 tensor-core kernel (bf16 operands only).
+ */
+int streambp_gemm(int op, int64_t M, int64_t N, int64_t K, const void *A, int64_t lda,
+                  const void *B, int64_t ldb, void *C, int64_t ldc, int32_t in_dtype,
+                  int32_t out_dtype, int accumulate, int engine, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* STREAMBP_H_ */

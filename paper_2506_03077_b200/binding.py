@@ -1,0 +1,276 @@
+"""ctypes binding of libstreambp.so: the same entry points as include/streambp.h.
+
+Only argument marshalling happens here (torch tensors -> device pointers, Python
+dataclasses -> C structs); every step of the computation runs in the CUDA library.
+There is no fallback: if the library is missing or cannot be loaded, importing
+`lib()` raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Dict, List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libstreambp.so")
+
+STREAMBP_F32, STREAMBP_BF16 = 0, 1
+OK = 0
+E_NULL, E_SHAPE, E_ALIGN, E_WORKSPACE, E_DTYPE, E_CUDA, E_BAD_LABEL, E_NO_VALID_LABELS, E_DEVICE_TIMEOUT = range(-1, -10, -1)
+OP_NT, OP_NN, OP_TN = 0, 1, 2
+
+WEIGHT_FIELDS = ("g1", "wq", "bq", "wk", "bk", "wv", "bv", "wo", "g2", "w_gate", "w_up", "w_down")
+
+EXPORTS = (
+    "streambp_layer_workspace_bytes", "streambp_layer_backward",
+    "streambp_lmhead_workspace_bytes", "streambp_lmhead_ce_backward",
+    "streambp_model_workspace_bytes", "streambp_model_backward",
+    "streambp_last_device_status", "streambp_status_string",
+    "streambp_last_cuda_error", "streambp_last_launch_count", "streambp_gemm",
+)
+
+
+class LayerCfgC(C.Structure):
+    _fields_ = [("d_model", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("d_ff", C.c_int32), ("qkv_bias", C.c_int32),
+                ("rope_theta", C.c_float), ("rms_eps", C.c_float), ("dtype", C.c_int32)]
+
+
+class LayerPtrsC(C.Structure):
+    _fields_ = [(f, C.c_void_p) for f in WEIGHT_FIELDS]
+
+
+class HeadCfgC(C.Structure):
+    _fields_ = [("d_model", C.c_int32), ("vocab", C.c_int64), ("rms_eps", C.c_float),
+                ("ignore_index", C.c_int64), ("dtype", C.c_int32)]
+
+
+class ModelCfgC(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("layer", LayerCfgC), ("head", HeadCfgC)]
+
+
+class StreamBPError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: status {status} ({status_string(status)})")
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load libstreambp.so (built by paper_2506_03077_b200.build). Raises if it is absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise FileNotFoundError(
+            f"{LIB_PATH} not found: build it with `python -m paper_2506_03077_b200.build` "
+            "(there is no CPU or PyTorch fallback)")
+    L = C.CDLL(LIB_PATH)
+    vp, i64, sz, i32 = C.c_void_p, C.c_int64, C.c_size_t, C.c_int32
+    L.streambp_layer_workspace_bytes.restype = sz
+    L.streambp_layer_workspace_bytes.argtypes = [C.POINTER(LayerCfgC), i64, i64]
+    L.streambp_layer_backward.restype = C.c_int
+    L.streambp_layer_backward.argtypes = [C.POINTER(LayerCfgC), C.POINTER(LayerPtrsC), vp, vp, i64, i64, i64, C.c_int,
+                                          C.POINTER(LayerPtrsC), vp, vp, sz, vp]
+    L.streambp_lmhead_workspace_bytes.restype = sz
+    L.streambp_lmhead_workspace_bytes.argtypes = [C.POINTER(HeadCfgC), i64, i64]
+    L.streambp_lmhead_ce_backward.restype = C.c_int
+    L.streambp_lmhead_ce_backward.argtypes = [C.POINTER(HeadCfgC), vp, vp, vp, vp, i64, i64, C.c_int, vp, vp, vp, vp,
+                                              vp, vp, sz, vp]
+    L.streambp_model_workspace_bytes.restype = sz
+    L.streambp_model_workspace_bytes.argtypes = [C.POINTER(ModelCfgC), i64, i64, i64]
+    L.streambp_model_backward.restype = C.c_int
+    L.streambp_model_backward.argtypes = [C.POINTER(ModelCfgC), vp, C.POINTER(LayerPtrsC), vp, vp, vp, vp, vp, i64,
+                                          i64, i64, C.c_int, vp, vp, C.POINTER(LayerPtrsC), vp, vp, vp, vp, sz, vp]
+    L.streambp_last_device_status.restype = C.c_int
+    L.streambp_last_device_status.argtypes = [vp, vp]
+    L.streambp_status_string.restype = C.c_char_p
+    L.streambp_status_string.argtypes = [C.c_int]
+    L.streambp_last_cuda_error.restype = C.c_int
+    L.streambp_last_cuda_error.argtypes = []
+    L.streambp_last_launch_count.restype = i64
+    L.streambp_last_launch_count.argtypes = []
+    L.streambp_gemm.restype = C.c_int
+    L.streambp_gemm.argtypes = [C.c_int, i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, i32, C.c_int, C.c_int, vp]
+    _lib = L
+    return L
+
+
+def status_string(status: int) -> str:
+    return lib().streambp_status_string(int(status)).decode()
+
+
+def _check(status: int, what: str):
+    if status != OK:
+        extra = ""
+        if status == E_CUDA:
+            extra = f" [cuda error {lib().streambp_last_cuda_error()}]"
+        raise StreamBPError(status, what + extra)
+
+
+def _dtype_code(dt: torch.dtype) -> int:
+    if dt == torch.float32:
+        return STREAMBP_F32
+    if dt == torch.bfloat16:
+        return STREAMBP_BF16
+    raise TypeError(f"unsupported storage dtype {dt}")
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "tensors must be contiguous CUDA tensors"
+    return t.data_ptr()
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream
+
+
+@dataclass
+class LayerConfig:
+    d_model: int
+    n_q_heads: int
+    n_kv_heads: int
+    head_dim: int
+    d_ff: int
+    qkv_bias: bool
+    rope_theta: float
+    rms_eps: float = 1e-6
+    dtype: torch.dtype = torch.bfloat16
+
+    def c(self) -> LayerCfgC:
+        return LayerCfgC(self.d_model, self.n_q_heads, self.n_kv_heads, self.head_dim, self.d_ff,
+                         1 if self.qkv_bias else 0, self.rope_theta, self.rms_eps, _dtype_code(self.dtype))
+
+
+@dataclass
+class HeadConfig:
+    d_model: int
+    vocab: int
+    rms_eps: float = 1e-6
+    ignore_index: int = -100
+    dtype: torch.dtype = torch.bfloat16
+
+    def c(self) -> HeadCfgC:
+        return HeadCfgC(self.d_model, self.vocab, self.rms_eps, self.ignore_index, _dtype_code(self.dtype))
+
+
+def _ptr_struct(tensors: Dict[str, torch.Tensor]) -> LayerPtrsC:
+    return LayerPtrsC(**{f: _ptr(tensors.get(f)) for f in WEIGHT_FIELDS})
+
+
+def layer_grad_shapes(cfg: LayerConfig) -> Dict[str, tuple]:
+    dq, dkv, d, I = cfg.n_q_heads * cfg.head_dim, cfg.n_kv_heads * cfg.head_dim, cfg.d_model, cfg.d_ff
+    shp = {"g1": (d,), "wq": (dq, d), "wk": (dkv, d), "wv": (dkv, d), "wo": (d, dq), "g2": (d,),
+           "w_gate": (I, d), "w_up": (I, d), "w_down": (d, I)}
+    if cfg.qkv_bias:
+        shp.update({"bq": (dq,), "bk": (dkv,), "bv": (dkv,)})
+    return shp
+
+
+def alloc_layer_grads(cfg: LayerConfig, device="cuda") -> Dict[str, torch.Tensor]:
+    return {k: torch.zeros(s, dtype=torch.float32, device=device) for k, s in layer_grad_shapes(cfg).items()}
+
+
+def layer_workspace_bytes(cfg: LayerConfig, T: int, chunk: int) -> int:
+    c = cfg.c()
+    return int(lib().streambp_layer_workspace_bytes(C.byref(c), T, chunk))
+
+
+def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def layer_backward(cfg: LayerConfig, weights: Dict[str, torch.Tensor], X: torch.Tensor, dY: torch.Tensor,
+                   chunk: int, grads: Dict[str, torch.Tensor], dX: torch.Tensor, workspace: torch.Tensor,
+                   pos0: int = 0, accumulate: bool = False, stream=None, check: bool = True) -> int:
+    """streambp_layer_backward; returns the status (raises on error when check=True)."""
+    c = cfg.c()
+    w, g = _ptr_struct(weights), _ptr_struct(grads)
+    st = lib().streambp_layer_backward(C.byref(c), C.byref(w), _ptr(X), _ptr(dY), X.shape[0], chunk, pos0,
+                                       1 if accumulate else 0, C.byref(g), _ptr(dX), _ptr(workspace),
+                                       workspace.numel(), _stream_ptr(stream))
+    if check:
+        _check(st, "streambp_layer_backward")
+    return st
+
+
+def lmhead_workspace_bytes(cfg: HeadConfig, T: int, chunk: int) -> int:
+    c = cfg.c()
+    return int(lib().streambp_lmhead_workspace_bytes(C.byref(c), T, chunk))
+
+
+def lmhead_ce_backward(cfg: HeadConfig, g_final, w_vocab, H, labels, chunk: int, loss, n_valid, dH, d_w_vocab,
+                       d_g_final, workspace, accumulate: bool = False, stream=None, check: bool = True) -> int:
+    c = cfg.c()
+    st = lib().streambp_lmhead_ce_backward(C.byref(c), _ptr(g_final), _ptr(w_vocab), _ptr(H), _ptr(labels),
+                                           H.shape[0], chunk, 1 if accumulate else 0, _ptr(loss), _ptr(n_valid),
+                                           _ptr(dH), _ptr(d_w_vocab), _ptr(d_g_final), _ptr(workspace),
+                                           workspace.numel(), _stream_ptr(stream))
+    if check:
+        _check(st, "streambp_lmhead_ce_backward")
+    return st
+
+
+def _model_cfg(n_layers: int, layer: LayerConfig, head: HeadConfig) -> ModelCfgC:
+    return ModelCfgC(n_layers, layer.c(), head.c())
+
+
+def model_workspace_bytes(n_layers: int, layer: LayerConfig, head: HeadConfig, T: int, chunk_layer: int,
+                          chunk_head: int) -> int:
+    c = _model_cfg(n_layers, layer, head)
+    return int(lib().streambp_model_workspace_bytes(C.byref(c), T, chunk_layer, chunk_head))
+
+
+def model_backward(layer: LayerConfig, head: HeadConfig, layers: Sequence[Dict[str, torch.Tensor]], g_final, w_vocab,
+                   labels, chunk_layer: int, chunk_head: int, loss, layer_grads: Sequence[Dict[str, torch.Tensor]],
+                   d_g_final, d_w_vocab, workspace, embed=None, ids=None, X0=None, d_embed=None, dX0=None,
+                   accumulate: bool = False, stream=None, check: bool = True) -> int:
+    L = len(layers)
+    c = _model_cfg(L, layer, head)
+    W = (LayerPtrsC * L)(*[_ptr_struct(w) for w in layers])
+    G = (LayerPtrsC * L)(*[_ptr_struct(g) for g in layer_grads])
+    T = labels.shape[0]
+    st = lib().streambp_model_backward(C.byref(c), _ptr(embed), W, _ptr(g_final), _ptr(w_vocab), _ptr(ids), _ptr(X0),
+                                       _ptr(labels), T, chunk_layer, chunk_head, 1 if accumulate else 0, _ptr(loss),
+                                       _ptr(d_embed), G, _ptr(d_g_final), _ptr(d_w_vocab), _ptr(dX0), _ptr(workspace),
+                                       workspace.numel(), _stream_ptr(stream))
+    if check:
+        _check(st, "streambp_model_backward")
+    return st
+
+
+def last_device_status(workspace: torch.Tensor, stream=None) -> int:
+    return int(lib().streambp_last_device_status(_ptr(workspace), _stream_ptr(stream)))
+
+
+def last_launch_count() -> int:
+    return int(lib().streambp_last_launch_count())
+
+
+def gemm(op: int, A: torch.Tensor, B: torch.Tensor, C_out: torch.Tensor, accumulate: bool = False, engine: int = 0,
+         stream=None, check: bool = True) -> int:
+    """streambp_gemm on 2-D row-major tensors (leading dimension = stride(0))."""
+    if op == OP_NT:
+        M, K = A.shape
+        N = B.shape[0]
+    elif op == OP_NN:
+        M, K = A.shape
+        N = B.shape[1]
+    else:
+        K, M = A.shape
+        N = B.shape[1]
+    assert A.stride(1) == 1 and B.stride(1) == 1 and C_out.stride(1) == 1
+    st = lib().streambp_gemm(op, M, N, K, A.data_ptr(), A.stride(0), B.data_ptr(), B.stride(0), C_out.data_ptr(),
+                             C_out.stride(0), _dtype_code(A.dtype), _dtype_code(C_out.dtype), 1 if accumulate else 0,
+                             engine, _stream_ptr(stream))
+    if check:
+        _check(st, "streambp_gemm")
+    return st

@@ -1,0 +1,290 @@
+// extern "C" boundary: argument validation, dtype dispatch, status handling.
+#include <cstdlib>
+#include <cstring>
+#include <vector>
+
+#include "common.cuh"
+
+namespace sbp {
+
+CallState &call_state() {
+    static thread_local CallState s;
+    return s;
+}
+
+namespace {
+int g_engine = -1;
+}
+int gemm_engine() {
+    if (g_engine < 0) {
+        const char *e = std::getenv("STREAMBP_GEMM_ENGINE");
+        g_engine = 0;
+        if (e && !std::strcmp(e, "simt")) g_engine = 1;
+        if (e && !std::strcmp(e, "tc")) g_engine = 2;
+    }
+    return g_engine;
+}
+void set_gemm_engine(int e) { g_engine = e; }
+
+template <typename TI, typename TC>
+int mm(GemmOp op, int64_t M, int64_t N, int64_t K, const TI *A, int64_t lda, const TI *B, int64_t ldb, TC *C,
+       int64_t ldc, const TI *bias, bool accumulate, cudaStream_t st) {
+    return gemm<TI, TC>(op, M, N, K, A, lda, B, ldb, C, ldc, bias, accumulate, st);
+}
+template <>
+int mm<bf16, float>(GemmOp op, int64_t M, int64_t N, int64_t K, const bf16 *A, int64_t lda, const bf16 *B, int64_t ldb,
+                    float *C, int64_t ldc, const bf16 *bias, bool accumulate, cudaStream_t st) {
+    const int e = gemm_engine();
+    if (e != 1 && gemm_tc_supported(op, M, N, K, lda, ldb, ldc, A, B, C, true))
+        return gemm_tc(op, M, N, K, A, lda, B, ldb, C, ldc, true, bias, accumulate, st);
+    if (e == 2) return STREAMBP_E_SHAPE;
+    return gemm<bf16, float>(op, M, N, K, A, lda, B, ldb, C, ldc, bias, accumulate, st);
+}
+template <>
+int mm<bf16, bf16>(GemmOp op, int64_t M, int64_t N, int64_t K, const bf16 *A, int64_t lda, const bf16 *B, int64_t ldb,
+                   bf16 *C, int64_t ldc, const bf16 *bias, bool accumulate, cudaStream_t st) {
+    const int e = gemm_engine();
+    if (e != 1 && !accumulate && gemm_tc_supported(op, M, N, K, lda, ldb, ldc, A, B, C, false))
+        return gemm_tc(op, M, N, K, A, lda, B, ldb, C, ldc, false, bias, false, st);
+    if (e == 2) return STREAMBP_E_SHAPE;
+    return gemm<bf16, bf16>(op, M, N, K, A, lda, B, ldb, C, ldc, bias, accumulate, st);
+}
+template int mm<float, float>(GemmOp, int64_t, int64_t, int64_t, const float *, int64_t, const float *, int64_t,
+                              float *, int64_t, const float *, bool, cudaStream_t);
+
+namespace {
+
+inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+int check_layer_cfg(const streambp_layer_cfg *c) {
+    if (!c) return STREAMBP_E_NULL;
+    if (c->dtype != STREAMBP_F32 && c->dtype != STREAMBP_BF16) return STREAMBP_E_DTYPE;
+    if (c->d_model < 8 || c->d_model % 8) return STREAMBP_E_SHAPE;
+    if (c->head_dim != 64 && c->head_dim != 128) return STREAMBP_E_SHAPE;
+    if (c->n_q_heads < 1 || c->n_kv_heads < 1 || c->n_q_heads % c->n_kv_heads) return STREAMBP_E_SHAPE;
+    if (c->d_ff < 8 || c->d_ff % 8) return STREAMBP_E_SHAPE;
+    if (!(c->rope_theta > 0.f) || !(c->rms_eps >= 0.f)) return STREAMBP_E_SHAPE;
+    return STREAMBP_OK;
+}
+int check_head_cfg(const streambp_head_cfg *c) {
+    if (!c) return STREAMBP_E_NULL;
+    if (c->dtype != STREAMBP_F32 && c->dtype != STREAMBP_BF16) return STREAMBP_E_DTYPE;
+    if (c->d_model < 8 || c->d_model % 8) return STREAMBP_E_SHAPE;
+    if (c->vocab < 1) return STREAMBP_E_SHAPE;
+    if (!(c->rms_eps >= 0.f)) return STREAMBP_E_SHAPE;
+    return STREAMBP_OK;
+}
+int check_layer_weights(const streambp_layer_cfg *c, const streambp_layer_weights *w) {
+    if (!w) return STREAMBP_E_NULL;
+    const void *req[] = {w->g1, w->wq, w->wk, w->wv, w->wo, w->g2, w->w_gate, w->w_up, w->w_down};
+    for (const void *p : req) {
+        if (!p) return STREAMBP_E_NULL;
+        if (!aligned(p, 16)) return STREAMBP_E_ALIGN;
+    }
+    if (c->qkv_bias) {
+        const void *b[] = {w->bq, w->bk, w->bv};
+        for (const void *p : b) {
+            if (!p) return STREAMBP_E_NULL;
+            if (!aligned(p, 16)) return STREAMBP_E_ALIGN;
+        }
+    }
+    return STREAMBP_OK;
+}
+int check_layer_grads(const streambp_layer_cfg *c, const streambp_layer_grads *g) {
+    if (!g) return STREAMBP_E_NULL;
+    float *req[] = {g->g1, g->wq, g->wk, g->wv, g->wo, g->g2, g->w_gate, g->w_up, g->w_down};
+    for (float *p : req) {
+        if (!p) return STREAMBP_E_NULL;
+        if (!aligned(p, 16)) return STREAMBP_E_ALIGN;
+    }
+    if (c->qkv_bias) {
+        float *b[] = {g->bq, g->bk, g->bv};
+        for (float *p : b) {
+            if (!p) return STREAMBP_E_NULL;
+            if (!aligned(p, 16)) return STREAMBP_E_ALIGN;
+        }
+    }
+    return STREAMBP_OK;
+}
+// weights with the bias pointers dropped when the configuration has no bias
+streambp_layer_weights effective(const streambp_layer_cfg *c, const streambp_layer_weights *w) {
+    streambp_layer_weights e = *w;
+    if (!c->qkv_bias) e.bq = e.bk = e.bv = nullptr;
+    return e;
+}
+int begin_call(void *ws, cudaStream_t st) {
+    call_state().cuda_error = 0;
+    call_state().launches = 0;
+    return fill_zero(ws, kHeaderBytes, st);
+}
+
+}  // namespace
+}  // namespace sbp
+
+using namespace sbp;
+
+extern "C" {
+
+size_t streambp_layer_workspace_bytes(const streambp_layer_cfg *cfg, int64_t T, int64_t chunk) {
+    if (check_layer_cfg(cfg) != STREAMBP_OK || T < 1 || chunk < 1) return 0;
+    return cfg->dtype == STREAMBP_F32 ? layer_workspace<float>(*cfg, T, chunk) : layer_workspace<bf16>(*cfg, T, chunk);
+}
+
+int streambp_layer_backward(const streambp_layer_cfg *cfg, const streambp_layer_weights *w, const void *X,
+                            const void *dY, int64_t T, int64_t chunk, int64_t pos0, int accumulate,
+                            const streambp_layer_grads *grads, void *dX, void *workspace, size_t workspace_bytes,
+                            void *cuda_stream) {
+    SBP_TRY(check_layer_cfg(cfg));
+    if (T < 1 || chunk < 1 || pos0 < 0) return STREAMBP_E_SHAPE;
+    SBP_TRY(check_layer_weights(cfg, w));
+    SBP_TRY(check_layer_grads(cfg, grads));
+    if (!X || !dY || !dX || !workspace) return STREAMBP_E_NULL;
+    if (!aligned(X, 16) || !aligned(dY, 16) || !aligned(dX, 16) || !aligned(workspace, 256)) return STREAMBP_E_ALIGN;
+    if (dX == X || dX == dY) return STREAMBP_E_SHAPE;
+    if (workspace_bytes < streambp_layer_workspace_bytes(cfg, T, chunk)) return STREAMBP_E_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    SBP_TRY(begin_call(workspace, st));
+    const streambp_layer_weights we = effective(cfg, w);
+    if (cfg->dtype == STREAMBP_F32)
+        return layer_backward<float>(*cfg, we, (const float *)X, (const float *)dY, T, chunk, pos0, accumulate != 0,
+                                     *grads, (float *)dX, workspace, st);
+    return layer_backward<bf16>(*cfg, we, (const bf16 *)X, (const bf16 *)dY, T, chunk, pos0, accumulate != 0, *grads,
+                                (bf16 *)dX, workspace, st);
+}
+
+size_t streambp_lmhead_workspace_bytes(const streambp_head_cfg *cfg, int64_t T, int64_t chunk) {
+    if (check_head_cfg(cfg) != STREAMBP_OK || T < 1 || chunk < 1) return 0;
+    return cfg->dtype == STREAMBP_F32 ? lmhead_workspace<float>(*cfg, T, chunk) : lmhead_workspace<bf16>(*cfg, T, chunk);
+}
+
+int streambp_lmhead_ce_backward(const streambp_head_cfg *cfg, const void *g_final, const void *w_vocab, const void *H,
+                                const int64_t *labels, int64_t T, int64_t chunk, int accumulate, float *loss,
+                                int64_t *n_valid, void *dH, float *d_w_vocab, float *d_g_final, void *workspace,
+                                size_t workspace_bytes, void *cuda_stream) {
+    SBP_TRY(check_head_cfg(cfg));
+    if (T < 1 || chunk < 1) return STREAMBP_E_SHAPE;
+    if (!g_final || !w_vocab || !H || !labels || !loss || !dH || !d_w_vocab || !d_g_final || !workspace)
+        return STREAMBP_E_NULL;
+    if (!aligned(g_final, 16) || !aligned(w_vocab, 16) || !aligned(H, 16) || !aligned(dH, 16) ||
+        !aligned(d_w_vocab, 16) || !aligned(d_g_final, 16) || !aligned(labels, 8) || !aligned(workspace, 256))
+        return STREAMBP_E_ALIGN;
+    if (workspace_bytes < streambp_lmhead_workspace_bytes(cfg, T, chunk)) return STREAMBP_E_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    SBP_TRY(begin_call(workspace, st));
+    if (cfg->dtype == STREAMBP_F32)
+        return lmhead_backward<float>(*cfg, (const float *)g_final, (const float *)w_vocab, (const float *)H, labels, T,
+                                      chunk, accumulate != 0, loss, n_valid, (float *)dH, d_w_vocab, d_g_final,
+                                      workspace, st);
+    return lmhead_backward<bf16>(*cfg, (const bf16 *)g_final, (const bf16 *)w_vocab, (const bf16 *)H, labels, T, chunk,
+                                 accumulate != 0, loss, n_valid, (bf16 *)dH, d_w_vocab, d_g_final, workspace, st);
+}
+
+static int check_model_cfg(const streambp_model_cfg *cfg) {
+    if (!cfg) return STREAMBP_E_NULL;
+    SBP_TRY(check_layer_cfg(&cfg->layer));
+    SBP_TRY(check_head_cfg(&cfg->head));
+    if (cfg->n_layers < 1) return STREAMBP_E_SHAPE;
+    if (cfg->layer.dtype != cfg->head.dtype) return STREAMBP_E_DTYPE;
+    if (cfg->layer.d_model != cfg->head.d_model) return STREAMBP_E_SHAPE;
+    return STREAMBP_OK;
+}
+
+size_t streambp_model_workspace_bytes(const streambp_model_cfg *cfg, int64_t T, int64_t chunk_layer,
+                                      int64_t chunk_head) {
+    if (check_model_cfg(cfg) != STREAMBP_OK || T < 1 || chunk_layer < 1 || chunk_head < 1) return 0;
+    return cfg->layer.dtype == STREAMBP_F32 ? model_workspace<float>(*cfg, T, chunk_layer, chunk_head)
+                                            : model_workspace<bf16>(*cfg, T, chunk_layer, chunk_head);
+}
+
+int streambp_model_backward(const streambp_model_cfg *cfg, const void *embed, const streambp_layer_weights *layers,
+                            const void *g_final, const void *w_vocab, const int64_t *ids, const void *X0,
+                            const int64_t *labels, int64_t T, int64_t chunk_layer, int64_t chunk_head, int accumulate,
+                            float *loss, float *d_embed, const streambp_layer_grads *layer_grads, float *d_g_final,
+                            float *d_w_vocab, void *dX0, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    SBP_TRY(check_model_cfg(cfg));
+    if (T < 1 || chunk_layer < 1 || chunk_head < 1) return STREAMBP_E_SHAPE;
+    if (!layers || !layer_grads || !g_final || !w_vocab || !labels || !loss || !d_g_final || !d_w_vocab || !workspace)
+        return STREAMBP_E_NULL;
+    if (ids ? !embed : !X0) return STREAMBP_E_NULL;
+    if (!aligned(g_final, 16) || !aligned(w_vocab, 16) || !aligned(d_g_final, 16) || !aligned(d_w_vocab, 16) ||
+        !aligned(workspace, 256) || (embed && !aligned(embed, 16)) || (X0 && !aligned(X0, 16)) ||
+        (dX0 && !aligned(dX0, 16)) || (d_embed && !aligned(d_embed, 16)))
+        return STREAMBP_E_ALIGN;
+    std::vector<streambp_layer_weights> eff(cfg->n_layers);
+    for (int l = 0; l < cfg->n_layers; l++) {
+        SBP_TRY(check_layer_weights(&cfg->layer, &layers[l]));
+        SBP_TRY(check_layer_grads(&cfg->layer, &layer_grads[l]));
+        eff[l] = effective(&cfg->layer, &layers[l]);
+    }
+    if (workspace_bytes < streambp_model_workspace_bytes(cfg, T, chunk_layer, chunk_head)) return STREAMBP_E_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    SBP_TRY(begin_call(workspace, st));
+    if (cfg->layer.dtype == STREAMBP_F32)
+        return model_backward<float>(*cfg, (const float *)embed, eff.data(), (const float *)g_final,
+                                     (const float *)w_vocab, ids, (const float *)X0, labels, T, chunk_layer, chunk_head,
+                                     accumulate != 0, loss, d_embed, layer_grads, d_g_final, d_w_vocab, (float *)dX0,
+                                     workspace, st);
+    return model_backward<bf16>(*cfg, (const bf16 *)embed, eff.data(), (const bf16 *)g_final, (const bf16 *)w_vocab,
+                                ids, (const bf16 *)X0, labels, T, chunk_layer, chunk_head, accumulate != 0, loss,
+                                d_embed, layer_grads, d_g_final, d_w_vocab, (bf16 *)dX0, workspace, st);
+}
+
+int streambp_last_device_status(void *workspace, void *cuda_stream) {
+    if (!workspace) return STREAMBP_E_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    WsHeader h;
+    if (!cuda_ok(cudaMemcpyAsync(&h, workspace, sizeof(h), cudaMemcpyDeviceToHost, st))) return STREAMBP_E_CUDA;
+    if (!cuda_ok(cudaStreamSynchronize(st))) return STREAMBP_E_CUDA;
+    return h.status;
+}
+
+const char *streambp_status_string(int s) {
+    switch (s) {
+        case STREAMBP_OK: return "ok";
+        case STREAMBP_E_NULL: return "a required pointer is NULL";
+        case STREAMBP_E_SHAPE: return "unsupported or inconsistent sizes";
+        case STREAMBP_E_ALIGN: return "pointer not sufficiently aligned";
+        case STREAMBP_E_WORKSPACE: return "workspace too small";
+        case STREAMBP_E_DTYPE: return "unknown dtype";
+        case STREAMBP_E_CUDA: return "CUDA call failed";
+        case STREAMBP_E_BAD_LABEL: return "label or token id out of range";
+        case STREAMBP_E_NO_VALID_LABELS: return "no unmasked label";
+        case STREAMBP_E_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+        default: return "unknown status";
+    }
+}
+
+int streambp_last_cuda_error(void) { return call_state().cuda_error; }
+int64_t streambp_last_launch_count(void) { return call_state().launches; }
+
+int streambp_gemm(int op, int64_t M, int64_t N, int64_t K, const void *A, int64_t lda, const void *B, int64_t ldb,
+                  void *C, int64_t ldc, int32_t in_dtype, int32_t out_dtype, int accumulate, int engine,
+                  void *cuda_stream) {
+    if (op < 0 || op > 2 || M < 1 || N < 1 || K < 1) return STREAMBP_E_SHAPE;
+    if (!A || !B || !C) return STREAMBP_E_NULL;
+    if (!aligned(A, 16) || !aligned(B, 16) || !aligned(C, 16)) return STREAMBP_E_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    call_state().cuda_error = 0;
+    call_state().launches = 0;
+    const GemmOp g = static_cast<GemmOp>(op);
+    const bool acc = accumulate != 0;
+    if (in_dtype == STREAMBP_F32) {
+        if (out_dtype != STREAMBP_F32 || engine == 2) return STREAMBP_E_DTYPE;
+        return gemm<float, float>(g, M, N, K, (const float *)A, lda, (const float *)B, ldb, (float *)C, ldc, nullptr,
+                                  acc, st);
+    }
+    if (in_dtype != STREAMBP_BF16) return STREAMBP_E_DTYPE;
+    const bool c32 = out_dtype == STREAMBP_F32;
+    if (!c32 && out_dtype != STREAMBP_BF16) return STREAMBP_E_DTYPE;
+    if (!c32 && acc) return STREAMBP_E_DTYPE;
+    const bool tc_ok = gemm_tc_supported(g, M, N, K, lda, ldb, ldc, A, B, C, c32);
+    if (engine == 2 && !tc_ok) return STREAMBP_E_SHAPE;
+    if (engine != 1 && tc_ok)
+        return gemm_tc(g, M, N, K, (const bf16 *)A, lda, (const bf16 *)B, ldb, C, ldc, c32, nullptr, acc, st);
+    if (c32)
+        return gemm<bf16, float>(g, M, N, K, (const bf16 *)A, lda, (const bf16 *)B, ldb, (float *)C, ldc, nullptr, acc,
+                                 st);
+    return gemm<bf16, bf16>(g, M, N, K, (const bf16 *)A, lda, (const bf16 *)B, ldb, (bf16 *)C, ldc, nullptr, false, st);
+}
+
+}  // extern "C"

@@ -1,0 +1,276 @@
+// Shared declarations of the streamed-backward CUDA library (internal).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/streambp.h"
+
+namespace sbp {
+
+typedef __nv_bfloat16 bf16;
+
+// ---- per-thread call context -------------------------------------------------
+struct CallState {
+    int cuda_error = 0;
+    int64_t launches = 0;
+};
+CallState &call_state();
+
+inline bool cuda_ok(cudaError_t e) {
+    if (e != cudaSuccess) {
+        call_state().cuda_error = (int)e;
+        return false;
+    }
+    return true;
+}
+
+// Every kernel launch goes through this so launches are counted and launch errors
+// are caught without synchronising.
+#define SBP_LAUNCH(kernel, grid, block, smem, stream, ...)                         \
+    do {                                                                           \
+        kernel<<<(grid), (block), (smem), (stream)>>>(__VA_ARGS__);                \
+        ::sbp::call_state().launches++;                                            \
+        if (!::sbp::cuda_ok(cudaGetLastError())) return STREAMBP_E_CUDA;           \
+    } while (0)
+
+#define SBP_TRY(expr)                         \
+    do {                                      \
+        int _st = (expr);                     \
+        if (_st != STREAMBP_OK) return _st;   \
+    } while (0)
+
+// ---- scalar conversion -------------------------------------------------------
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(bf16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f32<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+// ---- 16-byte vector access -----------------------------------------------------
+// Vec<T>::N elements of T in one 16-byte load/store.
+template <typename T> struct Vec;
+template <> struct Vec<float> {
+    static constexpr int N = 4;
+    float v[4];
+    __device__ __forceinline__ void load(const float *p) {
+        float4 t = *reinterpret_cast<const float4 *>(p);
+        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    }
+    __device__ __forceinline__ void store(float *p) const {
+        *reinterpret_cast<float4 *>(p) = make_float4(v[0], v[1], v[2], v[3]);
+    }
+};
+template <> struct Vec<bf16> {
+    static constexpr int N = 8;
+    float v[8];
+    __device__ __forceinline__ void load(const bf16 *p) {
+        uint4 t = *reinterpret_cast<const uint4 *>(p);
+        const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+        for (int i = 0; i < 4; i++) {
+            v[2 * i] = __uint_as_float(w[i] << 16);
+            v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        }
+    }
+    __device__ __forceinline__ void store(bf16 *p) const {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; i++) {
+            __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+            w[i] = *reinterpret_cast<uint32_t *>(&h);
+        }
+        *reinterpret_cast<uint4 *>(p) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+};
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// Block-wide sum for blocks of up to 1024 threads; `red` holds 33 floats of shared memory.
+__device__ __forceinline__ float block_sum(float v, float *red) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+    v = warp_sum(v);
+    __syncthreads();
+    if (lane == 0) red[w] = v;
+    __syncthreads();
+    if (w == 0) {
+        float t = lane < nw ? red[lane] : 0.f;
+        t = warp_sum(t);
+        if (lane == 0) red[32] = t;
+    }
+    __syncthreads();
+    return red[32];
+}
+__device__ __forceinline__ float block_max(float v, float *red) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+    v = warp_max(v);
+    __syncthreads();
+    if (lane == 0) red[w] = v;
+    __syncthreads();
+    if (w == 0) {
+        float t = lane < nw ? red[lane] : -INFINITY;
+        t = warp_max(t);
+        if (lane == 0) red[32] = t;
+    }
+    __syncthreads();
+    return red[32];
+}
+
+// ---- workspace header ----------------------------------------------------------
+// First 256 bytes of every workspace. `status` is the first non-OK device status.
+struct WsHeader {
+    int32_t status;
+    int32_t detail;
+    unsigned long long n_valid;
+    double loss_sum;
+};
+static constexpr size_t kHeaderBytes = 256;
+
+__device__ __forceinline__ void set_status(WsHeader *h, int st, int detail) {
+    if (atomicCAS(&h->status, 0, st) == 0) h->detail = detail;
+}
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Bump allocator over the caller's workspace; also used (with base == nullptr) to plan sizes.
+struct Arena {
+    char *base;
+    size_t off;
+    explicit Arena(void *b) : base(static_cast<char *>(b)), off(0) {}
+    template <typename T> T *take(size_t count) {
+        off = align_up(off, 256);
+        T *p = base ? reinterpret_cast<T *>(base + off) : nullptr;
+        off += count * sizeof(T);
+        return p;
+    }
+    void *take_bytes(size_t bytes) { return take<char>(bytes); }
+    size_t size() const { return align_up(off, 256); }
+};
+
+// ---- internal kernels (host launchers); T = storage dtype -----------------------
+enum GemmOp { OP_NT = 0, OP_NN = 1, OP_TN = 2 };
+
+// CUDA-core GEMM: C[M,N] (+)= op(A,B) (+ bias[N]); TC is the type of C. Returns a streambp_status.
+template <typename TI, typename TC>
+int gemm(GemmOp op, int64_t M, int64_t N, int64_t K, const TI *A, int64_t lda, const TI *B, int64_t ldb,
+         TC *C, int64_t ldc, const TI *bias, bool accumulate, cudaStream_t st);
+
+// tcgen05 GEMM (bf16 operands, fp32 accumulation in tensor memory).
+bool gemm_tc_supported(GemmOp op, int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb, int64_t ldc,
+                       const void *A, const void *B, const void *C, bool c_is_f32);
+int gemm_tc(GemmOp op, int64_t M, int64_t N, int64_t K, const bf16 *A, int64_t lda, const bf16 *B, int64_t ldb,
+            void *C, int64_t ldc, bool c_is_f32, const bf16 *bias, bool accumulate, cudaStream_t st);
+
+// Engine choice for the dispatching product below: 0 automatic, 1 CUDA cores only, 2 tensor cores required.
+int gemm_engine();
+void set_gemm_engine(int e);
+
+// Dispatching product used by the schedulers.
+template <typename TI, typename TC>
+int mm(GemmOp op, int64_t M, int64_t N, int64_t K, const TI *A, int64_t lda, const TI *B, int64_t ldb, TC *C,
+       int64_t ldc, const TI *bias, bool accumulate, cudaStream_t st);
+
+// h = x * rstd * gain ; rstd[t] saved. If res != nullptr: r = x + res is formed first, written to
+// r_out (fp32) and normalised instead of x.
+template <typename T>
+int rmsnorm_fwd(const T *x, const float *res, const T *gain, float eps, int64_t rows, int d, T *h, float *rstd,
+                float *r_out, cudaStream_t st);
+// out = add + ((dh*gain) - xhat*mean((dh*gain)*xhat)) * rstd ; x is given as xT (storage) or xF (fp32).
+// add: optional addT and/or addF. Outputs: optional outF (fp32) and outT (storage).
+// dgain += sum_t dh*xhat, reduced through partials[rmsnorm_bwd_partials_rows(rows), d].
+template <typename T>
+int rmsnorm_bwd(const float *dh, const T *xT, const float *xF, const float *rstd, const T *gain, const T *addT,
+                const float *addF, int64_t rows, int d, float *outF, T *outT, float *dgain, float *partials,
+                cudaStream_t st);
+int rmsnorm_bwd_partials_rows(int64_t rows);
+
+// cs[t, j] = (cos, sin)((pos0 + t) * theta^(-2j/dh)), j < dh/2
+int rope_table(float *cs, int64_t pos0, int64_t rows, int dh, float theta, cudaStream_t st);
+// out[t,h,:] = R(t) in[t,h,:] (transpose = false) or R(t)^T in[t,h,:]; cs row 0 belongs to in row 0.
+template <typename TO>
+int rope_apply(const float *in, const float *cs, int64_t rows, int heads, int dh, bool transpose, TO *out,
+               cudaStream_t st);
+template <typename T>
+int swiglu_fwd(const T *g, const T *u, int64_t n, T *m, cudaStream_t st);
+// in place: g := dg = dm*u*silu'(g), u := du = dm*silu(g)
+template <typename T>
+int swiglu_bwd(const T *dm, T *g, T *u, int64_t n, cudaStream_t st);
+// out (+)= column sums of a [rows, cols]; partials: [colsum_partial_rows(rows), cols]
+template <typename T>
+int colsum(const T *a, int64_t rows, int cols, float *out, bool accumulate, float *partials, cudaStream_t st);
+int colsum_partial_rows(int64_t rows);
+template <typename T>
+int cast_from_f32(const float *in, int64_t n, T *out, cudaStream_t st);
+// out = a + b (fp32 inputs)
+template <typename T>
+int add_cast(const float *a, const float *b, int64_t n, T *out, cudaStream_t st);
+int fill_zero(void *p, size_t bytes, cudaStream_t st);
+
+// Attention of one chunk of queries against the key/value prefix [0, q0 + n).
+// q,o,do: [n, Hq, dh]; k,v: [q0+n, Hkv, dh]; query row i sits at absolute row q0 + i and sees keys <= q0 + i.
+// lse: [Hq, n] (natural log, scores scaled by 1/sqrt(dh)).
+template <typename T>
+int attention_fwd(const T *q, const T *k, const T *v, int64_t n, int64_t q0, int Hq, int Hkv, int dh, T *o,
+                  float *lse, cudaStream_t st);
+// delta[h, i] = sum_j do*o (scratch [Hq, n]); dq fp32 [n,Hq,dh] overwritten; dk, dv fp32 [q0+n,Hkv,dh] accumulated.
+template <typename T>
+int attention_bwd(const T *q, const T *k, const T *v, const T *o, const T *dout, const float *lse, int64_t n,
+                  int64_t q0, int Hq, int Hkv, int dh, float *delta, float *dq, float *dk, float *dv,
+                  cudaStream_t st);
+
+// LM head pieces
+int count_valid_labels(const int64_t *labels, int64_t T, int64_t vocab, int64_t ignore, WsHeader *hdr,
+                       cudaStream_t st);
+// z: [rows, V] fp32 logits -> dz (storage dtype; may alias z when T == float); row_loss[rows] fp32.
+template <typename T>
+int ce_rows(const float *z, const int64_t *labels, int64_t rows, int64_t V, int64_t ignore, const WsHeader *hdr,
+            T *dz, float *row_loss, cudaStream_t st);
+int loss_accumulate(const float *row_loss, int64_t rows, WsHeader *hdr, cudaStream_t st);
+int loss_finalize(WsHeader *hdr, float *loss, int64_t *n_valid, cudaStream_t st);
+
+template <typename T>
+int embedding_gather(const T *embed, const int64_t *ids, int64_t rows, int d, int64_t vocab, T *out, WsHeader *hdr,
+                     cudaStream_t st);
+template <typename T>
+int embedding_scatter_add(const T *dx, const int64_t *ids, int64_t rows, int d, int64_t vocab, float *d_embed,
+                          cudaStream_t st);
+
+// ---- schedulers (T = storage dtype) --------------------------------------------------
+template <typename T>
+size_t layer_workspace(const streambp_layer_cfg &c, int64_t T_, int64_t chunk);
+template <typename T>
+int layer_backward(const streambp_layer_cfg &c, const streambp_layer_weights &w, const T *X, const T *dY, int64_t T_,
+                   int64_t chunk, int64_t pos0, bool accumulate, const streambp_layer_grads &g, T *dX, void *ws,
+                   cudaStream_t st);
+// Y = layer(X), chunked; uses the same workspace plan as layer_backward.
+template <typename T>
+int layer_forward(const streambp_layer_cfg &c, const streambp_layer_weights &w, const T *X, int64_t T_, int64_t chunk,
+                  int64_t pos0, T *Y, void *ws, cudaStream_t st);
+
+template <typename T>
+size_t lmhead_workspace(const streambp_head_cfg &c, int64_t T_, int64_t chunk);
+template <typename T>
+int lmhead_backward(const streambp_head_cfg &c, const T *g_final, const T *w_vocab, const T *H, const int64_t *labels,
+                    int64_t T_, int64_t chunk, bool accumulate, float *loss, int64_t *n_valid, T *dH, float *d_w_vocab,
+                    float *d_g_final, void *ws, cudaStream_t st);
+
+template <typename T>
+size_t model_workspace(const streambp_model_cfg &c, int64_t T_, int64_t chunk_layer, int64_t chunk_head);
+template <typename T>
+int model_backward(const streambp_model_cfg &c, const T *embed, const streambp_layer_weights *layers, const T *g_final,
+                   const T *w_vocab, const int64_t *ids, const T *X0, const int64_t *labels, int64_t T_,
+                   int64_t chunk_layer, int64_t chunk_head, bool accumulate, float *loss, float *d_embed,
+                   const streambp_layer_grads *layer_grads, float *d_g_final, float *d_w_vocab, T *dX0, void *ws,
+                   cudaStream_t st);
+
+}  // namespace sbp

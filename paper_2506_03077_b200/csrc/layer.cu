@@ -1,0 +1,212 @@
+// Host-side chunk scheduler of one decoder layer: the partitioned re-forward and the accumulation
+// of the paper's Sec. 3.2.2, as a fixed sequence of kernel launches on the caller's stream.
+//
+// K and V (rotated) are produced once for all T rows and cached; chunks are then processed from
+// the LAST to the first.  The order does not change the sum (any order of the terms of Eq. (1) is
+// exact); running backwards makes the fp32 dK/dV rows of chunk i final as soon as chunk i itself
+// has been processed (only chunks >= i attend to them), so the K/V-projection backward of chunk i
+// runs inside the same iteration, on the h1 rows that are already resident.
+#include "common.cuh"
+
+namespace sbp {
+
+namespace {
+
+template <typename T>
+struct LayerWs {
+    WsHeader *hdr;
+    float *cs;            // [T, dh/2] (cos, sin)
+    T *K, *V;             // [T, dkv]
+    float *dK, *dV;       // [T, dkv]
+    // one chunk
+    T *h1, *Q, *O, *h2, *g, *u, *m, *dr_s, *dO, *dk_s, *dv_s;
+    float *fa, *r, *dr, *rstd1, *rstd2, *lse, *delta, *partials;
+    size_t bytes;
+};
+
+template <typename T>
+LayerWs<T> plan(const streambp_layer_cfg &c, int64_t T_, int64_t chunk, void *base) {
+    const int64_t cn = chunk < T_ ? chunk : T_;
+    const int64_t d = c.d_model, dq = (int64_t)c.n_q_heads * c.head_dim, dkv = (int64_t)c.n_kv_heads * c.head_dim;
+    const int64_t I = c.d_ff, wide = dq > d ? dq : d;
+    Arena a(base);
+    LayerWs<T> w;
+    w.hdr = reinterpret_cast<WsHeader *>(a.take_bytes(kHeaderBytes));
+    w.cs = a.take<float>(T_ * c.head_dim);
+    w.K = a.take<T>(T_ * dkv);
+    w.V = a.take<T>(T_ * dkv);
+    w.dK = a.take<float>(T_ * dkv);
+    w.dV = a.take<float>(T_ * dkv);
+    w.h1 = a.take<T>(cn * d);
+    w.Q = a.take<T>(cn * dq);
+    w.O = a.take<T>(cn * dq);
+    w.h2 = a.take<T>(cn * d);
+    w.g = a.take<T>(cn * I);
+    w.u = a.take<T>(cn * I);
+    w.m = a.take<T>(cn * I);
+    w.dr_s = a.take<T>(cn * d);
+    w.dO = a.take<T>(cn * dq);
+    w.dk_s = a.take<T>(cn * dkv);
+    w.dv_s = a.take<T>(cn * dkv);
+    w.fa = a.take<float>(cn * wide);
+    w.r = a.take<float>(cn * d);
+    w.dr = a.take<float>(cn * d);
+    w.rstd1 = a.take<float>(cn);
+    w.rstd2 = a.take<float>(cn);
+    w.lse = a.take<float>(cn * c.n_q_heads);
+    w.delta = a.take<float>(cn * c.n_q_heads);
+    w.partials = a.take<float>(64 * wide);
+    w.bytes = a.size();
+    return w;
+}
+
+// K/V for all rows, chunk by chunk: h1 = RMSNorm1(X), K = RoPE(h1 Wk^T + bk), V = h1 Wv^T + bv
+template <typename T>
+int kv_prologue(const streambp_layer_cfg &c, const streambp_layer_weights &w, const T *X, int64_t T_, int64_t cn,
+                int64_t pos0, LayerWs<T> &s, cudaStream_t st) {
+    const int d = c.d_model, dh = c.head_dim, Hkv = c.n_kv_heads;
+    const int64_t dkv = (int64_t)Hkv * dh;
+    SBP_TRY(rope_table(s.cs, pos0, T_, dh, c.rope_theta, st));
+    for (int64_t r0 = 0; r0 < T_; r0 += cn) {
+        const int64_t n = (T_ - r0 < cn) ? T_ - r0 : cn;
+        SBP_TRY(rmsnorm_fwd<T>(X + r0 * d, nullptr, (const T *)w.g1, c.rms_eps, n, d, s.h1, s.rstd1, nullptr, st));
+        SBP_TRY((mm<T, float>(OP_NT, n, dkv, d, s.h1, d, (const T *)w.wk, d, s.fa, dkv, (const T *)w.bk, false, st)));
+        SBP_TRY(rope_apply<T>(s.fa, s.cs + r0 * dh, n, Hkv, dh, false, s.K + r0 * dkv, st));
+        SBP_TRY((mm<T, T>(OP_NT, n, dkv, d, s.h1, d, (const T *)w.wv, d, s.V + r0 * dkv, dkv, (const T *)w.bv, false, st)));
+    }
+    return STREAMBP_OK;
+}
+
+// Re-forward of one chunk up to m = silu(g) * u. Leaves h1, rstd1, Q, O, lse, r, h2, rstd2, g, u, m.
+template <typename T>
+int chunk_forward(const streambp_layer_cfg &c, const streambp_layer_weights &w, const T *X, int64_t r0, int64_t n,
+                  LayerWs<T> &s, cudaStream_t st) {
+    const int d = c.d_model, dh = c.head_dim, Hq = c.n_q_heads, Hkv = c.n_kv_heads;
+    const int64_t dq = (int64_t)Hq * dh, I = c.d_ff;
+    const T *Xi = X + r0 * d;
+    SBP_TRY(rmsnorm_fwd<T>(Xi, nullptr, (const T *)w.g1, c.rms_eps, n, d, s.h1, s.rstd1, nullptr, st));
+    SBP_TRY((mm<T, float>(OP_NT, n, dq, d, s.h1, d, (const T *)w.wq, d, s.fa, dq, (const T *)w.bq, false, st)));
+    SBP_TRY(rope_apply<T>(s.fa, s.cs + r0 * dh, n, Hq, dh, false, s.Q, st));
+    SBP_TRY(attention_fwd<T>(s.Q, s.K, s.V, n, r0, Hq, Hkv, dh, s.O, s.lse, st));
+    SBP_TRY((mm<T, float>(OP_NT, n, d, dq, s.O, dq, (const T *)w.wo, dq, s.fa, d, nullptr, false, st)));
+    SBP_TRY(rmsnorm_fwd<T>(Xi, s.fa, (const T *)w.g2, c.rms_eps, n, d, s.h2, s.rstd2, s.r, st));
+    SBP_TRY((mm<T, T>(OP_NT, n, I, d, s.h2, d, (const T *)w.w_gate, d, s.g, I, nullptr, false, st)));
+    SBP_TRY((mm<T, T>(OP_NT, n, I, d, s.h2, d, (const T *)w.w_up, d, s.u, I, nullptr, false, st)));
+    SBP_TRY(swiglu_fwd<T>(s.g, s.u, n * I, s.m, st));
+    return STREAMBP_OK;
+}
+
+}  // namespace
+
+template <typename T>
+size_t layer_workspace(const streambp_layer_cfg &c, int64_t T_, int64_t chunk) {
+    return plan<T>(c, T_, chunk, nullptr).bytes;
+}
+
+template <typename T>
+int layer_forward(const streambp_layer_cfg &c, const streambp_layer_weights &w, const T *X, int64_t T_, int64_t chunk,
+                  int64_t pos0, T *Y, void *ws, cudaStream_t st) {
+    const int64_t cn = chunk < T_ ? chunk : T_;
+    LayerWs<T> s = plan<T>(c, T_, chunk, ws);
+    const int d = c.d_model;
+    const int64_t I = c.d_ff;
+    SBP_TRY(kv_prologue<T>(c, w, X, T_, cn, pos0, s, st));
+    for (int64_t r0 = 0; r0 < T_; r0 += cn) {
+        const int64_t n = (T_ - r0 < cn) ? T_ - r0 : cn;
+        SBP_TRY(chunk_forward<T>(c, w, X, r0, n, s, st));
+        SBP_TRY((mm<T, float>(OP_NT, n, d, I, s.m, I, (const T *)w.w_down, I, s.fa, d, nullptr, false, st)));
+        SBP_TRY(add_cast<T>(s.r, s.fa, n * d, Y + r0 * d, st));
+    }
+    return STREAMBP_OK;
+}
+
+template <typename T>
+int layer_backward(const streambp_layer_cfg &c, const streambp_layer_weights &w, const T *X, const T *dY, int64_t T_,
+                   int64_t chunk, int64_t pos0, bool accumulate, const streambp_layer_grads &G, T *dX, void *ws,
+                   cudaStream_t st) {
+    const int64_t cn = chunk < T_ ? chunk : T_;
+    LayerWs<T> s = plan<T>(c, T_, chunk, ws);
+    const int d = c.d_model, dh = c.head_dim, Hq = c.n_q_heads, Hkv = c.n_kv_heads;
+    const int64_t dq = (int64_t)Hq * dh, dkv = (int64_t)Hkv * dh, I = c.d_ff;
+    constexpr bool kF32 = sizeof(T) == 4;
+
+    SBP_TRY(kv_prologue<T>(c, w, X, T_, cn, pos0, s, st));
+    SBP_TRY(fill_zero(s.dK, sizeof(float) * T_ * dkv, st));
+    SBP_TRY(fill_zero(s.dV, sizeof(float) * T_ * dkv, st));
+    if (!accumulate) {  // vectors are always added to; matrices are overwritten by the first chunk's product
+        SBP_TRY(fill_zero(G.g1, sizeof(float) * d, st));
+        SBP_TRY(fill_zero(G.g2, sizeof(float) * d, st));
+        if (c.qkv_bias) {
+            SBP_TRY(fill_zero(G.bq, sizeof(float) * dq, st));
+            SBP_TRY(fill_zero(G.bk, sizeof(float) * dkv, st));
+            SBP_TRY(fill_zero(G.bv, sizeof(float) * dkv, st));
+        }
+    }
+    const int64_t D = (T_ + cn - 1) / cn;
+    for (int64_t i = D - 1; i >= 0; i--) {
+        const int64_t r0 = i * cn;
+        const int64_t n = (T_ - r0 < cn) ? T_ - r0 : cn;
+        const bool acc = accumulate || i != D - 1;
+        const T *Xi = X + r0 * d, *dYi = dY + r0 * d;
+        SBP_TRY(chunk_forward<T>(c, w, X, r0, n, s, st));
+
+        // ---- MLP backward ----
+        SBP_TRY((mm<T, float>(OP_TN, d, I, n, dYi, d, s.m, I, G.w_down, I, nullptr, acc, st)));       // dWd += dY^T m
+        SBP_TRY((mm<T, T>(OP_NN, n, I, d, dYi, d, (const T *)w.w_down, I, s.m, I, nullptr, false, st)));  // dm = dY Wd
+        SBP_TRY(swiglu_bwd<T>(s.m, s.g, s.u, n * I, st));                                             // g := dg, u := du
+        SBP_TRY((mm<T, float>(OP_TN, I, d, n, s.g, I, s.h2, d, G.w_gate, d, nullptr, acc, st)));
+        SBP_TRY((mm<T, float>(OP_TN, I, d, n, s.u, I, s.h2, d, G.w_up, d, nullptr, acc, st)));
+        SBP_TRY((mm<T, float>(OP_NN, n, d, I, s.g, I, (const T *)w.w_gate, d, s.fa, d, nullptr, false, st)));
+        SBP_TRY((mm<T, float>(OP_NN, n, d, I, s.u, I, (const T *)w.w_up, d, s.fa, d, nullptr, true, st)));   // dh2
+        // dr = dY + norm2_bwd(dh2)
+        SBP_TRY(rmsnorm_bwd<T>(s.fa, nullptr, s.r, s.rstd2, (const T *)w.g2, dYi, nullptr, n, d, s.dr,
+                               kF32 ? nullptr : s.dr_s, G.g2, s.partials, st));
+        const T *dr_op = kF32 ? reinterpret_cast<const T *>(s.dr) : s.dr_s;
+
+        // ---- attention output projection backward ----
+        SBP_TRY((mm<T, float>(OP_TN, d, dq, n, dr_op, d, s.O, dq, G.wo, dq, nullptr, acc, st)));       // dWo += dr^T O
+        SBP_TRY((mm<T, T>(OP_NN, n, dq, d, dr_op, d, (const T *)w.wo, dq, s.dO, dq, nullptr, false, st)));  // dO = dr Wo
+
+        // ---- partitioned attention backward: dQ (into fa), dK/dV prefix += ----
+        SBP_TRY(attention_bwd<T>(s.Q, s.K, s.V, s.O, s.dO, s.lse, n, r0, Hq, Hkv, dh, s.delta, s.fa, s.dK, s.dV, st));
+
+        // ---- Q projection backward ----
+        T *dq_s = s.Q;  // Q is dead after the attention backward
+        SBP_TRY(rope_apply<T>(s.fa, s.cs + r0 * dh, n, Hq, dh, true, dq_s, st));
+        SBP_TRY((mm<T, float>(OP_TN, dq, d, n, dq_s, dq, s.h1, d, G.wq, d, nullptr, acc, st)));
+        if (c.qkv_bias) SBP_TRY(colsum<T>(dq_s, n, (int)dq, G.bq, true, s.partials, st));
+        SBP_TRY((mm<T, float>(OP_NN, n, d, dq, dq_s, dq, (const T *)w.wq, d, s.fa, d, nullptr, false, st)));   // dh1
+
+        // ---- K/V projection backward of this chunk's rows (their dK/dV are final now) ----
+        SBP_TRY(rope_apply<T>(s.dK + r0 * dkv, s.cs + r0 * dh, n, Hkv, dh, true, s.dk_s, st));
+        SBP_TRY(cast_from_f32<T>(s.dV + r0 * dkv, n * dkv, s.dv_s, st));
+        SBP_TRY((mm<T, float>(OP_TN, dkv, d, n, s.dk_s, dkv, s.h1, d, G.wk, d, nullptr, acc, st)));
+        SBP_TRY((mm<T, float>(OP_TN, dkv, d, n, s.dv_s, dkv, s.h1, d, G.wv, d, nullptr, acc, st)));
+        if (c.qkv_bias) {
+            SBP_TRY(colsum<T>(s.dk_s, n, (int)dkv, G.bk, true, s.partials, st));
+            SBP_TRY(colsum<T>(s.dv_s, n, (int)dkv, G.bv, true, s.partials, st));
+        }
+        SBP_TRY((mm<T, float>(OP_NN, n, d, dkv, s.dk_s, dkv, (const T *)w.wk, d, s.fa, d, nullptr, true, st)));
+        SBP_TRY((mm<T, float>(OP_NN, n, d, dkv, s.dv_s, dkv, (const T *)w.wv, d, s.fa, d, nullptr, true, st)));
+
+        // ---- dX = dr + norm1_bwd(dh1) ----
+        SBP_TRY(rmsnorm_bwd<T>(s.fa, Xi, nullptr, s.rstd1, (const T *)w.g1, nullptr, s.dr, n, d, nullptr, dX + r0 * d,
+                               G.g1, s.partials, st));
+    }
+    return STREAMBP_OK;
+}
+
+template size_t layer_workspace<float>(const streambp_layer_cfg &, int64_t, int64_t);
+template size_t layer_workspace<bf16>(const streambp_layer_cfg &, int64_t, int64_t);
+template int layer_forward<float>(const streambp_layer_cfg &, const streambp_layer_weights &, const float *, int64_t,
+                                  int64_t, int64_t, float *, void *, cudaStream_t);
+template int layer_forward<bf16>(const streambp_layer_cfg &, const streambp_layer_weights &, const bf16 *, int64_t,
+                                 int64_t, int64_t, bf16 *, void *, cudaStream_t);
+template int layer_backward<float>(const streambp_layer_cfg &, const streambp_layer_weights &, const float *,
+                                   const float *, int64_t, int64_t, int64_t, bool, const streambp_layer_grads &,
+                                   float *, void *, cudaStream_t);
+template int layer_backward<bf16>(const streambp_layer_cfg &, const streambp_layer_weights &, const bf16 *,
+                                  const bf16 *, int64_t, int64_t, int64_t, bool, const streambp_layer_grads &, bf16 *,
+                                  void *, cudaStream_t);
+
+}  // namespace sbp

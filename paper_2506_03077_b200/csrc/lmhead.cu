@@ -1,0 +1,80 @@
+// Host-side scheduler of the streamed final-norm + LM-head + cross-entropy backward
+// (Sec. 3.2.1: logits are formed, used and dropped one sequence chunk at a time).
+#include "common.cuh"
+
+namespace sbp {
+
+namespace {
+template <typename T>
+struct HeadWs {
+    WsHeader *hdr;
+    T *hn, *dz;
+    float *z, *dhn, *rstd, *row_loss, *partials;
+    size_t bytes;
+};
+
+template <typename T>
+HeadWs<T> plan(const streambp_head_cfg &c, int64_t T_, int64_t chunk, void *base) {
+    const int64_t cn = chunk < T_ ? chunk : T_;
+    const int64_t d = c.d_model, V = c.vocab;
+    Arena a(base);
+    HeadWs<T> w;
+    w.hdr = reinterpret_cast<WsHeader *>(a.take_bytes(kHeaderBytes));
+    w.hn = a.take<T>(cn * d);
+    w.z = a.take<float>(cn * V);
+    // fp32 storage: dlogits overwrite the logits in place
+    w.dz = sizeof(T) == 4 ? reinterpret_cast<T *>(w.z) : a.take<T>(cn * V);
+    w.dhn = a.take<float>(cn * d);
+    w.rstd = a.take<float>(cn);
+    w.row_loss = a.take<float>(cn);
+    w.partials = a.take<float>(64 * d);
+    w.bytes = a.size();
+    return w;
+}
+}  // namespace
+
+template <typename T>
+size_t lmhead_workspace(const streambp_head_cfg &c, int64_t T_, int64_t chunk) {
+    return plan<T>(c, T_, chunk, nullptr).bytes;
+}
+
+template <typename T>
+int lmhead_backward(const streambp_head_cfg &c, const T *g_final, const T *w_vocab, const T *H, const int64_t *labels,
+                    int64_t T_, int64_t chunk, bool accumulate, float *loss, int64_t *n_valid, T *dH, float *d_w_vocab,
+                    float *d_g_final, void *ws, cudaStream_t st) {
+    const int64_t cn = chunk < T_ ? chunk : T_;
+    HeadWs<T> s = plan<T>(c, T_, chunk, ws);
+    const int d = c.d_model;
+    const int64_t V = c.vocab;
+    // N is global: it is counted before the chunk loop so that every chunk scales by the same 1/N
+    SBP_TRY(count_valid_labels(labels, T_, V, c.ignore_index, s.hdr, st));
+    if (!accumulate) SBP_TRY(fill_zero(d_g_final, sizeof(float) * d, st));
+    const int64_t D = (T_ + cn - 1) / cn;
+    for (int64_t i = 0; i < D; i++) {
+        const int64_t r0 = i * cn;
+        const int64_t n = (T_ - r0 < cn) ? T_ - r0 : cn;
+        const bool acc = accumulate || i != 0;
+        const T *Hi = H + r0 * d;
+        SBP_TRY(rmsnorm_fwd<T>(Hi, nullptr, g_final, c.rms_eps, n, d, s.hn, s.rstd, nullptr, st));
+        SBP_TRY((mm<T, float>(OP_NT, n, V, d, s.hn, d, w_vocab, d, s.z, V, nullptr, false, st)));           // logits
+        SBP_TRY(ce_rows<T>(s.z, labels + r0, n, V, c.ignore_index, s.hdr, s.dz, s.row_loss, st));
+        SBP_TRY(loss_accumulate(s.row_loss, n, s.hdr, st));
+        SBP_TRY((mm<T, float>(OP_TN, V, d, n, s.dz, V, s.hn, d, d_w_vocab, d, nullptr, acc, st)));          // dW += dZ^T hn
+        SBP_TRY((mm<T, float>(OP_NN, n, d, V, s.dz, V, w_vocab, d, s.dhn, d, nullptr, false, st)));         // dhn = dZ W
+        SBP_TRY(rmsnorm_bwd<T>(s.dhn, Hi, nullptr, s.rstd, g_final, nullptr, nullptr, n, d, nullptr, dH + r0 * d,
+                               d_g_final, s.partials, st));
+    }
+    SBP_TRY(loss_finalize(s.hdr, loss, n_valid, st));
+    return STREAMBP_OK;
+}
+
+template size_t lmhead_workspace<float>(const streambp_head_cfg &, int64_t, int64_t);
+template size_t lmhead_workspace<bf16>(const streambp_head_cfg &, int64_t, int64_t);
+template int lmhead_backward<float>(const streambp_head_cfg &, const float *, const float *, const float *,
+                                    const int64_t *, int64_t, int64_t, bool, float *, int64_t *, float *, float *,
+                                    float *, void *, cudaStream_t);
+template int lmhead_backward<bf16>(const streambp_head_cfg &, const bf16 *, const bf16 *, const bf16 *,
+                                   const int64_t *, int64_t, int64_t, bool, float *, int64_t *, bf16 *, float *,
+                                   float *, void *, cudaStream_t);
+
+}  // namespace sbp

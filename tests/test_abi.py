@@ -1,0 +1,110 @@
+"""The C-ABI library loads, exports what include/streambp.h declares, and rejects bad
+arguments on the host (no GPU needed: validation precedes every CUDA call)."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2506_03077_b200 import binding as B
+from paper_2506_03077_b200 import build as build_mod
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    if not os.path.exists(B.LIB_PATH):
+        build_mod.build()
+    return B.lib()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "streambp.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(streambp_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = declared_functions()
+    assert {"streambp_layer_backward", "streambp_lmhead_ce_backward", "streambp_model_backward",
+            "streambp_layer_workspace_bytes", "streambp_last_device_status"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), n
+    assert set(names) == set(B.EXPORTS)
+
+
+def test_status_strings(lib):
+    assert B.status_string(0) == "ok"
+    seen = {B.status_string(s) for s in range(-9, 1)}
+    assert len(seen) == 10 and "unknown status" not in seen
+    assert B.status_string(-77) == "unknown status"
+
+
+def cfg(**kw):
+    base = dict(d_model=256, n_q_heads=4, n_kv_heads=2, head_dim=64, d_ff=688, qkv_bias=False, rope_theta=1e4)
+    base.update(kw)
+    import torch
+    return B.LayerConfig(dtype=torch.float32, **base)
+
+
+def test_workspace_query_rejects_bad_shapes(lib):
+    assert B.layer_workspace_bytes(cfg(), 512, 128) > 0
+    assert B.layer_workspace_bytes(cfg(head_dim=96), 512, 128) == 0
+    assert B.layer_workspace_bytes(cfg(n_kv_heads=3), 512, 128) == 0
+    assert B.layer_workspace_bytes(cfg(d_model=250), 512, 128) == 0
+    assert B.layer_workspace_bytes(cfg(), 0, 128) == 0
+    assert B.layer_workspace_bytes(cfg(), 512, 0) == 0
+    # chunk >= T is the un-partitioned mode and needs the most memory
+    small, full = B.layer_workspace_bytes(cfg(), 512, 128), B.layer_workspace_bytes(cfg(), 512, 512)
+    assert full > small and B.layer_workspace_bytes(cfg(), 512, 4096) == full
+
+
+def test_workspace_matches_memory_model(lib):
+    """Per-chunk activations scale with the chunk, the K/V set with T (Sec. 3.2.2, memory efficiency)."""
+    import torch
+    c = B.LayerConfig(4096, 32, 8, 128, 14336, False, 5e5, dtype=torch.bfloat16)
+    T = 32768
+    kv_set = T * 1024 * (2 + 2 + 4 + 4) + T * 128 * 4     # K, V bf16; dK, dV fp32; rope table
+    w1, w2 = B.layer_workspace_bytes(c, T, 1024), B.layer_workspace_bytes(c, T, 2048)
+    per_row = (w2 - w1) / 1024
+    assert abs((w1 - 1024 * per_row) - kv_set) < (1 << 21)
+    # one chunk row: 3 [I] + h1,h2,dr_s [d] + Q,O,dO [dq] + dk,dv [dkv] in bf16; fa, r, dr fp32; small vectors
+    expect = 2 * (3 * 14336 + 3 * 4096 + 3 * 4096 + 2 * 1024) + 4 * (3 * 4096) + 4 * (2 + 2 * 32)
+    assert abs(per_row - expect) < 64
+
+
+def test_host_side_errors(lib):
+    import torch
+    c = cfg().c()
+    w = B.LayerPtrsC(**{f: 4096 for f in B.WEIGHT_FIELDS})
+    g = B.LayerPtrsC(**{f: 4096 for f in B.WEIGHT_FIELDS})
+    call = lambda **kw: lib.streambp_layer_backward(
+        C.byref(kw.get("c", c)), C.byref(kw.get("w", w)), kw.get("X", 4096), kw.get("dY", 8192), kw.get("T", 512),
+        kw.get("chunk", 128), 0, 0, C.byref(kw.get("g", g)), kw.get("dX", 12288), kw.get("ws", 1 << 20),
+        kw.get("wsb", 16), None)
+    assert call() == B.E_WORKSPACE
+    assert call(X=None) == B.E_NULL
+    assert call(X=4100) == B.E_ALIGN
+    assert call(ws=(1 << 20) + 16) == B.E_ALIGN
+    assert call(T=0) == B.E_SHAPE
+    assert call(dX=4096) == B.E_SHAPE            # dX aliases X
+    bad = cfg().c()
+    bad.dtype = 7
+    assert call(c=bad) == B.E_DTYPE
+    wnull = B.LayerPtrsC(**{f: (None if f == "wo" else 4096) for f in B.WEIGHT_FIELDS})
+    assert call(w=wnull) == B.E_NULL
+    # biases are required only when the configuration says so
+    wnob = B.LayerPtrsC(**{f: (None if f in ("bq", "bk", "bv") else 4096) for f in B.WEIGHT_FIELDS})
+    assert call(w=wnob, g=wnob) == B.E_WORKSPACE
+    cb = cfg(qkv_bias=True).c()
+    assert call(c=cb, w=wnob) == B.E_NULL
+    h = B.HeadConfig(256, 4096, dtype=torch.float32).c()
+    st = lib.streambp_lmhead_ce_backward(C.byref(h), 4096, 4096, 4096, 4096, 512, 128, 0, 4096, 4096, 4096, 4096,
+                                         4096, 1 << 20, 16, None)
+    assert st == B.E_WORKSPACE
+    st = lib.streambp_lmhead_ce_backward(C.byref(h), 4096, 4096, 4096, None, 512, 128, 0, 4096, 4096, 4096, 4096,
+                                         4096, 1 << 20, 1 << 30, None)
+    assert st == B.E_NULL
+    assert lib.streambp_gemm(5, 8, 8, 8, 4096, 8, 4096, 8, 4096, 8, 1, 0, 0, 0, None) == B.E_SHAPE
+    assert lib.streambp_last_device_status(None, None) == B.E_NULL

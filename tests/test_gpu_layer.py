@@ -1,0 +1,87 @@
+"""GPU parity: streambp_layer_backward (through the C ABI) against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import streambp_oracle as O
+from paper_2506_03077_b200 import binding as B
+from paper_2506_03077_b200 import synth
+from helpers import TOL, assert_close, compare_layer, layer_case, run_layer, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def test_tiny_config_layer_fp32_matches_oracle():
+    # configuration "tiny": d 256, 4 query / 2 KV heads of 64, d_ff 688, T 512, chunk 128, fp32
+    cfgs = synth.CONFIGS["tiny"]
+    ocfg, bcfg, W, X, dY = layer_case(cfgs.layer, cfgs.seed, cfgs.T, torch.float32)
+    dX, grads = run_layer(bcfg, W, X, dY, cfgs.chunk)
+    compare_layer(ocfg, W, X, dY, dX, grads, TOL[torch.float32])
+
+
+@pytest.mark.parametrize("bias,Hq,Hkv,dh,T,chunk,pos0", [
+    (True, 4, 2, 64, 200, 64, 0),        # ragged last chunk (200 = 3*64 + 8), bias
+    (False, 2, 1, 128, 96, 40, 17),      # head_dim 128, ragged, position offset
+    (True, 6, 2, 64, 130, 1, 0),         # chunk of one row
+    (True, 4, 4, 64, 77, 1000, 5),       # chunk >= T: un-partitioned mode
+])
+def test_layer_fp32_shapes(bias, Hq, Hkv, dh, T, chunk, pos0):
+    shape = synth.LayerShape(64 * 2, Hq, Hkv, dh, 168, bias, 1e4)
+    ocfg, bcfg, W, X, dY = layer_case(shape, 7, T, torch.float32, dy_std=1.0, wstd=0.05)
+    dX, grads = run_layer(bcfg, W, X, dY, chunk, pos0=pos0)
+    compare_layer(ocfg, W, X, dY, dX, grads, TOL[torch.float32], pos0=pos0)
+
+
+def test_chunk_invariance_fp32():
+    # Eq. (1): any partition gives the same gradient -- divisors and non-divisors of T
+    shape = synth.LayerShape(128, 4, 2, 64, 168, True, 1e4)
+    ocfg, bcfg, W, X, dY = layer_case(shape, 3, 192, torch.float32, dy_std=1.0, wstd=0.05)
+    base_dX, base = run_layer(bcfg, W, X, dY, 192)
+    for chunk in (96, 64, 48, 32, 50, 7):
+        dX, grads = run_layer(bcfg, W, X, dY, chunk)
+        assert O.rel_frobenius(dX.cpu().numpy(), base_dX.cpu().numpy()) < 1e-5, chunk
+        for k in base:
+            assert O.rel_frobenius(grads[k].cpu().numpy(), base[k].cpu().numpy()) < 1e-5, (chunk, k)
+
+
+def test_accumulate_adds_to_existing_gradients():
+    shape = synth.LayerShape(128, 4, 2, 64, 168, True, 1e4)
+    ocfg, bcfg, W, X, dY = layer_case(shape, 4, 100, torch.float32, dy_std=1.0, wstd=0.05)
+    _, once = run_layer(bcfg, W, X, dY, 32)
+    grads = {k: v.clone() for k, v in once.items()}
+    run_layer(bcfg, W, X, dY, 32, accumulate=True, grads=grads)
+    for k in once:
+        assert O.rel_frobenius(grads[k].cpu().numpy(), 2.0 * once[k].cpu().numpy()) < 1e-6, k
+
+
+def test_reruns_are_bit_identical():
+    shape = synth.LayerShape(128, 4, 2, 64, 168, True, 1e4)
+    ocfg, bcfg, W, X, dY = layer_case(shape, 5, 150, torch.bfloat16)
+    dX1, g1 = run_layer(bcfg, W, X, dY, 64)
+    dX2, g2 = run_layer(bcfg, W, X, dY, 64)
+    assert torch.equal(dX1, dX2)
+    for k in g1:
+        assert torch.equal(g1[k], g2[k]), k
+
+
+def test_causality_zero_upstream_tail():
+    shape = synth.LayerShape(128, 4, 2, 64, 168, False, 1e4)
+    ocfg, bcfg, W, X, dY = layer_case(shape, 6, 160, torch.float32, dy_std=1.0, wstd=0.05)
+    dY[100:] = 0.0
+    dX, _ = run_layer(bcfg, W, X, dY, 48)
+    assert torch.count_nonzero(dX[100:]) == 0
+    assert torch.count_nonzero(dX[:100]) > 0
+
+
+@pytest.mark.parametrize("shape,T,chunk", [
+    (synth.LayerShape(512, 8, 2, 64, 1376, True, 1e6), 640, 256),
+    (synth.LayerShape(1024, 8, 2, 128, 2816, False, 5e5), 1100, 512),     # several tiles, ragged tail
+])
+def test_layer_bf16_matches_oracle(shape, T, chunk):
+    ocfg, bcfg, W, X, dY = layer_case(shape, 8, T, torch.bfloat16)
+    dX, grads = run_layer(bcfg, W, X, dY, chunk)
+    errs = compare_layer(ocfg, W, X, dY, dX, grads, TOL[torch.bfloat16])
+    print({k: f"{v:.2e}" for k, v in errs.items()})
+    # chunk invariance in bf16 within the same tolerance
+    dX2, grads2 = run_layer(bcfg, W, X, dY, T)
+    compare_layer(ocfg, W, X, dY, dX2, grads2, TOL[torch.bfloat16])

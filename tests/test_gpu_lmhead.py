@@ -1,0 +1,108 @@
+"""GPU parity: streambp_lmhead_ce_backward against the CPU oracle, closed forms and invariants."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import streambp_oracle as O
+from paper_2506_03077_b200 import binding as B
+from paper_2506_03077_b200 import synth
+from helpers import TOL, assert_close, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def run_head(hs: synth.HeadShape, g, W, H, labels, chunk, dtype, accumulate=False, prior=None):
+    cfg = B.HeadConfig(hs.d_model, hs.vocab, hs.rms_eps, hs.ignore_index, dtype)
+    gd, Wd, Hd = to_dev(g, dtype), to_dev(W, dtype), to_dev(H, dtype)
+    ld = torch.from_numpy(labels).cuda()
+    T = H.shape[0]
+    loss = torch.full((1,), float("nan"), device="cuda")
+    nv = torch.full((1,), -1, dtype=torch.int64, device="cuda")
+    dH = torch.full_like(Hd, float("nan"))
+    if prior is None:
+        dW = torch.full((hs.vocab, hs.d_model), float("nan"), device="cuda")
+        dg = torch.full((hs.d_model,), float("nan"), device="cuda")
+    else:
+        dW, dg = prior
+    ws = B.alloc_workspace(B.lmhead_workspace_bytes(cfg, T, chunk))
+    B.lmhead_ce_backward(cfg, gd, Wd, Hd, ld, chunk, loss, nv, dH, dW, dg, ws, accumulate=accumulate)
+    return loss, nv, dH, dW, dg, B.last_device_status(ws)
+
+
+def test_tiny_config_head_fp32():
+    c = synth.CONFIGS["tiny"]
+    g, W, H, labels = synth.make_head_inputs(c.head, c.seed, c.T, False, c.masked_prefix)
+    loss, nv, dH, dW, dg, st = run_head(c.head, g, W, H, labels, c.chunk_head, torch.float32)
+    assert st == B.OK
+    ref = O.lmhead_ce_backward(O.HeadCfg(c.head.d_model, c.head.vocab), g, W, H, labels)
+    assert int(nv.item()) == ref[1] == c.T - c.masked_prefix
+    assert abs(loss.item() - ref[0]) <= 1e-5 * abs(ref[0])
+    assert_close("dH", dH, ref[2], TOL[torch.float32])
+    assert_close("dW", dW, ref[3], TOL[torch.float32])
+    assert_close("dg", dg, ref[4], TOL[torch.float32])
+    assert torch.count_nonzero(dH[: c.masked_prefix]) == 0       # ignored rows: exactly zero
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("V,T,chunk", [(1000, 150, 64), (1003, 90, 32), (2048, 64, 64)])
+def test_head_shapes_and_chunk_invariance(dtype, V, T, chunk):
+    hs = synth.HeadShape(128, V)
+    g, W, H, labels = synth.make_head_inputs(hs, 11, T, dtype == torch.bfloat16, T // 4)
+    labels[T // 2] = -100
+    ref = O.lmhead_ce_backward(O.HeadCfg(128, V), g, W, H, labels)
+    for ch in (chunk, T, 1 if T <= 64 else 17):
+        loss, nv, dH, dW, dg, st = run_head(hs, g, W, H, labels, ch, dtype)
+        assert st == B.OK and int(nv.item()) == ref[1]
+        assert abs(loss.item() - ref[0]) <= (1e-5 if dtype == torch.float32 else 2e-3) * abs(ref[0])
+        assert_close("dH", dH, ref[2], TOL[dtype])
+        assert_close("dW", dW, ref[3], TOL[dtype])
+        assert_close("dg", dg, ref[4], TOL[dtype])
+
+
+def test_zero_head_weights_closed_form():
+    # W = 0: loss = ln V, dH = 0, dW[v] = (1/N) sum_t (1/V - [v = y_t]) hn_t
+    hs = synth.HeadShape(64, 4096)
+    g, W, H, labels = synth.make_head_inputs(hs, 2, 40, False, 8)
+    W[:] = 0.0
+    loss, nv, dH, dW, dg, st = run_head(hs, g, W, H, labels, 16, torch.float32)
+    assert abs(loss.item() - 8.317766166719343) < 2e-6
+    assert torch.count_nonzero(dH) == 0 and torch.count_nonzero(dg) == 0
+    hn = H / np.sqrt((H.astype(np.float64) ** 2).mean(-1, keepdims=True) + 1e-6) * g
+    N = 32
+    expect = np.tile(hn[8:].sum(0) / (4096 * N), (4096, 1))
+    for t in range(8, 40):
+        expect[labels[t]] -= hn[t] / N
+    assert_close("dW", dW, expect, 1e-5)
+
+
+def test_vocab_sum_of_weight_gradient_vanishes():
+    hs = synth.HeadShape(128, 3000)
+    g, W, H, labels = synth.make_head_inputs(hs, 5, 96, True, 10)
+    _, _, _, dW, _, _ = run_head(hs, g, W, H, labels, 32, torch.bfloat16)
+    col = dW.double().sum(0).abs().max().item()
+    scale = dW.double().abs().sum(0).max().item()
+    assert col <= 1e-2 * scale
+
+
+def test_device_status_bad_label_and_no_valid_label():
+    hs = synth.HeadShape(64, 500)
+    g, W, H, labels = synth.make_head_inputs(hs, 1, 32, False, 0)
+    bad = labels.copy()
+    bad[5] = 500
+    *_, st = run_head(hs, g, W, H, bad, 16, torch.float32)
+    assert st == B.E_BAD_LABEL
+    none = np.full_like(labels, -100)
+    loss, nv, dH, dW, dg, st = run_head(hs, g, W, H, none, 16, torch.float32)
+    assert st == B.E_NO_VALID_LABELS
+    assert loss.item() == 0.0 and int(nv.item()) == 0
+    assert torch.count_nonzero(dH) == 0 and torch.count_nonzero(dW) == 0 and torch.count_nonzero(dg) == 0
+
+
+def test_head_accumulate():
+    hs = synth.HeadShape(64, 512)
+    g, W, H, labels = synth.make_head_inputs(hs, 3, 48, False, 4)
+    _, _, _, dW, dg, _ = run_head(hs, g, W, H, labels, 16, torch.float32)
+    prior = (dW.clone(), dg.clone())
+    run_head(hs, g, W, H, labels, 16, torch.float32, accumulate=True, prior=prior)
+    assert O.rel_frobenius(prior[0].cpu().numpy(), 2 * dW.cpu().numpy()) < 1e-6
+    assert O.rel_frobenius(prior[1].cpu().numpy(), 2 * dg.cpu().numpy()) < 1e-6

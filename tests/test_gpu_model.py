@@ -1,0 +1,86 @@
+"""GPU parity: streambp_model_backward against the CPU oracle (tiny configuration end to end,
+and a small multi-layer model with embedding)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import streambp_oracle as O
+from paper_2506_03077_b200 import binding as B
+from paper_2506_03077_b200 import synth
+from helpers import TOL, assert_close, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def run_model(ls, hs, layers, g, Wv, labels, chunk_l, chunk_h, dtype, E=None, ids=None, X0=None):
+    lc = B.LayerConfig(ls.d_model, ls.n_q_heads, ls.n_kv_heads, ls.head_dim, ls.d_ff, ls.qkv_bias, ls.rope_theta,
+                       ls.rms_eps, dtype)
+    hc = B.HeadConfig(hs.d_model, hs.vocab, hs.rms_eps, hs.ignore_index, dtype)
+    Wd = [{k: to_dev(v, dtype) for k, v in W.items()} for W in layers]
+    Gd = [B.alloc_layer_grads(lc) for _ in layers]
+    for G in Gd:
+        for t in G.values():
+            t.fill_(float("nan"))
+    T = labels.shape[0]
+    loss = torch.zeros(1, device="cuda")
+    dg = torch.full((hs.d_model,), float("nan"), device="cuda")
+    dWv = torch.full((hs.vocab, hs.d_model), float("nan"), device="cuda")
+    dX0 = torch.full((T, ls.d_model), float("nan"), device="cuda", dtype=dtype)
+    dE = torch.full((hs.vocab, ls.d_model), float("nan"), device="cuda") if ids is not None else None
+    ws = B.alloc_workspace(B.model_workspace_bytes(len(layers), lc, hc, T, chunk_l, chunk_h))
+    B.model_backward(lc, hc, Wd, to_dev(g, dtype), to_dev(Wv, dtype), torch.from_numpy(labels).cuda(), chunk_l, chunk_h,
+                     loss, Gd, dg, dWv, ws,
+                     embed=None if E is None else to_dev(E, dtype),
+                     ids=None if ids is None else torch.from_numpy(ids).cuda(),
+                     X0=None if X0 is None else to_dev(X0, dtype), d_embed=dE, dX0=dX0)
+    assert B.last_device_status(ws) == B.OK
+    return loss, Gd, dg, dWv, dX0, dE
+
+
+def test_tiny_configuration_end_to_end_fp32():
+    """Tiny single decoder layer + LM head, fp32, seed 0: dX plus all weight gradients."""
+    c = synth.CONFIGS["tiny"]
+    W = synth.make_layer_weights(c.layer, c.seed, False)
+    X, _ = synth.make_layer_io(c.layer, c.seed, c.T, False)
+    g, Wv, _, labels = synth.make_head_inputs(c.head, c.seed, c.T, False, c.masked_prefix)
+    loss, Gd, dg, dWv, dX0, _ = run_model(c.layer, c.head, [W], g, Wv, labels, c.chunk, c.chunk_head, torch.float32, X0=X)
+    ls, hs = c.layer, c.head
+    ref = O.model_backward(O.LayerCfg(ls.d_model, ls.n_q_heads, ls.n_kv_heads, ls.head_dim, ls.d_ff, ls.qkv_bias,
+                                      ls.rope_theta, ls.rms_eps),
+                           O.HeadCfg(hs.d_model, hs.vocab), [W], g, Wv, labels, X0=X)
+    tol = TOL[torch.float32]
+    assert abs(loss.item() - ref["loss"]) <= 1e-5 * ref["loss"]
+    assert_close("dX0", dX0, ref["dX0"], tol)
+    assert_close("d_w_vocab", dWv, ref["w_vocab"], tol)
+    assert_close("d_g_final", dg, ref["g_final"], tol)
+    for k, v in ref["layers"][0].items():
+        assert_close(k, Gd[0][k], v, tol)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_small_model_with_embedding(dtype):
+    ls = synth.LayerShape(128, 4, 2, 64, 168, True, 1e4)
+    hs = synth.HeadShape(128, 777)
+    bf = dtype == torch.bfloat16
+    T, L = 150, 3
+    layers = [synth.make_layer_weights(ls, 30, bf, prefix=f"layer{l}") for l in range(L)]
+    E = synth.normal(30, "embed", (hs.vocab, ls.d_model), 0.0, 1.0)
+    g = synth.normal(30, "g_final", (ls.d_model,), 1.0, 0.02)
+    Wv = synth.normal(30, "w_vocab", (hs.vocab, ls.d_model), 0.0, 0.02)
+    if bf:
+        E, g, Wv = synth.round_bf16(E), synth.round_bf16(g), synth.round_bf16(Wv)
+    ids, labels = synth.make_model_tokens(hs.vocab, 30, T, 0.1)
+    ids[7] = ids[3]
+    loss, Gd, dg, dWv, dX0, dE = run_model(ls, hs, layers, g, Wv, labels, 64, 50, dtype, E=E, ids=ids)
+    ref = O.model_backward(O.LayerCfg(ls.d_model, ls.n_q_heads, ls.n_kv_heads, ls.head_dim, ls.d_ff, ls.qkv_bias,
+                                      ls.rope_theta, ls.rms_eps),
+                           O.HeadCfg(hs.d_model, hs.vocab), layers, g, Wv, labels, embed=E, ids=ids)
+    tol = TOL[dtype]
+    assert abs(loss.item() - ref["loss"]) <= (1e-5 if not bf else 3e-3) * ref["loss"]
+    assert_close("d_embed", dE, ref["d_embed"], tol)
+    assert_close("dX0", dX0, ref["dX0"], tol)
+    assert_close("d_w_vocab", dWv, ref["w_vocab"], tol)
+    assert_close("d_g_final", dg, ref["g_final"], tol)
+    for l in range(L):
+        for k, v in ref["layers"][l].items():
+            assert_close(f"layer{l}.{k}", Gd[l][k], v, tol)
