@@ -1,0 +1,293 @@
+#!/usr/bin/env python
+"""Benchmark of the streamed layer backward on one B200 (or N independent replicas).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--chunk C] [--impl reference]
+
+A step is one streambp_layer_backward call (K/V prologue, every chunk's re-forward and
+backward, all weight gradients) over one synthetic sequence.  Prints ONE JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "streamed_layer_backward_tokens_per_s"
+UNIT = "tokens/s"
+
+
+def layer_flops(s, T):
+    """Algorithmic FLOPs of one streamed layer backward: 6 forward products (no down projection),
+    14 backward products, attention (2 forward + 5 backward products) over the causal half."""
+    d, dq, dkv, I = s.d_model, s.dq, s.dkv, s.d_ff
+    P = d * dq + 2 * d * dkv + dq * d + 3 * d * I
+    fwd = 2 * T * (P - d * I)
+    bwd = 4 * T * P
+    pairs = T * (T + 1) / 2
+    att = 7 * 2 * s.head_dim * s.n_q_heads * pairs
+    return fwd + bwd + att
+
+
+def read_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        j = json.load(open(p))
+        return dict(hbm=j["hbm_gbs"], burst=j["bf16_tflops"], sustained=j["bf16_tflops_sustained"], source="measured")
+    return dict(hbm=6650.0, burst=1590.0, sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+_ORACLE_INPUTS = {}
+
+
+def oracle_sample(cfg, T_sample):
+    """Times the CPU oracle (as it stands) on the first T_sample tokens of the workload.
+    Input generation is outside the timed region."""
+    from oracle import streambp_oracle as O
+    from paper_2506_03077_b200 import synth
+    s = cfg.layer
+    key = (cfg.name, T_sample)
+    if key not in _ORACLE_INPUTS:
+        W = synth.make_layer_weights(s, cfg.seed, cfg.bf16)
+        X, dY = synth.make_layer_io(s, cfg.seed, T_sample, cfg.bf16)
+        _ORACLE_INPUTS[key] = (W, X, dY)
+    W, X, dY = _ORACLE_INPUTS[key]
+    oc = O.LayerCfg(s.d_model, s.n_q_heads, s.n_kv_heads, s.head_dim, s.d_ff, s.qkv_bias, s.rope_theta, s.rms_eps)
+    t0 = time.perf_counter()
+    O.layer_backward(oc, W, X, dY)
+    return time.perf_counter() - t0
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    T_sample = args.ref_tokens
+    for _ in range(args.warmup):
+        oracle_sample(cfg, T_sample)
+    times = [oracle_sample(cfg, T_sample) for _ in range(args.steps)]
+    total = sum(times)
+    value = T_sample * args.steps / total
+    cores = os.cpu_count()
+    sample = f"first {T_sample} tokens of {cfg.name} (full widths), fp64 numpy oracle, full-sequence backward"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "T": cfg.T, "chunk": cfg.chunk, "sample_tokens": T_sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="qwen7b_layer", choices=["qwen7b_layer", "llama8b_layer"])
+    ap.add_argument("--chunk", type=int, default=0)
+    ap.add_argument("--T", type=int, default=0, help="override the sequence length (profiling on small cases)")
+    ap.add_argument("--ref-tokens", type=int, default=512)
+    ap.add_argument("--cpu-baseline-tokens", type=int, default=1024)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+
+    from paper_2506_03077_b200 import synth
+    import copy
+    cfg = copy.copy(synth.CONFIGS[args.config])
+    if args.chunk:
+        cfg.chunk = args.chunk
+    if args.T:
+        cfg.T = args.T
+    if args.impl == "reference":
+        return run_reference(args, cfg)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2506_03077_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the streamed backward has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    B.lib()   # fail loudly if the CUDA library is absent
+
+    s = cfg.layer
+    dt = torch.bfloat16 if cfg.bf16 else torch.float32
+    T, chunk = cfg.T, cfg.chunk
+    bcfg = B.LayerConfig(s.d_model, s.n_q_heads, s.n_kv_heads, s.head_dim, s.d_ff, s.qkv_bias, s.rope_theta,
+                         s.rms_eps, dt)
+    seed = cfg.seed + 1000 * rank          # replicas see different sequences
+    Wn = synth.make_layer_weights(s, cfg.seed, cfg.bf16)
+    Xn, dYn = synth.make_layer_io(s, seed, T, cfg.bf16)
+    W = {k: torch.from_numpy(v).to("cuda", dt) for k, v in Wn.items()}
+    X_host = torch.from_numpy(Xn).to(dt).pin_memory()
+    dY_host = torch.from_numpy(dYn).to(dt).pin_memory()
+    dX_host = torch.empty_like(X_host).pin_memory()
+    X, dY = X_host.cuda(), dY_host.cuda()
+    dX = torch.empty_like(X)
+    grads = B.alloc_layer_grads(bcfg)
+    ws_bytes = B.layer_workspace_bytes(bcfg, T, chunk)
+    ws_full = B.layer_workspace_bytes(bcfg, T, T)
+    ws = B.alloc_workspace(ws_bytes)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        B.layer_backward(bcfg, W, X, dY, chunk, grads, dX, ws)
+
+    def step_e2e():
+        X.copy_(X_host, non_blocking=True)
+        dY.copy_(dY_host, non_blocking=True)
+        B.layer_backward(bcfg, W, X, dY, chunk, grads, dX, ws)
+        dX_host.copy_(dX, non_blocking=True)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            fn()
+        e1.record(stream)
+        barrier()
+        ms = torch.tensor([e0.elapsed_time(e1)], device="cuda")
+        if world > 1:
+            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+        return float(ms.item())
+
+    for _ in range(args.warmup):
+        step()
+    assert B.last_device_status(ws) == B.OK
+    launches_per_step = B.last_launch_count()
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    B.profile_enable(True)
+    total_ms = timed(step, args.steps)
+    prof = {k: B.profile_read(k) for k in B.KERNEL_CLASSES}
+    B.profile_enable(False)
+    clocks = sampler.stop() if rank == 0 else None
+
+    e2e_ms = None
+    if not args.no_e2e:
+        step_e2e()
+        e2e_ms = timed(step_e2e, args.steps)
+
+    ms_per_step = total_ms / args.steps
+    value = world * T / (ms_per_step * 1e-3)
+    peaks = read_peaks()
+    flops = layer_flops(s, T)
+    gemm_ms, gemm_calls, gemm_flops = prof["gemm"]
+    af_ms, af_calls, af_flops = prof["attention_fwd"]
+    ab_ms, ab_calls, ab_flops = prof["attention_bwd"]
+    achieved = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
+    # the bracketed kernels run inside a long step: compare with the sustained measured peak
+    peak = peaks["sustained"]
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if cfg.bf16 else "f32", "data": "synthetic",
+        "config": {"workload": cfg.name, "T": T, "chunk": chunk, "d_model": s.d_model, "n_q_heads": s.n_q_heads,
+                   "n_kv_heads": s.n_kv_heads, "head_dim": s.head_dim, "d_ff": s.d_ff, "qkv_bias": s.qkv_bias,
+                   "l2": "inputs larger than L2 (weights + gradients > 1 GB per step)",
+                   "multi_gpu": "replicas only"},
+        "algorithmic_tflop_per_step": flops / 1e12,
+        "tflops": flops / (ms_per_step * 1e-3) / 1e12,
+        "frac_of_measured_sustained_bf16": flops / (ms_per_step * 1e-3) / 1e12 / peaks["sustained"],
+        "frac_of_measured_burst_bf16": flops / (ms_per_step * 1e-3) / 1e12 / peaks["burst"],
+        "frac_of_nominal_bf16": flops / (ms_per_step * 1e-3) / 1e12 / 2250.0,
+        "peak_activation_gb": ws_bytes / 1e9, "peak_activation_gb_unchunked": ws_full / 1e9,
+        "gpu_launches": int(launches_per_step * args.steps),
+        "roofline": {"bound": "tensor", "kernel": "linear products (all GEMM launches of the step)",
+                     "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                     "peak_source": peaks["source"] + " sustained bf16", "traffic": None,
+                     "launches": int(gemm_calls), "ms_per_step": gemm_ms / args.steps},
+        "kernel_classes": {
+            "gemm": {"ms_per_step": gemm_ms / args.steps, "tflops": achieved},
+            "attention_fwd": {"ms_per_step": af_ms / args.steps,
+                              "tflops": af_flops / (af_ms * 1e-3) / 1e12 if af_ms > 0 else 0.0},
+            "attention_bwd": {"ms_per_step": ab_ms / args.steps,
+                              "tflops": ab_flops / (ab_ms * 1e-3) / 1e12 if ab_ms > 0 else 0.0},
+        },
+        "clocks": clocks,
+    }
+    if e2e_ms is not None:
+        nbytes = X_host.numel() * X_host.element_size()
+        out["e2e"] = {"value": world * T / (e2e_ms / args.steps * 1e-3), "unit": UNIT,
+                      "h2d_bytes_per_step": 2 * nbytes, "d2h_bytes_per_step": nbytes}
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        Ts = min(args.cpu_baseline_tokens, T)
+        sec = oracle_sample(cfg, Ts)
+        out["cpu_baseline"] = {"value": Ts / sec, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+                               "sample": f"first {Ts} tokens of {cfg.name} (full widths), fp64 numpy oracle, "
+                                         f"full-sequence backward, {sec:.1f} s"}
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

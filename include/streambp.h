@@ -188,6 +188,18 @@ int streambp_gemm(int op, int64_t M, int64_t N, int64_t K, const void *A, int64_
                   const void *B, int64_t ldb, void *C, int64_t ldc, int32_t in_dtype,
                   int32_t out_dtype, int accumulate, int engine, void *cuda_stream);
 
+/*
+ * Optional device timing by kernel class (0 = linear products, 1 = attention forward,
+ * 2 = attention backward).  While enabled, each launch of those classes is bracketed by CUDA
+ * events on the caller's stream.  streambp_profile_enable(1) also clears earlier records;
+ * streambp_profile_read() waits for the recorded events and returns, for one class, the summed
+ * device time, the number of bracketed launches and their algorithmic FLOPs (products: 2MNK;
+ * attention: 2 * head_dim per causal (query, key) pair and product).  Not thread-safe; meant for
+ * benchmarks.
+ */
+void streambp_profile_enable(int on);
+int streambp_profile_read(int kernel_class, double *milliseconds, int64_t *calls, double *flops);
+
 #ifdef __cplusplus
 }
 #endif

@@ -30,6 +30,7 @@ EXPORTS = (
     "streambp_model_workspace_bytes", "streambp_model_backward",
     "streambp_last_device_status", "streambp_status_string",
     "streambp_last_cuda_error", "streambp_last_launch_count", "streambp_gemm",
+    "streambp_profile_enable", "streambp_profile_read",
 )
 
 
@@ -97,6 +98,10 @@ def lib() -> C.CDLL:
     L.streambp_last_launch_count.argtypes = []
     L.streambp_gemm.restype = C.c_int
     L.streambp_gemm.argtypes = [C.c_int, i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, i32, C.c_int, C.c_int, vp]
+    L.streambp_profile_enable.restype = None
+    L.streambp_profile_enable.argtypes = [C.c_int]
+    L.streambp_profile_read.restype = C.c_int
+    L.streambp_profile_read.argtypes = [C.c_int, C.POINTER(C.c_double), C.POINTER(i64), C.POINTER(C.c_double)]
     _lib = L
     return L
 
@@ -274,3 +279,18 @@ def gemm(op: int, A: torch.Tensor, B: torch.Tensor, C_out: torch.Tensor, accumul
     if check:
         _check(st, "streambp_gemm")
     return st
+
+
+KERNEL_CLASSES = {"gemm": 0, "attention_fwd": 1, "attention_bwd": 2}
+
+
+def profile_enable(on: bool) -> None:
+    lib().streambp_profile_enable(1 if on else 0)
+
+
+def profile_read(kernel_class: str):
+    """(milliseconds, launches, algorithmic FLOPs) recorded for one kernel class."""
+    ms, n, fl = C.c_double(), C.c_int64(), C.c_double()
+    _check(lib().streambp_profile_read(KERNEL_CLASSES[kernel_class], C.byref(ms), C.byref(n), C.byref(fl)),
+           "streambp_profile_read")
+    return ms.value, n.value, fl.value

@@ -14,7 +14,33 @@ CallState &call_state() {
 
 namespace {
 int g_engine = -1;
+
+struct ProfRec {
+    cudaEvent_t a, b;
+    int cls;
+    double flops;
+};
+bool g_prof_on = false;
+std::vector<ProfRec> g_prof;      // event pairs, reused across resets
+size_t g_prof_used = 0;
+}  // namespace
+
+ProfScope::ProfScope(int cls, double flops, cudaStream_t stream) : idx(-1), st(stream) {
+    if (!g_prof_on) return;
+    if (g_prof_used == g_prof.size()) {
+        ProfRec r;
+        if (cudaEventCreate(&r.a) != cudaSuccess || cudaEventCreate(&r.b) != cudaSuccess) return;
+        g_prof.push_back(r);
+    }
+    idx = (int)g_prof_used++;
+    g_prof[idx].cls = cls;
+    g_prof[idx].flops = flops;
+    cudaEventRecord(g_prof[idx].a, st);
 }
+ProfScope::~ProfScope() {
+    if (idx >= 0) cudaEventRecord(g_prof[idx].b, st);
+}
+
 int gemm_engine() {
     if (g_engine < 0) {
         const char *e = std::getenv("STREAMBP_GEMM_ENGINE");
@@ -29,11 +55,13 @@ void set_gemm_engine(int e) { g_engine = e; }
 template <typename TI, typename TC>
 int mm(GemmOp op, int64_t M, int64_t N, int64_t K, const TI *A, int64_t lda, const TI *B, int64_t ldb, TC *C,
        int64_t ldc, const TI *bias, bool accumulate, cudaStream_t st) {
+    ProfScope prof(KC_GEMM, 2.0 * (double)M * (double)N * (double)K, st);
     return gemm<TI, TC>(op, M, N, K, A, lda, B, ldb, C, ldc, bias, accumulate, st);
 }
 template <>
 int mm<bf16, float>(GemmOp op, int64_t M, int64_t N, int64_t K, const bf16 *A, int64_t lda, const bf16 *B, int64_t ldb,
                     float *C, int64_t ldc, const bf16 *bias, bool accumulate, cudaStream_t st) {
+    ProfScope prof(KC_GEMM, 2.0 * (double)M * (double)N * (double)K, st);
     const int e = gemm_engine();
     if (e != 1 && gemm_tc_supported(op, M, N, K, lda, ldb, ldc, A, B, C, true))
         return gemm_tc(op, M, N, K, A, lda, B, ldb, C, ldc, true, bias, accumulate, st);
@@ -43,6 +71,7 @@ int mm<bf16, float>(GemmOp op, int64_t M, int64_t N, int64_t K, const bf16 *A, i
 template <>
 int mm<bf16, bf16>(GemmOp op, int64_t M, int64_t N, int64_t K, const bf16 *A, int64_t lda, const bf16 *B, int64_t ldb,
                    bf16 *C, int64_t ldc, const bf16 *bias, bool accumulate, cudaStream_t st) {
+    ProfScope prof(KC_GEMM, 2.0 * (double)M * (double)N * (double)K, st);
     const int e = gemm_engine();
     if (e != 1 && !accumulate && gemm_tc_supported(op, M, N, K, lda, ldb, ldc, A, B, C, false))
         return gemm_tc(op, M, N, K, A, lda, B, ldb, C, ldc, false, bias, false, st);
@@ -256,6 +285,30 @@ const char *streambp_status_string(int s) {
 
 int streambp_last_cuda_error(void) { return call_state().cuda_error; }
 int64_t streambp_last_launch_count(void) { return call_state().launches; }
+
+void streambp_profile_enable(int on) {
+    g_prof_on = on != 0;
+    g_prof_used = 0;
+}
+
+int streambp_profile_read(int kernel_class, double *milliseconds, int64_t *calls, double *flops) {
+    if (kernel_class < 0 || kernel_class >= KC_CLASSES) return STREAMBP_E_SHAPE;
+    double ms = 0.0, fl = 0.0;
+    int64_t n = 0;
+    for (size_t i = 0; i < g_prof_used; i++) {
+        if (g_prof[i].cls != kernel_class) continue;
+        if (!cuda_ok(cudaEventSynchronize(g_prof[i].b))) return STREAMBP_E_CUDA;
+        float t = 0.f;
+        if (!cuda_ok(cudaEventElapsedTime(&t, g_prof[i].a, g_prof[i].b))) return STREAMBP_E_CUDA;
+        ms += t;
+        fl += g_prof[i].flops;
+        n++;
+    }
+    if (milliseconds) *milliseconds = ms;
+    if (calls) *calls = n;
+    if (flops) *flops = fl;
+    return STREAMBP_OK;
+}
 
 int streambp_gemm(int op, int64_t M, int64_t N, int64_t K, const void *A, int64_t lda, const void *B, int64_t ldb,
                   void *C, int64_t ldc, int32_t in_dtype, int32_t out_dtype, int accumulate, int engine,

@@ -41,6 +41,17 @@ inline bool cuda_ok(cudaError_t e) {
         if (_st != STREAMBP_OK) return _st;   \
     } while (0)
 
+// ---- optional per-class device timing (off by default) -----------------------------
+// When enabled through streambp_profile_enable(), every product and attention launch is bracketed
+// by CUDA events on the caller's stream; the algorithmic FLOPs of the bracketed work are summed.
+enum KernelClass { KC_GEMM = 0, KC_ATTN_FWD = 1, KC_ATTN_BWD = 2, KC_CLASSES = 3 };
+struct ProfScope {
+    int idx;
+    cudaStream_t st;
+    ProfScope(int cls, double flops, cudaStream_t stream);
+    ~ProfScope();
+};
+
 // ---- scalar conversion -------------------------------------------------------
 __device__ __forceinline__ float to_f32(float v) { return v; }
 __device__ __forceinline__ float to_f32(bf16 v) { return __bfloat162float(v); }

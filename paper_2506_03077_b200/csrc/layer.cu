@@ -87,7 +87,12 @@ int chunk_forward(const streambp_layer_cfg &c, const streambp_layer_weights &w, 
     SBP_TRY(rmsnorm_fwd<T>(Xi, nullptr, (const T *)w.g1, c.rms_eps, n, d, s.h1, s.rstd1, nullptr, st));
     SBP_TRY((mm<T, float>(OP_NT, n, dq, d, s.h1, d, (const T *)w.wq, d, s.fa, dq, (const T *)w.bq, false, st)));
     SBP_TRY(rope_apply<T>(s.fa, s.cs + r0 * dh, n, Hq, dh, false, s.Q, st));
-    SBP_TRY(attention_fwd<T>(s.Q, s.K, s.V, n, r0, Hq, Hkv, dh, s.O, s.lse, st));
+    {
+        // causal pairs (query, key) of this chunk: n * r0 + n (n + 1) / 2; two products forward
+        const double pairs = (double)n * (double)r0 + 0.5 * (double)n * (double)(n + 1);
+        ProfScope prof(KC_ATTN_FWD, 2.0 * 2.0 * pairs * dh * Hq, st);
+        SBP_TRY(attention_fwd<T>(s.Q, s.K, s.V, n, r0, Hq, Hkv, dh, s.O, s.lse, st));
+    }
     SBP_TRY((mm<T, float>(OP_NT, n, d, dq, s.O, dq, (const T *)w.wo, dq, s.fa, d, nullptr, false, st)));
     SBP_TRY(rmsnorm_fwd<T>(Xi, s.fa, (const T *)w.g2, c.rms_eps, n, d, s.h2, s.rstd2, s.r, st));
     SBP_TRY((mm<T, T>(OP_NT, n, I, d, s.h2, d, (const T *)w.w_gate, d, s.g, I, nullptr, false, st)));
@@ -168,7 +173,12 @@ int layer_backward(const streambp_layer_cfg &c, const streambp_layer_weights &w,
         SBP_TRY((mm<T, T>(OP_NN, n, dq, d, dr_op, d, (const T *)w.wo, dq, s.dO, dq, nullptr, false, st)));  // dO = dr Wo
 
         // ---- partitioned attention backward: dQ (into fa), dK/dV prefix += ----
-        SBP_TRY(attention_bwd<T>(s.Q, s.K, s.V, s.O, s.dO, s.lse, n, r0, Hq, Hkv, dh, s.delta, s.fa, s.dK, s.dV, st));
+        {
+            const double pairs = (double)n * (double)r0 + 0.5 * (double)n * (double)(n + 1);
+            ProfScope prof(KC_ATTN_BWD, 5.0 * 2.0 * pairs * dh * Hq, st);   // five products backward
+            SBP_TRY(attention_bwd<T>(s.Q, s.K, s.V, s.O, s.dO, s.lse, n, r0, Hq, Hkv, dh, s.delta, s.fa, s.dK, s.dV,
+                                     st));
+        }
 
         // ---- Q projection backward ----
         T *dq_s = s.Q;  // Q is dead after the attention backward
