@@ -264,6 +264,9 @@ int streambp_last_device_status(void *workspace, void *cuda_stream) {
     WsHeader h;
     if (!cuda_ok(cudaMemcpyAsync(&h, workspace, sizeof(h), cudaMemcpyDeviceToHost, st))) return STREAMBP_E_CUDA;
     if (!cuda_ok(cudaStreamSynchronize(st))) return STREAMBP_E_CUDA;
+    const int fault = gemm_tc_take_fault();
+    if (fault < 0) return STREAMBP_E_CUDA;
+    if (fault > 0) return STREAMBP_E_DEVICE_TIMEOUT;
     return h.status;
 }
 

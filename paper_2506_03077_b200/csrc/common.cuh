@@ -182,6 +182,9 @@ bool gemm_tc_supported(GemmOp op, int64_t M, int64_t N, int64_t K, int64_t lda, 
 int gemm_tc(GemmOp op, int64_t M, int64_t N, int64_t K, const bf16 *A, int64_t lda, const bf16 *B, int64_t ldb,
             void *C, int64_t ldc, bool c_is_f32, const bf16 *bias, bool accumulate, cudaStream_t st);
 
+// Reads and clears the flag a tensor-core kernel raises when one of its bounded waits expires.
+int gemm_tc_take_fault();
+
 // Engine choice for the dispatching product below: 0 automatic, 1 CUDA cores only, 2 tensor cores required.
 int gemm_engine();
 void set_gemm_engine(int e);

@@ -1,13 +1,430 @@
-// tcgen05 tensor-core GEMM (placeholder until the kernel lands): reports every shape as unsupported.
+// tcgen05 tensor-core GEMM for sm_100a: bf16 operands staged in shared memory by TMA
+// (128-byte swizzle), fp32 accumulation in tensor memory, three operand layouts.
+//
+//   persistent grid, one CTA per SM, output tile 128 x 256, K slices of 64
+//   warp 0      : TMA producer (one elected lane)
+//   warp 1      : allocates tensor memory, issues tcgen05.mma (one elected lane)
+//   warps 2..5  : epilogue -- tcgen05.ld of a 32-lane quarter, bias / accumulate, 16-byte stores
+//   tensor memory holds two 128 x 256 fp32 accumulators, so the epilogue of tile i overlaps
+//   the main loop of tile i+1.
+//
+// Operand layouts (GemmOp): K-major operands are loaded as [rows][64 k] boxes, MN-major operands
+// (the B of "NN", both operands of "TN") as [64 k][64 mn] boxes; the shared-memory matrix
+// descriptors tell the tensor core which of the two it is looking at, so no operand is ever
+// transposed in memory.
+//
+// Every mbarrier wait is bounded (2 s of %globaltimer): on expiry the CTA raises a fault flag that
+// streambp_last_device_status() reports as STREAMBP_E_DEVICE_TIMEOUT, all roles leave their loops,
+// tensor memory is released and the kernel returns.
+#include <cuda.h>
+
 #include "common.cuh"
 
 namespace sbp {
-bool gemm_tc_supported(GemmOp, int64_t, int64_t, int64_t, int64_t, int64_t, int64_t, const void *, const void *,
-                       const void *, bool) {
-    return false;
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;   // 16 KiB
+constexpr int B_BYTES = BN * BK * 2;   // 32 KiB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr int NUM_THREADS = 192;
+constexpr uint32_t TMEM_COLS = 512;
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
+
+__device__ int g_tc_fault = 0;
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ unsigned long long global_timer() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
 }
-int gemm_tc(GemmOp, int64_t, int64_t, int64_t, const bf16 *, int64_t, const bf16 *, int64_t, void *, int64_t, bool,
-            const bf16 *, bool, cudaStream_t) {
-    return STREAMBP_E_SHAPE;
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait. Returns false if the CTA is aborting or the time limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_timer();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 255u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_timer() - t0 > WAIT_LIMIT_NS) {
+                *abort_flag = 1;
+                atomicExch(&g_tc_fault, 1);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+        : "memory");
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1 (sm_100).
+//   K-major : rows of 64 bf16 (128 B); 8-row groups 1024 B apart (stride offset); leading offset unused.
+//   MN-major: [k][64 mn] rows of 128 B; 8-k groups 1024 B apart (stride offset);
+//             64-element mn blocks 8192 B apart (leading offset).
+__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr, bool mn_major) {
+    const uint64_t lbo = mn_major ? (8192u >> 4) : 1u;
+    const uint64_t sbo = 1024u >> 4;
+    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | (lbo << 16) | (sbo << 32) | (1ull << 46) | (2ull << 61);
+}
+
+struct TcParams {
+    int M, N, K;
+    void *C;
+    long long ldc;
+    const bf16 *bias;
+    int accumulate;
+};
+
+template <bool A_MN, bool B_MN, bool OUT_F32>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+    gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                   const TcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;          // 1024-byte aligned operand stages
+    uint8_t *aux = smem_raw + (tiles - raw) + STAGES * STAGE_BYTES;
+    const uint32_t bar_full = smem_u32(aux);                 // STAGES x 8 B
+    const uint32_t bar_empty = bar_full + 8 * STAGES;        // STAGES x 8 B
+    const uint32_t bar_tfull = bar_empty + 8 * STAGES;       // 2 x 8 B
+    const uint32_t bar_tempty = bar_tfull + 16;              // 2 x 8 B
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux + 8 * STAGES * 2 + 32);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(aux + 8 * STAGES * 2 + 40);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + BN - 1) / BN;
+    const int num_tiles = tiles_m * tiles_n;
+    const int num_kb = (p.K + BK - 1) / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; s++) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int b = 0; b < 2; b++) {
+            mbar_init(bar_tfull + 8 * b, 1);
+            mbar_init(bar_tempty + 8 * b, 4);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"(TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------ TMA producer ------------------------------
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            bool alive = true;
+            for (int tile = blockIdx.x; tile < num_tiles && alive; tile += gridDim.x) {
+                const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
+                for (int kb = 0; kb < num_kb; kb++) {
+                    if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { alive = false; break; }
+                    const uint32_t full = bar_full + 8 * stage;
+                    const uint32_t sa = tiles + stage * STAGE_BYTES, sb = sa + A_BYTES;
+                    mbar_expect_tx(full, STAGE_BYTES);
+                    const int k0 = kb * BK;
+                    if (A_MN) {
+#pragma unroll
+                        for (int j = 0; j < BM / 64; j++) tma_load_2d(sa + j * 8192, &map_a, full, m0 + 64 * j, k0);
+                    } else {
+                        tma_load_2d(sa, &map_a, full, k0, m0);
+                    }
+                    if (B_MN) {
+#pragma unroll
+                        for (int j = 0; j < BN / 64; j++) tma_load_2d(sb + j * 8192, &map_b, full, n0 + 64 * j, k0);
+                    } else {
+                        tma_load_2d(sb, &map_b, full, k0, n0);
+                    }
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer ------------------------------
+        if (lane == 0) {
+            constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) |
+                                       ((B_MN ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) |
+                                       ((uint32_t)(BM >> 4) << 24);
+            constexpr uint32_t a_step = A_MN ? 2048u : 32u, b_step = B_MN ? 2048u : 32u;  // bytes per 16 k
+            uint32_t stage = 0, phase = 0, local = 0;
+            bool alive = true;
+            for (int tile = blockIdx.x; tile < num_tiles && alive; tile += gridDim.x, local++) {
+                const uint32_t buf = local & 1u, use = local >> 1;
+                if (!mbar_wait(bar_tempty + 8 * buf, (use & 1u) ^ 1u, abort_flag)) { alive = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * BN;
+                for (int kb = 0; kb < num_kb; kb++) {
+                    if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { alive = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = tiles + stage * STAGE_BYTES, sb = sa + A_BYTES;
+#pragma unroll
+                    for (int kk = 0; kk < BK / 16; kk++) {
+                        umma_bf16(d_tmem, make_desc(sa + kk * a_step, A_MN), make_desc(sb + kk * b_step, B_MN), idesc,
+                                  (kb | kk) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(bar_empty + 8 * stage);   // frees the stage once these MMAs have read it
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (alive) umma_commit(bar_tfull + 8 * buf);   // accumulator complete
+            }
+        }
+    } else {
+        // ------------------------------ epilogue ------------------------------
+        const int quarter = warp & 3;                 // TMEM lanes 32*quarter .. +31
+        uint32_t local = 0;
+        bool alive = true;
+        for (int tile = blockIdx.x; tile < num_tiles && alive; tile += gridDim.x, local++) {
+            const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
+            const uint32_t buf = local & 1u, use = local >> 1;
+            if (!mbar_wait(bar_tfull + 8 * buf, use & 1u, abort_flag)) { alive = false; break; }
+            tc_fence_after();
+            const int row = m0 + quarter * 32 + lane;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * BN;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; c++) {
+                const int col0 = n0 + c * 32;
+                if (col0 >= p.N) break;               // uniform across the warp
+                uint32_t r[32];
+                tmem_ld32(taddr + c * 32, r);
+                if (row < p.M) {
+                    if (OUT_F32) {
+                        float *out = reinterpret_cast<float *>(p.C) + (long long)row * p.ldc + col0;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            float v[4];
+#pragma unroll
+                            for (int e = 0; e < 4; e++) {
+                                v[e] = __uint_as_float(r[j + e]);
+                                if (p.bias && col0 + j + e < p.N) v[e] += __bfloat162float(p.bias[col0 + j + e]);
+                            }
+                            if (col0 + j + 3 < p.N) {
+                                if (p.accumulate) {
+                                    const float4 o = *reinterpret_cast<const float4 *>(out + j);
+                                    v[0] += o.x; v[1] += o.y; v[2] += o.z; v[3] += o.w;
+                                }
+                                *reinterpret_cast<float4 *>(out + j) = make_float4(v[0], v[1], v[2], v[3]);
+                            } else {
+                                for (int e = 0; e < 4; e++)
+                                    if (col0 + j + e < p.N) out[j + e] = p.accumulate ? out[j + e] + v[e] : v[e];
+                            }
+                        }
+                    } else {
+                        bf16 *out = reinterpret_cast<bf16 *>(p.C) + (long long)row * p.ldc + col0;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 8) {
+                            float v[8];
+#pragma unroll
+                            for (int e = 0; e < 8; e++) {
+                                v[e] = __uint_as_float(r[j + e]);
+                                if (p.bias && col0 + j + e < p.N) v[e] += __bfloat162float(p.bias[col0 + j + e]);
+                            }
+                            if (col0 + j + 7 < p.N) {
+                                uint32_t w[4];
+#pragma unroll
+                                for (int e = 0; e < 4; e++) {
+                                    __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]);
+                                    w[e] = *reinterpret_cast<uint32_t *>(&h);
+                                }
+                                *reinterpret_cast<uint4 *>(out + j) = make_uint4(w[0], w[1], w[2], w[3]);
+                            } else {
+                                for (int e = 0; e < 8; e++)
+                                    if (col0 + j + e < p.N) out[j + e] = __float2bfloat16_rn(v[e]);
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
+        }
+    }
+
+    __syncwarp();
+    if (*abort_flag) {
+        // give copies that are still in flight time to land before shared memory is released
+        const unsigned long long t0 = global_timer();
+        while (global_timer() - t0 < 200000ull) { }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 2-D bf16 tensor map over a row-major [rows, cols] matrix with leading dimension ld (elements).
+bool make_map(CUtensorMap *map, const void *base, int64_t rows, int64_t cols, int64_t ld, uint32_t box_cols,
+              uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    const cuuint32_t box[2] = {box_cols, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        call_state().cuda_error = (int)r;
+        return false;
+    }
+    return true;
+}
+
+int sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            n = 148;
+    }
+    return n;
+}
+
+template <bool A_MN, bool B_MN, bool OUT_F32>
+int launch(const CUtensorMap &ma, const CUtensorMap &mb, const TcParams &p, cudaStream_t st) {
+    auto kernel = gemm_tc_kernel<A_MN, B_MN, OUT_F32>;
+    static bool configured = false;
+    if (!configured) {
+        if (!cuda_ok(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES)))
+            return STREAMBP_E_CUDA;
+        configured = true;
+    }
+    const int tiles = ((p.M + BM - 1) / BM) * ((p.N + BN - 1) / BN);
+    const int grid = tiles < sm_count() ? tiles : sm_count();
+    SBP_LAUNCH(kernel, grid, NUM_THREADS, SMEM_BYTES, st, ma, mb, p);
+    return STREAMBP_OK;
+}
+
+}  // namespace
+
+bool gemm_tc_supported(GemmOp op, int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb, int64_t ldc,
+                       const void *A, const void *B, const void *C, bool c_is_f32) {
+    (void)op;
+    if (M < 1 || N < 1 || K < 1 || M > (1ll << 30) || N > (1ll << 30) || K > (1ll << 30)) return false;
+    if ((lda % 8) || (ldb % 8)) return false;                       // TMA: 16-byte row pitch
+    if (ldc % (c_is_f32 ? 4 : 8)) return false;                     // 16-byte vector stores
+    auto al = [](const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; };
+    if (!al(A) || !al(B) || !al(C)) return false;
+    return encode_fn() != nullptr;
+}
+
+int gemm_tc(GemmOp op, int64_t M, int64_t N, int64_t K, const bf16 *A, int64_t lda, const bf16 *B, int64_t ldb,
+            void *C, int64_t ldc, bool c_is_f32, const bf16 *bias, bool accumulate, cudaStream_t st) {
+    CUtensorMap ma, mb;
+    bool ok = true;
+    switch (op) {
+        case OP_NT:   // A [M,K] K-major, B [N,K] K-major
+            ok = make_map(&ma, A, M, K, lda, BK, BM) && make_map(&mb, B, N, K, ldb, BK, BN);
+            break;
+        case OP_NN:   // A [M,K] K-major, B [K,N] N-major
+            ok = make_map(&ma, A, M, K, lda, BK, BM) && make_map(&mb, B, K, N, ldb, 64, BK);
+            break;
+        case OP_TN:   // A [K,M] M-major, B [K,N] N-major
+            ok = make_map(&ma, A, K, M, lda, 64, BK) && make_map(&mb, B, K, N, ldb, 64, BK);
+            break;
+    }
+    if (!ok) return STREAMBP_E_CUDA;
+    TcParams p{(int)M, (int)N, (int)K, C, (long long)ldc, bias, accumulate ? 1 : 0};
+    if (op == OP_NT) return c_is_f32 ? launch<false, false, true>(ma, mb, p, st) : launch<false, false, false>(ma, mb, p, st);
+    if (op == OP_NN) return c_is_f32 ? launch<false, true, true>(ma, mb, p, st) : launch<false, true, false>(ma, mb, p, st);
+    return c_is_f32 ? launch<true, true, true>(ma, mb, p, st) : launch<true, true, false>(ma, mb, p, st);
+}
+
+// Reads and clears the fault flag raised by an expired bounded wait. Returns < 0 on a CUDA error.
+int gemm_tc_take_fault() {
+    int v = 0, zero = 0;
+    if (cudaMemcpyFromSymbol(&v, g_tc_fault, sizeof(int)) != cudaSuccess) return -1;
+    if (v && cudaMemcpyToSymbol(g_tc_fault, &zero, sizeof(int)) != cudaSuccess) return -1;
+    return v;
+}
+
 }  // namespace sbp
