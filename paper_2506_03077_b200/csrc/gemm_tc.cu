@@ -4,7 +4,11 @@
 //   persistent grid, one CTA per SM, output tile 128 x 256, K slices of 64
 //   warp 0      : TMA producer (one elected lane)
 //   warp 1      : allocates tensor memory, issues tcgen05.mma (one elected lane)
-//   warps 2..5  : epilogue -- tcgen05.ld of a 32-lane quarter, bias / accumulate, 16-byte stores
+//   warps 2..5  : epilogue -- tcgen05.ld of a 32-lane quarter, bias, then
+//                 fp32 output: 32x32 blocks staged in shared memory (128-byte swizzle) and written
+//                 by TMA store, or added into C by TMA reduce-add when accumulating, so the
+//                 read-modify-write of a weight-gradient tile never passes through the SM;
+//                 bf16 output: 16-byte stores from registers
 //   tensor memory holds two 128 x 256 fp32 accumulators, so the epilogue of tile i overlaps
 //   the main loop of tile i+1.
 //
@@ -27,7 +31,9 @@ constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
 constexpr int A_BYTES = BM * BK * 2;   // 16 KiB
 constexpr int B_BYTES = BN * BK * 2;   // 32 KiB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr int EPI_BUF_BYTES = 32 * 128;                  // one 32 x 32 fp32 block
+constexpr int EPI_BYTES = 4 * 2 * EPI_BUF_BYTES;          // 4 epilogue warps, double-buffered
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
 constexpr int NUM_THREADS = 192;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
@@ -86,6 +92,18 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         : "memory");
 }
 
+// C block [32 rows][32 fp32] in shared memory -> global, plain store or element-wise add at the destination
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int c0, int c1) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(src), "r"(c0), "r"(c1)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap *map, uint32_t src, int c0, int c1) {
+    asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(src), "r"(c0), "r"(c1)
+                 : "memory");
+}
+
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                           uint32_t accumulate) {
     asm volatile(
@@ -135,11 +153,12 @@ struct TcParams {
 template <bool A_MN, bool B_MN, bool OUT_F32>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
     gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                   const TcParams p) {
+                   const __grid_constant__ CUtensorMap map_c, const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;          // 1024-byte aligned operand stages
-    uint8_t *aux = smem_raw + (tiles - raw) + STAGES * STAGE_BYTES;
+    const uint32_t epi = tiles + STAGES * STAGE_BYTES;      // fp32 staging blocks, 1024-byte aligned
+    uint8_t *aux = smem_raw + (tiles - raw) + STAGES * STAGE_BYTES + EPI_BYTES;
     const uint32_t bar_full = smem_u32(aux);                 // STAGES x 8 B
     const uint32_t bar_empty = bar_full + 8 * STAGES;        // STAGES x 8 B
     const uint32_t bar_tfull = bar_empty + 8 * STAGES;       // 2 x 8 B
@@ -236,7 +255,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
     } else {
         // ------------------------------ epilogue ------------------------------
         const int quarter = warp & 3;                 // TMEM lanes 32*quarter .. +31
-        uint32_t local = 0;
+        uint32_t local = 0, staged = 0;               // staged: fp32 blocks this warp has sent so far
         bool alive = true;
         for (int tile = blockIdx.x; tile < num_tiles && alive; tile += gridDim.x, local++) {
             const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
@@ -251,29 +270,34 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
                 if (col0 >= p.N) break;               // uniform across the warp
                 uint32_t r[32];
                 tmem_ld32(taddr + c * 32, r);
-                if (row < p.M) {
-                    if (OUT_F32) {
-                        float *out = reinterpret_cast<float *>(p.C) + (long long)row * p.ldc + col0;
+                if (OUT_F32) {
+                    // stage the warp's 32 x 32 block (row = lane) with the 128-byte swizzle the tensor map expects
+                    const uint32_t buf_s = epi + (uint32_t)(quarter * 2 + (staged & 1u)) * EPI_BUF_BYTES;
+                    staged++;
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                    __syncwarp();
 #pragma unroll
-                        for (int j = 0; j < 32; j += 4) {
-                            float v[4];
+                    for (int j = 0; j < 8; j++) {
+                        float v[4];
 #pragma unroll
-                            for (int e = 0; e < 4; e++) {
-                                v[e] = __uint_as_float(r[j + e]);
-                                if (p.bias && col0 + j + e < p.N) v[e] += __bfloat162float(p.bias[col0 + j + e]);
-                            }
-                            if (col0 + j + 3 < p.N) {
-                                if (p.accumulate) {
-                                    const float4 o = *reinterpret_cast<const float4 *>(out + j);
-                                    v[0] += o.x; v[1] += o.y; v[2] += o.z; v[3] += o.w;
-                                }
-                                *reinterpret_cast<float4 *>(out + j) = make_float4(v[0], v[1], v[2], v[3]);
-                            } else {
-                                for (int e = 0; e < 4; e++)
-                                    if (col0 + j + e < p.N) out[j + e] = p.accumulate ? out[j + e] + v[e] : v[e];
-                            }
+                        for (int e = 0; e < 4; e++) {
+                            v[e] = __uint_as_float(r[4 * j + e]);
+                            if (p.bias && col0 + 4 * j + e < p.N) v[e] += __bfloat162float(p.bias[col0 + 4 * j + e]);
                         }
-                    } else {
+                        const uint32_t dst = buf_s + lane * 128 + ((j ^ (lane & 7)) << 4);
+                        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v[0]), "f"(v[1]),
+                                     "f"(v[2]), "f"(v[3])
+                                     : "memory");
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (p.accumulate) tma_reduce_add_2d(&map_c, buf_s, col0, m0 + quarter * 32);
+                        else tma_store_2d(&map_c, buf_s, col0, m0 + quarter * 32);
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    }
+                } else if (row < p.M) {
+                    {
                         bf16 *out = reinterpret_cast<bf16 *>(p.C) + (long long)row * p.ldc + col0;
 #pragma unroll
                         for (int j = 0; j < 32; j += 8) {
@@ -305,6 +329,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
         }
     }
 
+    if (OUT_F32 && warp >= 2 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     __syncwarp();
     if (*abort_flag) {
         // give copies that are still in flight time to land before shared memory is released
@@ -342,14 +367,14 @@ EncodeTiledFn encode_fn() {
 
 // 2-D bf16 tensor map over a row-major [rows, cols] matrix with leading dimension ld (elements).
 bool make_map(CUtensorMap *map, const void *base, int64_t rows, int64_t cols, int64_t ld, uint32_t box_cols,
-              uint32_t box_rows) {
+              uint32_t box_rows, bool f32 = false) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * (f32 ? 4 : 2)};
     const cuuint32_t box[2] = {box_cols, box_rows};
     const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+    const CUresult r = fn(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -370,7 +395,7 @@ int sm_count() {
 }
 
 template <bool A_MN, bool B_MN, bool OUT_F32>
-int launch(const CUtensorMap &ma, const CUtensorMap &mb, const TcParams &p, cudaStream_t st) {
+int launch(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &mc, const TcParams &p, cudaStream_t st) {
     auto kernel = gemm_tc_kernel<A_MN, B_MN, OUT_F32>;
     static bool configured = false;
     if (!configured) {
@@ -380,7 +405,7 @@ int launch(const CUtensorMap &ma, const CUtensorMap &mb, const TcParams &p, cuda
     }
     const int tiles = ((p.M + BM - 1) / BM) * ((p.N + BN - 1) / BN);
     const int grid = tiles < sm_count() ? tiles : sm_count();
-    SBP_LAUNCH(kernel, grid, NUM_THREADS, SMEM_BYTES, st, ma, mb, p);
+    SBP_LAUNCH(kernel, grid, NUM_THREADS, SMEM_BYTES, st, ma, mb, mc, p);
     return STREAMBP_OK;
 }
 
@@ -412,11 +437,13 @@ int gemm_tc(GemmOp op, int64_t M, int64_t N, int64_t K, const bf16 *A, int64_t l
             ok = make_map(&ma, A, K, M, lda, 64, BK) && make_map(&mb, B, K, N, ldb, 64, BK);
             break;
     }
+    CUtensorMap mc = ma;   // unused by the bf16-output kernels
+    if (ok && c_is_f32) ok = make_map(&mc, C, M, N, ldc, 32, 32, true);
     if (!ok) return STREAMBP_E_CUDA;
     TcParams p{(int)M, (int)N, (int)K, C, (long long)ldc, bias, accumulate ? 1 : 0};
-    if (op == OP_NT) return c_is_f32 ? launch<false, false, true>(ma, mb, p, st) : launch<false, false, false>(ma, mb, p, st);
-    if (op == OP_NN) return c_is_f32 ? launch<false, true, true>(ma, mb, p, st) : launch<false, true, false>(ma, mb, p, st);
-    return c_is_f32 ? launch<true, true, true>(ma, mb, p, st) : launch<true, true, false>(ma, mb, p, st);
+    if (op == OP_NT) return c_is_f32 ? launch<false, false, true>(ma, mb, mc, p, st) : launch<false, false, false>(ma, mb, mc, p, st);
+    if (op == OP_NN) return c_is_f32 ? launch<false, true, true>(ma, mb, mc, p, st) : launch<false, true, false>(ma, mb, mc, p, st);
+    return c_is_f32 ? launch<true, true, true>(ma, mb, mc, p, st) : launch<true, true, false>(ma, mb, mc, p, st);
 }
 
 // Reads and clears the fault flag raised by an expired bounded wait. Returns < 0 on a CUDA error.
