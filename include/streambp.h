@@ -189,6 +189,24 @@ int streambp_gemm(int op, int64_t M, int64_t N, int64_t K, const void *A, int64_
                   int32_t out_dtype, int accumulate, int engine, void *cuda_stream);
 
 /*
+ * Building blocks exposed for tests and profiling: the partitioned attention of Sec. 3.2.2
+ * (S^(i) = Q^(i) K^(:i)T, causal softmax, O^(i) = P^(i) V^(:i)) for one chunk of n query rows that
+ * sit at absolute rows q0 .. q0+n-1 and attend to keys 0 .. q0+n-1, and its backward.
+ * q, o, d_o: [n, n_q_heads, head_dim]; k, v: [q0+n, n_kv_heads, head_dim] (storage dtype);
+ * lse: [n_q_heads, n] fp32 (natural log of the row sums of exp(score / sqrt(head_dim)));
+ * delta: scratch [n_q_heads, n] fp32; dq: [n, n_q_heads, head_dim] fp32, overwritten;
+ * dk, dv: [q0+n, n_kv_heads, head_dim] fp32, ADDED to (the key-prefix accumulators).
+ * engine: 0 automatic, 1 CUDA cores, 2 tensor cores (bf16, head_dim 128 only).
+ */
+int streambp_attention_forward(const void *q, const void *k, const void *v, int64_t n, int64_t q0,
+                               int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, int32_t dtype,
+                               void *o, float *lse, int engine, void *cuda_stream);
+int streambp_attention_backward(const void *q, const void *k, const void *v, const void *o, const void *d_o,
+                                const float *lse, int64_t n, int64_t q0, int32_t n_q_heads, int32_t n_kv_heads,
+                                int32_t head_dim, int32_t dtype, float *delta, float *dq, float *dk, float *dv,
+                                int engine, void *cuda_stream);
+
+/*
  * Optional device timing by kernel class (0 = linear products, 1 = attention forward,
  * 2 = attention backward).  While enabled, each launch of those classes is bracketed by CUDA
  * events on the caller's stream.  streambp_profile_enable(1) also clears earlier records;

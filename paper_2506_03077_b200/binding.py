@@ -31,6 +31,7 @@ EXPORTS = (
     "streambp_last_device_status", "streambp_status_string",
     "streambp_last_cuda_error", "streambp_last_launch_count", "streambp_gemm",
     "streambp_profile_enable", "streambp_profile_read",
+    "streambp_attention_forward", "streambp_attention_backward",
 )
 
 
@@ -98,6 +99,11 @@ def lib() -> C.CDLL:
     L.streambp_last_launch_count.argtypes = []
     L.streambp_gemm.restype = C.c_int
     L.streambp_gemm.argtypes = [C.c_int, i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, i32, C.c_int, C.c_int, vp]
+    L.streambp_attention_forward.restype = C.c_int
+    L.streambp_attention_forward.argtypes = [vp, vp, vp, i64, i64, i32, i32, i32, i32, vp, vp, C.c_int, vp]
+    L.streambp_attention_backward.restype = C.c_int
+    L.streambp_attention_backward.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i32, i32, i32, i32, vp, vp, vp, vp,
+                                              C.c_int, vp]
     L.streambp_profile_enable.restype = None
     L.streambp_profile_enable.argtypes = [C.c_int]
     L.streambp_profile_read.restype = C.c_int
@@ -294,3 +300,26 @@ def profile_read(kernel_class: str):
     _check(lib().streambp_profile_read(KERNEL_CLASSES[kernel_class], C.byref(ms), C.byref(n), C.byref(fl)),
            "streambp_profile_read")
     return ms.value, n.value, fl.value
+
+
+def attention_forward(q, k, v, q0: int, o, lse, engine: int = 0, stream=None, check: bool = True) -> int:
+    """streambp_attention_forward; q, o: [n, Hq, dh], k, v: [q0+n, Hkv, dh], lse: [Hq, n] fp32."""
+    n, Hq, dh = q.shape
+    st = lib().streambp_attention_forward(_ptr(q), _ptr(k), _ptr(v), n, q0, Hq, k.shape[1], dh, _dtype_code(q.dtype),
+                                          _ptr(o), _ptr(lse), engine, _stream_ptr(stream))
+    if check:
+        _check(st, "streambp_attention_forward")
+    return st
+
+
+def attention_backward(q, k, v, o, d_o, lse, q0: int, dq, dk, dv, engine: int = 0, stream=None,
+                       check: bool = True) -> int:
+    """streambp_attention_backward; dq fp32 overwritten, dk / dv fp32 accumulated."""
+    n, Hq, dh = q.shape
+    delta = torch.empty(Hq, n, dtype=torch.float32, device=q.device)
+    st = lib().streambp_attention_backward(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(d_o), _ptr(lse), n, q0, Hq,
+                                           k.shape[1], dh, _dtype_code(q.dtype), _ptr(delta), _ptr(dq), _ptr(dk),
+                                           _ptr(dv), engine, _stream_ptr(stream))
+    if check:
+        _check(st, "streambp_attention_backward")
+    return st

@@ -78,6 +78,33 @@ int mm<bf16, bf16>(GemmOp op, int64_t M, int64_t N, int64_t K, const bf16 *A, in
     if (e == 2) return STREAMBP_E_SHAPE;
     return gemm<bf16, bf16>(op, M, N, K, A, lda, B, ldb, C, ldc, bias, accumulate, st);
 }
+template <>
+int attn_fwd<float>(const float *q, const float *k, const float *v, int64_t n, int64_t q0, int Hq, int Hkv, int dh,
+                    float *o, float *lse, cudaStream_t st) {
+    return attention_fwd<float>(q, k, v, n, q0, Hq, Hkv, dh, o, lse, st);
+}
+template <>
+int attn_fwd<bf16>(const bf16 *q, const bf16 *k, const bf16 *v, int64_t n, int64_t q0, int Hq, int Hkv, int dh,
+                   bf16 *o, float *lse, cudaStream_t st) {
+    const int e = gemm_engine();
+    if (e != 1 && attention_tc_supported(n, q0, Hq, Hkv, dh, q, k, v))
+        return attention_fwd_tc(q, k, v, n, q0, Hq, Hkv, o, lse, st);
+    if (e == 2) return STREAMBP_E_SHAPE;
+    return attention_fwd<bf16>(q, k, v, n, q0, Hq, Hkv, dh, o, lse, st);
+}
+template <>
+int attn_bwd<float>(const float *q, const float *k, const float *v, const float *o, const float *dout,
+                    const float *lse, int64_t n, int64_t q0, int Hq, int Hkv, int dh, float *delta, float *dq,
+                    float *dk, float *dv, cudaStream_t st) {
+    return attention_bwd<float>(q, k, v, o, dout, lse, n, q0, Hq, Hkv, dh, delta, dq, dk, dv, st);
+}
+template <>
+int attn_bwd<bf16>(const bf16 *q, const bf16 *k, const bf16 *v, const bf16 *o, const bf16 *dout, const float *lse,
+                   int64_t n, int64_t q0, int Hq, int Hkv, int dh, float *delta, float *dq, float *dk, float *dv,
+                   cudaStream_t st) {
+    return attention_bwd<bf16>(q, k, v, o, dout, lse, n, q0, Hq, Hkv, dh, delta, dq, dk, dv, st);
+}
+
 template int mm<float, float>(GemmOp, int64_t, int64_t, int64_t, const float *, int64_t, const float *, int64_t,
                               float *, int64_t, const float *, bool, cudaStream_t);
 
@@ -264,9 +291,9 @@ int streambp_last_device_status(void *workspace, void *cuda_stream) {
     WsHeader h;
     if (!cuda_ok(cudaMemcpyAsync(&h, workspace, sizeof(h), cudaMemcpyDeviceToHost, st))) return STREAMBP_E_CUDA;
     if (!cuda_ok(cudaStreamSynchronize(st))) return STREAMBP_E_CUDA;
-    const int fault = gemm_tc_take_fault();
-    if (fault < 0) return STREAMBP_E_CUDA;
-    if (fault > 0) return STREAMBP_E_DEVICE_TIMEOUT;
+    const int f1 = gemm_tc_take_fault(), f2 = attention_tc_take_fault();
+    if (f1 < 0 || f2 < 0) return STREAMBP_E_CUDA;
+    if (f1 > 0 || f2 > 0) return STREAMBP_E_DEVICE_TIMEOUT;
     return h.status;
 }
 
@@ -288,6 +315,57 @@ const char *streambp_status_string(int s) {
 
 int streambp_last_cuda_error(void) { return call_state().cuda_error; }
 int64_t streambp_last_launch_count(void) { return call_state().launches; }
+
+int streambp_attention_forward(const void *q, const void *k, const void *v, int64_t n, int64_t q0, int32_t n_q_heads,
+                               int32_t n_kv_heads, int32_t head_dim, int32_t dtype, void *o, float *lse, int engine,
+                               void *cuda_stream) {
+    if (!q || !k || !v || !o || !lse) return STREAMBP_E_NULL;
+    if (n < 1 || q0 < 0 || n_q_heads < 1 || n_kv_heads < 1 || n_q_heads % n_kv_heads ||
+        (head_dim != 64 && head_dim != 128))
+        return STREAMBP_E_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    call_state().cuda_error = 0;
+    call_state().launches = 0;
+    if (dtype == STREAMBP_F32) {
+        if (engine == 2) return STREAMBP_E_DTYPE;
+        return attention_fwd<float>((const float *)q, (const float *)k, (const float *)v, n, q0, n_q_heads, n_kv_heads,
+                                    head_dim, (float *)o, lse, st);
+    }
+    if (dtype != STREAMBP_BF16) return STREAMBP_E_DTYPE;
+    const bool tc_ok = attention_tc_supported(n, q0, n_q_heads, n_kv_heads, head_dim, q, k, v);
+    if (engine == 2 && !tc_ok) return STREAMBP_E_SHAPE;
+    if (engine != 1 && tc_ok)
+        return attention_fwd_tc((const bf16 *)q, (const bf16 *)k, (const bf16 *)v, n, q0, n_q_heads, n_kv_heads,
+                                (bf16 *)o, lse, st);
+    return attention_fwd<bf16>((const bf16 *)q, (const bf16 *)k, (const bf16 *)v, n, q0, n_q_heads, n_kv_heads,
+                               head_dim, (bf16 *)o, lse, st);
+}
+
+int streambp_attention_backward(const void *q, const void *k, const void *v, const void *o, const void *d_o,
+                                const float *lse, int64_t n, int64_t q0, int32_t n_q_heads, int32_t n_kv_heads,
+                                int32_t head_dim, int32_t dtype, float *delta, float *dq, float *dk, float *dv,
+                                int engine, void *cuda_stream) {
+    if (!q || !k || !v || !o || !d_o || !lse || !delta || !dq || !dk || !dv) return STREAMBP_E_NULL;
+    if (n < 1 || q0 < 0 || n_q_heads < 1 || n_kv_heads < 1 || n_q_heads % n_kv_heads ||
+        (head_dim != 64 && head_dim != 128))
+        return STREAMBP_E_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    call_state().cuda_error = 0;
+    call_state().launches = 0;
+    if (dtype == STREAMBP_F32) {
+        if (engine == 2) return STREAMBP_E_DTYPE;
+        return attention_bwd<float>((const float *)q, (const float *)k, (const float *)v, (const float *)o,
+                                    (const float *)d_o, lse, n, q0, n_q_heads, n_kv_heads, head_dim, delta, dq, dk, dv,
+                                    st);
+    }
+    if (dtype != STREAMBP_BF16) return STREAMBP_E_DTYPE;
+    const int saved = gemm_engine();
+    set_gemm_engine(engine);
+    const int rc = attn_bwd<bf16>((const bf16 *)q, (const bf16 *)k, (const bf16 *)v, (const bf16 *)o,
+                                  (const bf16 *)d_o, lse, n, q0, n_q_heads, n_kv_heads, head_dim, delta, dq, dk, dv, st);
+    set_gemm_engine(saved);
+    return rc;
+}
 
 void streambp_profile_enable(int on) {
     g_prof_on = on != 0;

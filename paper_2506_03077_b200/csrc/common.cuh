@@ -242,6 +242,20 @@ int attention_bwd(const T *q, const T *k, const T *v, const T *o, const T *dout,
                   int64_t q0, int Hq, int Hkv, int dh, float *delta, float *dq, float *dk, float *dv,
                   cudaStream_t st);
 
+// tcgen05 attention (bf16, head_dim 128)
+bool attention_tc_supported(int64_t n, int64_t q0, int Hq, int Hkv, int dh, const void *q, const void *k,
+                            const void *v);
+int attention_fwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, int64_t n, int64_t q0, int Hq, int Hkv, bf16 *o,
+                     float *lse, cudaStream_t st);
+int attention_tc_take_fault();
+// Dispatching attention used by the schedulers (tensor cores when supported, else CUDA cores).
+template <typename T>
+int attn_fwd(const T *q, const T *k, const T *v, int64_t n, int64_t q0, int Hq, int Hkv, int dh, T *o, float *lse,
+             cudaStream_t st);
+template <typename T>
+int attn_bwd(const T *q, const T *k, const T *v, const T *o, const T *dout, const float *lse, int64_t n, int64_t q0,
+             int Hq, int Hkv, int dh, float *delta, float *dq, float *dk, float *dv, cudaStream_t st);
+
 // LM head pieces
 int count_valid_labels(const int64_t *labels, int64_t T, int64_t vocab, int64_t ignore, WsHeader *hdr,
                        cudaStream_t st);

@@ -91,7 +91,7 @@ int chunk_forward(const streambp_layer_cfg &c, const streambp_layer_weights &w, 
         // causal pairs (query, key) of this chunk: n * r0 + n (n + 1) / 2; two products forward
         const double pairs = (double)n * (double)r0 + 0.5 * (double)n * (double)(n + 1);
         ProfScope prof(KC_ATTN_FWD, 2.0 * 2.0 * pairs * dh * Hq, st);
-        SBP_TRY(attention_fwd<T>(s.Q, s.K, s.V, n, r0, Hq, Hkv, dh, s.O, s.lse, st));
+        SBP_TRY(attn_fwd<T>(s.Q, s.K, s.V, n, r0, Hq, Hkv, dh, s.O, s.lse, st));
     }
     SBP_TRY((mm<T, float>(OP_NT, n, d, dq, s.O, dq, (const T *)w.wo, dq, s.fa, d, nullptr, false, st)));
     SBP_TRY(rmsnorm_fwd<T>(Xi, s.fa, (const T *)w.g2, c.rms_eps, n, d, s.h2, s.rstd2, s.r, st));
@@ -176,8 +176,7 @@ int layer_backward(const streambp_layer_cfg &c, const streambp_layer_weights &w,
         {
             const double pairs = (double)n * (double)r0 + 0.5 * (double)n * (double)(n + 1);
             ProfScope prof(KC_ATTN_BWD, 5.0 * 2.0 * pairs * dh * Hq, st);   // five products backward
-            SBP_TRY(attention_bwd<T>(s.Q, s.K, s.V, s.O, s.dO, s.lse, n, r0, Hq, Hkv, dh, s.delta, s.fa, s.dK, s.dV,
-                                     st));
+            SBP_TRY(attn_bwd<T>(s.Q, s.K, s.V, s.O, s.dO, s.lse, n, r0, Hq, Hkv, dh, s.delta, s.fa, s.dK, s.dV, st));
         }
 
         // ---- Q projection backward ----

@@ -1,0 +1,120 @@
+"""GPU parity of the partitioned-attention building blocks (CUDA-core and tensor-core engines)
+against the CPU oracle's attention."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import streambp_oracle as O
+from paper_2506_03077_b200 import binding as B
+from paper_2506_03077_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def make_qkv(seed, n, q0, Hq, Hkv, dh, dtype, scale=1.0):
+    kv = q0 + n
+    q = synth.normal(seed, "q", (kv, Hq, dh), 0.0, scale)
+    k = synth.normal(seed, "k", (kv, Hkv, dh), 0.0, scale)
+    v = synth.normal(seed, "v", (kv, Hkv, dh))
+    do = synth.normal(seed, "do", (kv, Hq, dh))
+    if dtype == torch.bfloat16:
+        q, k, v, do = (synth.round_bf16(a) for a in (q, k, v, do))
+    return q, k, v, do
+
+
+def oracle_chunk(q, k, v, do, q0):
+    """Oracle attention on the whole prefix; the rows of the chunk are those from q0 on.
+    Upstream gradient is zero outside the chunk, so dk/dv hold the chunk's contribution only."""
+    o = O.attention_forward(q.astype(np.float64), k.astype(np.float64), v.astype(np.float64))
+    do_chunk = do.astype(np.float64).copy()
+    do_chunk[:q0] = 0.0
+    dq, dk, dv = O.attention_backward(q.astype(np.float64), k.astype(np.float64), v.astype(np.float64), do_chunk)
+    return o[q0:], dq[q0:], dk, dv
+
+
+def oracle_lse(q, k, q0, dh):
+    T, Hq, _ = q.shape
+    G = Hq // k.shape[1]
+    out = np.empty((Hq, T - q0))
+    for h in range(Hq):
+        s = (q[q0:, h].astype(np.float64) @ k[:, h // G].astype(np.float64).T) / np.sqrt(dh)
+        for i in range(T - q0):
+            row = s[i, : q0 + i + 1]
+            out[h, i] = row.max() + np.log(np.exp(row - row.max()).sum())
+    return out
+
+
+CASES = [
+    # n, q0, Hq, Hkv
+    (128, 0, 2, 1),        # one tile, diagonal only
+    (256, 0, 4, 2),        # two query tiles
+    (128, 384, 2, 2),      # chunk deep inside the sequence: full tiles then the diagonal
+    (200, 300, 4, 1),      # ragged chunk, offset not a tile multiple
+    (77, 1000, 2, 1),      # short chunk against a long prefix
+    (640, 0, 2, 1),        # un-partitioned
+]
+
+
+@pytest.mark.parametrize("engine", [1, 2])
+@pytest.mark.parametrize("n,q0,Hq,Hkv", CASES)
+def test_attention_forward_bf16(engine, n, q0, Hq, Hkv):
+    dh, dt = 128, torch.bfloat16
+    q, k, v, do = make_qkv(n + q0, n, q0, Hq, Hkv, dh, dt, scale=1.5)
+    o_ref, _, _, _ = oracle_chunk(q, k, v, do, q0)
+    qd = torch.from_numpy(q[q0:]).to("cuda", dt).contiguous()
+    kd, vd = torch.from_numpy(k).to("cuda", dt), torch.from_numpy(v).to("cuda", dt)
+    o = torch.full((n, Hq, dh), float("nan"), device="cuda", dtype=dt)
+    lse = torch.full((Hq, n), float("nan"), device="cuda")
+    B.attention_forward(qd, kd, vd, q0, o, lse, engine=engine)
+    torch.cuda.synchronize()
+    got = o.float().cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    assert O.rel_frobenius(got, o_ref) < 6e-3
+    assert np.abs(got - o_ref).max() < 0.06
+    lse_ref = oracle_lse(q, k, q0, dh)
+    assert np.abs(lse.cpu().numpy() - lse_ref).max() < 2e-3
+
+
+@pytest.mark.parametrize("engine", [1, 2])
+@pytest.mark.parametrize("n,q0,Hq,Hkv", CASES)
+def test_attention_backward_bf16(engine, n, q0, Hq, Hkv):
+    dh, dt = 128, torch.bfloat16
+    q, k, v, do = make_qkv(n + q0 + 1, n, q0, Hq, Hkv, dh, dt, scale=1.5)
+    o_ref, dq_ref, dk_ref, dv_ref = oracle_chunk(q, k, v, do, q0)
+    qd = torch.from_numpy(q[q0:]).to("cuda", dt).contiguous()
+    dod = torch.from_numpy(do[q0:]).to("cuda", dt).contiguous()
+    kd, vd = torch.from_numpy(k).to("cuda", dt), torch.from_numpy(v).to("cuda", dt)
+    o = torch.empty((n, Hq, dh), device="cuda", dtype=dt)
+    lse = torch.empty((Hq, n), device="cuda")
+    B.attention_forward(qd, kd, vd, q0, o, lse, engine=1)
+    dq = torch.full((n, Hq, dh), float("nan"), device="cuda")
+    dk = torch.ones((q0 + n, Hkv, dh), device="cuda")       # accumulated into: start from a known value
+    dv = torch.ones((q0 + n, Hkv, dh), device="cuda")
+    B.attention_backward(qd, kd, vd, o, dod, lse, q0, dq, dk, dv, engine=engine)
+    torch.cuda.synchronize()
+    assert O.rel_frobenius(dq.cpu().numpy(), dq_ref) < 1.5e-2
+    assert O.rel_frobenius(dk.cpu().numpy() - 1.0, dk_ref) < 1.5e-2
+    assert O.rel_frobenius(dv.cpu().numpy() - 1.0, dv_ref) < 1.5e-2
+
+
+@pytest.mark.parametrize("dh,dtype", [(64, torch.float32), (128, torch.float32), (64, torch.bfloat16)])
+def test_attention_cuda_core_variants(dh, dtype):
+    n, q0, Hq, Hkv = 100, 60, 4, 2
+    q, k, v, do = make_qkv(5, n, q0, Hq, Hkv, dh, dtype)
+    o_ref, dq_ref, dk_ref, dv_ref = oracle_chunk(q, k, v, do, q0)
+    qd = torch.from_numpy(q[q0:]).to("cuda", dtype).contiguous()
+    dod = torch.from_numpy(do[q0:]).to("cuda", dtype).contiguous()
+    kd, vd = torch.from_numpy(k).to("cuda", dtype), torch.from_numpy(v).to("cuda", dtype)
+    o = torch.empty((n, Hq, dh), device="cuda", dtype=dtype)
+    lse = torch.empty((Hq, n), device="cuda")
+    B.attention_forward(qd, kd, vd, q0, o, lse, engine=1)
+    tol = 1e-5 if dtype == torch.float32 else 6e-3
+    assert O.rel_frobenius(o.float().cpu().numpy(), o_ref) < tol
+    dq = torch.empty((n, Hq, dh), device="cuda")
+    dk = torch.zeros((q0 + n, Hkv, dh), device="cuda")
+    dv = torch.zeros((q0 + n, Hkv, dh), device="cuda")
+    B.attention_backward(qd, kd, vd, o, dod, lse, q0, dq, dk, dv, engine=1)
+    tol = 2e-5 if dtype == torch.float32 else 1.5e-2
+    assert O.rel_frobenius(dq.cpu().numpy(), dq_ref) < tol
+    assert O.rel_frobenius(dk.cpu().numpy(), dk_ref) < tol
+    assert O.rel_frobenius(dv.cpu().numpy(), dv_ref) < tol
