@@ -102,6 +102,12 @@ template <>
 int attn_bwd<bf16>(const bf16 *q, const bf16 *k, const bf16 *v, const bf16 *o, const bf16 *dout, const float *lse,
                    int64_t n, int64_t q0, int Hq, int Hkv, int dh, float *delta, float *dq, float *dk, float *dv,
                    cudaStream_t st) {
+    const int e = gemm_engine();
+    if (e != 1 && attention_tc_supported(n, q0, Hq, Hkv, dh, q, k, v)) {
+        SBP_TRY(attention_delta<bf16>(o, dout, n, Hq, dh, delta, st));
+        return attention_bwd_tc(q, k, v, dout, lse, delta, n, q0, Hq, Hkv, dq, dk, dv, st);
+    }
+    if (e == 2) return STREAMBP_E_SHAPE;
     return attention_bwd<bf16>(q, k, v, o, dout, lse, n, q0, Hq, Hkv, dh, delta, dq, dk, dv, st);
 }
 

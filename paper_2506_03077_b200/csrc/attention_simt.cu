@@ -327,6 +327,16 @@ int attention_bwd(const T *q, const T *k, const T *v, const T *o, const T *dout,
     return STREAMBP_OK;
 }
 
+template <typename T>
+int attention_delta(const T *o, const T *dout, int64_t n, int Hq, int dh, float *delta, cudaStream_t st) {
+    if (n <= 0) return STREAMBP_OK;
+    const int64_t warps = n * Hq;
+    SBP_LAUNCH(attn_delta_kernel<T>, (unsigned)((warps * 32 + 255) / 256), 256, 0, st, o, dout, n, Hq, dh, delta);
+    return STREAMBP_OK;
+}
+template int attention_delta<float>(const float *, const float *, int64_t, int, int, float *, cudaStream_t);
+template int attention_delta<bf16>(const bf16 *, const bf16 *, int64_t, int, int, float *, cudaStream_t);
+
 template int attention_fwd<float>(const float *, const float *, const float *, int64_t, int64_t, int, int, int, float *,
                                   float *, cudaStream_t);
 template int attention_fwd<bf16>(const bf16 *, const bf16 *, const bf16 *, int64_t, int64_t, int, int, int, bf16 *,

@@ -15,6 +15,8 @@
 //
 // All mbarrier waits are bounded (see sm100.cuh); on expiry the CTA leaves its loops, frees its
 // tensor memory and returns, and the host sees STREAMBP_E_DEVICE_TIMEOUT.
+#include <cstdlib>
+
 #include "sm100.cuh"
 
 namespace sbp {
@@ -64,6 +66,7 @@ struct FwdParams {
 
 constexpr int FWD_SMEM = TILE_BYTES /*Q*/ + 2 * TILE_BYTES /*K*/ + 2 * TILE_BYTES /*V*/ + TILE_BYTES /*P*/ + 1024 + 256;
 
+template <bool P_TMEM>
 __global__ void __launch_bounds__(192, 1)
     attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                        const __grid_constant__ CUtensorMap map_v, const FwdParams p) {
@@ -107,6 +110,7 @@ __global__ void __launch_bounds__(192, 1)
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
     const uint32_t tS = tmem, tO = tmem + 256;     // S buffers at columns 0 and 128, O at 256
+    const uint32_t tP = tmem + 384;                // P as packed bf16 pairs (64 columns) when P_TMEM
 
     if (warp == 0) {
         if (lane == 0) {
@@ -151,9 +155,13 @@ __global__ void __launch_bounds__(192, 1)
                 if (!mbar_wait(v_full + 8 * st, ph, abort_flag)) { alive = false; break; }
                 tc_fence_after();
 #pragma unroll
-                for (int kk = 0; kk < 8; kk++)
-                    umma_bf16(tO, desc_kmajor(sP, kk), desc_mnmajor(sV + st * TILE_BYTES, kk), idesc_pv,
-                              (j | kk) != 0);
+                for (int kk = 0; kk < 8; kk++) {
+                    if (P_TMEM)
+                        umma_bf16_ts(tO, tP + kk * 8, desc_mnmajor(sV + st * TILE_BYTES, kk), idesc_pv, (j | kk) != 0);
+                    else
+                        umma_bf16(tO, desc_kmajor(sP, kk), desc_mnmajor(sV + st * TILE_BYTES, kk), idesc_pv,
+                                  (j | kk) != 0);
+                }
                 umma_commit(v_empty + 8 * st);
                 umma_commit(pv_done);
             }
@@ -230,10 +238,21 @@ __global__ void __launch_bounds__(192, 1)
                     tmem_wait_st();
                 }
             }
+            if (P_TMEM) {
 #pragma unroll
-            for (int cc = 0; cc < 16; cc++)
-                st_shared_v4(swz_addr(sP, row, cc), pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                for (int c = 0; c < 2; c++) {
+                    uint32_t r[32];
+#pragma unroll
+                    for (int e = 0; e < 32; e++) r[e] = pk[c * 32 + e];
+                    tmem_st32(tP + lane_base + c * 32, r);
+                }
+                tmem_wait_st();
+            } else {
+#pragma unroll
+                for (int cc = 0; cc < 16; cc++)
+                    st_shared_v4(swz_addr(sP, row, cc), pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(p_full);
@@ -276,6 +295,382 @@ __global__ void __launch_bounds__(192, 1)
     }
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Backward.  Two kernels, both deterministic (no floating-point atomics):
+//   dK/dV: one CTA per (128-key tile, KV head); K and V tiles stay in shared memory; loops over the
+//          G query heads of the group and over the query tiles that can see the key tile.
+//          S^T = K Q^T and dP^T = V dO^T land in tensor memory with keys on the lanes, so a thread owns
+//          one key row; P^T and dS^T are packed to bf16 in place and feed dV += P^T dO and dK += dS^T Q
+//          as tensor-memory A operands.  The Q / dO tiles serve both as K-major B operands (first two
+//          products) and as MN-major B operands (last two) without being moved.
+//   dQ   : one CTA per (128-query tile, query head); Q and dO tiles stay resident, K / V tiles stream;
+//          S = Q K^T, dP = dO V^T, dS packed in place, dQ += dS K.
+// ---------------------------------------------------------------------------------------------
+struct BwdParams {
+    int n;
+    long long q0;
+    int Hq, Hkv;
+    const float *lse;     // [Hq, n]
+    const float *delta;   // [Hq, n]
+    float *dq;            // [n, Hq, 128]
+    float *dk, *dv;       // [q0 + n, Hkv, 128]
+    float scale, scale_log2;
+};
+
+constexpr int BWD_SMEM = 6 * TILE_BYTES + 4 * TILE * 4 /* lse, delta x 2 stages */ + 1024 + 256;
+
+__global__ void __launch_bounds__(192, 1)
+    attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                            const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
+                            const BwdParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    const uint32_t sK = base, sV = sK + TILE_BYTES, sQ = sV + TILE_BYTES, sdO = sQ + 2 * TILE_BYTES;
+    uint8_t *tail = smem_raw + (base - raw) + 6 * TILE_BYTES;
+    float *s_lse = reinterpret_cast<float *>(tail);           // [2][128], pre-multiplied by log2(e)
+    float *s_delta = s_lse + 2 * TILE;                        // [2][128]
+    uint8_t *aux = tail + 4 * TILE * 4;
+    const uint32_t bars = smem_u32(aux);
+    const uint32_t kv_full = bars, in_full = bars + 8, in_empty = bars + 24, s_full = bars + 40, p_full = bars + 48,
+                   acc_full = bars + 56;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux + 64);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(aux + 72);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = blockIdx.y, G = p.Hq / p.Hkv;
+    const long long k_abs0 = (long long)blockIdx.x * TILE;
+    const int nqt = (p.n + TILE - 1) / TILE;
+    const int first_qt = k_abs0 > p.q0 ? (int)((k_abs0 - p.q0) / TILE) : 0;
+    const int per_head = nqt - first_qt;
+    const int iters = G * per_head;
+
+    if (threadIdx.x == 0) {
+        mbar_init(kv_full, 1);
+        for (int s = 0; s < 2; s++) {
+            mbar_init(in_full + 8 * s, 1);
+            mbar_init(in_empty + 8 * s, 1);
+        }
+        mbar_init(s_full, 1);
+        mbar_init(p_full, 4);
+        mbar_init(acc_full, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    const uint32_t tST = tmem, tDPT = tmem + 128, tDV = tmem + 256, tDK = tmem + 384;
+
+    if (warp == 0) {
+        // ---- producer: K, V once; then per iteration lse / delta (plain loads) and the Q, dO tiles (TMA)
+        if (lane == 0) {
+            mbar_expect_tx(kv_full, 2 * TILE_BYTES);
+            tma_load_2d(sK, &map_k, kv_full, g * TILE, (int)k_abs0);
+            tma_load_2d(sK + HALF_BYTES, &map_k, kv_full, g * TILE + 64, (int)k_abs0);
+            tma_load_2d(sV, &map_v, kv_full, g * TILE, (int)k_abs0);
+            tma_load_2d(sV + HALF_BYTES, &map_v, kv_full, g * TILE + 64, (int)k_abs0);
+        }
+        bool alive = true;
+        for (int it = 0; it < iters && alive; it++) {
+            const int h = g * G + it / per_head, qt0 = (first_qt + it % per_head) * TILE;
+            const uint32_t st = it & 1, ph = (it >> 1) & 1;
+            int ok = 1;
+            if (lane == 0) ok = mbar_wait(in_empty + 8 * st, ph ^ 1u, abort_flag) ? 1 : 0;
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) { alive = false; break; }
+#pragma unroll
+            for (int e = 0; e < 4; e++) {
+                const int col = lane * 4 + e, r = qt0 + col;
+                s_lse[st * TILE + col] = r < p.n ? p.lse[(long long)h * p.n + r] * kLog2e : 0.f;
+                s_delta[st * TILE + col] = r < p.n ? p.delta[(long long)h * p.n + r] : 0.f;
+            }
+            __syncwarp();
+            if (lane == 0) {
+                const uint32_t full = in_full + 8 * st;
+                mbar_expect_tx(full, 2 * TILE_BYTES);
+                tma_load_2d(sQ + st * TILE_BYTES, &map_q, full, h * TILE, qt0);
+                tma_load_2d(sQ + st * TILE_BYTES + HALF_BYTES, &map_q, full, h * TILE + 64, qt0);
+                tma_load_2d(sdO + st * TILE_BYTES, &map_do, full, h * TILE, qt0);
+                tma_load_2d(sdO + st * TILE_BYTES + HALF_BYTES, &map_do, full, h * TILE + 64, qt0);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc_kk = make_idesc(TILE, TILE, false, false);
+            constexpr uint32_t idesc_kmn = make_idesc(TILE, TILE, false, true);
+            bool alive = mbar_wait(kv_full, 0, abort_flag);
+            for (int it = 0; it < iters && alive; it++) {
+                const uint32_t st = it & 1, ph = (it >> 1) & 1;
+                if (!mbar_wait(in_full + 8 * st, ph, abort_flag)) { alive = false; break; }
+                tc_fence_after();
+                const uint32_t q_t = sQ + st * TILE_BYTES, do_t = sdO + st * TILE_BYTES;
+#pragma unroll
+                for (int kk = 0; kk < 8; kk++)
+                    umma_bf16(tST, desc_kmajor(sK, kk), desc_kmajor(q_t, kk), idesc_kk, kk != 0);
+#pragma unroll
+                for (int kk = 0; kk < 8; kk++)
+                    umma_bf16(tDPT, desc_kmajor(sV, kk), desc_kmajor(do_t, kk), idesc_kk, kk != 0);
+                umma_commit(s_full);
+                if (!mbar_wait(p_full, it & 1, abort_flag)) { alive = false; break; }
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < 8; kk++)
+                    umma_bf16_ts(tDV, tST + kk * 8, desc_mnmajor(do_t, kk), idesc_kmn, (it | kk) != 0);
+#pragma unroll
+                for (int kk = 0; kk < 8; kk++)
+                    umma_bf16_ts(tDK, tDPT + kk * 8, desc_mnmajor(q_t, kk), idesc_kmn, (it | kk) != 0);
+                umma_commit(in_empty + 8 * st);
+            }
+            if (alive) umma_commit(acc_full);
+        }
+    } else {
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;                      // key row within the tile
+        const long long k_abs = k_abs0 + row;
+        const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+        bool alive = true;
+        for (int it = 0; it < iters && alive; it++) {
+            const int qt0 = (first_qt + it % per_head) * TILE;
+            const uint32_t st = it & 1;
+            // the producer's lse / delta rows of this stage are published together with the tiles
+            if (!mbar_wait(in_full + 8 * st, (it >> 1) & 1, abort_flag)) { alive = false; break; }
+            if (!mbar_wait(s_full, it & 1, abort_flag)) { alive = false; break; }
+            tc_fence_after();
+            const long long q_abs0 = p.q0 + qt0;
+            // query column c is visible to this key iff q_abs0 + c >= k_abs
+            const int first_col = (k_abs > q_abs0) ? (int)((k_abs - q_abs0) > TILE ? TILE : (k_abs - q_abs0)) : 0;
+            const float *lse2 = s_lse + st * TILE, *dl = s_delta + st * TILE;
+#pragma unroll 1
+            for (int c = 0; c < 4; c++) {
+                uint32_t rs[32], rp[32];
+                tmem_ld32(tST + lane_base + c * 32, rs);
+                tmem_ld32(tDPT + lane_base + c * 32, rp);
+                uint32_t pp[16], ds[16];
+#pragma unroll
+                for (int e = 0; e < 32; e += 4) {
+                    const float4 l4 = *reinterpret_cast<const float4 *>(lse2 + c * 32 + e);
+                    const float4 d4 = *reinterpret_cast<const float4 *>(dl + c * 32 + e);
+                    const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, dv[4] = {d4.x, d4.y, d4.z, d4.w};
+                    float pv[4], dsv[4];
+#pragma unroll
+                    for (int t = 0; t < 4; t++) {
+                        const int col = c * 32 + e + t;
+                        float x = __uint_as_float(rs[e + t]) * p.scale_log2 - lv[t];
+                        if (col < first_col) x = -INFINITY;
+                        pv[t] = fast_exp2(x);
+                        dsv[t] = pv[t] * (__uint_as_float(rp[e + t]) - dv[t]) * p.scale;
+                    }
+                    pp[e / 2] = pack_bf16(pv[0], pv[1]);
+                    pp[e / 2 + 1] = pack_bf16(pv[2], pv[3]);
+                    ds[e / 2] = pack_bf16(dsv[0], dsv[1]);
+                    ds[e / 2 + 1] = pack_bf16(dsv[2], dsv[3]);
+                }
+                tmem_st16(tST + lane_base + c * 16, pp);
+                tmem_st16(tDPT + lane_base + c * 16, ds);
+            }
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(p_full);
+        }
+        if (alive && iters > 0 && mbar_wait(acc_full, 0, abort_flag)) {
+            tc_fence_after();
+            const bool in_range = k_abs < p.q0 + p.n;
+#pragma unroll 1
+            for (int c = 0; c < 4; c++) {
+                uint32_t rv[32], rk[32];
+                tmem_ld32(tDV + lane_base + c * 32, rv);
+                tmem_ld32(tDK + lane_base + c * 32, rk);
+                if (in_range) {
+                    float *pv = p.dv + (k_abs * p.Hkv + g) * TILE + c * 32;
+                    float *pk = p.dk + (k_abs * p.Hkv + g) * TILE + c * 32;
+#pragma unroll
+                    for (int e = 0; e < 32; e += 4) {
+                        float4 a = *reinterpret_cast<float4 *>(pv + e);
+                        a.x += __uint_as_float(rv[e]); a.y += __uint_as_float(rv[e + 1]);
+                        a.z += __uint_as_float(rv[e + 2]); a.w += __uint_as_float(rv[e + 3]);
+                        *reinterpret_cast<float4 *>(pv + e) = a;
+                        float4 b = *reinterpret_cast<float4 *>(pk + e);
+                        b.x += __uint_as_float(rk[e]); b.y += __uint_as_float(rk[e + 1]);
+                        b.z += __uint_as_float(rk[e + 2]); b.w += __uint_as_float(rk[e + 3]);
+                        *reinterpret_cast<float4 *>(pk + e) = b;
+                    }
+                }
+            }
+        }
+    }
+
+    __syncwarp();
+    if (*abort_flag) {
+        const unsigned long long t0 = global_timer();
+        while (global_timer() - t0 < 200000ull) { }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem, 512);
+    }
+}
+
+__global__ void __launch_bounds__(192, 1)
+    attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                          const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
+                          const BwdParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    const uint32_t sQ = base, sdO = sQ + TILE_BYTES, sK = sdO + TILE_BYTES, sV = sK + 2 * TILE_BYTES;
+    uint8_t *aux = smem_raw + (base - raw) + 6 * TILE_BYTES + 4 * TILE * 4;
+    const uint32_t bars = smem_u32(aux);
+    const uint32_t q_full = bars, kv_full = bars + 8, kv_empty = bars + 24, s_full = bars + 40, p_full = bars + 48,
+                   acc_full = bars + 56;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux + 64);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(aux + 72);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int h = blockIdx.y, g = h / (p.Hq / p.Hkv);
+    const int qt0 = blockIdx.x * TILE;
+    const long long q_abs0 = p.q0 + qt0;
+    const int rows_here = (p.n - qt0) < TILE ? (p.n - qt0) : TILE;
+    const long long kv_end = q_abs0 + rows_here;
+    const int nkv = (int)((kv_end + TILE - 1) / TILE);
+
+    if (threadIdx.x == 0) {
+        mbar_init(q_full, 1);
+        for (int s = 0; s < 2; s++) {
+            mbar_init(kv_full + 8 * s, 1);
+            mbar_init(kv_empty + 8 * s, 1);
+        }
+        mbar_init(s_full, 1);
+        mbar_init(p_full, 4);
+        mbar_init(acc_full, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    const uint32_t tS = tmem, tDP = tmem + 128, tDQ = tmem + 256;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            mbar_expect_tx(q_full, 2 * TILE_BYTES);
+            tma_load_2d(sQ, &map_q, q_full, h * TILE, qt0);
+            tma_load_2d(sQ + HALF_BYTES, &map_q, q_full, h * TILE + 64, qt0);
+            tma_load_2d(sdO, &map_do, q_full, h * TILE, qt0);
+            tma_load_2d(sdO + HALF_BYTES, &map_do, q_full, h * TILE + 64, qt0);
+            for (int j = 0; j < nkv; j++) {
+                const uint32_t st = j & 1, ph = (j >> 1) & 1;
+                if (!mbar_wait(kv_empty + 8 * st, ph ^ 1u, abort_flag)) break;
+                const uint32_t full = kv_full + 8 * st;
+                mbar_expect_tx(full, 2 * TILE_BYTES);
+                tma_load_2d(sK + st * TILE_BYTES, &map_k, full, g * TILE, j * TILE);
+                tma_load_2d(sK + st * TILE_BYTES + HALF_BYTES, &map_k, full, g * TILE + 64, j * TILE);
+                tma_load_2d(sV + st * TILE_BYTES, &map_v, full, g * TILE, j * TILE);
+                tma_load_2d(sV + st * TILE_BYTES + HALF_BYTES, &map_v, full, g * TILE + 64, j * TILE);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc_kk = make_idesc(TILE, TILE, false, false);
+            constexpr uint32_t idesc_kmn = make_idesc(TILE, TILE, false, true);
+            bool alive = mbar_wait(q_full, 0, abort_flag);
+            for (int j = 0; j < nkv && alive; j++) {
+                const uint32_t st = j & 1, ph = (j >> 1) & 1;
+                if (!mbar_wait(kv_full + 8 * st, ph, abort_flag)) { alive = false; break; }
+                tc_fence_after();
+                const uint32_t k_t = sK + st * TILE_BYTES, v_t = sV + st * TILE_BYTES;
+#pragma unroll
+                for (int kk = 0; kk < 8; kk++)
+                    umma_bf16(tS, desc_kmajor(sQ, kk), desc_kmajor(k_t, kk), idesc_kk, kk != 0);
+#pragma unroll
+                for (int kk = 0; kk < 8; kk++)
+                    umma_bf16(tDP, desc_kmajor(sdO, kk), desc_kmajor(v_t, kk), idesc_kk, kk != 0);
+                umma_commit(s_full);
+                if (!mbar_wait(p_full, j & 1, abort_flag)) { alive = false; break; }
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < 8; kk++)
+                    umma_bf16_ts(tDQ, tDP + kk * 8, desc_mnmajor(k_t, kk), idesc_kmn, (j | kk) != 0);
+                umma_commit(kv_empty + 8 * st);
+            }
+            if (alive) umma_commit(acc_full);
+        }
+    } else {
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;
+        const int qr = qt0 + row;
+        const long long q_abs = q_abs0 + row;
+        const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+        const float lse2 = qr < p.n ? p.lse[(long long)h * p.n + qr] * kLog2e : 0.f;
+        const float delta = qr < p.n ? p.delta[(long long)h * p.n + qr] : 0.f;
+        bool alive = true;
+        for (int j = 0; j < nkv && alive; j++) {
+            if (!mbar_wait(s_full, j & 1, abort_flag)) { alive = false; break; }
+            tc_fence_after();
+            const long long k_abs0 = (long long)j * TILE;
+            const bool diag = k_abs0 + TILE - 1 > q_abs0;
+            const int lim = diag ? (int)(q_abs - k_abs0) : (1 << 30);
+#pragma unroll 1
+            for (int c = 0; c < 4; c++) {
+                uint32_t rs[32], rp[32], ds[16];
+                tmem_ld32(tS + lane_base + c * 32, rs);
+                tmem_ld32(tDP + lane_base + c * 32, rp);
+#pragma unroll
+                for (int e = 0; e < 32; e += 2) {
+                    float x0 = __uint_as_float(rs[e]) * p.scale_log2 - lse2;
+                    float x1 = __uint_as_float(rs[e + 1]) * p.scale_log2 - lse2;
+                    if (c * 32 + e > lim) x0 = -INFINITY;
+                    if (c * 32 + e + 1 > lim) x1 = -INFINITY;
+                    const float d0 = fast_exp2(x0) * (__uint_as_float(rp[e]) - delta) * p.scale;
+                    const float d1 = fast_exp2(x1) * (__uint_as_float(rp[e + 1]) - delta) * p.scale;
+                    ds[e / 2] = pack_bf16(d0, d1);
+                }
+                tmem_st16(tDP + lane_base + c * 16, ds);
+            }
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(p_full);
+        }
+        if (alive && mbar_wait(acc_full, 0, abort_flag)) {
+            tc_fence_after();
+#pragma unroll 1
+            for (int c = 0; c < 4; c++) {
+                uint32_t r[32];
+                tmem_ld32(tDQ + lane_base + c * 32, r);
+                if (qr < p.n) {
+                    float *out = p.dq + ((long long)qr * p.Hq + h) * TILE + c * 32;
+#pragma unroll
+                    for (int e = 0; e < 32; e += 4)
+                        *reinterpret_cast<float4 *>(out + e) =
+                            make_float4(__uint_as_float(r[e]), __uint_as_float(r[e + 1]), __uint_as_float(r[e + 2]),
+                                        __uint_as_float(r[e + 3]));
+                }
+            }
+        }
+    }
+
+    __syncwarp();
+    if (*abort_flag) {
+        const unsigned long long t0 = global_timer();
+        while (global_timer() - t0 < 200000ull) { }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem, 512);
+    }
+}
+
 template <typename K>
 bool opt_in_smem(K kernel, int bytes) {
     return cuda_ok(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
@@ -293,6 +688,7 @@ bool attention_tc_supported(int64_t n, int64_t q0, int Hq, int Hkv, int dh, cons
 
 int attention_fwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, int64_t n, int64_t q0, int Hq, int Hkv, bf16 *o,
                      float *lse, cudaStream_t st) {
+    static const bool p_smem = std::getenv("STREAMBP_ATTN_P_SMEM") != nullptr;
     CUtensorMap mq, mk, mv;
     const int64_t kv_len = q0 + n;
     if (!make_tensor_map(&mq, q, n, (int64_t)Hq * TILE, (int64_t)Hq * TILE, 64, TILE, false) ||
@@ -301,12 +697,41 @@ int attention_fwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, int64_t n, int
         return STREAMBP_E_CUDA;
     static bool configured = false;
     if (!configured) {
-        if (!opt_in_smem(attn_fwd_tc_kernel, FWD_SMEM)) return STREAMBP_E_CUDA;
+        if (!opt_in_smem(attn_fwd_tc_kernel<true>, FWD_SMEM) || !opt_in_smem(attn_fwd_tc_kernel<false>, FWD_SMEM))
+            return STREAMBP_E_CUDA;
         configured = true;
     }
     FwdParams p{(int)n, (long long)q0, Hq, Hkv, o, lse, kLog2e / sqrtf((float)TILE)};
     dim3 grid((unsigned)((n + TILE - 1) / TILE), Hq);
-    SBP_LAUNCH(attn_fwd_tc_kernel, grid, 192, FWD_SMEM, st, mq, mk, mv, p);
+    if (p_smem)
+        SBP_LAUNCH(attn_fwd_tc_kernel<false>, grid, 192, FWD_SMEM, st, mq, mk, mv, p);
+    else
+        SBP_LAUNCH(attn_fwd_tc_kernel<true>, grid, 192, FWD_SMEM, st, mq, mk, mv, p);
+    return STREAMBP_OK;
+}
+
+int attention_bwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, const bf16 *dout, const float *lse,
+                     const float *delta, int64_t n, int64_t q0, int Hq, int Hkv, float *dq, float *dk, float *dv,
+                     cudaStream_t st) {
+    CUtensorMap mq, mk, mv, mdo;
+    const int64_t kv_len = q0 + n;
+    if (!make_tensor_map(&mq, q, n, (int64_t)Hq * TILE, (int64_t)Hq * TILE, 64, TILE, false) ||
+        !make_tensor_map(&mdo, dout, n, (int64_t)Hq * TILE, (int64_t)Hq * TILE, 64, TILE, false) ||
+        !make_tensor_map(&mk, k, kv_len, (int64_t)Hkv * TILE, (int64_t)Hkv * TILE, 64, TILE, false) ||
+        !make_tensor_map(&mv, v, kv_len, (int64_t)Hkv * TILE, (int64_t)Hkv * TILE, 64, TILE, false))
+        return STREAMBP_E_CUDA;
+    static bool configured = false;
+    if (!configured) {
+        if (!opt_in_smem(attn_bwd_dkdv_tc_kernel, BWD_SMEM) || !opt_in_smem(attn_bwd_dq_tc_kernel, BWD_SMEM))
+            return STREAMBP_E_CUDA;
+        configured = true;
+    }
+    const float scale = 1.f / sqrtf((float)TILE);
+    BwdParams p{(int)n, (long long)q0, Hq, Hkv, lse, delta, dq, dk, dv, scale, scale * kLog2e};
+    dim3 gkv((unsigned)((kv_len + TILE - 1) / TILE), Hkv);
+    dim3 gq((unsigned)((n + TILE - 1) / TILE), Hq);
+    SBP_LAUNCH(attn_bwd_dkdv_tc_kernel, gkv, 192, BWD_SMEM, st, mq, mk, mv, mdo, p);
+    SBP_LAUNCH(attn_bwd_dq_tc_kernel, gq, 192, BWD_SMEM, st, mq, mk, mv, mdo, p);
     return STREAMBP_OK;
 }
 

@@ -247,6 +247,12 @@ bool attention_tc_supported(int64_t n, int64_t q0, int Hq, int Hkv, int dh, cons
                             const void *v);
 int attention_fwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, int64_t n, int64_t q0, int Hq, int Hkv, bf16 *o,
                      float *lse, cudaStream_t st);
+// delta [Hq, n] must already hold rowsum(dO * O) (attention_delta below).
+int attention_bwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, const bf16 *dout, const float *lse,
+                     const float *delta, int64_t n, int64_t q0, int Hq, int Hkv, float *dq, float *dk, float *dv,
+                     cudaStream_t st);
+template <typename T>
+int attention_delta(const T *o, const T *dout, int64_t n, int Hq, int dh, float *delta, cudaStream_t st);
 int attention_tc_take_fault();
 // Dispatching attention used by the schedulers (tensor cores when supported, else CUDA cores).
 template <typename T>
