@@ -35,6 +35,32 @@ def layer_flops(s, T):
     return fwd + bwd + att
 
 
+# DRAM bytes (read + write) of one representative launch of the dominant kernel, from the ncu capture
+# summarised in profiles/gemm_tc_kernel_qwen7b_chunk1024.md (the per-chunk product dh2 += du Wu:
+# M 1024, N 3584, K 18944; algorithmic bytes 189.3e6).  Launch shapes depend on the chunk, not on T.
+NCU_TRAFFIC_BYTES = {("qwen7b_layer", 1024): 192.9e6}
+
+
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """Timing rule for N > 1: every rank reports the slowest rank's device time."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_seed(base_seed: int, rank: int) -> int:
+    """Replicas see different sequences; the weights are the same on every rank."""
+    return base_seed + 1000 * rank
+
+
+def aggregate_tokens_per_s(T: int, world: int, ms_per_step: float) -> float:
+    """Whole-job throughput: tokens all replicas processed in a step / the slowest replica's step time."""
+    return world * T / (ms_per_step * 1e-3)
+
+
 def read_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -174,7 +200,7 @@ def main():
     T, chunk = cfg.T, cfg.chunk
     bcfg = B.LayerConfig(s.d_model, s.n_q_heads, s.n_kv_heads, s.head_dim, s.d_ff, s.qkv_bias, s.rope_theta,
                          s.rms_eps, dt)
-    seed = cfg.seed + 1000 * rank          # replicas see different sequences
+    seed = replica_seed(cfg.seed, rank)
     Wn = synth.make_layer_weights(s, cfg.seed, cfg.bf16)
     Xn, dYn = synth.make_layer_io(s, seed, T, cfg.bf16)
     W = {k: torch.from_numpy(v).to("cuda", dt) for k, v in Wn.items()}
@@ -211,10 +237,7 @@ def main():
             fn()
         e1.record(stream)
         barrier()
-        ms = torch.tensor([e0.elapsed_time(e1)], device="cuda")
-        if world > 1:
-            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-        return float(ms.item())
+        return max_over_ranks(e0.elapsed_time(e1), world, "cuda")
 
     for _ in range(args.warmup):
         step()
@@ -236,7 +259,7 @@ def main():
         e2e_ms = timed(step_e2e, args.steps)
 
     ms_per_step = total_ms / args.steps
-    value = world * T / (ms_per_step * 1e-3)
+    value = aggregate_tokens_per_s(T, world, ms_per_step)
     peaks = read_peaks()
     flops = layer_flops(s, T)
     gemm_ms, gemm_calls, gemm_flops = prof["gemm"]
@@ -262,7 +285,9 @@ def main():
         "gpu_launches": int(launches_per_step * args.steps),
         "roofline": {"bound": "tensor", "kernel": "linear products (all GEMM launches of the step)",
                      "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-                     "peak_source": peaks["source"] + " sustained bf16", "traffic": None,
+                     "peak_source": peaks["source"] + " sustained bf16",
+                     "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, chunk)),
+                     "traffic_note": "dram bytes of one representative product launch under ncu (see profiles/)",
                      "launches": int(gemm_calls), "ms_per_step": gemm_ms / args.steps},
         "kernel_classes": {
             "gemm": {"ms_per_step": gemm_ms / args.steps, "tflops": achieved},
@@ -275,7 +300,7 @@ def main():
     }
     if e2e_ms is not None:
         nbytes = X_host.numel() * X_host.element_size()
-        out["e2e"] = {"value": world * T / (e2e_ms / args.steps * 1e-3), "unit": UNIT,
+        out["e2e"] = {"value": aggregate_tokens_per_s(T, world, e2e_ms / args.steps), "unit": UNIT,
                       "h2d_bytes_per_step": 2 * nbytes, "d2h_bytes_per_step": nbytes}
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         Ts = min(args.cpu_baseline_tokens, T)

@@ -1,0 +1,65 @@
+"""Host-side logic of bench.py on CPU: FLOP accounting, replica bookkeeping and the
+max-over-ranks timing rule with two gloo ranks."""
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+import bench  # noqa: E402
+from paper_2506_03077_b200 import synth  # noqa: E402
+
+
+def test_layer_flops_match_the_published_totals():
+    # qwen7b layer T 8192 -> 12.03 TFLOP, llama8b layer T 32768 -> 69.82 TFLOP
+    assert abs(bench.layer_flops(synth.QWEN7B_LAYER, 8192) / 1e12 - 12.03) < 0.01
+    assert abs(bench.layer_flops(synth.LLAMA8B_LAYER, 32768) / 1e12 - 69.82) < 0.01
+
+
+def test_replica_bookkeeping():
+    assert bench.replica_seed(1, 0) == 1 and bench.replica_seed(1, 3) == 3001
+    assert bench.aggregate_tokens_per_s(8192, 4, 20.0) == pytest.approx(4 * 8192 / 0.02)
+    p = bench.read_peaks()
+    assert p["sustained"] > 0 and p["source"] in ("measured", "fallback")
+
+
+def _rank_main(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    mine = 10.0 + 5.0 * rank                     # rank 1 is the slow replica
+    agreed = bench.max_over_ranks(mine, world, "cpu")
+    dist.barrier()
+    out.put((rank, agreed))
+    dist.destroy_process_group()
+
+
+def test_max_over_ranks_with_two_gloo_ranks():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = 29500 + os.getpid() % 1000
+    procs = [ctx.Process(target=_rank_main, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = dict(q.get(timeout=120) for _ in range(2))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert got == {0: 15.0, 1: 15.0}
+
+
+def test_reference_arm_prints_one_json_line():
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1",
+                        "--warmup", "0", "--ref-tokens", "32", "--config", "qwen7b_layer"],
+                       capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr
+    lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    j = json.loads(lines[0])
+    assert j["impl"] == "reference" and j["cpu_baseline"]["kind"] == "oracle"
+    assert j["e2e"]["h2d_bytes_per_step"] == 0 and j["value"] > 0
