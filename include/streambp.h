@@ -207,6 +207,28 @@ int streambp_attention_backward(const void *q, const void *k, const void *v, con
                                 int engine, void *cuda_stream);
 
 /*
+ * (No counterpart in the paper.)  streambp_attention_backward for callers that have no device buffer
+ * to offer for `delta` and cannot obtain one when they call: host code in a latency-critical loop
+ * where cudaMalloc / cudaFree would stall the whole device, a plug-in whose host framework already owns
+ * all device memory, a process whose memory budget is frozen after start-up.  Same arguments and results
+ * as streambp_attention_backward minus `delta`: the row sums live in a fixed array inside the library
+ * image, STREAMBP_STATIC_DELTA_MAX_FLOATS floats (4 MiB) that every GPU loading the library holds until
+ * the process exits.  The call performs no device-memory allocation of any kind.
+ *   - Limit: n * n_q_heads <= STREAMBP_STATIC_DELTA_MAX_FLOATS, else STREAMBP_E_WORKSPACE is returned
+ *     and nothing is enqueued.
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ *     that device current); make that first call before starting any stream capture.
+ *   - All calls on a device share the one array.  Its previous contents are irrelevant (every row sum
+ *     used by a call is rewritten by that call first), but two calls whose kernels overlap on the GPU
+ *     (different streams, or several host threads) race on it: serialise them on one stream.
+ */
+#define STREAMBP_STATIC_DELTA_MAX_FLOATS (1 << 20)
+int streambp_attention_backward_static(const void *q, const void *k, const void *v, const void *o, const void *d_o,
+                                       const float *lse, int64_t n, int64_t q0, int32_t n_q_heads,
+                                       int32_t n_kv_heads, int32_t head_dim, int32_t dtype, float *dq, float *dk,
+                                       float *dv, int engine, void *cuda_stream);
+
+/*
  * Optional device timing by kernel class (0 = linear products, 1 = attention forward,
  * 2 = attention backward).  While enabled, each launch of those classes is bracketed by CUDA
  * events on the caller's stream.  streambp_profile_enable(1) also clears earlier records;

@@ -31,7 +31,7 @@ EXPORTS = (
     "streambp_last_device_status", "streambp_status_string",
     "streambp_last_cuda_error", "streambp_last_launch_count", "streambp_gemm",
     "streambp_profile_enable", "streambp_profile_read",
-    "streambp_attention_forward", "streambp_attention_backward",
+    "streambp_attention_forward", "streambp_attention_backward", "streambp_attention_backward_static",
 )
 
 
@@ -104,6 +104,9 @@ def lib() -> C.CDLL:
     L.streambp_attention_backward.restype = C.c_int
     L.streambp_attention_backward.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i32, i32, i32, i32, vp, vp, vp, vp,
                                               C.c_int, vp]
+    L.streambp_attention_backward_static.restype = C.c_int
+    L.streambp_attention_backward_static.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i32, i32, i32, i32, vp, vp, vp,
+                                                     C.c_int, vp]
     L.streambp_profile_enable.restype = None
     L.streambp_profile_enable.argtypes = [C.c_int]
     L.streambp_profile_read.restype = C.c_int
@@ -322,4 +325,22 @@ def attention_backward(q, k, v, o, d_o, lse, q0: int, dq, dk, dv, engine: int = 
                                            _ptr(dv), engine, _stream_ptr(stream))
     if check:
         _check(st, "streambp_attention_backward")
+    return st
+
+
+STATIC_DELTA_MAX_FLOATS = 1 << 20
+
+
+def attention_backward_static(q, k, v, o, d_o, lse, q0: int, dq, dk, dv, engine: int = 0, stream=None,
+                              check: bool = True) -> int:
+    """streambp_attention_backward_static: like attention_backward, but the row-sum scratch is the
+    library's fixed 4 MiB array, so neither this wrapper nor the library allocates device memory.
+    For callers that cannot allocate at call time.  Requires n * Hq <= STATIC_DELTA_MAX_FLOATS;
+    calls that overlap on the GPU race on the shared array."""
+    n, Hq, dh = q.shape
+    st = lib().streambp_attention_backward_static(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(d_o), _ptr(lse), n, q0, Hq,
+                                                  k.shape[1], dh, _dtype_code(q.dtype), _ptr(dq), _ptr(dk), _ptr(dv),
+                                                  engine, _stream_ptr(stream))
+    if check:
+        _check(st, "streambp_attention_backward_static")
     return st
