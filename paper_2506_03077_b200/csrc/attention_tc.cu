@@ -181,19 +181,21 @@ __global__ void __launch_bounds__(192, 1)
             const long long k_abs0 = (long long)j * TILE;
             const bool diag = k_abs0 + TILE - 1 > q_abs0;       // some (query, key) pair of the tile is masked
             const int lim = diag ? (int)(q_abs - k_abs0) : (1 << 30);   // keys 0..lim of the tile are visible
-            // pass 1: row maximum of the scaled scores
+            // pass 1: row maximum of the raw scores (the scale is positive, so it commutes with max)
             float mt = -INFINITY;
 #pragma unroll 1
             for (int c = 0; c < 4; c++) {
                 uint32_t r[32];
                 tmem_ld32(tSj + c * 32, r);
+                if (diag) {
 #pragma unroll
-                for (int e = 0; e < 32; e++) {
-                    float x = __uint_as_float(r[e]) * p.scale_log2;
-                    if (c * 32 + e > lim) x = -INFINITY;
-                    mt = fmaxf(mt, x);
+                    for (int e = 0; e < 32; e++) mt = fmaxf(mt, c * 32 + e > lim ? -INFINITY : __uint_as_float(r[e]));
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 32; e++) mt = fmaxf(mt, __uint_as_float(r[e]));
                 }
             }
+            mt *= p.scale_log2;
             float factor = 1.f;
             const bool grow = mt > m_used + 8.f;                 // also true on the first tile (m_used = -inf)
             if (grow) {
@@ -201,18 +203,21 @@ __global__ void __launch_bounds__(192, 1)
                 m_used = mt;
                 l *= factor;
             }
-            // pass 2: P = exp2(x - m_used), packed to bf16
+            // pass 2: P = exp2(s * scale - m_used), packed to bf16
             uint32_t pk[64];
+            const float neg_m = -m_used;
 #pragma unroll
             for (int c = 0; c < 4; c++) {
                 uint32_t r[32];
                 tmem_ld32(tSj + c * 32, r);
 #pragma unroll
                 for (int e = 0; e < 32; e += 2) {
-                    float x0 = __uint_as_float(r[e]) * p.scale_log2 - m_used;
-                    float x1 = __uint_as_float(r[e + 1]) * p.scale_log2 - m_used;
-                    if (c * 32 + e > lim) x0 = -INFINITY;
-                    if (c * 32 + e + 1 > lim) x1 = -INFINITY;
+                    float x0 = fmaf(__uint_as_float(r[e]), p.scale_log2, neg_m);
+                    float x1 = fmaf(__uint_as_float(r[e + 1]), p.scale_log2, neg_m);
+                    if (diag) {
+                        if (c * 32 + e > lim) x0 = -INFINITY;
+                        if (c * 32 + e + 1 > lim) x1 = -INFINITY;
+                    }
                     const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
                     l += p0 + p1;
                     pk[c * 16 + e / 2] = pack_bf16(p0, p1);
@@ -306,6 +311,12 @@ __global__ void __launch_bounds__(192, 1)
 //          products) and as MN-major B operands (last two) without being moved.
 //   dQ   : one CTA per (128-query tile, query head); Q and dO tiles stay resident, K / V tiles stream;
 //          S = Q K^T, dP = dO V^T, dS packed in place, dQ += dS K.
+// Both split every 128-wide tile of the streamed operand into two 64-wide halves with their own
+// tensor-memory buffers; each half is turned into P / dS by two softmax warpgroups of 32 columns
+// each (16 softmax warps per CTA, four per scheduler, to hide the tensor-memory load latency).
+// The MMA thread interleaves: as soon as a half's P / dS is consumed by the accumulating products it
+// issues the NEXT tile's S / dP for that half, so each half's softmax warps always have work queued
+// while the tensor pipe serves the other half.
 // ---------------------------------------------------------------------------------------------
 struct BwdParams {
     int n;
@@ -319,8 +330,17 @@ struct BwdParams {
 };
 
 constexpr int BWD_SMEM = 6 * TILE_BYTES + 4 * TILE * 4 /* lse, delta x 2 stages */ + 1024 + 256;
+constexpr int BWD_THREADS = 64 + 512;
+constexpr int HALF = 64;
 
-__global__ void __launch_bounds__(192, 1)
+__device__ __forceinline__ void abort_drain(volatile int *abort_flag) {
+    if (*abort_flag) {   // give copies that are still in flight time to land before shared memory is released
+        const unsigned long long t0 = global_timer();
+        while (global_timer() - t0 < 200000ull) { }
+    }
+}
+
+__global__ void __launch_bounds__(BWD_THREADS, 1)
     attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                             const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
                             const BwdParams p) {
@@ -333,10 +353,10 @@ __global__ void __launch_bounds__(192, 1)
     float *s_delta = s_lse + 2 * TILE;                        // [2][128]
     uint8_t *aux = tail + 4 * TILE * 4;
     const uint32_t bars = smem_u32(aux);
-    const uint32_t kv_full = bars, in_full = bars + 8, in_empty = bars + 24, s_full = bars + 40, p_full = bars + 48,
-                   acc_full = bars + 56;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux + 64);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(aux + 72);
+    const uint32_t kv_full = bars, in_full = bars + 8, in_empty = bars + 24, s_full = bars + 40, p_full = bars + 56,
+                   acc_full = bars + 72;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux + 80);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(aux + 88);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = blockIdx.y, G = p.Hq / p.Hkv;
@@ -351,9 +371,9 @@ __global__ void __launch_bounds__(192, 1)
         for (int s = 0; s < 2; s++) {
             mbar_init(in_full + 8 * s, 1);
             mbar_init(in_empty + 8 * s, 1);
+            mbar_init(s_full + 8 * s, 1);
+            mbar_init(p_full + 8 * s, 8);
         }
-        mbar_init(s_full, 1);
-        mbar_init(p_full, 4);
         mbar_init(acc_full, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -363,6 +383,7 @@ __global__ void __launch_bounds__(192, 1)
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    // columns: S^T halves at 0 / 64, dP^T halves at 128 / 192, dV at 256, dK at 384
     const uint32_t tST = tmem, tDPT = tmem + 128, tDV = tmem + 256, tDK = tmem + 384;
 
     if (warp == 0) {
@@ -374,19 +395,18 @@ __global__ void __launch_bounds__(192, 1)
             tma_load_2d(sV, &map_v, kv_full, g * TILE, (int)k_abs0);
             tma_load_2d(sV + HALF_BYTES, &map_v, kv_full, g * TILE + 64, (int)k_abs0);
         }
-        bool alive = true;
-        for (int it = 0; it < iters && alive; it++) {
+        for (int it = 0; it < iters; it++) {
             const int h = g * G + it / per_head, qt0 = (first_qt + it % per_head) * TILE;
             const uint32_t st = it & 1, ph = (it >> 1) & 1;
             int ok = 1;
             if (lane == 0) ok = mbar_wait(in_empty + 8 * st, ph ^ 1u, abort_flag) ? 1 : 0;
             ok = __shfl_sync(0xffffffffu, ok, 0);
-            if (!ok) { alive = false; break; }
+            if (!ok) break;
 #pragma unroll
             for (int e = 0; e < 4; e++) {
                 const int col = lane * 4 + e, r = qt0 + col;
                 s_lse[st * TILE + col] = r < p.n ? p.lse[(long long)h * p.n + r] * kLog2e : 0.f;
-                s_delta[st * TILE + col] = r < p.n ? p.delta[(long long)h * p.n + r] : 0.f;
+                s_delta[st * TILE + col] = r < p.n ? p.delta[(long long)h * p.n + r] * p.scale : 0.f;
             }
             __syncwarp();
             if (lane == 0) {
@@ -400,115 +420,138 @@ __global__ void __launch_bounds__(192, 1)
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc_kk = make_idesc(TILE, TILE, false, false);
-            constexpr uint32_t idesc_kmn = make_idesc(TILE, TILE, false, true);
+            constexpr uint32_t idesc_half = make_idesc(TILE, HALF, false, false);   // N = 64 queries
+            constexpr uint32_t idesc_acc = make_idesc(TILE, TILE, false, true);     // N = 128 head dims
             bool alive = mbar_wait(kv_full, 0, abort_flag);
+            // S^T and dP^T of one 64-query half of iteration `it`
+            auto issue_sdp = [&](int it, int hf) {
+                const uint32_t st = it & 1;
+                const uint32_t q_t = sQ + st * TILE_BYTES + hf * 8192, do_t = sdO + st * TILE_BYTES + hf * 8192;
+#pragma unroll
+                for (int kk = 0; kk < 8; kk++)
+                    umma_bf16(tST + hf * HALF, desc_kmajor(sK, kk), desc_kmajor(q_t, kk), idesc_half, kk != 0);
+#pragma unroll
+                for (int kk = 0; kk < 8; kk++)
+                    umma_bf16(tDPT + hf * HALF, desc_kmajor(sV, kk), desc_kmajor(do_t, kk), idesc_half, kk != 0);
+                umma_commit(s_full + 8 * hf);
+            };
+            if (alive && iters > 0) {
+                alive = mbar_wait(in_full, 0, abort_flag);
+                if (alive) {
+                    tc_fence_after();
+                    issue_sdp(0, 0);
+                    issue_sdp(0, 1);
+                }
+            }
             for (int it = 0; it < iters && alive; it++) {
-                const uint32_t st = it & 1, ph = (it >> 1) & 1;
-                if (!mbar_wait(in_full + 8 * st, ph, abort_flag)) { alive = false; break; }
-                tc_fence_after();
+                const uint32_t st = it & 1;
                 const uint32_t q_t = sQ + st * TILE_BYTES, do_t = sdO + st * TILE_BYTES;
 #pragma unroll
-                for (int kk = 0; kk < 8; kk++)
-                    umma_bf16(tST, desc_kmajor(sK, kk), desc_kmajor(q_t, kk), idesc_kk, kk != 0);
+                for (int hf = 0; hf < 2; hf++) {
+                    if (!mbar_wait(p_full + 8 * hf, it & 1, abort_flag)) { alive = false; break; }
+                    tc_fence_after();
 #pragma unroll
-                for (int kk = 0; kk < 8; kk++)
-                    umma_bf16(tDPT, desc_kmajor(sV, kk), desc_kmajor(do_t, kk), idesc_kk, kk != 0);
-                umma_commit(s_full);
-                if (!mbar_wait(p_full, it & 1, abort_flag)) { alive = false; break; }
-                tc_fence_after();
+                    for (int kk = 0; kk < 4; kk++)
+                        umma_bf16_ts(tDV, tST + hf * HALF + (kk >> 1) * 32 + (kk & 1) * 8, desc_mnmajor(do_t, hf * 4 + kk),
+                                     idesc_acc, (it | hf | kk) != 0);
 #pragma unroll
-                for (int kk = 0; kk < 8; kk++)
-                    umma_bf16_ts(tDV, tST + kk * 8, desc_mnmajor(do_t, kk), idesc_kmn, (it | kk) != 0);
-#pragma unroll
-                for (int kk = 0; kk < 8; kk++)
-                    umma_bf16_ts(tDK, tDPT + kk * 8, desc_mnmajor(q_t, kk), idesc_kmn, (it | kk) != 0);
-                umma_commit(in_empty + 8 * st);
+                    for (int kk = 0; kk < 4; kk++)
+                        umma_bf16_ts(tDK, tDPT + hf * HALF + (kk >> 1) * 32 + (kk & 1) * 8, desc_mnmajor(q_t, hf * 4 + kk),
+                                     idesc_acc, (it | hf | kk) != 0);
+                    if (hf == 1) umma_commit(in_empty + 8 * st);       // both halves of this stage are consumed
+                    if (it + 1 < iters) {
+                        // the half's buffers are free again (the products above read them, in order)
+                        if (hf == 0) {
+                            if (!mbar_wait(in_full + 8 * ((it + 1) & 1), ((it + 1) >> 1) & 1, abort_flag)) {
+                                alive = false;
+                                break;
+                            }
+                            tc_fence_after();
+                        }
+                        issue_sdp(it + 1, hf);
+                    }
+                }
             }
             if (alive) umma_commit(acc_full);
         }
     } else {
         const int quarter = warp & 3;
+        const int wg = (warp - 2) >> 2;                           // 0..3: 32-query group of the tile
+        const int hf = wg >> 1, col_base = wg * 32;               // half (tensor-memory buffer) and first query column
         const int row = quarter * 32 + lane;                      // key row within the tile
         const long long k_abs = k_abs0 + row;
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+        const uint32_t tS_g = tST + col_base + lane_base, tP_g = tDPT + col_base + lane_base;
+        // packed bf16 pairs overwrite the front of the group's OWN fp32 columns (already consumed);
+        // the MMA thread addresses each 16-query slice of the A operand separately
         bool alive = true;
         for (int it = 0; it < iters && alive; it++) {
             const int qt0 = (first_qt + it % per_head) * TILE;
             const uint32_t st = it & 1;
             // the producer's lse / delta rows of this stage are published together with the tiles
             if (!mbar_wait(in_full + 8 * st, (it >> 1) & 1, abort_flag)) { alive = false; break; }
-            if (!mbar_wait(s_full, it & 1, abort_flag)) { alive = false; break; }
+            if (!mbar_wait(s_full + 8 * hf, it & 1, abort_flag)) { alive = false; break; }
             tc_fence_after();
             const long long q_abs0 = p.q0 + qt0;
-            // query column c is visible to this key iff q_abs0 + c >= k_abs
+            const bool diag = k_abs0 + TILE - 1 > q_abs0;          // the tile pair holds masked (query, key) pairs
+            // query column c of the tile is visible to this key iff q_abs0 + c >= k_abs
             const int first_col = (k_abs > q_abs0) ? (int)((k_abs - q_abs0) > TILE ? TILE : (k_abs - q_abs0)) : 0;
-            const float *lse2 = s_lse + st * TILE, *dl = s_delta + st * TILE;
-#pragma unroll 1
-            for (int c = 0; c < 4; c++) {
-                uint32_t rs[32], rp[32];
-                tmem_ld32(tST + lane_base + c * 32, rs);
-                tmem_ld32(tDPT + lane_base + c * 32, rp);
-                uint32_t pp[16], ds[16];
+            const float *lse2 = s_lse + st * TILE + col_base, *dl = s_delta + st * TILE + col_base;
+            uint32_t rs[32], rp[32], pp[16], ds[16];
+            tmem_ld32(tS_g, rs);
+            tmem_ld32(tP_g, rp);
 #pragma unroll
-                for (int e = 0; e < 32; e += 4) {
-                    const float4 l4 = *reinterpret_cast<const float4 *>(lse2 + c * 32 + e);
-                    const float4 d4 = *reinterpret_cast<const float4 *>(dl + c * 32 + e);
-                    const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, dv[4] = {d4.x, d4.y, d4.z, d4.w};
-                    float pv[4], dsv[4];
+            for (int e = 0; e < 32; e += 4) {
+                const float4 l4 = *reinterpret_cast<const float4 *>(lse2 + e);
+                const float4 d4 = *reinterpret_cast<const float4 *>(dl + e);
+                const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, dv[4] = {d4.x, d4.y, d4.z, d4.w};
+                float pv[4], dsv[4];
 #pragma unroll
-                    for (int t = 0; t < 4; t++) {
-                        const int col = c * 32 + e + t;
-                        float x = __uint_as_float(rs[e + t]) * p.scale_log2 - lv[t];
-                        if (col < first_col) x = -INFINITY;
-                        pv[t] = fast_exp2(x);
-                        dsv[t] = pv[t] * (__uint_as_float(rp[e + t]) - dv[t]) * p.scale;
-                    }
-                    pp[e / 2] = pack_bf16(pv[0], pv[1]);
-                    pp[e / 2 + 1] = pack_bf16(pv[2], pv[3]);
-                    ds[e / 2] = pack_bf16(dsv[0], dsv[1]);
-                    ds[e / 2 + 1] = pack_bf16(dsv[2], dsv[3]);
+                for (int t = 0; t < 4; t++) {
+                    float x = fmaf(__uint_as_float(rs[e + t]), p.scale_log2, -lv[t]);
+                    if (diag && col_base + e + t < first_col) x = -INFINITY;
+                    pv[t] = fast_exp2(x);
+                    dsv[t] = pv[t] * fmaf(__uint_as_float(rp[e + t]), p.scale, -dv[t]);
                 }
-                tmem_st16(tST + lane_base + c * 16, pp);
-                tmem_st16(tDPT + lane_base + c * 16, ds);
+                pp[e / 2] = pack_bf16(pv[0], pv[1]);
+                pp[e / 2 + 1] = pack_bf16(pv[2], pv[3]);
+                ds[e / 2] = pack_bf16(dsv[0], dsv[1]);
+                ds[e / 2 + 1] = pack_bf16(dsv[2], dsv[3]);
             }
+            tmem_st16(tS_g, pp);
+            tmem_st16(tP_g, ds);
             tmem_wait_st();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(p_full);
+            if (lane == 0) mbar_arrive(p_full + 8 * hf);
         }
-        if (alive && iters > 0 && mbar_wait(acc_full, 0, abort_flag)) {
+        if (alive && mbar_wait(acc_full, 0, abort_flag)) {
             tc_fence_after();
             const bool in_range = k_abs < p.q0 + p.n;
-#pragma unroll 1
-            for (int c = 0; c < 4; c++) {
-                uint32_t rv[32], rk[32];
-                tmem_ld32(tDV + lane_base + c * 32, rv);
-                tmem_ld32(tDK + lane_base + c * 32, rk);
-                if (in_range) {
-                    float *pv = p.dv + (k_abs * p.Hkv + g) * TILE + c * 32;
-                    float *pk = p.dk + (k_abs * p.Hkv + g) * TILE + c * 32;
+            // group wg writes head dims 32*wg .. 32*wg+31
+            uint32_t rv[32], rk[32];
+            tmem_ld32(tDV + lane_base + col_base, rv);
+            tmem_ld32(tDK + lane_base + col_base, rk);
+            if (in_range) {
+                float *pv = p.dv + (k_abs * p.Hkv + g) * TILE + col_base;
+                float *pk = p.dk + (k_abs * p.Hkv + g) * TILE + col_base;
 #pragma unroll
-                    for (int e = 0; e < 32; e += 4) {
-                        float4 a = *reinterpret_cast<float4 *>(pv + e);
-                        a.x += __uint_as_float(rv[e]); a.y += __uint_as_float(rv[e + 1]);
-                        a.z += __uint_as_float(rv[e + 2]); a.w += __uint_as_float(rv[e + 3]);
-                        *reinterpret_cast<float4 *>(pv + e) = a;
-                        float4 b = *reinterpret_cast<float4 *>(pk + e);
-                        b.x += __uint_as_float(rk[e]); b.y += __uint_as_float(rk[e + 1]);
-                        b.z += __uint_as_float(rk[e + 2]); b.w += __uint_as_float(rk[e + 3]);
-                        *reinterpret_cast<float4 *>(pk + e) = b;
-                    }
+                for (int e = 0; e < 32; e += 4) {
+                    float4 a = *reinterpret_cast<float4 *>(pv + e);
+                    a.x += __uint_as_float(rv[e]); a.y += __uint_as_float(rv[e + 1]);
+                    a.z += __uint_as_float(rv[e + 2]); a.w += __uint_as_float(rv[e + 3]);
+                    *reinterpret_cast<float4 *>(pv + e) = a;
+                    float4 b = *reinterpret_cast<float4 *>(pk + e);
+                    b.x += __uint_as_float(rk[e]); b.y += __uint_as_float(rk[e + 1]);
+                    b.z += __uint_as_float(rk[e + 2]); b.w += __uint_as_float(rk[e + 3]);
+                    *reinterpret_cast<float4 *>(pk + e) = b;
                 }
             }
         }
     }
 
     __syncwarp();
-    if (*abort_flag) {
-        const unsigned long long t0 = global_timer();
-        while (global_timer() - t0 < 200000ull) { }
-    }
+    abort_drain(abort_flag);
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -517,7 +560,7 @@ __global__ void __launch_bounds__(192, 1)
     }
 }
 
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(BWD_THREADS, 1)
     attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                           const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
                           const BwdParams p) {
@@ -527,10 +570,10 @@ __global__ void __launch_bounds__(192, 1)
     const uint32_t sQ = base, sdO = sQ + TILE_BYTES, sK = sdO + TILE_BYTES, sV = sK + 2 * TILE_BYTES;
     uint8_t *aux = smem_raw + (base - raw) + 6 * TILE_BYTES + 4 * TILE * 4;
     const uint32_t bars = smem_u32(aux);
-    const uint32_t q_full = bars, kv_full = bars + 8, kv_empty = bars + 24, s_full = bars + 40, p_full = bars + 48,
-                   acc_full = bars + 56;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux + 64);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(aux + 72);
+    const uint32_t q_full = bars, kv_full = bars + 8, kv_empty = bars + 24, s_full = bars + 40, p_full = bars + 56,
+                   acc_full = bars + 72;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux + 80);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(aux + 88);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int h = blockIdx.y, g = h / (p.Hq / p.Hkv);
@@ -545,9 +588,9 @@ __global__ void __launch_bounds__(192, 1)
         for (int s = 0; s < 2; s++) {
             mbar_init(kv_full + 8 * s, 1);
             mbar_init(kv_empty + 8 * s, 1);
+            mbar_init(s_full + 8 * s, 1);
+            mbar_init(p_full + 8 * s, 8);
         }
-        mbar_init(s_full, 1);
-        mbar_init(p_full, 4);
         mbar_init(acc_full, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -557,6 +600,7 @@ __global__ void __launch_bounds__(192, 1)
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    // columns: S halves at 0 / 64 (keys 0-63 / 64-127 of the tile), dP halves at 128 / 192, dQ at 256
     const uint32_t tS = tmem, tDP = tmem + 128, tDQ = tmem + 256;
 
     if (warp == 0) {
@@ -579,90 +623,111 @@ __global__ void __launch_bounds__(192, 1)
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc_kk = make_idesc(TILE, TILE, false, false);
-            constexpr uint32_t idesc_kmn = make_idesc(TILE, TILE, false, true);
+            constexpr uint32_t idesc_half = make_idesc(TILE, HALF, false, false);   // N = 64 keys
+            constexpr uint32_t idesc_acc = make_idesc(TILE, TILE, false, true);     // N = 128 head dims
             bool alive = mbar_wait(q_full, 0, abort_flag);
+            // S and dP of one 64-key half of tile j
+            auto issue_sdp = [&](int j, int hf) {
+                const uint32_t st = j & 1;
+                const uint32_t k_t = sK + st * TILE_BYTES + hf * 8192, v_t = sV + st * TILE_BYTES + hf * 8192;
+#pragma unroll
+                for (int kk = 0; kk < 8; kk++)
+                    umma_bf16(tS + hf * HALF, desc_kmajor(sQ, kk), desc_kmajor(k_t, kk), idesc_half, kk != 0);
+#pragma unroll
+                for (int kk = 0; kk < 8; kk++)
+                    umma_bf16(tDP + hf * HALF, desc_kmajor(sdO, kk), desc_kmajor(v_t, kk), idesc_half, kk != 0);
+                umma_commit(s_full + 8 * hf);
+            };
+            if (alive) {
+                alive = mbar_wait(kv_full, 0, abort_flag);
+                if (alive) {
+                    tc_fence_after();
+                    issue_sdp(0, 0);
+                    issue_sdp(0, 1);
+                }
+            }
             for (int j = 0; j < nkv && alive; j++) {
-                const uint32_t st = j & 1, ph = (j >> 1) & 1;
-                if (!mbar_wait(kv_full + 8 * st, ph, abort_flag)) { alive = false; break; }
-                tc_fence_after();
-                const uint32_t k_t = sK + st * TILE_BYTES, v_t = sV + st * TILE_BYTES;
+                const uint32_t st = j & 1;
+                const uint32_t k_t = sK + st * TILE_BYTES;
 #pragma unroll
-                for (int kk = 0; kk < 8; kk++)
-                    umma_bf16(tS, desc_kmajor(sQ, kk), desc_kmajor(k_t, kk), idesc_kk, kk != 0);
+                for (int hf = 0; hf < 2; hf++) {
+                    if (!mbar_wait(p_full + 8 * hf, j & 1, abort_flag)) { alive = false; break; }
+                    tc_fence_after();
 #pragma unroll
-                for (int kk = 0; kk < 8; kk++)
-                    umma_bf16(tDP, desc_kmajor(sdO, kk), desc_kmajor(v_t, kk), idesc_kk, kk != 0);
-                umma_commit(s_full);
-                if (!mbar_wait(p_full, j & 1, abort_flag)) { alive = false; break; }
-                tc_fence_after();
-#pragma unroll
-                for (int kk = 0; kk < 8; kk++)
-                    umma_bf16_ts(tDQ, tDP + kk * 8, desc_mnmajor(k_t, kk), idesc_kmn, (j | kk) != 0);
-                umma_commit(kv_empty + 8 * st);
+                    for (int kk = 0; kk < 4; kk++)
+                        umma_bf16_ts(tDQ, tDP + hf * HALF + (kk >> 1) * 32 + (kk & 1) * 8, desc_mnmajor(k_t, hf * 4 + kk),
+                                     idesc_acc, (j | hf | kk) != 0);
+                    if (hf == 1) umma_commit(kv_empty + 8 * st);
+                    if (j + 1 < nkv) {
+                        if (hf == 0) {
+                            if (!mbar_wait(kv_full + 8 * ((j + 1) & 1), ((j + 1) >> 1) & 1, abort_flag)) {
+                                alive = false;
+                                break;
+                            }
+                            tc_fence_after();
+                        }
+                        issue_sdp(j + 1, hf);
+                    }
+                }
             }
             if (alive) umma_commit(acc_full);
         }
     } else {
         const int quarter = warp & 3;
+        const int wg = (warp - 2) >> 2;                           // 0..3: 32-key group of the tile
+        const int hf = wg >> 1, key_base = wg * 32;
         const int row = quarter * 32 + lane;
         const int qr = qt0 + row;
         const long long q_abs = q_abs0 + row;
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-        const float lse2 = qr < p.n ? p.lse[(long long)h * p.n + qr] * kLog2e : 0.f;
-        const float delta = qr < p.n ? p.delta[(long long)h * p.n + qr] : 0.f;
+        const uint32_t tS_g = tS + key_base + lane_base, tP_g = tDP + key_base + lane_base;
+        const float neg_lse2 = qr < p.n ? -p.lse[(long long)h * p.n + qr] * kLog2e : 0.f;
+        const float neg_delta_s = qr < p.n ? -p.delta[(long long)h * p.n + qr] * p.scale : 0.f;
         bool alive = true;
         for (int j = 0; j < nkv && alive; j++) {
-            if (!mbar_wait(s_full, j & 1, abort_flag)) { alive = false; break; }
+            if (!mbar_wait(s_full + 8 * hf, j & 1, abort_flag)) { alive = false; break; }
             tc_fence_after();
             const long long k_abs0 = (long long)j * TILE;
             const bool diag = k_abs0 + TILE - 1 > q_abs0;
-            const int lim = diag ? (int)(q_abs - k_abs0) : (1 << 30);
-#pragma unroll 1
-            for (int c = 0; c < 4; c++) {
-                uint32_t rs[32], rp[32], ds[16];
-                tmem_ld32(tS + lane_base + c * 32, rs);
-                tmem_ld32(tDP + lane_base + c * 32, rp);
+            const int lim = (int)(q_abs - k_abs0);                // keys 0..lim of the tile are visible (diag tiles)
+            uint32_t rs[32], rp[32], ds[16];
+            tmem_ld32(tS_g, rs);
+            tmem_ld32(tP_g, rp);
 #pragma unroll
-                for (int e = 0; e < 32; e += 2) {
-                    float x0 = __uint_as_float(rs[e]) * p.scale_log2 - lse2;
-                    float x1 = __uint_as_float(rs[e + 1]) * p.scale_log2 - lse2;
-                    if (c * 32 + e > lim) x0 = -INFINITY;
-                    if (c * 32 + e + 1 > lim) x1 = -INFINITY;
-                    const float d0 = fast_exp2(x0) * (__uint_as_float(rp[e]) - delta) * p.scale;
-                    const float d1 = fast_exp2(x1) * (__uint_as_float(rp[e + 1]) - delta) * p.scale;
-                    ds[e / 2] = pack_bf16(d0, d1);
+            for (int e = 0; e < 32; e += 2) {
+                float x0 = fmaf(__uint_as_float(rs[e]), p.scale_log2, neg_lse2);
+                float x1 = fmaf(__uint_as_float(rs[e + 1]), p.scale_log2, neg_lse2);
+                if (diag) {
+                    if (key_base + e > lim) x0 = -INFINITY;
+                    if (key_base + e + 1 > lim) x1 = -INFINITY;
                 }
-                tmem_st16(tDP + lane_base + c * 16, ds);
+                const float d0 = fast_exp2(x0) * fmaf(__uint_as_float(rp[e]), p.scale, neg_delta_s);
+                const float d1 = fast_exp2(x1) * fmaf(__uint_as_float(rp[e + 1]), p.scale, neg_delta_s);
+                ds[e / 2] = pack_bf16(d0, d1);
             }
+            tmem_st16(tP_g, ds);       // front of the group's own fp32 columns
             tmem_wait_st();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(p_full);
+            if (lane == 0) mbar_arrive(p_full + 8 * hf);
         }
         if (alive && mbar_wait(acc_full, 0, abort_flag)) {
             tc_fence_after();
-#pragma unroll 1
-            for (int c = 0; c < 4; c++) {
-                uint32_t r[32];
-                tmem_ld32(tDQ + lane_base + c * 32, r);
-                if (qr < p.n) {
-                    float *out = p.dq + ((long long)qr * p.Hq + h) * TILE + c * 32;
+            uint32_t r[32];
+            tmem_ld32(tDQ + lane_base + key_base, r);
+            if (qr < p.n) {
+                float *out = p.dq + ((long long)qr * p.Hq + h) * TILE + key_base;
 #pragma unroll
-                    for (int e = 0; e < 32; e += 4)
-                        *reinterpret_cast<float4 *>(out + e) =
-                            make_float4(__uint_as_float(r[e]), __uint_as_float(r[e + 1]), __uint_as_float(r[e + 2]),
-                                        __uint_as_float(r[e + 3]));
-                }
+                for (int e = 0; e < 32; e += 4)
+                    *reinterpret_cast<float4 *>(out + e) =
+                        make_float4(__uint_as_float(r[e]), __uint_as_float(r[e + 1]), __uint_as_float(r[e + 2]),
+                                    __uint_as_float(r[e + 3]));
             }
         }
     }
 
     __syncwarp();
-    if (*abort_flag) {
-        const unsigned long long t0 = global_timer();
-        while (global_timer() - t0 < 200000ull) { }
-    }
+    abort_drain(abort_flag);
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -730,8 +795,8 @@ int attention_bwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, const bf16 *do
     BwdParams p{(int)n, (long long)q0, Hq, Hkv, lse, delta, dq, dk, dv, scale, scale * kLog2e};
     dim3 gkv((unsigned)((kv_len + TILE - 1) / TILE), Hkv);
     dim3 gq((unsigned)((n + TILE - 1) / TILE), Hq);
-    SBP_LAUNCH(attn_bwd_dkdv_tc_kernel, gkv, 192, BWD_SMEM, st, mq, mk, mv, mdo, p);
-    SBP_LAUNCH(attn_bwd_dq_tc_kernel, gq, 192, BWD_SMEM, st, mq, mk, mv, mdo, p);
+    SBP_LAUNCH(attn_bwd_dkdv_tc_kernel, gkv, BWD_THREADS, BWD_SMEM, st, mq, mk, mv, mdo, p);
+    SBP_LAUNCH(attn_bwd_dq_tc_kernel, gq, BWD_THREADS, BWD_SMEM, st, mq, mk, mv, mdo, p);
     return STREAMBP_OK;
 }
 
