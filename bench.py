@@ -156,13 +156,108 @@ def run_reference(args, cfg):
     }))
 
 
+def head_flops(h, T):
+    """Three products of 2 T d V each (logits, dH, dW_vocab)."""
+    return 3 * 2 * T * h.d_model * h.vocab
+
+
+def run_head_or_model(args, cfg):
+    """Secondary workloads (one JSON line, same keys where they apply): the streamed LM head alone
+    (qwen7b_head) and the whole model on layer-input checkpoints (qwen7b_model).  Weights of the model
+    workload are drawn on the device (7.6 G parameters), everything else as in the layer workloads."""
+    import torch
+    from paper_2506_03077_b200 import binding as B
+    from paper_2506_03077_b200 import synth
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+        raise SystemExit("head / model workloads run on one GPU")
+    torch.cuda.set_device(0)
+    B.lib()
+    dt = torch.bfloat16
+    h, T = cfg.head, cfg.T
+    hc = B.HeadConfig(h.d_model, h.vocab, h.rms_eps, h.ignore_index, dt)
+    gen = torch.Generator(device="cuda").manual_seed(cfg.seed)
+    rn = lambda *shape, mean=0.0, std=1.0: (torch.randn(*shape, generator=gen, device="cuda") * std + mean).to(dt)
+    loss = torch.zeros(1, device="cuda")
+    peaks = read_peaks()
+    if cfg.n_layers == 0:
+        g, Wv, H, labels = synth.make_head_inputs(h, cfg.seed, T, True, cfg.masked_prefix)
+        gd, Wd, Hd = (torch.from_numpy(a).to("cuda", dt) for a in (g, Wv, H))
+        ld = torch.from_numpy(labels).cuda()
+        nv = torch.zeros(1, dtype=torch.int64, device="cuda")
+        dH, dW, dg = torch.empty_like(Hd), torch.empty(h.vocab, h.d_model, device="cuda"), torch.empty(h.d_model, device="cuda")
+        ws_bytes = B.lmhead_workspace_bytes(hc, T, cfg.chunk)
+        ws_full = B.lmhead_workspace_bytes(hc, T, T)
+        ws = B.alloc_workspace(ws_bytes)
+        step = lambda: B.lmhead_ce_backward(hc, gd, Wd, Hd, ld, cfg.chunk, loss, nv, dH, dW, dg, ws)
+        flops, name = head_flops(h, T), "streamed_lmhead_ce_backward_tokens_per_s"
+    else:
+        s, L = cfg.layer, cfg.n_layers
+        lc = B.LayerConfig(s.d_model, s.n_q_heads, s.n_kv_heads, s.head_dim, s.d_ff, s.qkv_bias, s.rope_theta, s.rms_eps, dt)
+        shapes = B.layer_grad_shapes(lc)
+        layers = [{k: rn(*shp, mean=1.0 if k in ("g1", "g2") else 0.0, std=0.02) for k, shp in shapes.items()}
+                  for _ in range(L)]
+        grads = [B.alloc_layer_grads(lc) for _ in range(L)]
+        E, Wv, gf = rn(h.vocab, h.d_model, std=0.02), rn(h.vocab, h.d_model, std=0.02), rn(h.d_model, mean=1.0, std=0.02)
+        ids, labels = synth.make_model_tokens(h.vocab, cfg.seed, T, cfg.prompt_frac)
+        idd, ld = torch.from_numpy(ids).cuda(), torch.from_numpy(labels).cuda()
+        dE, dWv, dg = torch.empty(h.vocab, h.d_model, device="cuda"), torch.empty(h.vocab, h.d_model, device="cuda"), torch.empty(h.d_model, device="cuda")
+        ch = cfg.chunk_head or cfg.chunk
+        ws_bytes = B.model_workspace_bytes(L, lc, hc, T, cfg.chunk, ch)
+        ws_full = B.model_workspace_bytes(L, lc, hc, T, T, T)
+        ws = B.alloc_workspace(ws_bytes)
+        step = lambda: B.model_backward(lc, hc, layers, gf, Wv, ld, cfg.chunk, ch, loss, grads, dg, dWv, ws,
+                                        embed=E, ids=idd, d_embed=dE)
+        P = s.d_model * s.dq + 2 * s.d_model * s.dkv + s.dq * s.d_model + 3 * s.d_model * s.d_ff
+        fwd_extra = 2 * T * P + 4 * s.head_dim * s.n_q_heads * T * (T + 1) / 2      # checkpointing forward
+        flops = L * (layer_flops(s, T) + fwd_extra) + head_flops(h, T)
+        name = "streamed_model_backward_tokens_per_s"
+    for _ in range(args.warmup):
+        step()
+    assert B.last_device_status(ws) == B.OK
+    launches = B.last_launch_count()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(0)
+    sampler.start()
+    B.profile_enable(True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    prof = {k: B.profile_read(k) for k in B.KERNEL_CLASSES}
+    B.profile_enable(False)
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / args.steps
+    gemm_ms, gemm_calls, gemm_flops = prof["gemm"]
+    achieved = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
+    print(json.dumps({
+        "metric": name, "value": T / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic", "loss": loss.item(),
+        "config": {"workload": cfg.name, "T": T, "chunk": cfg.chunk, "n_layers": cfg.n_layers, "vocab": h.vocab,
+                   "l2": "inputs larger than L2"},
+        "algorithmic_tflop_per_step": flops / 1e12, "tflops": flops / (ms * 1e-3) / 1e12,
+        "frac_of_measured_sustained_bf16": flops / (ms * 1e-3) / 1e12 / peaks["sustained"],
+        "peak_activation_gb": ws_bytes / 1e9, "peak_activation_gb_unchunked": ws_full / 1e9,
+        "gpu_launches": int(launches * args.steps),
+        "roofline": {"bound": "tensor", "kernel": "linear products", "achieved": achieved, "peak": peaks["sustained"],
+                     "unit": "TFLOP/s", "frac": achieved / peaks["sustained"], "traffic": None,
+                     "launches": int(gemm_calls), "ms_per_step": gemm_ms / args.steps},
+        "kernel_classes": {k: {"ms_per_step": v[0] / args.steps} for k, v in prof.items()},
+        "clocks": clocks,
+    }))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="qwen7b_layer", choices=["qwen7b_layer", "llama8b_layer"])
+    ap.add_argument("--config", default="qwen7b_layer",
+                    choices=["qwen7b_layer", "llama8b_layer", "qwen7b_head", "qwen7b_model"])
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count of the model configuration")
     ap.add_argument("--chunk", type=int, default=0)
     ap.add_argument("--T", type=int, default=0, help="override the sequence length (profiling on small cases)")
     ap.add_argument("--ref-tokens", type=int, default=512)
@@ -178,8 +273,14 @@ def main():
         cfg.chunk = args.chunk
     if args.T:
         cfg.T = args.T
+    if args.layers:
+        cfg.n_layers = args.layers
     if args.impl == "reference":
+        if cfg.layer is None or cfg.n_layers:
+            raise SystemExit("--impl reference times the oracle on the layer workloads only")
         return run_reference(args, cfg)
+    if cfg.layer is None or cfg.n_layers:
+        return run_head_or_model(args, cfg)
 
     import torch
     import torch.distributed as dist

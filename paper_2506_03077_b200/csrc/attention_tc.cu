@@ -28,15 +28,13 @@ constexpr int TILE_BYTES = 2 * HALF_BYTES;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
-// A / B descriptors for a [128 rows][128 cols] bf16 tile stored as two 64-column swizzled sub-tiles.
+// Descriptor low words for a [128 rows][128 cols] bf16 tile stored as two 64-column swizzled sub-tiles.
 // K-major use (contraction along the 128 columns): slice kk covers columns 16kk .. 16kk+15.
-__device__ __forceinline__ uint64_t desc_kmajor(uint32_t tile, int kk) {
-    return make_desc_sw128(tile + (kk >> 2) * HALF_BYTES + (kk & 3) * 32, 16, 1024);
-}
+__device__ __forceinline__ uint32_t klo(uint32_t tile) { return desc_lo(tile, 16); }
+__host__ __device__ constexpr uint32_t kstep(int kk) { return (uint32_t)((kk >> 2) * (HALF_BYTES >> 4) + (kk & 3) * 2); }
 // MN-major use as B (contraction along the 128 rows, N = the 128 columns): slice kk covers rows 16kk .. 16kk+15.
-__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t tile, int kk) {
-    return make_desc_sw128(tile + kk * 2048, HALF_BYTES, 1024);
-}
+__device__ __forceinline__ uint32_t mnlo(uint32_t tile) { return desc_lo(tile, HALF_BYTES); }
+__host__ __device__ constexpr uint32_t mnstep(int kk) { return (uint32_t)(kk * 128); }
 
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
@@ -140,9 +138,10 @@ __global__ void __launch_bounds__(192, 1)
                 if (!mbar_wait(k_full + 8 * st, ph, abort_flag)) return false;
                 tc_fence_after();
 #pragma unroll
+                const uint32_t q_lo = klo(sQ), k_lo = klo(sK + st * TILE_BYTES);
+#pragma unroll
                 for (int kk = 0; kk < 8; kk++)
-                    umma_bf16(tS + st * TILE, desc_kmajor(sQ, kk), desc_kmajor(sK + st * TILE_BYTES, kk), idesc_s,
-                              kk != 0);
+                    umma_ss(tS + st * TILE, q_lo + kstep(kk), k_lo + kstep(kk), idesc_s, kk != 0);
                 umma_commit(k_empty + 8 * st);
                 umma_commit(s_full + 8 * st);
                 return true;
@@ -154,13 +153,13 @@ __global__ void __launch_bounds__(192, 1)
                 if (!mbar_wait(p_full, j & 1, abort_flag)) { alive = false; break; }
                 if (!mbar_wait(v_full + 8 * st, ph, abort_flag)) { alive = false; break; }
                 tc_fence_after();
+                const uint32_t v_lo = mnlo(sV + st * TILE_BYTES), p_lo = klo(sP);
 #pragma unroll
                 for (int kk = 0; kk < 8; kk++) {
                     if (P_TMEM)
-                        umma_bf16_ts(tO, tP + kk * 8, desc_mnmajor(sV + st * TILE_BYTES, kk), idesc_pv, (j | kk) != 0);
+                        umma_ts(tO, tP + kk * 8, v_lo + mnstep(kk), idesc_pv, (j | kk) != 0);
                     else
-                        umma_bf16(tO, desc_kmajor(sP, kk), desc_mnmajor(sV + st * TILE_BYTES, kk), idesc_pv,
-                                  (j | kk) != 0);
+                        umma_ss(tO, p_lo + kstep(kk), v_lo + mnstep(kk), idesc_pv, (j | kk) != 0);
                 }
                 umma_commit(v_empty + 8 * st);
                 umma_commit(pv_done);
@@ -423,16 +422,17 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
             constexpr uint32_t idesc_half = make_idesc(TILE, HALF, false, false);   // N = 64 queries
             constexpr uint32_t idesc_acc = make_idesc(TILE, TILE, false, true);     // N = 128 head dims
             bool alive = mbar_wait(kv_full, 0, abort_flag);
+            const uint32_t k_lo = klo(sK), v_lo = klo(sV);
             // S^T and dP^T of one 64-query half of iteration `it`
             auto issue_sdp = [&](int it, int hf) {
                 const uint32_t st = it & 1;
-                const uint32_t q_t = sQ + st * TILE_BYTES + hf * 8192, do_t = sdO + st * TILE_BYTES + hf * 8192;
+                const uint32_t q_lo = klo(sQ + st * TILE_BYTES + hf * 8192), do_lo = klo(sdO + st * TILE_BYTES + hf * 8192);
 #pragma unroll
                 for (int kk = 0; kk < 8; kk++)
-                    umma_bf16(tST + hf * HALF, desc_kmajor(sK, kk), desc_kmajor(q_t, kk), idesc_half, kk != 0);
+                    umma_ss(tST + hf * HALF, k_lo + kstep(kk), q_lo + kstep(kk), idesc_half, kk != 0);
 #pragma unroll
                 for (int kk = 0; kk < 8; kk++)
-                    umma_bf16(tDPT + hf * HALF, desc_kmajor(sV, kk), desc_kmajor(do_t, kk), idesc_half, kk != 0);
+                    umma_ss(tDPT + hf * HALF, v_lo + kstep(kk), do_lo + kstep(kk), idesc_half, kk != 0);
                 umma_commit(s_full + 8 * hf);
             };
             if (alive && iters > 0) {
@@ -445,19 +445,19 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
             }
             for (int it = 0; it < iters && alive; it++) {
                 const uint32_t st = it & 1;
-                const uint32_t q_t = sQ + st * TILE_BYTES, do_t = sdO + st * TILE_BYTES;
+                const uint32_t q_mn = mnlo(sQ + st * TILE_BYTES), do_mn = mnlo(sdO + st * TILE_BYTES);
 #pragma unroll
                 for (int hf = 0; hf < 2; hf++) {
                     if (!mbar_wait(p_full + 8 * hf, it & 1, abort_flag)) { alive = false; break; }
                     tc_fence_after();
 #pragma unroll
                     for (int kk = 0; kk < 4; kk++)
-                        umma_bf16_ts(tDV, tST + hf * HALF + (kk >> 1) * 32 + (kk & 1) * 8, desc_mnmajor(do_t, hf * 4 + kk),
-                                     idesc_acc, (it | hf | kk) != 0);
+                        umma_ts(tDV, tST + hf * HALF + (kk >> 1) * 32 + (kk & 1) * 8, do_mn + mnstep(hf * 4 + kk),
+                                idesc_acc, (it | hf | kk) != 0);
 #pragma unroll
                     for (int kk = 0; kk < 4; kk++)
-                        umma_bf16_ts(tDK, tDPT + hf * HALF + (kk >> 1) * 32 + (kk & 1) * 8, desc_mnmajor(q_t, hf * 4 + kk),
-                                     idesc_acc, (it | hf | kk) != 0);
+                        umma_ts(tDK, tDPT + hf * HALF + (kk >> 1) * 32 + (kk & 1) * 8, q_mn + mnstep(hf * 4 + kk),
+                                idesc_acc, (it | hf | kk) != 0);
                     if (hf == 1) umma_commit(in_empty + 8 * st);       // both halves of this stage are consumed
                     if (it + 1 < iters) {
                         // the half's buffers are free again (the products above read them, in order)
@@ -626,16 +626,17 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
             constexpr uint32_t idesc_half = make_idesc(TILE, HALF, false, false);   // N = 64 keys
             constexpr uint32_t idesc_acc = make_idesc(TILE, TILE, false, true);     // N = 128 head dims
             bool alive = mbar_wait(q_full, 0, abort_flag);
+            const uint32_t q_lo = klo(sQ), do_lo = klo(sdO);
             // S and dP of one 64-key half of tile j
             auto issue_sdp = [&](int j, int hf) {
                 const uint32_t st = j & 1;
-                const uint32_t k_t = sK + st * TILE_BYTES + hf * 8192, v_t = sV + st * TILE_BYTES + hf * 8192;
+                const uint32_t kh_lo = klo(sK + st * TILE_BYTES + hf * 8192), vh_lo = klo(sV + st * TILE_BYTES + hf * 8192);
 #pragma unroll
                 for (int kk = 0; kk < 8; kk++)
-                    umma_bf16(tS + hf * HALF, desc_kmajor(sQ, kk), desc_kmajor(k_t, kk), idesc_half, kk != 0);
+                    umma_ss(tS + hf * HALF, q_lo + kstep(kk), kh_lo + kstep(kk), idesc_half, kk != 0);
 #pragma unroll
                 for (int kk = 0; kk < 8; kk++)
-                    umma_bf16(tDP + hf * HALF, desc_kmajor(sdO, kk), desc_kmajor(v_t, kk), idesc_half, kk != 0);
+                    umma_ss(tDP + hf * HALF, do_lo + kstep(kk), vh_lo + kstep(kk), idesc_half, kk != 0);
                 umma_commit(s_full + 8 * hf);
             };
             if (alive) {
@@ -648,15 +649,15 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
             }
             for (int j = 0; j < nkv && alive; j++) {
                 const uint32_t st = j & 1;
-                const uint32_t k_t = sK + st * TILE_BYTES;
+                const uint32_t k_mn = mnlo(sK + st * TILE_BYTES);
 #pragma unroll
                 for (int hf = 0; hf < 2; hf++) {
                     if (!mbar_wait(p_full + 8 * hf, j & 1, abort_flag)) { alive = false; break; }
                     tc_fence_after();
 #pragma unroll
                     for (int kk = 0; kk < 4; kk++)
-                        umma_bf16_ts(tDQ, tDP + hf * HALF + (kk >> 1) * 32 + (kk & 1) * 8, desc_mnmajor(k_t, hf * 4 + kk),
-                                     idesc_acc, (j | hf | kk) != 0);
+                        umma_ts(tDQ, tDP + hf * HALF + (kk >> 1) * 32 + (kk & 1) * 8, k_mn + mnstep(hf * 4 + kk), idesc_acc,
+                                (j | hf | kk) != 0);
                     if (hf == 1) umma_commit(kv_empty + 8 * st);
                     if (j + 1 < nkv) {
                         if (hf == 0) {

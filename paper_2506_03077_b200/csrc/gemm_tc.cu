@@ -191,11 +191,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
                     if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { alive = false; break; }
                     tc_fence_after();
                     const uint32_t sa = tiles + stage * STAGE_BYTES, sb = sa + A_BYTES;
+                    const uint32_t a_lo = desc_lo(sa, A_MN ? 8192u : 16u), b_lo = desc_lo(sb, B_MN ? 8192u : 16u);
 #pragma unroll
-                    for (int kk = 0; kk < BK / 16; kk++) {
-                        umma_bf16(d_tmem, make_desc(sa + kk * a_step, A_MN), make_desc(sb + kk * b_step, B_MN), idesc,
-                                  (kb | kk) != 0 ? 1u : 0u);
-                    }
+                    for (int kk = 0; kk < BK / 16; kk++)
+                        umma_ss(d_tmem, a_lo + kk * (a_step >> 4), b_lo + kk * (b_step >> 4), idesc,
+                                (kb | kk) != 0 ? 1u : 0u);
                     umma_commit(bar_empty + 8 * stage);   // frees the stage once these MMAs have read it
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
