@@ -310,12 +310,12 @@ __global__ void __launch_bounds__(192, 1)
 //          products) and as MN-major B operands (last two) without being moved.
 //   dQ   : one CTA per (128-query tile, query head); Q and dO tiles stay resident, K / V tiles stream;
 //          S = Q K^T, dP = dO V^T, dS packed in place, dQ += dS K.
-// Both split every 128-wide tile of the streamed operand into two 64-wide halves with their own
-// tensor-memory buffers; each half is turned into P / dS by two softmax warpgroups of 32 columns
-// each (16 softmax warps per CTA, four per scheduler, to hide the tensor-memory load latency).
-// The MMA thread interleaves: as soon as a half's P / dS is consumed by the accumulating products it
-// issues the NEXT tile's S / dP for that half, so each half's softmax warps always have work queued
-// while the tensor pipe serves the other half.
+// Work inside a tile pair is split in TIME, not in space, so every product is a full 128 x 128 x 128 one
+// (an N = 64 product is limited by shared-memory bandwidth to 2/3 of the tensor rate): the softmax
+// warps (16 per CTA, each thread owns 32 columns of one row) first turn S into P -- which is all the dV
+// product needs -- and only then combine it with dP into dS.  The MMA thread interleaves accordingly:
+// dV_i, then S_{i+1} (its buffer is free again), then dK_i, then dP_{i+1}; the tensor pipe therefore
+// always has the next tile's products queued while the softmax warps work.
 // ---------------------------------------------------------------------------------------------
 struct BwdParams {
     int n;
@@ -352,8 +352,8 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
     float *s_delta = s_lse + 2 * TILE;                        // [2][128]
     uint8_t *aux = tail + 4 * TILE * 4;
     const uint32_t bars = smem_u32(aux);
-    const uint32_t kv_full = bars, in_full = bars + 8, in_empty = bars + 24, s_full = bars + 40, p_full = bars + 56,
-                   acc_full = bars + 72;
+    const uint32_t kv_full = bars, in_full = bars + 8, in_empty = bars + 24, s_full = bars + 40, dp_full = bars + 48,
+                   p1_full = bars + 56, p2_full = bars + 64, acc_full = bars + 72;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux + 80);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(aux + 88);
 
@@ -370,9 +370,11 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
         for (int s = 0; s < 2; s++) {
             mbar_init(in_full + 8 * s, 1);
             mbar_init(in_empty + 8 * s, 1);
-            mbar_init(s_full + 8 * s, 1);
-            mbar_init(p_full + 8 * s, 8);
         }
+        mbar_init(s_full, 1);
+        mbar_init(dp_full, 1);
+        mbar_init(p1_full, 16);
+        mbar_init(p2_full, 16);
         mbar_init(acc_full, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -382,7 +384,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    // columns: S^T halves at 0 / 64, dP^T halves at 128 / 192, dV at 256, dK at 384
+    // columns: S^T at 0, dP^T at 128, dV at 256, dK at 384
     const uint32_t tST = tmem, tDPT = tmem + 128, tDV = tmem + 256, tDK = tmem + 384;
 
     if (warp == 0) {
@@ -419,111 +421,123 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc_half = make_idesc(TILE, HALF, false, false);   // N = 64 queries
-            constexpr uint32_t idesc_acc = make_idesc(TILE, TILE, false, true);     // N = 128 head dims
+            constexpr uint32_t idesc_kk = make_idesc(TILE, TILE, false, false);     // both operands K-major
+            constexpr uint32_t idesc_acc = make_idesc(TILE, TILE, false, true);     // B MN-major (N = head dims)
             bool alive = mbar_wait(kv_full, 0, abort_flag);
             const uint32_t k_lo = klo(sK), v_lo = klo(sV);
-            // S^T and dP^T of one 64-query half of iteration `it`
-            auto issue_sdp = [&](int it, int hf) {
-                const uint32_t st = it & 1;
-                const uint32_t q_lo = klo(sQ + st * TILE_BYTES + hf * 8192), do_lo = klo(sdO + st * TILE_BYTES + hf * 8192);
+            auto issue_st = [&](int it) {      // S^T = K Q^T
+                const uint32_t q_lo = klo(sQ + (it & 1) * TILE_BYTES);
 #pragma unroll
-                for (int kk = 0; kk < 8; kk++)
-                    umma_ss(tST + hf * HALF, k_lo + kstep(kk), q_lo + kstep(kk), idesc_half, kk != 0);
-#pragma unroll
-                for (int kk = 0; kk < 8; kk++)
-                    umma_ss(tDPT + hf * HALF, v_lo + kstep(kk), do_lo + kstep(kk), idesc_half, kk != 0);
-                umma_commit(s_full + 8 * hf);
+                for (int kk = 0; kk < 8; kk++) umma_ss(tST, k_lo + kstep(kk), q_lo + kstep(kk), idesc_kk, kk != 0);
+                umma_commit(s_full);
             };
-            if (alive && iters > 0) {
-                alive = mbar_wait(in_full, 0, abort_flag);
-                if (alive) {
-                    tc_fence_after();
-                    issue_sdp(0, 0);
-                    issue_sdp(0, 1);
-                }
+            auto issue_dpt = [&](int it) {     // dP^T = V dO^T
+                const uint32_t do_lo = klo(sdO + (it & 1) * TILE_BYTES);
+#pragma unroll
+                for (int kk = 0; kk < 8; kk++) umma_ss(tDPT, v_lo + kstep(kk), do_lo + kstep(kk), idesc_kk, kk != 0);
+                umma_commit(dp_full);
+            };
+            if (alive) alive = mbar_wait(in_full, 0, abort_flag);
+            if (alive) {
+                tc_fence_after();
+                issue_st(0);
+                issue_dpt(0);
             }
             for (int it = 0; it < iters && alive; it++) {
                 const uint32_t st = it & 1;
                 const uint32_t q_mn = mnlo(sQ + st * TILE_BYTES), do_mn = mnlo(sdO + st * TILE_BYTES);
+                // dV += P^T dO as soon as P^T is packed
+                if (!mbar_wait(p1_full, it & 1, abort_flag)) { alive = false; break; }
+                tc_fence_after();
 #pragma unroll
-                for (int hf = 0; hf < 2; hf++) {
-                    if (!mbar_wait(p_full + 8 * hf, it & 1, abort_flag)) { alive = false; break; }
+                for (int kk = 0; kk < 8; kk++)
+                    umma_ts(tDV, tST + (kk >> 1) * 32 + (kk & 1) * 8, do_mn + mnstep(kk), idesc_acc, (it | kk) != 0);
+                // the S^T columns are free again once dV has read them (in order): next tile's S^T
+                if (it + 1 < iters) {
+                    if (!mbar_wait(in_full + 8 * ((it + 1) & 1), ((it + 1) >> 1) & 1, abort_flag)) { alive = false; break; }
                     tc_fence_after();
-#pragma unroll
-                    for (int kk = 0; kk < 4; kk++)
-                        umma_ts(tDV, tST + hf * HALF + (kk >> 1) * 32 + (kk & 1) * 8, do_mn + mnstep(hf * 4 + kk),
-                                idesc_acc, (it | hf | kk) != 0);
-#pragma unroll
-                    for (int kk = 0; kk < 4; kk++)
-                        umma_ts(tDK, tDPT + hf * HALF + (kk >> 1) * 32 + (kk & 1) * 8, q_mn + mnstep(hf * 4 + kk),
-                                idesc_acc, (it | hf | kk) != 0);
-                    if (hf == 1) umma_commit(in_empty + 8 * st);       // both halves of this stage are consumed
-                    if (it + 1 < iters) {
-                        // the half's buffers are free again (the products above read them, in order)
-                        if (hf == 0) {
-                            if (!mbar_wait(in_full + 8 * ((it + 1) & 1), ((it + 1) >> 1) & 1, abort_flag)) {
-                                alive = false;
-                                break;
-                            }
-                            tc_fence_after();
-                        }
-                        issue_sdp(it + 1, hf);
-                    }
+                    issue_st(it + 1);
                 }
+                // dK += dS^T Q
+                if (!mbar_wait(p2_full, it & 1, abort_flag)) { alive = false; break; }
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < 8; kk++)
+                    umma_ts(tDK, tDPT + (kk >> 1) * 32 + (kk & 1) * 8, q_mn + mnstep(kk), idesc_acc, (it | kk) != 0);
+                umma_commit(in_empty + 8 * st);            // Q and dO of this stage are consumed
+                if (it + 1 < iters) issue_dpt(it + 1);
             }
             if (alive) umma_commit(acc_full);
         }
     } else {
         const int quarter = warp & 3;
         const int wg = (warp - 2) >> 2;                           // 0..3: 32-query group of the tile
-        const int hf = wg >> 1, col_base = wg * 32;               // half (tensor-memory buffer) and first query column
+        const int col_base = wg * 32;
         const int row = quarter * 32 + lane;                      // key row within the tile
         const long long k_abs = k_abs0 + row;
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-        const uint32_t tS_g = tST + col_base + lane_base, tP_g = tDPT + col_base + lane_base;
         // packed bf16 pairs overwrite the front of the group's OWN fp32 columns (already consumed);
         // the MMA thread addresses each 16-query slice of the A operand separately
+        const uint32_t tS_g = tST + col_base + lane_base, tP_g = tDPT + col_base + lane_base;
         bool alive = true;
         for (int it = 0; it < iters && alive; it++) {
             const int qt0 = (first_qt + it % per_head) * TILE;
             const uint32_t st = it & 1;
             // the producer's lse / delta rows of this stage are published together with the tiles
             if (!mbar_wait(in_full + 8 * st, (it >> 1) & 1, abort_flag)) { alive = false; break; }
-            if (!mbar_wait(s_full + 8 * hf, it & 1, abort_flag)) { alive = false; break; }
+            if (!mbar_wait(s_full, it & 1, abort_flag)) { alive = false; break; }
             tc_fence_after();
             const long long q_abs0 = p.q0 + qt0;
             const bool diag = k_abs0 + TILE - 1 > q_abs0;          // the tile pair holds masked (query, key) pairs
             // query column c of the tile is visible to this key iff q_abs0 + c >= k_abs
             const int first_col = (k_abs > q_abs0) ? (int)((k_abs - q_abs0) > TILE ? TILE : (k_abs - q_abs0)) : 0;
             const float *lse2 = s_lse + st * TILE + col_base, *dl = s_delta + st * TILE + col_base;
-            uint32_t rs[32], rp[32], pp[16], ds[16];
-            tmem_ld32(tS_g, rs);
-            tmem_ld32(tP_g, rp);
+            // phase 1: P^T = exp2(S^T * scale - lse), all the dV product needs
+            float pv[32];
+            {
+                uint32_t rs[32], pp[16];
+                tmem_ld32(tS_g, rs);
 #pragma unroll
-            for (int e = 0; e < 32; e += 4) {
-                const float4 l4 = *reinterpret_cast<const float4 *>(lse2 + e);
-                const float4 d4 = *reinterpret_cast<const float4 *>(dl + e);
-                const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, dv[4] = {d4.x, d4.y, d4.z, d4.w};
-                float pv[4], dsv[4];
+                for (int e = 0; e < 32; e += 4) {
+                    const float4 l4 = *reinterpret_cast<const float4 *>(lse2 + e);
+                    const float lv[4] = {l4.x, l4.y, l4.z, l4.w};
 #pragma unroll
-                for (int t = 0; t < 4; t++) {
-                    float x = fmaf(__uint_as_float(rs[e + t]), p.scale_log2, -lv[t]);
-                    if (diag && col_base + e + t < first_col) x = -INFINITY;
-                    pv[t] = fast_exp2(x);
-                    dsv[t] = pv[t] * fmaf(__uint_as_float(rp[e + t]), p.scale, -dv[t]);
+                    for (int t = 0; t < 4; t++) {
+                        float x = fmaf(__uint_as_float(rs[e + t]), p.scale_log2, -lv[t]);
+                        if (diag && col_base + e + t < first_col) x = -INFINITY;
+                        pv[e + t] = fast_exp2(x);
+                    }
+                    pp[e / 2] = pack_bf16(pv[e], pv[e + 1]);
+                    pp[e / 2 + 1] = pack_bf16(pv[e + 2], pv[e + 3]);
                 }
-                pp[e / 2] = pack_bf16(pv[0], pv[1]);
-                pp[e / 2 + 1] = pack_bf16(pv[2], pv[3]);
-                ds[e / 2] = pack_bf16(dsv[0], dsv[1]);
-                ds[e / 2 + 1] = pack_bf16(dsv[2], dsv[3]);
+                tmem_st16(tS_g, pp);
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(p1_full);
             }
-            tmem_st16(tS_g, pp);
-            tmem_st16(tP_g, ds);
-            tmem_wait_st();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(p_full + 8 * hf);
+            // phase 2: dS^T = P^T * (dP^T * scale - delta * scale)
+            if (!mbar_wait(dp_full, it & 1, abort_flag)) { alive = false; break; }
+            tc_fence_after();
+            {
+                uint32_t rp[32], ds[16];
+                tmem_ld32(tP_g, rp);
+#pragma unroll
+                for (int e = 0; e < 32; e += 4) {
+                    const float4 d4 = *reinterpret_cast<const float4 *>(dl + e);
+                    const float dv[4] = {d4.x, d4.y, d4.z, d4.w};
+                    float dsv[4];
+#pragma unroll
+                    for (int t = 0; t < 4; t++) dsv[t] = pv[e + t] * fmaf(__uint_as_float(rp[e + t]), p.scale, -dv[t]);
+                    ds[e / 2] = pack_bf16(dsv[0], dsv[1]);
+                    ds[e / 2 + 1] = pack_bf16(dsv[2], dsv[3]);
+                }
+                tmem_st16(tP_g, ds);
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(p2_full);
+            }
         }
         if (alive && mbar_wait(acc_full, 0, abort_flag)) {
             tc_fence_after();
@@ -570,8 +584,8 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
     const uint32_t sQ = base, sdO = sQ + TILE_BYTES, sK = sdO + TILE_BYTES, sV = sK + 2 * TILE_BYTES;
     uint8_t *aux = smem_raw + (base - raw) + 6 * TILE_BYTES + 4 * TILE * 4;
     const uint32_t bars = smem_u32(aux);
-    const uint32_t q_full = bars, kv_full = bars + 8, kv_empty = bars + 24, s_full = bars + 40, p_full = bars + 56,
-                   acc_full = bars + 72;
+    const uint32_t q_full = bars, kv_full = bars + 8, kv_empty = bars + 24, s_full = bars + 40, dp_full = bars + 48,
+                   s_free = bars + 56, p2_full = bars + 64, acc_full = bars + 72;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux + 80);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(aux + 88);
 
@@ -588,9 +602,11 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
         for (int s = 0; s < 2; s++) {
             mbar_init(kv_full + 8 * s, 1);
             mbar_init(kv_empty + 8 * s, 1);
-            mbar_init(s_full + 8 * s, 1);
-            mbar_init(p_full + 8 * s, 8);
         }
+        mbar_init(s_full, 1);
+        mbar_init(dp_full, 1);
+        mbar_init(s_free, 16);
+        mbar_init(p2_full, 16);
         mbar_init(acc_full, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -600,7 +616,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    // columns: S halves at 0 / 64 (keys 0-63 / 64-127 of the tile), dP halves at 128 / 192, dQ at 256
+    // columns: S at 0, dP at 128, dQ at 256
     const uint32_t tS = tmem, tDP = tmem + 128, tDQ = tmem + 256;
 
     if (warp == 0) {
@@ -623,60 +639,52 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc_half = make_idesc(TILE, HALF, false, false);   // N = 64 keys
-            constexpr uint32_t idesc_acc = make_idesc(TILE, TILE, false, true);     // N = 128 head dims
+            constexpr uint32_t idesc_kk = make_idesc(TILE, TILE, false, false);
+            constexpr uint32_t idesc_acc = make_idesc(TILE, TILE, false, true);
             bool alive = mbar_wait(q_full, 0, abort_flag);
             const uint32_t q_lo = klo(sQ), do_lo = klo(sdO);
-            // S and dP of one 64-key half of tile j
-            auto issue_sdp = [&](int j, int hf) {
-                const uint32_t st = j & 1;
-                const uint32_t kh_lo = klo(sK + st * TILE_BYTES + hf * 8192), vh_lo = klo(sV + st * TILE_BYTES + hf * 8192);
+            auto issue_s = [&](int j) {        // S = Q K^T
+                const uint32_t k_lo = klo(sK + (j & 1) * TILE_BYTES);
 #pragma unroll
-                for (int kk = 0; kk < 8; kk++)
-                    umma_ss(tS + hf * HALF, q_lo + kstep(kk), kh_lo + kstep(kk), idesc_half, kk != 0);
-#pragma unroll
-                for (int kk = 0; kk < 8; kk++)
-                    umma_ss(tDP + hf * HALF, do_lo + kstep(kk), vh_lo + kstep(kk), idesc_half, kk != 0);
-                umma_commit(s_full + 8 * hf);
+                for (int kk = 0; kk < 8; kk++) umma_ss(tS, q_lo + kstep(kk), k_lo + kstep(kk), idesc_kk, kk != 0);
+                umma_commit(s_full);
             };
+            auto issue_dp = [&](int j) {       // dP = dO V^T
+                const uint32_t v_lo = klo(sV + (j & 1) * TILE_BYTES);
+#pragma unroll
+                for (int kk = 0; kk < 8; kk++) umma_ss(tDP, do_lo + kstep(kk), v_lo + kstep(kk), idesc_kk, kk != 0);
+                umma_commit(dp_full);
+            };
+            if (alive) alive = mbar_wait(kv_full, 0, abort_flag);
             if (alive) {
-                alive = mbar_wait(kv_full, 0, abort_flag);
-                if (alive) {
-                    tc_fence_after();
-                    issue_sdp(0, 0);
-                    issue_sdp(0, 1);
-                }
+                tc_fence_after();
+                issue_s(0);
+                issue_dp(0);
             }
             for (int j = 0; j < nkv && alive; j++) {
                 const uint32_t st = j & 1;
+                if (j + 1 < nkv) {
+                    // next tile's S as soon as the softmax warps have read this tile's S into registers
+                    if (!mbar_wait(kv_full + 8 * ((j + 1) & 1), ((j + 1) >> 1) & 1, abort_flag)) { alive = false; break; }
+                    if (!mbar_wait(s_free, j & 1, abort_flag)) { alive = false; break; }
+                    tc_fence_after();
+                    issue_s(j + 1);
+                }
+                if (!mbar_wait(p2_full, j & 1, abort_flag)) { alive = false; break; }
+                tc_fence_after();
                 const uint32_t k_mn = mnlo(sK + st * TILE_BYTES);
 #pragma unroll
-                for (int hf = 0; hf < 2; hf++) {
-                    if (!mbar_wait(p_full + 8 * hf, j & 1, abort_flag)) { alive = false; break; }
-                    tc_fence_after();
-#pragma unroll
-                    for (int kk = 0; kk < 4; kk++)
-                        umma_ts(tDQ, tDP + hf * HALF + (kk >> 1) * 32 + (kk & 1) * 8, k_mn + mnstep(hf * 4 + kk), idesc_acc,
-                                (j | hf | kk) != 0);
-                    if (hf == 1) umma_commit(kv_empty + 8 * st);
-                    if (j + 1 < nkv) {
-                        if (hf == 0) {
-                            if (!mbar_wait(kv_full + 8 * ((j + 1) & 1), ((j + 1) >> 1) & 1, abort_flag)) {
-                                alive = false;
-                                break;
-                            }
-                            tc_fence_after();
-                        }
-                        issue_sdp(j + 1, hf);
-                    }
-                }
+                for (int kk = 0; kk < 8; kk++)
+                    umma_ts(tDQ, tDP + (kk >> 1) * 32 + (kk & 1) * 8, k_mn + mnstep(kk), idesc_acc, (j | kk) != 0);
+                umma_commit(kv_empty + 8 * st);            // K and V of this stage are consumed
+                if (j + 1 < nkv) issue_dp(j + 1);          // the dP columns are free once dQ has read dS (in order)
             }
             if (alive) umma_commit(acc_full);
         }
     } else {
         const int quarter = warp & 3;
         const int wg = (warp - 2) >> 2;                           // 0..3: 32-key group of the tile
-        const int hf = wg >> 1, key_base = wg * 32;
+        const int key_base = wg * 32;
         const int row = quarter * 32 + lane;
         const int qr = qt0 + row;
         const long long q_abs = q_abs0 + row;
@@ -686,31 +694,44 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
         const float neg_delta_s = qr < p.n ? -p.delta[(long long)h * p.n + qr] * p.scale : 0.f;
         bool alive = true;
         for (int j = 0; j < nkv && alive; j++) {
-            if (!mbar_wait(s_full + 8 * hf, j & 1, abort_flag)) { alive = false; break; }
+            if (!mbar_wait(s_full, j & 1, abort_flag)) { alive = false; break; }
             tc_fence_after();
             const long long k_abs0 = (long long)j * TILE;
             const bool diag = k_abs0 + TILE - 1 > q_abs0;
             const int lim = (int)(q_abs - k_abs0);                // keys 0..lim of the tile are visible (diag tiles)
-            uint32_t rs[32], rp[32], ds[16];
-            tmem_ld32(tS_g, rs);
-            tmem_ld32(tP_g, rp);
+            // phase 1: P from S; the S columns are handed back to the tensor pipe right after the load
+            float pv[32];
+            {
+                uint32_t rs[32];
+                tmem_ld32(tS_g, rs);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(s_free);
 #pragma unroll
-            for (int e = 0; e < 32; e += 2) {
-                float x0 = fmaf(__uint_as_float(rs[e]), p.scale_log2, neg_lse2);
-                float x1 = fmaf(__uint_as_float(rs[e + 1]), p.scale_log2, neg_lse2);
-                if (diag) {
-                    if (key_base + e > lim) x0 = -INFINITY;
-                    if (key_base + e + 1 > lim) x1 = -INFINITY;
+                for (int e = 0; e < 32; e++) {
+                    float x = fmaf(__uint_as_float(rs[e]), p.scale_log2, neg_lse2);
+                    if (diag && key_base + e > lim) x = -INFINITY;
+                    pv[e] = fast_exp2(x);
                 }
-                const float d0 = fast_exp2(x0) * fmaf(__uint_as_float(rp[e]), p.scale, neg_delta_s);
-                const float d1 = fast_exp2(x1) * fmaf(__uint_as_float(rp[e + 1]), p.scale, neg_delta_s);
-                ds[e / 2] = pack_bf16(d0, d1);
             }
-            tmem_st16(tP_g, ds);       // front of the group's own fp32 columns
-            tmem_wait_st();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(p_full + 8 * hf);
+            // phase 2: dS = P * (dP * scale - delta * scale), packed in place
+            if (!mbar_wait(dp_full, j & 1, abort_flag)) { alive = false; break; }
+            tc_fence_after();
+            {
+                uint32_t rp[32], ds[16];
+                tmem_ld32(tP_g, rp);
+#pragma unroll
+                for (int e = 0; e < 32; e += 2) {
+                    const float d0 = pv[e] * fmaf(__uint_as_float(rp[e]), p.scale, neg_delta_s);
+                    const float d1 = pv[e + 1] * fmaf(__uint_as_float(rp[e + 1]), p.scale, neg_delta_s);
+                    ds[e / 2] = pack_bf16(d0, d1);
+                }
+                tmem_st16(tP_g, ds);       // front of the group's own fp32 columns
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(p2_full);
+            }
         }
         if (alive && mbar_wait(acc_full, 0, abort_flag)) {
             tc_fence_after();
