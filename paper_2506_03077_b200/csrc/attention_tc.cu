@@ -2,21 +2,19 @@
 // the queries of one chunk against the key/value prefix that ends with the chunk.
 //
 // Forward, one CTA per (128-query tile, query head):
-//   warp 0     : TMA producer -- Q once, then K and V tiles of 128 keys through two-stage rings
-//   warp 1     : MMA issuer   -- S_j = Q K_j^T into one of two tensor-memory buffers (so S_{j+1} is
-//                computed while the softmax of S_j runs), then O += P_j V_j
-//   warps 2..5 : softmax      -- one query row per thread: row max and sum need no shuffles;
-//                P_j is written to shared memory in the swizzled K-major layout the MMA reads;
-//                the running output in tensor memory is rescaled only when a row's maximum
-//                grows by more than 2^8 (exact: the final division by the row sum uses the same
-//                reference), which after the first tiles is rare
+//   warp 0      : TMA producer -- Q once, then K and V tiles of 128 keys through two-stage rings
+//   warp 1      : MMA issuer   -- S_j = Q K_j^T into one of two tensor-memory buffers (so S_{j+1} is
+//                 computed while the softmax of S_j runs), then O += P_j V_j with P_j read from
+//                 tensor memory as the A operand
+//   warps 2..17 : softmax      -- a thread owns 32 key columns of one query row (see the kernel);
+//                 the running output in tensor memory is rescaled only when a row's maximum grows
+//                 by more than 2^8 (exact: the final division by the row sum uses the same
+//                 reference), which after the first tiles is rare
 //   Key tiles beyond the diagonal are never loaded; the causal predicate is evaluated only in
 //   tiles the diagonal crosses.
 //
 // All mbarrier waits are bounded (see sm100.cuh); on expiry the CTA leaves its loops, frees its
 // tensor memory and returns, and the host sees STREAMBP_E_DEVICE_TIMEOUT.
-#include <cstdlib>
-
 #include "sm100.cuh"
 
 namespace sbp {
@@ -45,14 +43,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&h);
 }
-// 16-byte chunk `chunk` (0..15) of row `row` in a two-sub-tile swizzled [128][128] bf16 tile
-__device__ __forceinline__ uint32_t swz_addr(uint32_t tile, int row, int chunk) {
-    return tile + (chunk >> 3) * HALF_BYTES + row * 128 + (((chunk & 7) ^ (row & 7)) << 4);
-}
-__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
-
 struct FwdParams {
     int n;              // query rows in this chunk
     long long q0;       // absolute row of query 0
@@ -62,29 +52,42 @@ struct FwdParams {
     float scale_log2;   // log2(e) / sqrt(head_dim)
 };
 
-constexpr int FWD_SMEM = TILE_BYTES /*Q*/ + 2 * TILE_BYTES /*K*/ + 2 * TILE_BYTES /*V*/ + TILE_BYTES /*P*/ + 1024 + 256;
+// ---------------------------------------------------------------------------------------------
+// Forward with sixteen softmax warps: the 128 key columns of a tile are split over four warpgroups
+// (32 columns per thread), so four warps per scheduler hide the tensor-memory load latency that one
+// warp per scheduler leaves exposed.  The four threads that share a query row exchange their partial
+// row maxima through shared memory (an mbarrier with a bounded wait, not bar.sync, so that a CTA that
+// is giving up cannot dead-lock on it); they then take identical rescale decisions, keep partial row
+// sums that are only combined in the epilogue, and each warpgroup rescales / writes its own 32 head
+// dims of the output.
+// ---------------------------------------------------------------------------------------------
+constexpr int FWD16_THREADS = 64 + 512;
+constexpr int FWD16_SMEM = 5 * TILE_BYTES + 3 * 4 * TILE * 4 /* row max x2, row sum */ + 1024 + 256;
 
-template <bool P_TMEM>
-__global__ void __launch_bounds__(192, 1)
-    attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                       const __grid_constant__ CUtensorMap map_v, const FwdParams p) {
+__global__ void __launch_bounds__(FWD16_THREADS, 1)
+    attn_fwd_tc16_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                         const __grid_constant__ CUtensorMap map_v, const FwdParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
-    const uint32_t sQ = base, sK = sQ + TILE_BYTES, sV = sK + 2 * TILE_BYTES, sP = sV + 2 * TILE_BYTES;
-    uint8_t *aux = smem_raw + (base - raw) + 6 * TILE_BYTES;
+    const uint32_t sQ = base, sK = sQ + TILE_BYTES, sV = sK + 2 * TILE_BYTES;
+    uint8_t *tail = smem_raw + (base - raw) + 5 * TILE_BYTES;
+    float *s_max = reinterpret_cast<float *>(tail);            // [2 buffers][4 groups][128 rows]
+    float *s_sum = s_max + 2 * 4 * TILE;                       // [4 groups][128 rows]
+    uint8_t *aux = tail + 3 * 4 * TILE * 4;
     const uint32_t bars = smem_u32(aux);
     const uint32_t q_full = bars, k_full = bars + 8, k_empty = bars + 24, v_full = bars + 40, v_empty = bars + 56,
-                   s_full = bars + 72, s_empty = bars + 88, p_full = bars + 104, pv_done = bars + 112;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux + 128);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(aux + 136);
+                   s_full = bars + 72, s_empty = bars + 88, p_full = bars + 104, pv_done = bars + 112,
+                   mx_bar = bars + 120, sum_bar = bars + 136;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux + 144);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(aux + 152);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int h = blockIdx.y, g = h / (p.Hq / p.Hkv);
     const int qt0 = blockIdx.x * TILE;
-    const long long q_abs0 = p.q0 + qt0;                                      // absolute row of the tile's first query
+    const long long q_abs0 = p.q0 + qt0;
     const int rows_here = (p.n - qt0) < TILE ? (p.n - qt0) : TILE;
-    const long long kv_end = q_abs0 + rows_here;                              // keys 0 .. kv_end-1 are visible to the tile
+    const long long kv_end = q_abs0 + rows_here;
     const int nkv = (int)((kv_end + TILE - 1) / TILE);
 
     if (threadIdx.x == 0) {
@@ -95,10 +98,12 @@ __global__ void __launch_bounds__(192, 1)
             mbar_init(v_full + 8 * s, 1);
             mbar_init(v_empty + 8 * s, 1);
             mbar_init(s_full + 8 * s, 1);
-            mbar_init(s_empty + 8 * s, 4);
+            mbar_init(s_empty + 8 * s, 16);
+            mbar_init(mx_bar + 8 * s, 16);
         }
-        mbar_init(p_full, 4);
+        mbar_init(p_full, 16);
         mbar_init(pv_done, 1);
+        mbar_init(sum_bar, 16);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -107,8 +112,7 @@ __global__ void __launch_bounds__(192, 1)
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    const uint32_t tS = tmem, tO = tmem + 256;     // S buffers at columns 0 and 128, O at 256
-    const uint32_t tP = tmem + 384;                // P as packed bf16 pairs (64 columns) when P_TMEM
+    const uint32_t tS = tmem, tO = tmem + 256, tP = tmem + 384;   // S x2, O, packed P (64 columns)
 
     if (warp == 0) {
         if (lane == 0) {
@@ -132,16 +136,15 @@ __global__ void __launch_bounds__(192, 1)
             constexpr uint32_t idesc_s = make_idesc(TILE, TILE, false, false);
             constexpr uint32_t idesc_pv = make_idesc(TILE, TILE, false, true);
             bool alive = mbar_wait(q_full, 0, abort_flag);
+            const uint32_t q_lo = klo(sQ);
             auto issue_s = [&](int j) -> bool {
                 const uint32_t st = j & 1, ph = (j >> 1) & 1;
                 if (!mbar_wait(s_empty + 8 * st, ph ^ 1u, abort_flag)) return false;
                 if (!mbar_wait(k_full + 8 * st, ph, abort_flag)) return false;
                 tc_fence_after();
+                const uint32_t k_lo = klo(sK + st * TILE_BYTES);
 #pragma unroll
-                const uint32_t q_lo = klo(sQ), k_lo = klo(sK + st * TILE_BYTES);
-#pragma unroll
-                for (int kk = 0; kk < 8; kk++)
-                    umma_ss(tS + st * TILE, q_lo + kstep(kk), k_lo + kstep(kk), idesc_s, kk != 0);
+                for (int kk = 0; kk < 8; kk++) umma_ss(tS + st * TILE, q_lo + kstep(kk), k_lo + kstep(kk), idesc_s, kk != 0);
                 umma_commit(k_empty + 8 * st);
                 umma_commit(s_full + 8 * st);
                 return true;
@@ -153,136 +156,112 @@ __global__ void __launch_bounds__(192, 1)
                 if (!mbar_wait(p_full, j & 1, abort_flag)) { alive = false; break; }
                 if (!mbar_wait(v_full + 8 * st, ph, abort_flag)) { alive = false; break; }
                 tc_fence_after();
-                const uint32_t v_lo = mnlo(sV + st * TILE_BYTES), p_lo = klo(sP);
+                const uint32_t v_lo = mnlo(sV + st * TILE_BYTES);
 #pragma unroll
-                for (int kk = 0; kk < 8; kk++) {
-                    if (P_TMEM)
-                        umma_ts(tO, tP + kk * 8, v_lo + mnstep(kk), idesc_pv, (j | kk) != 0);
-                    else
-                        umma_ss(tO, p_lo + kstep(kk), v_lo + mnstep(kk), idesc_pv, (j | kk) != 0);
-                }
+                for (int kk = 0; kk < 8; kk++) umma_ts(tO, tP + kk * 8, v_lo + mnstep(kk), idesc_pv, (j | kk) != 0);
                 umma_commit(v_empty + 8 * st);
                 umma_commit(pv_done);
             }
         }
     } else {
         const int quarter = warp & 3;
-        const int row = quarter * 32 + lane;                     // query row within the tile
+        const int wg = (warp - 2) >> 2;                          // key-column group 0..3 (and head-dim group in O)
+        const int col_base = wg * 32;
+        const int row = quarter * 32 + lane;
         const long long q_abs = q_abs0 + row;
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-        float m_used = -INFINITY, l = 0.f;
+        float m_used = -INFINITY, l = 0.f;                       // l: partial row sum over this thread's columns
         bool alive = true;
         for (int j = 0; j < nkv && alive; j++) {
             const uint32_t st = j & 1, ph = (j >> 1) & 1;
             if (!mbar_wait(s_full + 8 * st, ph, abort_flag)) { alive = false; break; }
             tc_fence_after();
-            const uint32_t tSj = tS + st * TILE + lane_base;
             const long long k_abs0 = (long long)j * TILE;
-            const bool diag = k_abs0 + TILE - 1 > q_abs0;       // some (query, key) pair of the tile is masked
-            const int lim = diag ? (int)(q_abs - k_abs0) : (1 << 30);   // keys 0..lim of the tile are visible
-            // pass 1: row maximum of the raw scores (the scale is positive, so it commutes with max)
+            const bool diag = k_abs0 + TILE - 1 > q_abs0;
+            const int lim = (int)(q_abs - k_abs0);                // keys 0..lim of the tile are visible (diag tiles)
+            uint32_t r[32];
+            tmem_ld32(tS + st * TILE + col_base + lane_base, r);
+            // S buffer may be overwritten by S_{j+2}
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(s_empty + 8 * st);
             float mt = -INFINITY;
-#pragma unroll 1
-            for (int c = 0; c < 4; c++) {
-                uint32_t r[32];
-                tmem_ld32(tSj + c * 32, r);
-                if (diag) {
+            if (diag) {
 #pragma unroll
-                    for (int e = 0; e < 32; e++) mt = fmaxf(mt, c * 32 + e > lim ? -INFINITY : __uint_as_float(r[e]));
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 32; e++) mt = fmaxf(mt, __uint_as_float(r[e]));
+                for (int e = 0; e < 32; e++) {
+                    if (col_base + e > lim) r[e] = 0xff800000u;   // -inf
+                    mt = fmaxf(mt, __uint_as_float(r[e]));
                 }
+            } else {
+#pragma unroll
+                for (int e = 0; e < 32; e++) mt = fmaxf(mt, __uint_as_float(r[e]));
             }
-            mt *= p.scale_log2;
+            // exchange partial maxima with the three other threads of this row
+            s_max[(st * 4 + wg) * TILE + row] = mt;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(mx_bar + 8 * st);
+            if (!mbar_wait(mx_bar + 8 * st, ph, abort_flag)) { alive = false; break; }
+            const float *mx = s_max + st * 4 * TILE + row;
+            mt = fmaxf(fmaxf(mx[0], mx[TILE]), fmaxf(mx[2 * TILE], mx[3 * TILE])) * p.scale_log2;
             float factor = 1.f;
-            const bool grow = mt > m_used + 8.f;                 // also true on the first tile (m_used = -inf)
+            const bool grow = mt > m_used + 8.f;                  // also true on the first tile (m_used = -inf)
             if (grow) {
                 factor = fast_exp2(m_used - mt);
                 m_used = mt;
                 l *= factor;
             }
-            // pass 2: P = exp2(s * scale - m_used), packed to bf16
-            uint32_t pk[64];
+            uint32_t pk[16];
             const float neg_m = -m_used;
 #pragma unroll
-            for (int c = 0; c < 4; c++) {
-                uint32_t r[32];
-                tmem_ld32(tSj + c * 32, r);
-#pragma unroll
-                for (int e = 0; e < 32; e += 2) {
-                    float x0 = fmaf(__uint_as_float(r[e]), p.scale_log2, neg_m);
-                    float x1 = fmaf(__uint_as_float(r[e + 1]), p.scale_log2, neg_m);
-                    if (diag) {
-                        if (c * 32 + e > lim) x0 = -INFINITY;
-                        if (c * 32 + e + 1 > lim) x1 = -INFINITY;
-                    }
-                    const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
-                    l += p0 + p1;
-                    pk[c * 16 + e / 2] = pack_bf16(p0, p1);
-                }
+            for (int e = 0; e < 32; e += 2) {
+                const float p0 = fast_exp2(fmaf(__uint_as_float(r[e]), p.scale_log2, neg_m));
+                const float p1 = fast_exp2(fmaf(__uint_as_float(r[e + 1]), p.scale_log2, neg_m));
+                l += p0 + p1;
+                pk[e / 2] = pack_bf16(p0, p1);
             }
-            // S buffer may be overwritten by S_{j+2}
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(s_empty + 8 * st);
             // P buffer and O are free once P_{j-1} V_{j-1} has completed
             if (j > 0) {
                 if (!mbar_wait(pv_done, (j - 1) & 1, abort_flag)) { alive = false; break; }
                 tc_fence_after();
-                if (__any_sync(0xffffffffu, grow)) {
-#pragma unroll 1
-                    for (int c = 0; c < 4; c++) {
-                        uint32_t r[32];
-                        tmem_ld32(tO + lane_base + c * 32, r);
+                if (__any_sync(0xffffffffu, grow)) {              // this warpgroup rescales head dims col_base .. +31
+                    uint32_t o[32];
+                    tmem_ld32(tO + lane_base + col_base, o);
 #pragma unroll
-                        for (int e = 0; e < 32; e++) r[e] = __float_as_uint(__uint_as_float(r[e]) * factor);
-                        tmem_st32(tO + lane_base + c * 32, r);
-                    }
-                    tmem_wait_st();
+                    for (int e = 0; e < 32; e++) o[e] = __float_as_uint(__uint_as_float(o[e]) * factor);
+                    tmem_st32(tO + lane_base + col_base, o);
                 }
             }
-            if (P_TMEM) {
-#pragma unroll
-                for (int c = 0; c < 2; c++) {
-                    uint32_t r[32];
-#pragma unroll
-                    for (int e = 0; e < 32; e++) r[e] = pk[c * 32 + e];
-                    tmem_st32(tP + lane_base + c * 32, r);
-                }
-                tmem_wait_st();
-            } else {
-#pragma unroll
-                for (int cc = 0; cc < 16; cc++)
-                    st_shared_v4(swz_addr(sP, row, cc), pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            }
+            tmem_st16(tP + lane_base + wg * 16, pk);
+            tmem_wait_st();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(p_full);
         }
-        // epilogue: O / l and the log-sum-exp
-        if (alive && mbar_wait(pv_done, (nkv - 1) & 1, abort_flag)) {
-            tc_fence_after();
-            const float inv = 1.f / l;
-            const int qr = qt0 + row;
-#pragma unroll 1
-            for (int c = 0; c < 4; c++) {
-                uint32_t r[32];
-                tmem_ld32(tO + lane_base + c * 32, r);
+        // epilogue: combine the four partial row sums, then O / l and the log-sum-exp
+        if (alive) {
+            s_sum[wg * TILE + row] = l;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(sum_bar);
+            if (mbar_wait(sum_bar, 0, abort_flag) && mbar_wait(pv_done, (nkv - 1) & 1, abort_flag)) {
+                tc_fence_after();
+                const float lt = s_sum[row] + s_sum[TILE + row] + s_sum[2 * TILE + row] + s_sum[3 * TILE + row];
+                const float inv = 1.f / lt;
+                const int qr = qt0 + row;
+                uint32_t o[32];
+                tmem_ld32(tO + lane_base + col_base, o);
                 if (qr < p.n) {
-                    bf16 *out = p.o + ((long long)qr * p.Hq + h) * TILE + c * 32;
+                    bf16 *out = p.o + ((long long)qr * p.Hq + h) * TILE + col_base;
 #pragma unroll
                     for (int e = 0; e < 32; e += 8) {
                         uint32_t w[4];
 #pragma unroll
                         for (int t = 0; t < 4; t++)
-                            w[t] = pack_bf16(__uint_as_float(r[e + 2 * t]) * inv, __uint_as_float(r[e + 2 * t + 1]) * inv);
+                            w[t] = pack_bf16(__uint_as_float(o[e + 2 * t]) * inv, __uint_as_float(o[e + 2 * t + 1]) * inv);
                         *reinterpret_cast<uint4 *>(out + e) = make_uint4(w[0], w[1], w[2], w[3]);
                     }
+                    if (wg == 0) p.lse[(long long)h * p.n + qr] = (m_used + log2f(lt)) * kLn2;
                 }
             }
-            if (qr < p.n) p.lse[(long long)h * p.n + qr] = (m_used + log2f(l)) * kLn2;
         }
     }
 
@@ -298,7 +277,6 @@ __global__ void __launch_bounds__(192, 1)
         tmem_dealloc(tmem, 512);
     }
 }
-
 
 // ---------------------------------------------------------------------------------------------
 // Backward.  Two kernels, both deterministic (no floating-point atomics):
@@ -775,7 +753,6 @@ bool attention_tc_supported(int64_t n, int64_t q0, int Hq, int Hkv, int dh, cons
 
 int attention_fwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, int64_t n, int64_t q0, int Hq, int Hkv, bf16 *o,
                      float *lse, cudaStream_t st) {
-    static const bool p_smem = std::getenv("STREAMBP_ATTN_P_SMEM") != nullptr;
     CUtensorMap mq, mk, mv;
     const int64_t kv_len = q0 + n;
     if (!make_tensor_map(&mq, q, n, (int64_t)Hq * TILE, (int64_t)Hq * TILE, 64, TILE, false) ||
@@ -784,16 +761,12 @@ int attention_fwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, int64_t n, int
         return STREAMBP_E_CUDA;
     static bool configured = false;
     if (!configured) {
-        if (!opt_in_smem(attn_fwd_tc_kernel<true>, FWD_SMEM) || !opt_in_smem(attn_fwd_tc_kernel<false>, FWD_SMEM))
-            return STREAMBP_E_CUDA;
+        if (!opt_in_smem(attn_fwd_tc16_kernel, FWD16_SMEM)) return STREAMBP_E_CUDA;
         configured = true;
     }
     FwdParams p{(int)n, (long long)q0, Hq, Hkv, o, lse, kLog2e / sqrtf((float)TILE)};
     dim3 grid((unsigned)((n + TILE - 1) / TILE), Hq);
-    if (p_smem)
-        SBP_LAUNCH(attn_fwd_tc_kernel<false>, grid, 192, FWD_SMEM, st, mq, mk, mv, p);
-    else
-        SBP_LAUNCH(attn_fwd_tc_kernel<true>, grid, 192, FWD_SMEM, st, mq, mk, mv, p);
+    SBP_LAUNCH(attn_fwd_tc16_kernel, grid, FWD16_THREADS, FWD16_SMEM, st, mq, mk, mv, p);
     return STREAMBP_OK;
 }
 
