@@ -190,6 +190,9 @@ def run_head_or_model(args, cfg):
         ws = B.alloc_workspace(ws_bytes)
         step = lambda: B.lmhead_ce_backward(hc, gd, Wd, Hd, ld, cfg.chunk, loss, nv, dH, dW, dg, ws)
         flops, name = head_flops(h, T), "streamed_lmhead_ce_backward_tokens_per_s"
+        # chunks whose labels are all ignored are skipped on the device (their gradient is exactly zero)
+        live_chunks = sum(1 for r0 in range(0, T, cfg.chunk) if (labels[r0:r0 + cfg.chunk] != h.ignore_index).any())
+        executed_flops = head_flops(h, min(T, live_chunks * cfg.chunk))
     else:
         s, L = cfg.layer, cfg.n_layers
         lc = B.LayerConfig(s.d_model, s.n_q_heads, s.n_kv_heads, s.head_dim, s.d_ff, s.qkv_bias, s.rope_theta, s.rms_eps, dt)
@@ -210,6 +213,7 @@ def run_head_or_model(args, cfg):
         P = s.d_model * s.dq + 2 * s.d_model * s.dkv + s.dq * s.d_model + 3 * s.d_model * s.d_ff
         fwd_extra = 2 * T * P + 4 * s.head_dim * s.n_q_heads * T * (T + 1) / 2      # checkpointing forward
         flops = L * (layer_flops(s, T) + fwd_extra) + head_flops(h, T)
+        executed_flops = flops
         name = "streamed_model_backward_tokens_per_s"
     for _ in range(args.warmup):
         step()
@@ -239,6 +243,9 @@ def run_head_or_model(args, cfg):
                    "l2": "inputs larger than L2"},
         "algorithmic_tflop_per_step": flops / 1e12, "tflops": flops / (ms * 1e-3) / 1e12,
         "frac_of_measured_sustained_bf16": flops / (ms * 1e-3) / 1e12 / peaks["sustained"],
+        "executed_tflop_per_step": executed_flops / 1e12,
+        "tflops_executed": executed_flops / (ms * 1e-3) / 1e12,
+        "frac_of_measured_sustained_bf16_executed": executed_flops / (ms * 1e-3) / 1e12 / peaks["sustained"],
         "peak_activation_gb": ws_bytes / 1e9, "peak_activation_gb_unchunked": ws_full / 1e9,
         "gpu_launches": int(launches * args.steps),
         "roofline": {"bound": "tensor", "kernel": "linear products", "achieved": achieved, "peak": peaks["sustained"],

@@ -15,6 +15,10 @@ typedef __nv_bfloat16 bf16;
 struct CallState {
     int cuda_error = 0;
     int64_t launches = 0;
+    // Optional device-side gate for the launches that follow: kernels that honour it return at once
+    // (or write exact zeros, where an output must still be defined) when *gate == 0.  Used by the LM
+    // head to skip chunks whose labels are all ignored without a host round trip.
+    const int *gate = nullptr;
 };
 CallState &call_state();
 
@@ -51,6 +55,8 @@ struct ProfScope {
     ProfScope(int cls, double flops, cudaStream_t stream);
     ~ProfScope();
 };
+
+__device__ __forceinline__ bool gated_off(const int *gate) { return gate != nullptr && *gate == 0; }
 
 // ---- scalar conversion -------------------------------------------------------
 __device__ __forceinline__ float to_f32(float v) { return v; }
@@ -265,6 +271,9 @@ int attn_bwd(const T *q, const T *k, const T *v, const T *o, const T *dout, cons
 // LM head pieces
 int count_valid_labels(const int64_t *labels, int64_t T, int64_t vocab, int64_t ignore, WsHeader *hdr,
                        cudaStream_t st);
+// counts[i] = number of labels != ignore in rows [i*chunk, min(T, (i+1)*chunk))
+int count_valid_per_chunk(const int64_t *labels, int64_t T, int64_t chunk, int64_t ignore, int *counts,
+                          cudaStream_t st);
 // z: [rows, V] fp32 logits -> dz (storage dtype; may alias z when T == float); row_loss[rows] fp32.
 template <typename T>
 int ce_rows(const float *z, const int64_t *labels, int64_t rows, int64_t V, int64_t ignore, const WsHeader *hdr,

@@ -12,8 +12,9 @@ template <typename T>
 __global__ void __launch_bounds__(256) rmsnorm_fwd_kernel(const T *__restrict__ x, const float *__restrict__ res,
                                                           const T *__restrict__ gain, float eps, int d,
                                                           T *__restrict__ h, float *__restrict__ rstd_out,
-                                                          float *__restrict__ r_out) {
+                                                          float *__restrict__ r_out, const int *gate) {
     __shared__ float red[33];
+    if (gated_off(gate)) return;
     const int64_t row = blockIdx.x;
     const T *xr = x + row * d;
     constexpr int N = Vec<T>::N;
@@ -58,7 +59,8 @@ template <typename T>
 int rmsnorm_fwd(const T *x, const float *res, const T *gain, float eps, int64_t rows, int d, T *h, float *rstd,
                 float *r_out, cudaStream_t st) {
     if (rows <= 0) return STREAMBP_OK;
-    SBP_LAUNCH(rmsnorm_fwd_kernel<T>, (unsigned)rows, 256, 0, st, x, res, gain, eps, d, h, rstd, r_out);
+    SBP_LAUNCH(rmsnorm_fwd_kernel<T>, (unsigned)rows, 256, 0, st, x, res, gain, eps, d, h, rstd, r_out,
+               call_state().gate);
     return STREAMBP_OK;
 }
 template int rmsnorm_fwd<float>(const float *, const float *, const float *, float, int64_t, int, float *, float *,
@@ -74,9 +76,16 @@ __global__ void __launch_bounds__(256)
     rmsnorm_bwd_rows_kernel(const float *__restrict__ dh, const T *__restrict__ xT, const float *__restrict__ xF,
                             const float *__restrict__ rstd_in, const T *__restrict__ gain,
                             const T *__restrict__ addT, const float *__restrict__ addF, int d,
-                            float *__restrict__ outF, T *__restrict__ outT) {
+                            float *__restrict__ outF, T *__restrict__ outT, const int *gate) {
     __shared__ float red[33];
     const int64_t row = blockIdx.x;
+    if (gated_off(gate)) {   // the upstream gradient of this block of rows is exactly zero
+        for (int c = threadIdx.x; c < d; c += blockDim.x) {
+            if (outF) outF[row * d + c] = 0.f;
+            if (outT) outT[row * d + c] = from_f32<T>(0.f);
+        }
+        return;
+    }
     const float rstd = rstd_in[row];
     float dot = 0.f;
     for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
@@ -116,9 +125,9 @@ template <typename T>
 __global__ void __launch_bounds__(256)
     rmsnorm_dgain_partial_kernel(const float *__restrict__ dh, const T *__restrict__ xT, const float *__restrict__ xF,
                                  const float *__restrict__ rstd, int64_t rows, int d, int rows_per_split,
-                                 float *__restrict__ partial) {
+                                 float *__restrict__ partial, const int *gate) {
     const int col = blockIdx.x * 256 + threadIdx.x;
-    if (col >= d) return;
+    if (col >= d || gated_off(gate)) return;
     const int64_t r0 = (int64_t)blockIdx.y * rows_per_split;
     const int64_t r1 = min(rows, r0 + (int64_t)rows_per_split);
     float acc = 0.f;
@@ -131,9 +140,9 @@ __global__ void __launch_bounds__(256)
 
 __global__ void __launch_bounds__(256)
     partial_reduce_kernel(const float *__restrict__ partial, int nsplit, int cols, float *__restrict__ out,
-                          int accumulate) {
+                          int accumulate, const int *gate) {
     const int col = blockIdx.x * 256 + threadIdx.x;
-    if (col >= cols) return;
+    if (col >= cols || gated_off(gate)) return;
     float acc = 0.f;
     for (int s = 0; s < nsplit; s++) acc += partial[(int64_t)s * cols + col];
     out[col] = accumulate ? out[col] + acc : acc;
@@ -151,14 +160,15 @@ int rmsnorm_bwd(const float *dh, const T *xT, const float *xF, const float *rstd
                 const float *addF, int64_t rows, int d, float *outF, T *outT, float *dgain, float *partials,
                 cudaStream_t st) {
     if (rows <= 0) return STREAMBP_OK;
+    const int *gate = call_state().gate;
     SBP_LAUNCH(rmsnorm_bwd_rows_kernel<T>, (unsigned)rows, 256, 0, st, dh, xT, xF, rstd, gain, addT, addF, d, outF,
-               outT);
+               outT, gate);
     if (dgain) {
         const int ns = split_count(rows);
         const int rps = (int)((rows + ns - 1) / ns);
         dim3 grid((d + 255) / 256, ns);
-        SBP_LAUNCH(rmsnorm_dgain_partial_kernel<T>, grid, 256, 0, st, dh, xT, xF, rstd, rows, d, rps, partials);
-        SBP_LAUNCH(partial_reduce_kernel, (d + 255) / 256, 256, 0, st, partials, ns, d, dgain, 1);
+        SBP_LAUNCH(rmsnorm_dgain_partial_kernel<T>, grid, 256, 0, st, dh, xT, xF, rstd, rows, d, rps, partials, gate);
+        SBP_LAUNCH(partial_reduce_kernel, (d + 255) / 256, 256, 0, st, partials, ns, d, dgain, 1, gate);
     }
     return STREAMBP_OK;
 }
@@ -191,7 +201,8 @@ int colsum(const T *a, int64_t rows, int cols, float *out, bool accumulate, floa
     const int rps = (int)((rows + ns - 1) / ns);
     dim3 grid((cols + 255) / 256, ns);
     SBP_LAUNCH(colsum_partial_kernel<T>, grid, 256, 0, st, a, rows, cols, rps, partials);
-    SBP_LAUNCH(partial_reduce_kernel, (cols + 255) / 256, 256, 0, st, partials, ns, cols, out, accumulate ? 1 : 0);
+    SBP_LAUNCH(partial_reduce_kernel, (cols + 255) / 256, 256, 0, st, partials, ns, cols, out, accumulate ? 1 : 0,
+               (const int *)nullptr);
     return STREAMBP_OK;
 }
 template int colsum<float>(const float *, int64_t, int, float *, bool, float *, cudaStream_t);
@@ -400,13 +411,34 @@ int count_valid_labels(const int64_t *labels, int64_t T_, int64_t vocab, int64_t
     return STREAMBP_OK;
 }
 
+__global__ void __launch_bounds__(256)
+    count_chunk_labels_kernel(const int64_t *__restrict__ labels, int64_t T_, int64_t chunk, int64_t ignore,
+                              int *__restrict__ counts) {
+    __shared__ int cnt;
+    if (threadIdx.x == 0) cnt = 0;
+    __syncthreads();
+    const int64_t r0 = (int64_t)blockIdx.x * chunk, r1 = min(T_, r0 + chunk);
+    int mine = 0;
+    for (int64_t t = r0 + threadIdx.x; t < r1; t += blockDim.x) mine += labels[t] != ignore ? 1 : 0;
+    atomicAdd(&cnt, mine);
+    __syncthreads();
+    if (threadIdx.x == 0) counts[blockIdx.x] = cnt;
+}
+int count_valid_per_chunk(const int64_t *labels, int64_t T_, int64_t chunk, int64_t ignore, int *counts,
+                          cudaStream_t st) {
+    const int64_t D = (T_ + chunk - 1) / chunk;
+    SBP_LAUNCH(count_chunk_labels_kernel, (unsigned)D, 256, 0, st, labels, T_, chunk, ignore, counts);
+    return STREAMBP_OK;
+}
+
 // one block per logits row: online (max, sum-exp), then dz = (softmax - onehot) / N
 template <typename T>
 __global__ void __launch_bounds__(1024)
     ce_rows_kernel(const float *z, const int64_t *__restrict__ labels, int64_t V, int64_t ignore,
-                   const WsHeader *__restrict__ hdr, T *dz, float *__restrict__ row_loss) {
+                   const WsHeader *__restrict__ hdr, T *dz, float *__restrict__ row_loss, const int *gate) {
     __shared__ float red[33];
     __shared__ float zy_s;
+    if (gated_off(gate)) return;
     const int64_t row = blockIdx.x;
     const float *zr = z + row * V;
     T *dr = dz + row * V;
@@ -473,7 +505,7 @@ template <typename T>
 int ce_rows(const float *z, const int64_t *labels, int64_t rows, int64_t V, int64_t ignore, const WsHeader *hdr,
             T *dz, float *row_loss, cudaStream_t st) {
     if (rows <= 0) return STREAMBP_OK;
-    SBP_LAUNCH(ce_rows_kernel<T>, (unsigned)rows, 1024, 0, st, z, labels, V, ignore, hdr, dz, row_loss);
+    SBP_LAUNCH(ce_rows_kernel<T>, (unsigned)rows, 1024, 0, st, z, labels, V, ignore, hdr, dz, row_loss, call_state().gate);
     return STREAMBP_OK;
 }
 template int ce_rows<float>(const float *, const int64_t *, int64_t, int64_t, int64_t, const WsHeader *, float *,
@@ -482,8 +514,9 @@ template int ce_rows<bf16>(const float *, const int64_t *, int64_t, int64_t, int
                            float *, cudaStream_t);
 
 __global__ void __launch_bounds__(1024) loss_accumulate_kernel(const float *__restrict__ row_loss, int64_t rows,
-                                                               WsHeader *hdr) {
+                                                               WsHeader *hdr, const int *gate) {
     __shared__ double red[32];
+    if (gated_off(gate)) return;
     double acc = 0.0;
     for (int64_t r = threadIdx.x; r < rows; r += blockDim.x) acc += (double)row_loss[r];
 #pragma unroll
@@ -498,7 +531,7 @@ __global__ void __launch_bounds__(1024) loss_accumulate_kernel(const float *__re
 }
 int loss_accumulate(const float *row_loss, int64_t rows, WsHeader *hdr, cudaStream_t st) {
     if (rows <= 0) return STREAMBP_OK;
-    SBP_LAUNCH(loss_accumulate_kernel, 1, 1024, 0, st, row_loss, rows, hdr);
+    SBP_LAUNCH(loss_accumulate_kernel, 1, 1024, 0, st, row_loss, rows, hdr, call_state().gate);
     return STREAMBP_OK;
 }
 

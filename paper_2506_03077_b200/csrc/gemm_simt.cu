@@ -14,8 +14,9 @@ template <typename TI, typename TC, bool A_KCONTIG, bool B_KCONTIG>
 __global__ void __launch_bounds__(256)
     gemm_simt_kernel(int64_t M, int64_t N, int64_t K, const TI *__restrict__ A, int64_t sam, int64_t sak,
                      const TI *__restrict__ B, int64_t sbk, int64_t sbn, TC *C, int64_t ldc,
-                     const TI *__restrict__ bias, int accumulate) {
+                     const TI *__restrict__ bias, int accumulate, const int *gate) {
     __shared__ __align__(16) float As[BK][LDS];
+    if (gated_off(gate)) return;
     __shared__ __align__(16) float Bs[BK][LDS];
     const int tid = threadIdx.x;
     const int tx = tid & 15, ty = tid >> 4;
@@ -78,15 +79,15 @@ int gemm(GemmOp op, int64_t M, int64_t N, int64_t K, const TI *A, int64_t lda, c
     switch (op) {
         case OP_NT:
             SBP_LAUNCH((gemm_simt_kernel<TI, TC, true, true>), grid, 256, 0, st, M, N, K, A, lda, (int64_t)1, B,
-                       (int64_t)1, ldb, C, ldc, bias, acc);
+                       (int64_t)1, ldb, C, ldc, bias, acc, call_state().gate);
             break;
         case OP_NN:
             SBP_LAUNCH((gemm_simt_kernel<TI, TC, true, false>), grid, 256, 0, st, M, N, K, A, lda, (int64_t)1, B, ldb,
-                       (int64_t)1, C, ldc, bias, acc);
+                       (int64_t)1, C, ldc, bias, acc, call_state().gate);
             break;
         case OP_TN:
             SBP_LAUNCH((gemm_simt_kernel<TI, TC, false, false>), grid, 256, 0, st, M, N, K, A, (int64_t)1, lda, B, ldb,
-                       (int64_t)1, C, ldc, bias, acc);
+                       (int64_t)1, C, ldc, bias, acc, call_state().gate);
             break;
     }
     return STREAMBP_OK;

@@ -98,6 +98,7 @@ struct TcParams {
     long long ldc;
     const bf16 *bias;
     int accumulate;
+    const int *gate;      // optional: the kernel returns at once when *gate == 0
 };
 
 template <bool A_MN, bool B_MN, bool OUT_F32>
@@ -105,6 +106,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
     gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                    const __grid_constant__ CUtensorMap map_c, const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
+    if (gated_off(p.gate)) return;
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;          // 1024-byte aligned operand stages
     const uint32_t epi = tiles + STAGES * STAGE_BYTES;      // fp32 staging blocks, 1024-byte aligned
@@ -343,7 +345,7 @@ int gemm_tc(GemmOp op, int64_t M, int64_t N, int64_t K, const bf16 *A, int64_t l
     CUtensorMap mc = ma;   // unused by the bf16-output kernels
     if (ok && c_is_f32) ok = make_tensor_map(&mc, C, M, N, ldc, 32, 32, true);
     if (!ok) return STREAMBP_E_CUDA;
-    TcParams p{(int)M, (int)N, (int)K, C, (long long)ldc, bias, accumulate ? 1 : 0};
+    TcParams p{(int)M, (int)N, (int)K, C, (long long)ldc, bias, accumulate ? 1 : 0, call_state().gate};
     if (op == OP_NT) return c_is_f32 ? launch<false, false, true>(ma, mb, mc, p, st) : launch<false, false, false>(ma, mb, mc, p, st);
     if (op == OP_NN) return c_is_f32 ? launch<false, true, true>(ma, mb, mc, p, st) : launch<false, true, false>(ma, mb, mc, p, st);
     return c_is_f32 ? launch<true, true, true>(ma, mb, mc, p, st) : launch<true, true, false>(ma, mb, mc, p, st);

@@ -10,6 +10,7 @@ struct HeadWs {
     WsHeader *hdr;
     T *hn, *dz;
     float *z, *dhn, *rstd, *row_loss, *partials;
+    int *chunk_valid;     // [number of chunks] unmasked labels per chunk: the device-side gate of each chunk
     size_t bytes;
 };
 
@@ -28,6 +29,7 @@ HeadWs<T> plan(const streambp_head_cfg &c, int64_t T_, int64_t chunk, void *base
     w.rstd = a.take<float>(cn);
     w.row_loss = a.take<float>(cn);
     w.partials = a.take<float>(64 * d);
+    w.chunk_valid = a.take<int>((T_ + cn - 1) / cn);
     w.bytes = a.size();
     return w;
 }
@@ -48,13 +50,24 @@ int lmhead_backward(const streambp_head_cfg &c, const T *g_final, const T *w_voc
     const int64_t V = c.vocab;
     // N is global: it is counted before the chunk loop so that every chunk scales by the same 1/N
     SBP_TRY(count_valid_labels(labels, T_, V, c.ignore_index, s.hdr, st));
-    if (!accumulate) SBP_TRY(fill_zero(d_g_final, sizeof(float) * d, st));
+    SBP_TRY(count_valid_per_chunk(labels, T_, cn, c.ignore_index, s.chunk_valid, st));
+    if (!accumulate) {
+        // chunks whose labels are all ignored are skipped on the device (their dlogits are exactly zero),
+        // so no particular chunk can be relied on to overwrite the outputs: clear them and always add
+        SBP_TRY(fill_zero(d_g_final, sizeof(float) * d, st));
+        SBP_TRY(fill_zero(d_w_vocab, sizeof(float) * (size_t)V * d, st));
+    }
     const int64_t D = (T_ + cn - 1) / cn;
+    struct GateScope {      // every launch of a chunk is gated by that chunk's count of unmasked labels
+        explicit GateScope(const int *g) { call_state().gate = g; }
+        ~GateScope() { call_state().gate = nullptr; }
+    };
     for (int64_t i = 0; i < D; i++) {
         const int64_t r0 = i * cn;
         const int64_t n = (T_ - r0 < cn) ? T_ - r0 : cn;
-        const bool acc = accumulate || i != 0;
+        const bool acc = true;
         const T *Hi = H + r0 * d;
+        GateScope gate(s.chunk_valid + i);
         SBP_TRY(rmsnorm_fwd<T>(Hi, nullptr, g_final, c.rms_eps, n, d, s.hn, s.rstd, nullptr, st));
         SBP_TRY((mm<T, float>(OP_NT, n, V, d, s.hn, d, w_vocab, d, s.z, V, nullptr, false, st)));           // logits
         SBP_TRY(ce_rows<T>(s.z, labels + r0, n, V, c.ignore_index, s.hdr, s.dz, s.row_loss, st));

@@ -106,3 +106,24 @@ def test_head_accumulate():
     run_head(hs, g, W, H, labels, 16, torch.float32, accumulate=True, prior=prior)
     assert O.rel_frobenius(prior[0].cpu().numpy(), 2 * dW.cpu().numpy()) < 1e-6
     assert O.rel_frobenius(prior[1].cpu().numpy(), 2 * dg.cpu().numpy()) < 1e-6
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_fully_masked_chunks_are_skipped_exactly(dtype):
+    """Chunks whose labels are all ignored are gated off on the device; the result must still be the
+    oracle's, with exactly-zero dH rows there, also when the first chunk is one of them."""
+    hs = synth.HeadShape(128, 1536)
+    T, chunk = 256, 64
+    g, W, H, labels = synth.make_head_inputs(hs, 21, T, dtype == torch.bfloat16, 0)
+    labels[0:64] = -100        # chunk 0
+    labels[128:192] = -100     # chunk 2
+    labels[200] = -100         # a single ignored row inside a live chunk
+    ref = O.lmhead_ce_backward(O.HeadCfg(128, 1536), g, W, H, labels)
+    loss, nv, dH, dW, dg, st = run_head(hs, g, W, H, labels, chunk, dtype)
+    assert st == B.OK and int(nv.item()) == ref[1] == 127
+    assert abs(loss.item() - ref[0]) <= (1e-5 if dtype == torch.float32 else 2e-3) * abs(ref[0])
+    assert_close("dH", dH, ref[2], TOL[dtype])
+    assert_close("dW", dW, ref[3], TOL[dtype])
+    assert_close("dg", dg, ref[4], TOL[dtype])
+    for rows in (slice(0, 64), slice(128, 192), slice(200, 201)):
+        assert torch.count_nonzero(dH[rows]) == 0

@@ -84,3 +84,26 @@ def test_small_model_with_embedding(dtype):
     for l in range(L):
         for k, v in ref["layers"][l].items():
             assert_close(f"layer{l}.{k}", Gd[l][k], v, tol)
+
+
+def test_error_growth_through_28_layers_bf16():
+    """Depth of the full model configuration (28 layers) at small widths: the bf16 path must stay inside
+    the tolerance although every layer boundary rounds activations and gradients to bf16."""
+    ls = synth.LayerShape(256, 4, 2, 128, 688, True, 1e6)
+    hs = synth.HeadShape(256, 2048)
+    T, L = 384, 28
+    layers = [synth.make_layer_weights(ls, 31, True, prefix=f"layer{l}") for l in range(L)]
+    E = synth.round_bf16(synth.normal(31, "embed", (hs.vocab, ls.d_model), 0.0, 1.0))
+    g = synth.round_bf16(synth.normal(31, "g_final", (ls.d_model,), 1.0, 0.02))
+    Wv = synth.round_bf16(synth.normal(31, "w_vocab", (hs.vocab, ls.d_model), 0.0, 0.02))
+    ids, labels = synth.make_model_tokens(hs.vocab, 31, T, 0.1)
+    loss, Gd, dg, dWv, dX0, dE = run_model(ls, hs, layers, g, Wv, labels, 128, 128, torch.bfloat16, E=E, ids=ids)
+    ref = O.model_backward(O.LayerCfg(ls.d_model, ls.n_q_heads, ls.n_kv_heads, ls.head_dim, ls.d_ff, ls.qkv_bias,
+                                      ls.rope_theta, ls.rms_eps),
+                           O.HeadCfg(hs.d_model, hs.vocab), layers, g, Wv, labels, embed=E, ids=ids)
+    tol = TOL[torch.bfloat16]
+    assert_close("d_embed", dE, ref["d_embed"], tol)
+    assert_close("d_w_vocab", dWv, ref["w_vocab"], tol)
+    for l in (0, 13, 27):
+        for k, v in ref["layers"][l].items():
+            assert_close(f"layer{l}.{k}", Gd[l][k], v, tol)
