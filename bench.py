@@ -36,7 +36,7 @@ def layer_flops(s, T):
 
 
 # DRAM bytes (read + write) of one representative launch of the dominant kernel, from the ncu capture
-# summarised in profiles/gemm_tc_kernel_qwen7b_chunk1024.md (the per-chunk product dh2 += du Wu:
+# summarised in profiles/gemm_tc_kernel_chunk_products.md (the per-chunk product dh2 += du Wu:
 # M 1024, N 3584, K 18944; algorithmic bytes 189.3e6).  Launch shapes depend on the chunk, not on T.
 NCU_TRAFFIC_BYTES = {("qwen7b_layer", 1024): 192.9e6}
 
