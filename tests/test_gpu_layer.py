@@ -85,3 +85,17 @@ def test_layer_bf16_matches_oracle(shape, T, chunk):
     # chunk invariance in bf16 within the same tolerance
     dX2, grads2 = run_layer(bcfg, W, X, dY, T)
     compare_layer(ocfg, W, X, dY, dX2, grads2, TOL[torch.bfloat16])
+
+
+def test_layer_bf16_long_prefix_small_width():
+    """Few query tiles against a long prefix: the attention kernels split their key range into pieces
+    (merged in a fixed order) to fill the SMs; results must match the oracle and stay bit-reproducible."""
+    shape = synth.LayerShape(256, 2, 1, 128, 688, True, 1e6)
+    T, chunk = 4096 + 200, 512
+    ocfg, bcfg, W, X, dY = layer_case(shape, 12, T, torch.bfloat16)
+    dX, grads = run_layer(bcfg, W, X, dY, chunk)
+    compare_layer(ocfg, W, X, dY, dX, grads, TOL[torch.bfloat16])
+    dX2, grads2 = run_layer(bcfg, W, X, dY, chunk)
+    assert torch.equal(dX, dX2)
+    for k in grads:
+        assert torch.equal(grads[k], grads2[k]), k
