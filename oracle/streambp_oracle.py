@@ -11,7 +11,8 @@ full-sequence forward and backward of
     Sec. 3.2.2 with the normalisation, heads and residuals the paper leaves out
     "without loss of generality" put back in the usual Llama/Qwen form;
   * the final RMSNorm + language-modelling head + mean cross-entropy over the
-    unmasked tokens (Sec. 3.2.1, SFT objective, Eq. (2));
+    unmasked tokens (Sec. 3.2.1, SFT objective, Eq. (2)), and the same head under
+    the GRPO (Eq. (4)) and DPO (Eq. (5)) objectives;
   * a stack of such layers between an embedding lookup and that head.
 
 Everything is numpy float64.  `numpy.matmul`, `exp`, `log`, `cos`, `sin` are the
@@ -317,6 +318,112 @@ def lmhead_ce_backward(cfg: HeadCfg, g_final, w_vocab, H, labels, row_block=512)
         dH[t0:t1], dgi = rmsnorm_backward(dhn, xhat, rms, g_final)
         dg += dgi
     return total / N, N, dH, dW, dg
+
+
+# ---------------------------------------------------------------------------
+# LM head under the RL objectives of Sec. 3.2.1 (GRPO Eq. (4), DPO Eq. (5)).
+# Both depend on the logits only through log pi_theta(t) = z_t[o_t] - logsumexp(z_t) of the given
+# token o_t, so the gradient wrt the logits of row t is c_t * (e_{o_t} - softmax(z_t)) with a
+# per-token coefficient c_t = dL / dlog pi_theta(t).  Rows whose token equals ignore_index do not
+# take part.
+# ---------------------------------------------------------------------------
+
+def _token_logprobs(cfg: HeadCfg, g_final, w_vocab, H, tokens, row_block):
+    """log softmax(RMSNorm(H) W^T)[t, tokens[t]] for rows that take part (0 elsewhere)."""
+    T = H.shape[0]
+    part = tokens != cfg.ignore_index
+    logp = np.zeros(T)
+    for t0 in range(0, T, row_block):
+        t1 = min(T, t0 + row_block)
+        hn, _, _ = rmsnorm_forward(H[t0:t1], g_final, cfg.rms_eps)
+        z = hn @ w_vocab.T
+        zmax = z.max(axis=-1, keepdims=True)
+        lse = zmax[:, 0] + np.log(np.exp(z - zmax).sum(axis=-1))
+        idx = np.nonzero(part[t0:t1])[0]
+        logp[t0 + idx] = z[idx, tokens[t0:t1][idx]] - lse[idx]
+    return logp
+
+
+def _backprop_token_coefficients(cfg: HeadCfg, g_final, w_vocab, H, tokens, coef, row_block):
+    """Given c_t = dL/dlog pi(t), returns (dH, dW_vocab, dg_final): dz_t = c_t (e_{o_t} - softmax(z_t))."""
+    T = H.shape[0]
+    part = tokens != cfg.ignore_index
+    dH, dW, dg = np.zeros_like(H), np.zeros_like(w_vocab), np.zeros_like(g_final)
+    for t0 in range(0, T, row_block):
+        t1 = min(T, t0 + row_block)
+        hn, xhat, rms = rmsnorm_forward(H[t0:t1], g_final, cfg.rms_eps)
+        z = hn @ w_vocab.T
+        z = z - z.max(axis=-1, keepdims=True)
+        p = np.exp(z)
+        p /= p.sum(axis=-1, keepdims=True)
+        dz = -p
+        idx = np.nonzero(part[t0:t1])[0]
+        dz[idx, tokens[t0:t1][idx]] += 1.0
+        dz *= np.where(part[t0:t1], coef[t0:t1], 0.0)[:, None]
+        dW += dz.T @ hn
+        dH[t0:t1], dgi = rmsnorm_backward(dz @ w_vocab, xhat, rms, g_final)
+        dg += dgi
+    return dH, dW, dg
+
+
+def grpo_token_terms(logp, logp_old, logp_ref, advantage, beta, clip_eps):
+    """f(t) of Eq. (4) and df/dlog pi_theta(t):
+    f = min(r A, clip(r, 1-eps, 1+eps) A) - beta (log pi_theta - log pi_ref), r = pi_theta / pi_old."""
+    r = np.exp(logp - logp_old)
+    unclipped = r * advantage
+    clipped = np.clip(r, 1.0 - clip_eps, 1.0 + clip_eps) * advantage
+    f = np.minimum(unclipped, clipped) - beta * (logp - logp_ref)
+    # d(r A)/dlog pi = r A; the clipped branch is constant in log pi wherever the clip is active
+    inside = (r > 1.0 - clip_eps) & (r < 1.0 + clip_eps)
+    takes_unclipped = unclipped <= clipped
+    df = np.where(takes_unclipped | inside, unclipped, 0.0) - beta
+    return f, df
+
+
+def lmhead_grpo_forward(cfg: HeadCfg, g_final, w_vocab, H, tokens, logp_old, logp_ref, advantage, weight,
+                        beta, clip_eps, row_block=512):
+    """L = - sum_t weight_t f(t); weight_t carries the 1/(G T_o) of Eq. (4)."""
+    g_final, w_vocab, H = _f64(g_final), _f64(w_vocab), _f64(H)
+    tokens = np.asarray(tokens, dtype=np.int64)
+    part = tokens != cfg.ignore_index
+    logp = _token_logprobs(cfg, g_final, w_vocab, H, tokens, row_block)
+    f, _ = grpo_token_terms(logp, _f64(logp_old), _f64(logp_ref), _f64(advantage), beta, clip_eps)
+    return float(-np.sum(np.where(part, _f64(weight) * f, 0.0)))
+
+
+def lmhead_grpo_backward(cfg: HeadCfg, g_final, w_vocab, H, tokens, logp_old, logp_ref, advantage, weight,
+                         beta, clip_eps, row_block=512):
+    """Returns (loss, logp, dH, dW_vocab, dg_final) for the GRPO objective."""
+    g_final, w_vocab, H = _f64(g_final), _f64(w_vocab), _f64(H)
+    tokens = np.asarray(tokens, dtype=np.int64)
+    part = tokens != cfg.ignore_index
+    logp = _token_logprobs(cfg, g_final, w_vocab, H, tokens, row_block)
+    f, df = grpo_token_terms(logp, _f64(logp_old), _f64(logp_ref), _f64(advantage), beta, clip_eps)
+    w = _f64(weight)
+    loss = float(-np.sum(np.where(part, w * f, 0.0)))
+    dH, dW, dg = _backprop_token_coefficients(cfg, g_final, w_vocab, H, tokens, -w * df, row_block)
+    return loss, logp, dH, dW, dg
+
+
+def lmhead_dpo_forward(cfg: HeadCfg, g_final, w_vocab, H, tokens, logp_ref, sign, beta, row_block=512):
+    """L = -log sigmoid(beta * ell), ell = sum_t sign_t (log pi_theta(t) - log pi_ref(t)) with sign +1 on the
+    chosen response's tokens and -1 on the rejected one's (Eq. (5))."""
+    g_final, w_vocab, H = _f64(g_final), _f64(w_vocab), _f64(H)
+    tokens = np.asarray(tokens, dtype=np.int64)
+    part = tokens != cfg.ignore_index
+    logp = _token_logprobs(cfg, g_final, w_vocab, H, tokens, row_block)
+    ell = float(np.sum(np.where(part, _f64(sign) * (logp - _f64(logp_ref)), 0.0)))
+    return float(np.log1p(np.exp(-beta * ell))), ell
+
+
+def lmhead_dpo_backward(cfg: HeadCfg, g_final, w_vocab, H, tokens, logp_ref, sign, beta, row_block=512):
+    """Returns (loss, ell, dH, dW_vocab, dg_final): dL/dlog pi(t) = (sigmoid(beta ell) - 1) beta sign_t (Eq. (6))."""
+    g_final, w_vocab, H = _f64(g_final), _f64(w_vocab), _f64(H)
+    tokens = np.asarray(tokens, dtype=np.int64)
+    loss, ell = lmhead_dpo_forward(cfg, g_final, w_vocab, H, tokens, logp_ref, sign, beta, row_block)
+    factor = 1.0 / (1.0 + np.exp(-beta * ell)) - 1.0
+    dH, dW, dg = _backprop_token_coefficients(cfg, g_final, w_vocab, H, tokens, factor * beta * _f64(sign), row_block)
+    return loss, ell, dH, dW, dg
 
 
 # ---------------------------------------------------------------------------
