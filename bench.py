@@ -190,6 +190,24 @@ def run_head_or_model(args, cfg):
         ws = B.alloc_workspace(ws_bytes)
         step = lambda: B.lmhead_ce_backward(hc, gd, Wd, Hd, ld, cfg.chunk, loss, nv, dH, dW, dg, ws)
         flops, name = head_flops(h, T), "streamed_lmhead_ce_backward_tokens_per_s"
+        if args.objective != "sft":
+            # synthetic per-token inputs of the RL objectives: behaviour / reference log-probabilities around the
+            # ln V of a random-init policy, unit-variance advantages, uniform weights (GRPO) or +-1 signs (DPO)
+            n_part = int((labels != h.ignore_index).sum())
+            lp0 = -float(__import__("math").log(h.vocab))
+            old = torch.from_numpy(synth.normal(cfg.seed, "logp_old", (T,), lp0, 0.3)).cuda()
+            ref = torch.from_numpy(synth.normal(cfg.seed, "logp_ref", (T,), lp0, 0.3)).cuda()
+            adv = torch.from_numpy(synth.normal(cfg.seed, "advantage", (T,))).cuda()
+            if args.objective == "grpo":
+                wt = torch.full((T,), 1.0 / n_part, device="cuda")
+                obj, beta, eps = B.OBJ_GRPO, 0.04, 0.2
+            else:
+                half = (T + cfg.masked_prefix) // 2
+                wt = torch.where(torch.arange(T, device="cuda") < half, 1.0, -1.0).float()
+                obj, beta, eps = B.OBJ_DPO, 0.1, 0.0
+            step = lambda: B.lmhead_rl_backward(hc, obj, beta, eps, gd, Wd, Hd, ld, old, ref, adv, wt, cfg.chunk, loss,
+                                                dH, dW, dg, ws)
+            name = f"streamed_lmhead_{args.objective}_backward_tokens_per_s"
         # chunks whose labels are all ignored are skipped on the device (their gradient is exactly zero)
         live_chunks = sum(1 for r0 in range(0, T, cfg.chunk) if (labels[r0:r0 + cfg.chunk] != h.ignore_index).any())
         executed_flops = head_flops(h, min(T, live_chunks * cfg.chunk))
@@ -265,6 +283,8 @@ def main():
     ap.add_argument("--config", default="qwen7b_layer",
                     choices=["qwen7b_layer", "llama8b_layer", "qwen7b_head", "qwen7b_model"])
     ap.add_argument("--layers", type=int, default=0, help="override the layer count of the model configuration")
+    ap.add_argument("--objective", default="sft", choices=["sft", "grpo", "dpo"],
+                    help="objective of the qwen7b_head workload (Sec. 3.2.1)")
     ap.add_argument("--chunk", type=int, default=0)
     ap.add_argument("--T", type=int, default=0, help="override the sequence length (profiling on small cases)")
     ap.add_argument("--ref-tokens", type=int, default=512)

@@ -134,6 +134,41 @@ int streambp_lmhead_ce_backward(const streambp_head_cfg *cfg, const void *g_fina
                                 float *d_w_vocab, float *d_g_final,
                                 void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/*
+ * The same streamed head under the reinforcement-learning objectives of Sec. 3.2.1.  Both depend on the
+ * logits only through log pi_theta(t) = logits[t, token_t] - logsumexp(logits[t, :]), so each chunk's
+ * dlogits are c_t * (onehot(token_t) - softmax(logits[t, :])) with a per-token coefficient c_t, and the
+ * chunk loop, the two gradient products and the norm backward are those of the SFT head.
+ *
+ *   STREAMBP_OBJ_GRPO (Eq. (4)):  L = - sum_t weight_t f(t),
+ *       f(t) = min(r_t A_t, clip(r_t, 1-clip_eps, 1+clip_eps) A_t) - beta (log pi_theta(t) - logp_ref[t]),
+ *       r_t = exp(log pi_theta(t) - logp_old[t]).  weight_t carries the 1/(G T_o) of the objective
+ *       (any per-token weighting is allowed); advantage[t] = A_t.
+ *   STREAMBP_OBJ_DPO (Eq. (5)):   L = - log sigmoid(beta * ell),
+ *       ell = sum_t weight_t (log pi_theta(t) - logp_ref[t]) with weight_t = +1 on the chosen response's
+ *       tokens and -1 on the rejected one's.  As in the paper, ell and the un-corrected gradients
+ *       beta * sum_t d ell(t) are accumulated over the chunks and the outputs are then multiplied in place
+ *       by (sigmoid(beta ell) - 1); because of that in-place correction `accumulate` must be 0.
+ *
+ * tokens [T] int64 (ignore_index: the row takes no part); logp_old, logp_ref, advantage, weight: fp32 [T]
+ * device arrays (logp_old and advantage are not read for DPO).  Outputs: *loss; logp [T] fp32 (optional,
+ * log pi_theta of the given tokens, 0 on rows that take no part); *ell (optional, DPO); dH, d_w_vocab,
+ * d_g_final as in streambp_lmhead_ce_backward.  Workspace: streambp_lmhead_workspace_bytes().
+ */
+typedef enum { STREAMBP_OBJ_GRPO = 1, STREAMBP_OBJ_DPO = 2 } streambp_objective;
+typedef struct {
+    int32_t objective;   /* streambp_objective */
+    float beta;
+    float clip_eps;      /* GRPO only */
+} streambp_rl_cfg;
+
+int streambp_lmhead_rl_backward(const streambp_head_cfg *cfg, const streambp_rl_cfg *rl, const void *g_final,
+                                const void *w_vocab, const void *H, const int64_t *tokens, const float *logp_old,
+                                const float *logp_ref, const float *advantage, const float *weight, int64_t T,
+                                int64_t chunk, int accumulate, float *loss, float *logp, float *ell, void *dH,
+                                float *d_w_vocab, float *d_g_final, void *workspace, size_t workspace_bytes,
+                                void *cuda_stream);
+
 typedef struct {
     int32_t n_layers;
     streambp_layer_cfg layer;

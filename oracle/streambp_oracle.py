@@ -366,17 +366,31 @@ def _backprop_token_coefficients(cfg: HeadCfg, g_final, w_vocab, H, tokens, coef
     return dH, dW, dg
 
 
-def grpo_token_terms(logp, logp_old, logp_ref, advantage, beta, clip_eps):
+def grpo_token_terms(logp, logp_old, logp_ref, advantage, beta, clip_eps, branch_logp=None):
     """f(t) of Eq. (4) and df/dlog pi_theta(t):
-    f = min(r A, clip(r, 1-eps, 1+eps) A) - beta (log pi_theta - log pi_ref), r = pi_theta / pi_old."""
+    f = min(r A, clip(r, 1-eps, 1+eps) A) - beta (log pi_theta - log pi_ref), r = pi_theta / pi_old.
+
+    The min / clip is a branch decided by a floating-point comparison.  `branch_logp` (float32 log pi_theta
+    values, e.g. those a lower-precision implementation reports) lets a comparison take that decision from
+    the same numbers, in float32, as the implementation under test; the values of f and df are always
+    computed from `logp` in float64."""
     r = np.exp(logp - logp_old)
     unclipped = r * advantage
     clipped = np.clip(r, 1.0 - clip_eps, 1.0 + clip_eps) * advantage
-    f = np.minimum(unclipped, clipped) - beta * (logp - logp_ref)
+    if branch_logp is None:
+        inside = (r > 1.0 - clip_eps) & (r < 1.0 + clip_eps)
+        takes_unclipped = unclipped <= clipped
+    else:
+        f32 = np.float32
+        rb = np.exp(np.asarray(branch_logp, f32) - np.asarray(logp_old, f32))
+        adv32 = np.asarray(advantage, f32)
+        lo, hi = f32(1.0) - f32(clip_eps), f32(1.0) + f32(clip_eps)
+        inside = (rb > lo) & (rb < hi)
+        takes_unclipped = rb * adv32 <= np.minimum(np.maximum(rb, lo), hi) * adv32
     # d(r A)/dlog pi = r A; the clipped branch is constant in log pi wherever the clip is active
-    inside = (r > 1.0 - clip_eps) & (r < 1.0 + clip_eps)
-    takes_unclipped = unclipped <= clipped
-    df = np.where(takes_unclipped | inside, unclipped, 0.0) - beta
+    keeps = takes_unclipped | inside
+    f = np.where(keeps, unclipped, clipped) - beta * (logp - logp_ref)
+    df = np.where(keeps, unclipped, 0.0) - beta
     return f, df
 
 
@@ -392,13 +406,13 @@ def lmhead_grpo_forward(cfg: HeadCfg, g_final, w_vocab, H, tokens, logp_old, log
 
 
 def lmhead_grpo_backward(cfg: HeadCfg, g_final, w_vocab, H, tokens, logp_old, logp_ref, advantage, weight,
-                         beta, clip_eps, row_block=512):
+                         beta, clip_eps, row_block=512, branch_logp=None):
     """Returns (loss, logp, dH, dW_vocab, dg_final) for the GRPO objective."""
     g_final, w_vocab, H = _f64(g_final), _f64(w_vocab), _f64(H)
     tokens = np.asarray(tokens, dtype=np.int64)
     part = tokens != cfg.ignore_index
     logp = _token_logprobs(cfg, g_final, w_vocab, H, tokens, row_block)
-    f, df = grpo_token_terms(logp, _f64(logp_old), _f64(logp_ref), _f64(advantage), beta, clip_eps)
+    f, df = grpo_token_terms(logp, _f64(logp_old), _f64(logp_ref), _f64(advantage), beta, clip_eps, branch_logp)
     w = _f64(weight)
     loss = float(-np.sum(np.where(part, w * f, 0.0)))
     dH, dW, dg = _backprop_token_coefficients(cfg, g_final, w_vocab, H, tokens, -w * df, row_block)

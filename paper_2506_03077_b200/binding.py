@@ -32,6 +32,7 @@ EXPORTS = (
     "streambp_last_cuda_error", "streambp_last_launch_count", "streambp_gemm",
     "streambp_profile_enable", "streambp_profile_read",
     "streambp_attention_forward", "streambp_attention_backward", "streambp_attention_backward_static",
+    "streambp_lmhead_rl_backward",
 )
 
 
@@ -48,6 +49,10 @@ class LayerPtrsC(C.Structure):
 class HeadCfgC(C.Structure):
     _fields_ = [("d_model", C.c_int32), ("vocab", C.c_int64), ("rms_eps", C.c_float),
                 ("ignore_index", C.c_int64), ("dtype", C.c_int32)]
+
+
+class RlCfgC(C.Structure):
+    _fields_ = [("objective", C.c_int32), ("beta", C.c_float), ("clip_eps", C.c_float)]
 
 
 class ModelCfgC(C.Structure):
@@ -84,6 +89,9 @@ def lib() -> C.CDLL:
     L.streambp_lmhead_ce_backward.restype = C.c_int
     L.streambp_lmhead_ce_backward.argtypes = [C.POINTER(HeadCfgC), vp, vp, vp, vp, i64, i64, C.c_int, vp, vp, vp, vp,
                                               vp, vp, sz, vp]
+    L.streambp_lmhead_rl_backward.restype = C.c_int
+    L.streambp_lmhead_rl_backward.argtypes = [C.POINTER(HeadCfgC), C.POINTER(RlCfgC), vp, vp, vp, vp, vp, vp, vp, vp,
+                                              i64, i64, C.c_int, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     L.streambp_model_workspace_bytes.restype = sz
     L.streambp_model_workspace_bytes.argtypes = [C.POINTER(ModelCfgC), i64, i64, i64]
     L.streambp_model_backward.restype = C.c_int
@@ -343,4 +351,23 @@ def attention_backward_static(q, k, v, o, d_o, lse, q0: int, dq, dk, dv, engine:
                                                   engine, _stream_ptr(stream))
     if check:
         _check(st, "streambp_attention_backward_static")
+    return st
+
+
+OBJ_GRPO, OBJ_DPO = 1, 2
+
+
+def lmhead_rl_backward(cfg: HeadConfig, objective: int, beta: float, clip_eps: float, g_final, w_vocab, H, tokens,
+                       logp_old, logp_ref, advantage, weight, chunk: int, loss, dH, d_w_vocab, d_g_final, workspace,
+                       logp=None, ell=None, accumulate: bool = False, stream=None, check: bool = True) -> int:
+    """streambp_lmhead_rl_backward (GRPO / DPO objectives of the streamed LM head)."""
+    c = cfg.c()
+    rl = RlCfgC(objective, beta, clip_eps)
+    st = lib().streambp_lmhead_rl_backward(C.byref(c), C.byref(rl), _ptr(g_final), _ptr(w_vocab), _ptr(H),
+                                           _ptr(tokens), _ptr(logp_old), _ptr(logp_ref), _ptr(advantage),
+                                           _ptr(weight), H.shape[0], chunk, 1 if accumulate else 0, _ptr(loss),
+                                           _ptr(logp), _ptr(ell), _ptr(dH), _ptr(d_w_vocab), _ptr(d_g_final),
+                                           _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+    if check:
+        _check(st, "streambp_lmhead_rl_backward")
     return st

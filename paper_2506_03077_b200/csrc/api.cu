@@ -241,6 +241,38 @@ int streambp_lmhead_ce_backward(const streambp_head_cfg *cfg, const void *g_fina
                                  accumulate != 0, loss, n_valid, (bf16 *)dH, d_w_vocab, d_g_final, workspace, st);
 }
 
+int streambp_lmhead_rl_backward(const streambp_head_cfg *cfg, const streambp_rl_cfg *rl, const void *g_final,
+                                const void *w_vocab, const void *H, const int64_t *tokens, const float *logp_old,
+                                const float *logp_ref, const float *advantage, const float *weight, int64_t T,
+                                int64_t chunk, int accumulate, float *loss, float *logp, float *ell, void *dH,
+                                float *d_w_vocab, float *d_g_final, void *workspace, size_t workspace_bytes,
+                                void *cuda_stream) {
+    SBP_TRY(check_head_cfg(cfg));
+    if (!rl) return STREAMBP_E_NULL;
+    if (rl->objective != STREAMBP_OBJ_GRPO && rl->objective != STREAMBP_OBJ_DPO) return STREAMBP_E_SHAPE;
+    if (T < 1 || chunk < 1 || !(rl->beta >= 0.f)) return STREAMBP_E_SHAPE;
+    if (rl->objective == STREAMBP_OBJ_GRPO && !(rl->clip_eps >= 0.f && rl->clip_eps < 1.f)) return STREAMBP_E_SHAPE;
+    if (rl->objective == STREAMBP_OBJ_DPO && accumulate) return STREAMBP_E_SHAPE;   // in-place correction at the end
+    if (!g_final || !w_vocab || !H || !tokens || !logp_ref || !weight || !loss || !dH || !d_w_vocab || !d_g_final ||
+        !workspace)
+        return STREAMBP_E_NULL;
+    if (rl->objective == STREAMBP_OBJ_GRPO && (!logp_old || !advantage)) return STREAMBP_E_NULL;
+    if (!aligned(g_final, 16) || !aligned(w_vocab, 16) || !aligned(H, 16) || !aligned(dH, 16) ||
+        !aligned(d_w_vocab, 16) || !aligned(d_g_final, 16) || !aligned(tokens, 8) || !aligned(workspace, 256))
+        return STREAMBP_E_ALIGN;
+    if (workspace_bytes < streambp_lmhead_workspace_bytes(cfg, T, chunk)) return STREAMBP_E_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    SBP_TRY(begin_call(workspace, st));
+    const RlRows rows{rl->objective, rl->beta, rl->clip_eps, logp_old, logp_ref, advantage, weight, logp};
+    if (cfg->dtype == STREAMBP_F32)
+        return lmhead_backward<float>(*cfg, (const float *)g_final, (const float *)w_vocab, (const float *)H, tokens, T,
+                                      chunk, accumulate != 0, loss, nullptr, (float *)dH, d_w_vocab, d_g_final,
+                                      workspace, st, &rows, ell);
+    return lmhead_backward<bf16>(*cfg, (const bf16 *)g_final, (const bf16 *)w_vocab, (const bf16 *)H, tokens, T, chunk,
+                                 accumulate != 0, loss, nullptr, (bf16 *)dH, d_w_vocab, d_g_final, workspace, st, &rows,
+                                 ell);
+}
+
 static int check_model_cfg(const streambp_model_cfg *cfg) {
     if (!cfg) return STREAMBP_E_NULL;
     SBP_TRY(check_layer_cfg(&cfg->layer));

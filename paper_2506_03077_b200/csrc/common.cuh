@@ -150,6 +150,7 @@ struct WsHeader {
     int32_t detail;
     unsigned long long n_valid;
     double loss_sum;
+    float factor;       // DPO: sigmoid(beta * ell) - 1, the in-place correction applied after the chunk loop
 };
 static constexpr size_t kHeaderBytes = 256;
 
@@ -279,6 +280,24 @@ template <typename T>
 int ce_rows(const float *z, const int64_t *labels, int64_t rows, int64_t V, int64_t ignore, const WsHeader *hdr,
             T *dz, float *row_loss, cudaStream_t st);
 int loss_accumulate(const float *row_loss, int64_t rows, WsHeader *hdr, cudaStream_t st);
+// RL objectives of the LM head: per row, log pi(token) from the logits, then dz = c * (onehot - softmax) with the
+// objective's coefficient c.  row_val: the row's contribution to the loss (GRPO) or to ell (DPO).
+struct RlRows {
+    int objective;            // STREAMBP_OBJ_GRPO / STREAMBP_OBJ_DPO
+    float beta, clip_eps;
+    const float *logp_old;    // GRPO
+    const float *logp_ref;
+    const float *advantage;   // GRPO
+    const float *weight;      // GRPO: per-token weight; DPO: +1 chosen / -1 rejected
+    float *logp_out;          // optional
+};
+template <typename T>
+int rl_rows(const float *z, const int64_t *tokens, int64_t rows, int64_t V, int64_t ignore, const RlRows &rl,
+            int64_t row0, T *dz, float *row_val, cudaStream_t st);
+int rl_finalize(WsHeader *hdr, int objective, float beta, float *loss, float *ell, cudaStream_t st);
+// p[i] *= hdr->factor
+template <typename T>
+int scale_by_factor(T *p, int64_t n, const WsHeader *hdr, cudaStream_t st);
 int loss_finalize(WsHeader *hdr, float *loss, int64_t *n_valid, cudaStream_t st);
 
 template <typename T>
@@ -302,10 +321,12 @@ int layer_forward(const streambp_layer_cfg &c, const streambp_layer_weights &w, 
 
 template <typename T>
 size_t lmhead_workspace(const streambp_head_cfg &c, int64_t T_, int64_t chunk);
+// rl == nullptr: SFT cross-entropy (labels = targets); else the RL objective described by *rl (labels = the
+// sampled tokens, rl->logp_* etc. indexed by absolute row), `ell` optional (DPO).
 template <typename T>
 int lmhead_backward(const streambp_head_cfg &c, const T *g_final, const T *w_vocab, const T *H, const int64_t *labels,
                     int64_t T_, int64_t chunk, bool accumulate, float *loss, int64_t *n_valid, T *dH, float *d_w_vocab,
-                    float *d_g_final, void *ws, cudaStream_t st);
+                    float *d_g_final, void *ws, cudaStream_t st, const RlRows *rl = nullptr, float *ell = nullptr);
 
 template <typename T>
 size_t model_workspace(const streambp_model_cfg &c, int64_t T_, int64_t chunk_layer, int64_t chunk_head);

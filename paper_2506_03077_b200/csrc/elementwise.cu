@@ -513,6 +513,152 @@ template int ce_rows<float>(const float *, const int64_t *, int64_t, int64_t, in
 template int ce_rows<bf16>(const float *, const int64_t *, int64_t, int64_t, int64_t, const WsHeader *, bf16 *,
                            float *, cudaStream_t);
 
+// RL objectives: one block per logits row
+template <typename T>
+__global__ void __launch_bounds__(1024)
+    rl_rows_kernel(const float *z, const int64_t *__restrict__ tokens, int64_t V, int64_t ignore, RlRows rl, int64_t row0,
+                   T *dz, float *__restrict__ row_val, const int *gate) {
+    __shared__ float red[33];
+    __shared__ float zy_s;
+    if (gated_off(gate)) return;
+    const int64_t row = blockIdx.x, arow = row0 + row;
+    const float *zr = z + row * V;
+    T *dr = dz + row * V;
+    const int64_t y = tokens[row];
+    const bool part = (y != ignore) && y >= 0 && y < V;
+    const bool vec = (V & 3) == 0;
+    if (!part) {
+        for (int64_t c = threadIdx.x; c < V; c += blockDim.x) dr[c] = from_f32<T>(0.f);
+        if (threadIdx.x == 0) {
+            row_val[row] = 0.f;
+            if (rl.logp_out) rl.logp_out[arow] = 0.f;
+        }
+        return;
+    }
+    float m = -INFINITY, s = 0.f;
+    for (int64_t c = threadIdx.x * 4; c < V; c += blockDim.x * 4) {
+        float v[4];
+        if (vec && c + 3 < V) {
+            const float4 a = *reinterpret_cast<const float4 *>(zr + c);
+            v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+        } else {
+            for (int k = 0; k < 4; k++) v[k] = (c + k < V) ? zr[c + k] : -INFINITY;
+        }
+        const float mx = fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3]));
+        if (mx > m) {
+            s *= __expf(m - mx);
+            m = mx;
+        }
+        s += __expf(v[0] - m) + __expf(v[1] - m) + __expf(v[2] - m) + __expf(v[3] - m);
+    }
+    const float gm = block_max(m, red);
+    s = (m == -INFINITY) ? 0.f : s * __expf(m - gm);
+    const float gs = block_sum(s, red);
+    if (threadIdx.x == 0) zy_s = zr[y];
+    __syncthreads();
+    const float lse = gm + logf(gs);
+    const float logp = zy_s - lse;
+    // coefficient c = dL / dlog pi(token) (DPO: before the final sigmoid correction)
+    float coef, val;
+    if (rl.objective == STREAMBP_OBJ_GRPO) {
+        const float w = rl.weight[arow], adv = rl.advantage[arow];
+        const float r = expf(logp - rl.logp_old[arow]);
+        const float lo = 1.f - rl.clip_eps, hi = 1.f + rl.clip_eps;
+        const float unclipped = r * adv, clipped = fminf(fmaxf(r, lo), hi) * adv;
+        const bool keeps = (unclipped <= clipped) || (r > lo && r < hi);   // gradient flows through r A
+        const float kl = rl.beta * (logp - rl.logp_ref[arow]);
+        val = -w * ((keeps ? unclipped : clipped) - kl);
+        coef = -w * ((keeps ? unclipped : 0.f) - rl.beta);
+    } else {
+        const float sgn = rl.weight[arow];
+        val = sgn * (logp - rl.logp_ref[arow]);
+        coef = rl.beta * sgn;
+    }
+    if (threadIdx.x == 0) {
+        row_val[row] = val;
+        if (rl.logp_out) rl.logp_out[arow] = logp;
+    }
+    for (int64_t c = threadIdx.x * 4; c < V; c += blockDim.x * 4) {
+        float v[4];
+        if (vec && c + 3 < V) {
+            const float4 a = *reinterpret_cast<const float4 *>(zr + c);
+            v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+        } else {
+            for (int k = 0; k < 4; k++) v[k] = (c + k < V) ? zr[c + k] : -INFINITY;
+        }
+#pragma unroll
+        for (int k = 0; k < 4; k++) {
+            if (c + k < V) {
+                float pr = -__expf(v[k] - lse);
+                if (c + k == y) pr += 1.f;
+                dr[c + k] = from_f32<T>(coef * pr);
+            }
+        }
+    }
+}
+
+template <typename T>
+int rl_rows(const float *z, const int64_t *tokens, int64_t rows, int64_t V, int64_t ignore, const RlRows &rl,
+            int64_t row0, T *dz, float *row_val, cudaStream_t st) {
+    if (rows <= 0) return STREAMBP_OK;
+    SBP_LAUNCH(rl_rows_kernel<T>, (unsigned)rows, 1024, 0, st, z, tokens, V, ignore, rl, row0, dz, row_val,
+               call_state().gate);
+    return STREAMBP_OK;
+}
+template int rl_rows<float>(const float *, const int64_t *, int64_t, int64_t, int64_t, const RlRows &, int64_t, float *,
+                            float *, cudaStream_t);
+template int rl_rows<bf16>(const float *, const int64_t *, int64_t, int64_t, int64_t, const RlRows &, int64_t, bf16 *,
+                           float *, cudaStream_t);
+
+__global__ void rl_finalize_kernel(WsHeader *hdr, int objective, float beta, float *loss, float *ell) {
+    if (hdr->n_valid == 0) set_status(hdr, STREAMBP_E_NO_VALID_LABELS, 0);
+    const double acc = hdr->loss_sum;
+    if (objective == STREAMBP_OBJ_GRPO) {
+        hdr->factor = 1.f;
+        if (loss) *loss = (float)acc;
+        if (ell) *ell = 0.f;
+    } else {
+        // L = -log sigmoid(beta ell) = log(1 + exp(-beta ell)); correction factor sigmoid(beta ell) - 1
+        const double x = (double)beta * acc;
+        const double sg = 1.0 / (1.0 + exp(-x));
+        hdr->factor = hdr->n_valid == 0 ? 0.f : (float)(sg - 1.0);
+        if (loss) *loss = hdr->n_valid == 0 ? 0.f : (float)(x > 0 ? log1p(exp(-x)) : -x + log1p(exp(x)));
+        if (ell) *ell = (float)acc;
+    }
+}
+int rl_finalize(WsHeader *hdr, int objective, float beta, float *loss, float *ell, cudaStream_t st) {
+    SBP_LAUNCH(rl_finalize_kernel, 1, 1, 0, st, hdr, objective, beta, loss, ell);
+    return STREAMBP_OK;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) scale_by_factor_kernel(T *p, int64_t n, const WsHeader *hdr) {
+    const float f = hdr->factor;
+    constexpr int N = Vec<T>::N;
+    for (int64_t i0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * N; i0 < n; i0 += (int64_t)gridDim.x * blockDim.x * N) {
+        if (i0 + N <= n) {
+            Vec<T> a;
+            a.load(p + i0);
+#pragma unroll
+            for (int i = 0; i < N; i++) a.v[i] *= f;
+            a.store(p + i0);
+        } else {
+            for (int64_t i = i0; i < n; i++) p[i] = from_f32<T>(to_f32(p[i]) * f);
+        }
+    }
+}
+template <typename T>
+int scale_by_factor(T *p, int64_t n, const WsHeader *hdr, cudaStream_t st) {
+    if (n <= 0) return STREAMBP_OK;
+    int64_t blocks = (n / Vec<T>::N + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    if (blocks < 1) blocks = 1;
+    SBP_LAUNCH(scale_by_factor_kernel<T>, (unsigned)blocks, 256, 0, st, p, n, hdr);
+    return STREAMBP_OK;
+}
+template int scale_by_factor<float>(float *, int64_t, const WsHeader *, cudaStream_t);
+template int scale_by_factor<bf16>(bf16 *, int64_t, const WsHeader *, cudaStream_t);
+
 __global__ void __launch_bounds__(1024) loss_accumulate_kernel(const float *__restrict__ row_loss, int64_t rows,
                                                                WsHeader *hdr, const int *gate) {
     __shared__ double red[32];

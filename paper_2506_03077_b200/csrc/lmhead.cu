@@ -43,7 +43,7 @@ size_t lmhead_workspace(const streambp_head_cfg &c, int64_t T_, int64_t chunk) {
 template <typename T>
 int lmhead_backward(const streambp_head_cfg &c, const T *g_final, const T *w_vocab, const T *H, const int64_t *labels,
                     int64_t T_, int64_t chunk, bool accumulate, float *loss, int64_t *n_valid, T *dH, float *d_w_vocab,
-                    float *d_g_final, void *ws, cudaStream_t st) {
+                    float *d_g_final, void *ws, cudaStream_t st, const RlRows *rl, float *ell) {
     const int64_t cn = chunk < T_ ? chunk : T_;
     HeadWs<T> s = plan<T>(c, T_, chunk, ws);
     const int d = c.d_model;
@@ -57,6 +57,8 @@ int lmhead_backward(const streambp_head_cfg &c, const T *g_final, const T *w_voc
         SBP_TRY(fill_zero(d_g_final, sizeof(float) * d, st));
         SBP_TRY(fill_zero(d_w_vocab, sizeof(float) * (size_t)V * d, st));
     }
+    // rows of skipped chunks keep this zero
+    if (rl && rl->logp_out) SBP_TRY(fill_zero(rl->logp_out, sizeof(float) * T_, st));
     const int64_t D = (T_ + cn - 1) / cn;
     struct GateScope {      // every launch of a chunk is gated by that chunk's count of unmasked labels
         explicit GateScope(const int *g) { call_state().gate = g; }
@@ -70,14 +72,27 @@ int lmhead_backward(const streambp_head_cfg &c, const T *g_final, const T *w_voc
         GateScope gate(s.chunk_valid + i);
         SBP_TRY(rmsnorm_fwd<T>(Hi, nullptr, g_final, c.rms_eps, n, d, s.hn, s.rstd, nullptr, st));
         SBP_TRY((mm<T, float>(OP_NT, n, V, d, s.hn, d, w_vocab, d, s.z, V, nullptr, false, st)));           // logits
-        SBP_TRY(ce_rows<T>(s.z, labels + r0, n, V, c.ignore_index, s.hdr, s.dz, s.row_loss, st));
+        if (rl)
+            SBP_TRY(rl_rows<T>(s.z, labels + r0, n, V, c.ignore_index, *rl, r0, s.dz, s.row_loss, st));
+        else
+            SBP_TRY(ce_rows<T>(s.z, labels + r0, n, V, c.ignore_index, s.hdr, s.dz, s.row_loss, st));
         SBP_TRY(loss_accumulate(s.row_loss, n, s.hdr, st));
         SBP_TRY((mm<T, float>(OP_TN, V, d, n, s.dz, V, s.hn, d, d_w_vocab, d, nullptr, acc, st)));          // dW += dZ^T hn
         SBP_TRY((mm<T, float>(OP_NN, n, d, V, s.dz, V, w_vocab, d, s.dhn, d, nullptr, false, st)));         // dhn = dZ W
         SBP_TRY(rmsnorm_bwd<T>(s.dhn, Hi, nullptr, s.rstd, g_final, nullptr, nullptr, n, d, nullptr, dH + r0 * d,
                                d_g_final, s.partials, st));
     }
-    SBP_TRY(loss_finalize(s.hdr, loss, n_valid, st));
+    if (!rl) {
+        SBP_TRY(loss_finalize(s.hdr, loss, n_valid, st));
+        return STREAMBP_OK;
+    }
+    SBP_TRY(rl_finalize(s.hdr, rl->objective, rl->beta, loss, ell, st));
+    if (rl->objective == STREAMBP_OBJ_DPO) {
+        // the running sums hold beta * sum_t d ell(t); the exact gradient is (sigmoid(beta ell) - 1) times that
+        SBP_TRY(scale_by_factor<float>(d_w_vocab, V * d, s.hdr, st));
+        SBP_TRY(scale_by_factor<float>(d_g_final, d, s.hdr, st));
+        SBP_TRY(scale_by_factor<T>(dH, T_ * d, s.hdr, st));
+    }
     return STREAMBP_OK;
 }
 
@@ -85,9 +100,9 @@ template size_t lmhead_workspace<float>(const streambp_head_cfg &, int64_t, int6
 template size_t lmhead_workspace<bf16>(const streambp_head_cfg &, int64_t, int64_t);
 template int lmhead_backward<float>(const streambp_head_cfg &, const float *, const float *, const float *,
                                     const int64_t *, int64_t, int64_t, bool, float *, int64_t *, float *, float *,
-                                    float *, void *, cudaStream_t);
+                                    float *, void *, cudaStream_t, const RlRows *, float *);
 template int lmhead_backward<bf16>(const streambp_head_cfg &, const bf16 *, const bf16 *, const bf16 *,
                                    const int64_t *, int64_t, int64_t, bool, float *, int64_t *, bf16 *, float *,
-                                   float *, void *, cudaStream_t);
+                                   float *, void *, cudaStream_t, const RlRows *, float *);
 
 }  // namespace sbp

@@ -1,0 +1,117 @@
+"""GPU parity: streambp_lmhead_rl_backward (GRPO and DPO objectives, Sec. 3.2.1) against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import streambp_oracle as O
+from paper_2506_03077_b200 import binding as B
+from paper_2506_03077_b200 import synth
+from helpers import TOL, assert_close, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def make_case(seed, T, d, V, dtype, masked):
+    bf = dtype == torch.bfloat16
+    hs = synth.HeadShape(d, V)
+    g, W, H, tok = synth.make_head_inputs(hs, seed, T, bf, masked)
+    W = W * 4.0                                   # sharper policies: ratios and clip branches vary more
+    if bf:
+        W = synth.round_bf16(W)
+    cfg = O.HeadCfg(d, V)
+    lp = O._token_logprobs(cfg, g.astype(np.float64), W.astype(np.float64), H.astype(np.float64), tok, 256)
+    old = (lp + synth.normal(seed, "old", (T,), 0.0, 0.3)).astype(np.float32)
+    ref = (lp + synth.normal(seed, "ref", (T,), 0.0, 0.3)).astype(np.float32)
+    adv = synth.normal(seed, "adv", (T,)).astype(np.float32)
+    return hs, cfg, g, W, H, tok, old, ref, adv
+
+
+def run_rl(hs, objective, beta, eps, g, W, H, tok, old, ref, adv, wt, chunk, dtype, accumulate=False, check=True):
+    cfg = B.HeadConfig(hs.d_model, hs.vocab, hs.rms_eps, hs.ignore_index, dtype)
+    T = H.shape[0]
+    f32 = lambda a: None if a is None else torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).cuda()
+    loss = torch.full((1,), float("nan"), device="cuda")
+    ell = torch.full((1,), float("nan"), device="cuda")
+    logp = torch.full((T,), float("nan"), device="cuda")
+    dH = torch.full((T, hs.d_model), float("nan"), device="cuda", dtype=dtype)
+    dW = torch.full((hs.vocab, hs.d_model), float("nan"), device="cuda")
+    dg = torch.full((hs.d_model,), float("nan"), device="cuda")
+    ws = B.alloc_workspace(B.lmhead_workspace_bytes(cfg, T, chunk))
+    st = B.lmhead_rl_backward(cfg, objective, beta, eps, to_dev(g, dtype), to_dev(W, dtype), to_dev(H, dtype),
+                              torch.from_numpy(tok).cuda(), f32(old), f32(ref), f32(adv), f32(wt), chunk, loss, dH, dW,
+                              dg, ws, logp=logp, ell=ell, accumulate=accumulate, check=check)
+    if st != B.OK:
+        return st
+    assert B.last_device_status(ws) == B.OK
+    return loss.item(), ell.item(), logp, dH, dW, dg
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("T,V,chunk", [(200, 1000, 64), (96, 1003, 96)])
+def test_grpo_matches_oracle(dtype, T, V, chunk):
+    masked = T // 5
+    hs, cfg, g, W, H, tok, old, ref, adv = make_case(40 + T, T, 128, V, dtype, masked)
+    tok[T // 2] = -100
+    wt = np.full(T, 1.0 / (T - masked - 1), dtype=np.float32)
+    beta, eps = 0.04, 0.2
+    for ch in (chunk, 23):                         # chunk invariance, ragged
+        loss, _, logp, dH, dW, dg = run_rl(hs, B.OBJ_GRPO, beta, eps, g, W, H, tok, old, ref, adv, wt, ch, dtype)
+        # the clip / min branch is a floating-point decision: the oracle takes it from the log-probabilities the
+        # kernel reports, in float32, and computes every value itself in float64
+        ref_out = O.lmhead_grpo_backward(cfg, g, W, H, tok, old, ref, adv, wt, beta, eps,
+                                         branch_logp=logp.cpu().numpy())
+        part = tok != -100
+        lp_tol = 2e-5 if dtype == torch.float32 else 3e-2
+        assert np.abs(logp.cpu().numpy()[part] - ref_out[1][part]).max() < lp_tol
+        assert torch.count_nonzero(logp[torch.from_numpy(~part).cuda()]) == 0
+        assert abs(loss - ref_out[0]) <= (2e-5 if dtype == torch.float32 else 2e-2) * max(1.0, abs(ref_out[0]))
+        assert_close("dH", dH, ref_out[2], TOL[dtype])
+        assert_close("dW", dW, ref_out[3], TOL[dtype])
+        assert_close("dg", dg, ref_out[4], TOL[dtype])
+        assert torch.count_nonzero(dH[:masked]) == 0
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_dpo_matches_oracle(dtype):
+    T, V, chunk = 192, 1536, 64
+    hs, cfg, g, W, H, tok, old, ref, adv = make_case(77, T, 128, V, dtype, 0)
+    tok[:40] = -100                                # shared prompt; then chosen (+1) and rejected (-1) responses
+    tok[64:128] = -100                             # a whole chunk that takes no part
+    sign = np.where(np.arange(T) < 128, 1.0, -1.0).astype(np.float32)
+    beta = 0.25
+    ref_out = O.lmhead_dpo_backward(cfg, g, W, H, tok, ref, sign, beta)
+    for ch in (chunk, T, 50):
+        loss, ell, logp, dH, dW, dg = run_rl(hs, B.OBJ_DPO, beta, 0.0, g, W, H, tok, None, ref, None, sign, ch, dtype)
+        assert abs(ell - ref_out[1]) <= (1e-4 if dtype == torch.float32 else 0.3)
+        assert abs(loss - ref_out[0]) <= (1e-5 if dtype == torch.float32 else 5e-2)
+        # the correction factor sigmoid(beta ell) - 1 inherits ell's error in bf16; compare directions and scale
+        assert_close("dH", dH, ref_out[2], TOL[dtype] if dtype == torch.float32 else 6e-2)
+        assert_close("dW", dW, ref_out[3], TOL[dtype] if dtype == torch.float32 else 6e-2)
+        assert_close("dg", dg, ref_out[4], TOL[dtype] if dtype == torch.float32 else 6e-2)
+        if dtype == torch.bfloat16:
+            # with the oracle's own factor the gradients agree to the usual tolerance
+            f_gpu = 1.0 / (1.0 + np.exp(-beta * ell)) - 1.0
+            f_ref = 1.0 / (1.0 + np.exp(-beta * ref_out[1])) - 1.0
+            assert_close("dW rescaled", dW * (f_ref / f_gpu), ref_out[3], TOL[dtype])
+        assert torch.count_nonzero(dH[64:128]) == 0
+
+
+def test_rl_head_special_cases_and_errors():
+    T, V = 64, 512
+    hs, cfg, g, W, H, tok, old, ref, adv = make_case(5, T, 64, V, torch.float32, 8)
+    N = T - 8
+    lp = O._token_logprobs(cfg, g.astype(np.float64), W.astype(np.float64), H.astype(np.float64), tok, 64)
+    sft = O.lmhead_ce_backward(cfg, g, W, H, tok)
+    # on-policy, beta = 0, advantage 1, weight 1/N: the gradient of the mean cross-entropy (Eq. (2))
+    out = run_rl(hs, B.OBJ_GRPO, 0.0, 0.2, g, W, H, tok, lp, ref, np.ones(T), np.full(T, 1.0 / N), 16, torch.float32)
+    assert abs(out[0] + 1.0) < 1e-5
+    assert_close("dW", out[4], sft[3], 1e-4)
+    assert_close("dH", out[3], sft[2], 1e-4)
+    # DPO with pi_ref = pi_theta: ell = 0, loss = ln 2, factor -1/2
+    out = run_rl(hs, B.OBJ_DPO, 0.5, 0.0, g, W, H, tok, None, lp, None, np.ones(T), 16, torch.float32)
+    assert abs(out[0] - np.log(2.0)) < 1e-5 and abs(out[1]) < 1e-4
+    assert_close("dW", out[4], 0.25 * N * sft[3], 1e-4)
+    # DPO cannot accumulate (the correction is applied in place); unknown objectives are refused
+    assert run_rl(hs, B.OBJ_DPO, 0.5, 0.0, g, W, H, tok, None, lp, None, np.ones(T), 16, torch.float32,
+                  accumulate=True, check=False) == B.E_SHAPE
+    assert run_rl(hs, 7, 0.5, 0.0, g, W, H, tok, None, lp, None, np.ones(T), 16, torch.float32, check=False) == B.E_SHAPE

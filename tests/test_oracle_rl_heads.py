@@ -120,3 +120,18 @@ def test_special_cases_reduce_to_cross_entropy():
     kl_only = O._backprop_token_coefficients(cfg, g, W, H, tok, 0.1 * wt, 64)
     for a, b in zip(o2[2:], kl_only):
         assert O.rel_frobenius(a, b) < 1e-12
+
+
+def test_branch_logp_only_moves_the_decision():
+    cfg, g, W, H, tok, old, ref, adv, wt = setup(7)
+    base = O.lmhead_grpo_backward(cfg, g, W, H, tok, old, ref, adv, wt, 0.04, 0.2)
+    same = O.lmhead_grpo_backward(cfg, g, W, H, tok, old, ref, adv, wt, 0.04, 0.2, branch_logp=base[1].astype(np.float32))
+    assert same[0] == base[0] and np.array_equal(same[3], base[3])
+    # a perturbed log-probability that pushes one token across the clip boundary changes that token's term only
+    r = np.exp(base[1] - old)
+    t = int(np.argmax((tok != -100) & (r > 1.0) & (r < 1.2) & (adv > 0)))
+    bl = base[1].astype(np.float32).copy()
+    bl[t] = old[t] + np.log(1.3)
+    moved = O.lmhead_grpo_backward(cfg, g, W, H, tok, old, ref, adv, wt, 0.04, 0.2, branch_logp=bl)
+    diff_rows = np.nonzero(np.abs(moved[2] - base[2]).sum(-1) > 0)[0]
+    assert list(diff_rows) == [t]
