@@ -103,6 +103,23 @@ int streambp_layer_backward(const streambp_layer_cfg *cfg, const streambp_layer_
                             int accumulate, const streambp_layer_grads *grads, void *dX,
                             void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/*
+ * The same streamed backward for a PACKED BATCH: X and dY hold n_seqs sequences back to back
+ * (rows cu_seqlens[i] .. cu_seqlens[i+1]-1 are sequence i; cu_seqlens is a HOST array of n_seqs + 1
+ * increasing entries from 0 to T).  Tokens attend only to earlier tokens of their own sequence and
+ * rotary positions restart at pos0 in every sequence; every other step of the layer is row-wise, so a
+ * chunk may span sequences and the products keep the chunk as their row dimension however short the
+ * sequences are (the paper's transfer of sequence-length scaling to batch-size scaling, Sec. 4.1).
+ * The result equals the sum over the sequences of streambp_layer_backward on each of them.
+ * Workspace: streambp_layer_workspace_bytes(cfg, T, chunk).  Errors: additionally STREAMBP_E_SHAPE
+ * for malformed cu_seqlens.
+ */
+int streambp_layer_backward_packed(const streambp_layer_cfg *cfg, const streambp_layer_weights *w,
+                                   const void *X, const void *dY, int64_t T, int64_t chunk,
+                                   const int64_t *cu_seqlens, int32_t n_seqs, int64_t pos0, int accumulate,
+                                   const streambp_layer_grads *grads, void *dX,
+                                   void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 typedef struct {
     int32_t d_model;
     int64_t vocab;

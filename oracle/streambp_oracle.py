@@ -259,6 +259,19 @@ def layer_backward(cfg: LayerCfg, W, X, dY, pos0=0, row_block=1024):
     return dX, G
 
 
+def layer_backward_packed(cfg: LayerCfg, W, X, dY, cu_seqlens, pos0=0, row_block=1024):
+    """A packed batch is a set of independent sequences that share the weights: the input gradient of
+    each sequence is that of the sequence alone, the weight gradients are the sums over the sequences."""
+    X, dY = _f64(X), _f64(dY)
+    dX = np.empty_like(X)
+    G: Dict[str, np.ndarray] = {}
+    for a, e in zip(cu_seqlens[:-1], cu_seqlens[1:]):
+        dX[a:e], Gi = layer_backward(cfg, W, X[a:e], dY[a:e], pos0=pos0, row_block=row_block)
+        for k, v in Gi.items():
+            G[k] = v if k not in G else G[k] + v
+    return dX, G
+
+
 # ---------------------------------------------------------------------------
 # LM head + cross-entropy (SFT objective of Sec. 3.2.1, normalised by the number
 # of unmasked labels)

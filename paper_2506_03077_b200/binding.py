@@ -32,7 +32,7 @@ EXPORTS = (
     "streambp_last_cuda_error", "streambp_last_launch_count", "streambp_gemm",
     "streambp_profile_enable", "streambp_profile_read",
     "streambp_attention_forward", "streambp_attention_backward", "streambp_attention_backward_static",
-    "streambp_lmhead_rl_backward",
+    "streambp_lmhead_rl_backward", "streambp_layer_backward_packed",
 )
 
 
@@ -84,6 +84,9 @@ def lib() -> C.CDLL:
     L.streambp_layer_backward.restype = C.c_int
     L.streambp_layer_backward.argtypes = [C.POINTER(LayerCfgC), C.POINTER(LayerPtrsC), vp, vp, i64, i64, i64, C.c_int,
                                           C.POINTER(LayerPtrsC), vp, vp, sz, vp]
+    L.streambp_layer_backward_packed.restype = C.c_int
+    L.streambp_layer_backward_packed.argtypes = [C.POINTER(LayerCfgC), C.POINTER(LayerPtrsC), vp, vp, i64, i64,
+                                                 C.POINTER(i64), i32, i64, C.c_int, C.POINTER(LayerPtrsC), vp, vp, sz, vp]
     L.streambp_lmhead_workspace_bytes.restype = sz
     L.streambp_lmhead_workspace_bytes.argtypes = [C.POINTER(HeadCfgC), i64, i64]
     L.streambp_lmhead_ce_backward.restype = C.c_int
@@ -221,6 +224,21 @@ def layer_backward(cfg: LayerConfig, weights: Dict[str, torch.Tensor], X: torch.
                                        workspace.numel(), _stream_ptr(stream))
     if check:
         _check(st, "streambp_layer_backward")
+    return st
+
+
+def layer_backward_packed(cfg: LayerConfig, weights, X, dY, chunk: int, cu_seqlens: Sequence[int], grads, dX, workspace,
+                          pos0: int = 0, accumulate: bool = False, stream=None, check: bool = True) -> int:
+    """streambp_layer_backward_packed: X, dY hold the sequences back to back; cu_seqlens = [0, ..., T] on the host."""
+    c = cfg.c()
+    w, g = _ptr_struct(weights), _ptr_struct(grads)
+    n = len(cu_seqlens) - 1
+    cu = (C.c_int64 * (n + 1))(*[int(v) for v in cu_seqlens])
+    st = lib().streambp_layer_backward_packed(C.byref(c), C.byref(w), _ptr(X), _ptr(dY), X.shape[0], chunk, cu, n, pos0,
+                                              1 if accumulate else 0, C.byref(g), _ptr(dX), _ptr(workspace),
+                                              workspace.numel(), _stream_ptr(stream))
+    if check:
+        _check(st, "streambp_layer_backward_packed")
     return st
 
 

@@ -192,10 +192,10 @@ size_t streambp_layer_workspace_bytes(const streambp_layer_cfg *cfg, int64_t T, 
     return cfg->dtype == STREAMBP_F32 ? layer_workspace<float>(*cfg, T, chunk) : layer_workspace<bf16>(*cfg, T, chunk);
 }
 
-int streambp_layer_backward(const streambp_layer_cfg *cfg, const streambp_layer_weights *w, const void *X,
-                            const void *dY, int64_t T, int64_t chunk, int64_t pos0, int accumulate,
-                            const streambp_layer_grads *grads, void *dX, void *workspace, size_t workspace_bytes,
-                            void *cuda_stream) {
+static int layer_backward_checked(const streambp_layer_cfg *cfg, const streambp_layer_weights *w, const void *X,
+                                  const void *dY, int64_t T, int64_t chunk, const int64_t *cu_seqlens, int n_seqs,
+                                  int64_t pos0, int accumulate, const streambp_layer_grads *grads, void *dX,
+                                  void *workspace, size_t workspace_bytes, void *cuda_stream) {
     SBP_TRY(check_layer_cfg(cfg));
     if (T < 1 || chunk < 1 || pos0 < 0) return STREAMBP_E_SHAPE;
     SBP_TRY(check_layer_weights(cfg, w));
@@ -203,15 +203,37 @@ int streambp_layer_backward(const streambp_layer_cfg *cfg, const streambp_layer_
     if (!X || !dY || !dX || !workspace) return STREAMBP_E_NULL;
     if (!aligned(X, 16) || !aligned(dY, 16) || !aligned(dX, 16) || !aligned(workspace, 256)) return STREAMBP_E_ALIGN;
     if (dX == X || dX == dY) return STREAMBP_E_SHAPE;
+    if (cu_seqlens) {
+        if (n_seqs < 1 || cu_seqlens[0] != 0 || cu_seqlens[n_seqs] != T) return STREAMBP_E_SHAPE;
+        for (int i = 0; i < n_seqs; i++)
+            if (cu_seqlens[i + 1] <= cu_seqlens[i]) return STREAMBP_E_SHAPE;
+    }
     if (workspace_bytes < streambp_layer_workspace_bytes(cfg, T, chunk)) return STREAMBP_E_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     SBP_TRY(begin_call(workspace, st));
     const streambp_layer_weights we = effective(cfg, w);
     if (cfg->dtype == STREAMBP_F32)
         return layer_backward<float>(*cfg, we, (const float *)X, (const float *)dY, T, chunk, pos0, accumulate != 0,
-                                     *grads, (float *)dX, workspace, st);
+                                     *grads, (float *)dX, workspace, st, cu_seqlens, n_seqs);
     return layer_backward<bf16>(*cfg, we, (const bf16 *)X, (const bf16 *)dY, T, chunk, pos0, accumulate != 0, *grads,
-                                (bf16 *)dX, workspace, st);
+                                (bf16 *)dX, workspace, st, cu_seqlens, n_seqs);
+}
+
+int streambp_layer_backward(const streambp_layer_cfg *cfg, const streambp_layer_weights *w, const void *X,
+                            const void *dY, int64_t T, int64_t chunk, int64_t pos0, int accumulate,
+                            const streambp_layer_grads *grads, void *dX, void *workspace, size_t workspace_bytes,
+                            void *cuda_stream) {
+    return layer_backward_checked(cfg, w, X, dY, T, chunk, nullptr, 0, pos0, accumulate, grads, dX, workspace,
+                                  workspace_bytes, cuda_stream);
+}
+
+int streambp_layer_backward_packed(const streambp_layer_cfg *cfg, const streambp_layer_weights *w, const void *X,
+                                   const void *dY, int64_t T, int64_t chunk, const int64_t *cu_seqlens, int32_t n_seqs,
+                                   int64_t pos0, int accumulate, const streambp_layer_grads *grads, void *dX,
+                                   void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (!cu_seqlens) return STREAMBP_E_NULL;
+    return layer_backward_checked(cfg, w, X, dY, T, chunk, cu_seqlens, n_seqs, pos0, accumulate, grads, dX, workspace,
+                                  workspace_bytes, cuda_stream);
 }
 
 size_t streambp_lmhead_workspace_bytes(const streambp_head_cfg *cfg, int64_t T, int64_t chunk) {

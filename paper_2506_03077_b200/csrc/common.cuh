@@ -313,11 +313,12 @@ size_t layer_workspace(const streambp_layer_cfg &c, int64_t T_, int64_t chunk);
 template <typename T>
 int layer_backward(const streambp_layer_cfg &c, const streambp_layer_weights &w, const T *X, const T *dY, int64_t T_,
                    int64_t chunk, int64_t pos0, bool accumulate, const streambp_layer_grads &g, T *dX, void *ws,
-                   cudaStream_t st);
+                   cudaStream_t st, const int64_t *cu_seqlens = nullptr, int n_seqs = 0);
 // Y = layer(X), chunked; uses the same workspace plan as layer_backward.
 template <typename T>
+// cu_seqlens (host, n_seqs + 1 entries, 0 ... T): sequence boundaries of a packed batch, or nullptr.
 int layer_forward(const streambp_layer_cfg &c, const streambp_layer_weights &w, const T *X, int64_t T_, int64_t chunk,
-                  int64_t pos0, T *Y, void *ws, cudaStream_t st);
+                  int64_t pos0, T *Y, void *ws, cudaStream_t st, const int64_t *cu_seqlens = nullptr, int n_seqs = 0);
 
 template <typename T>
 size_t lmhead_workspace(const streambp_head_cfg &c, int64_t T_, int64_t chunk);

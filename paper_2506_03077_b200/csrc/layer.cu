@@ -6,11 +6,32 @@
 // exact); running backwards makes the fp32 dK/dV rows of chunk i final as soon as chunk i itself
 // has been processed (only chunks >= i attend to them), so the K/V-projection backward of chunk i
 // runs inside the same iteration, on the h1 rows that are already resident.
+#include <vector>
+
 #include "common.cuh"
 
 namespace sbp {
 
 namespace {
+
+// Sequence boundaries of a packed batch: rows [b[i], b[i+1]) form sequence i.  A single sequence [0, T)
+// when the caller passes none.  Only the attention and the rotary positions see the boundaries: every
+// other step of the layer is row-wise.
+struct Segments {
+    std::vector<int64_t> b;
+    Segments(const int64_t *cu, int n, int64_t T_) {
+        if (cu && n > 0) b.assign(cu, cu + n + 1);
+        else b = {0, T_};
+    }
+    // calls f(a, e, s) for every maximal run of rows [a, e) inside [r0, r1) that lies in one sequence (start s)
+    template <typename F> int for_each(int64_t r0, int64_t r1, F f) const {
+        for (size_t i = 0; i + 1 < b.size(); i++) {
+            const int64_t a = b[i] > r0 ? b[i] : r0, e = b[i + 1] < r1 ? b[i + 1] : r1;
+            if (a < e) SBP_TRY(f(a, e, b[i]));
+        }
+        return STREAMBP_OK;
+    }
+};
 
 template <typename T>
 struct LayerWs {
@@ -63,10 +84,13 @@ LayerWs<T> plan(const streambp_layer_cfg &c, int64_t T_, int64_t chunk, void *ba
 // K/V for all rows, chunk by chunk: h1 = RMSNorm1(X), K = RoPE(h1 Wk^T + bk), V = h1 Wv^T + bv
 template <typename T>
 int kv_prologue(const streambp_layer_cfg &c, const streambp_layer_weights &w, const T *X, int64_t T_, int64_t cn,
-                int64_t pos0, LayerWs<T> &s, cudaStream_t st) {
+                int64_t pos0, const Segments &seg, LayerWs<T> &s, cudaStream_t st) {
     const int d = c.d_model, dh = c.head_dim, Hkv = c.n_kv_heads;
     const int64_t dkv = (int64_t)Hkv * dh;
-    SBP_TRY(rope_table(s.cs, pos0, T_, dh, c.rope_theta, st));
+    // rotary positions restart at every sequence of a packed batch
+    SBP_TRY(seg.for_each(0, T_, [&](int64_t a, int64_t e, int64_t) {
+        return rope_table(s.cs + a * dh, pos0, e - a, dh, c.rope_theta, st);
+    }));
     for (int64_t r0 = 0; r0 < T_; r0 += cn) {
         const int64_t n = (T_ - r0 < cn) ? T_ - r0 : cn;
         SBP_TRY(rmsnorm_fwd<T>(X + r0 * d, nullptr, (const T *)w.g1, c.rms_eps, n, d, s.h1, s.rstd1, nullptr, st));
@@ -80,19 +104,23 @@ int kv_prologue(const streambp_layer_cfg &c, const streambp_layer_weights &w, co
 // Re-forward of one chunk up to m = silu(g) * u. Leaves h1, rstd1, Q, O, lse, r, h2, rstd2, g, u, m.
 template <typename T>
 int chunk_forward(const streambp_layer_cfg &c, const streambp_layer_weights &w, const T *X, int64_t r0, int64_t n,
-                  LayerWs<T> &s, cudaStream_t st) {
+                  const Segments &seg, LayerWs<T> &s, cudaStream_t st) {
     const int d = c.d_model, dh = c.head_dim, Hq = c.n_q_heads, Hkv = c.n_kv_heads;
     const int64_t dq = (int64_t)Hq * dh, I = c.d_ff;
     const T *Xi = X + r0 * d;
     SBP_TRY(rmsnorm_fwd<T>(Xi, nullptr, (const T *)w.g1, c.rms_eps, n, d, s.h1, s.rstd1, nullptr, st));
     SBP_TRY((mm<T, float>(OP_NT, n, dq, d, s.h1, d, (const T *)w.wq, d, s.fa, dq, (const T *)w.bq, false, st)));
     SBP_TRY(rope_apply<T>(s.fa, s.cs + r0 * dh, n, Hq, dh, false, s.Q, st));
-    {
-        // causal pairs (query, key) of this chunk: n * r0 + n (n + 1) / 2; two products forward
-        const double pairs = (double)n * (double)r0 + 0.5 * (double)n * (double)(n + 1);
+    // the chunk's queries against the key / value prefix of their own sequence, one call per sequence the
+    // chunk touches (a = first row, e = end row, q_seq = start of that sequence)
+    SBP_TRY(seg.for_each(r0, r0 + n, [&](int64_t a, int64_t e, int64_t q_seq) {
+        const int64_t m = e - a, off = a - r0, dkv = (int64_t)Hkv * dh;
+        // causal pairs (query, key): m * (a - q_seq) + m (m + 1) / 2; two products forward
+        const double pairs = (double)m * (double)(a - q_seq) + 0.5 * (double)m * (double)(m + 1);
         ProfScope prof(KC_ATTN_FWD, 2.0 * 2.0 * pairs * dh * Hq, st);
-        SBP_TRY(attn_fwd<T>(s.Q, s.K, s.V, n, r0, Hq, Hkv, dh, s.O, s.lse, st));
-    }
+        return attn_fwd<T>(s.Q + off * dq, s.K + q_seq * dkv, s.V + q_seq * dkv, m, a - q_seq, Hq, Hkv, dh,
+                           s.O + off * dq, s.lse + off * Hq, st);
+    }));
     SBP_TRY((mm<T, float>(OP_NT, n, d, dq, s.O, dq, (const T *)w.wo, dq, s.fa, d, nullptr, false, st)));
     SBP_TRY(rmsnorm_fwd<T>(Xi, s.fa, (const T *)w.g2, c.rms_eps, n, d, s.h2, s.rstd2, s.r, st));
     SBP_TRY((mm<T, T>(OP_NT, n, I, d, s.h2, d, (const T *)w.w_gate, d, s.g, I, nullptr, false, st)));
@@ -110,15 +138,16 @@ size_t layer_workspace(const streambp_layer_cfg &c, int64_t T_, int64_t chunk) {
 
 template <typename T>
 int layer_forward(const streambp_layer_cfg &c, const streambp_layer_weights &w, const T *X, int64_t T_, int64_t chunk,
-                  int64_t pos0, T *Y, void *ws, cudaStream_t st) {
+                  int64_t pos0, T *Y, void *ws, cudaStream_t st, const int64_t *cu_seqlens, int n_seqs) {
+    const Segments seg(cu_seqlens, n_seqs, T_);
     const int64_t cn = chunk < T_ ? chunk : T_;
     LayerWs<T> s = plan<T>(c, T_, chunk, ws);
     const int d = c.d_model;
     const int64_t I = c.d_ff;
-    SBP_TRY(kv_prologue<T>(c, w, X, T_, cn, pos0, s, st));
+    SBP_TRY(kv_prologue<T>(c, w, X, T_, cn, pos0, seg, s, st));
     for (int64_t r0 = 0; r0 < T_; r0 += cn) {
         const int64_t n = (T_ - r0 < cn) ? T_ - r0 : cn;
-        SBP_TRY(chunk_forward<T>(c, w, X, r0, n, s, st));
+        SBP_TRY(chunk_forward<T>(c, w, X, r0, n, seg, s, st));
         SBP_TRY((mm<T, float>(OP_NT, n, d, I, s.m, I, (const T *)w.w_down, I, s.fa, d, nullptr, false, st)));
         SBP_TRY(add_cast<T>(s.r, s.fa, n * d, Y + r0 * d, st));
     }
@@ -128,14 +157,15 @@ int layer_forward(const streambp_layer_cfg &c, const streambp_layer_weights &w, 
 template <typename T>
 int layer_backward(const streambp_layer_cfg &c, const streambp_layer_weights &w, const T *X, const T *dY, int64_t T_,
                    int64_t chunk, int64_t pos0, bool accumulate, const streambp_layer_grads &G, T *dX, void *ws,
-                   cudaStream_t st) {
+                   cudaStream_t st, const int64_t *cu_seqlens, int n_seqs) {
+    const Segments seg(cu_seqlens, n_seqs, T_);
     const int64_t cn = chunk < T_ ? chunk : T_;
     LayerWs<T> s = plan<T>(c, T_, chunk, ws);
     const int d = c.d_model, dh = c.head_dim, Hq = c.n_q_heads, Hkv = c.n_kv_heads;
     const int64_t dq = (int64_t)Hq * dh, dkv = (int64_t)Hkv * dh, I = c.d_ff;
     constexpr bool kF32 = sizeof(T) == 4;
 
-    SBP_TRY(kv_prologue<T>(c, w, X, T_, cn, pos0, s, st));
+    SBP_TRY(kv_prologue<T>(c, w, X, T_, cn, pos0, seg, s, st));
     SBP_TRY(fill_zero(s.dK, sizeof(float) * T_ * dkv, st));
     SBP_TRY(fill_zero(s.dV, sizeof(float) * T_ * dkv, st));
     if (!accumulate) {  // vectors are always added to; matrices are overwritten by the first chunk's product
@@ -153,7 +183,7 @@ int layer_backward(const streambp_layer_cfg &c, const streambp_layer_weights &w,
         const int64_t n = (T_ - r0 < cn) ? T_ - r0 : cn;
         const bool acc = accumulate || i != D - 1;
         const T *Xi = X + r0 * d, *dYi = dY + r0 * d;
-        SBP_TRY(chunk_forward<T>(c, w, X, r0, n, s, st));
+        SBP_TRY(chunk_forward<T>(c, w, X, r0, n, seg, s, st));
 
         // ---- MLP backward ----
         SBP_TRY((mm<T, float>(OP_TN, d, I, n, dYi, d, s.m, I, G.w_down, I, nullptr, acc, st)));       // dWd += dY^T m
@@ -173,11 +203,14 @@ int layer_backward(const streambp_layer_cfg &c, const streambp_layer_weights &w,
         SBP_TRY((mm<T, T>(OP_NN, n, dq, d, dr_op, d, (const T *)w.wo, dq, s.dO, dq, nullptr, false, st)));  // dO = dr Wo
 
         // ---- partitioned attention backward: dQ (into fa), dK/dV prefix += ----
-        {
-            const double pairs = (double)n * (double)r0 + 0.5 * (double)n * (double)(n + 1);
+        SBP_TRY(seg.for_each(r0, r0 + n, [&](int64_t a, int64_t e, int64_t q_seq) {
+            const int64_t m = e - a, off = a - r0;
+            const double pairs = (double)m * (double)(a - q_seq) + 0.5 * (double)m * (double)(m + 1);
             ProfScope prof(KC_ATTN_BWD, 5.0 * 2.0 * pairs * dh * Hq, st);   // five products backward
-            SBP_TRY(attn_bwd<T>(s.Q, s.K, s.V, s.O, s.dO, s.lse, n, r0, Hq, Hkv, dh, s.delta, s.fa, s.dK, s.dV, st));
-        }
+            return attn_bwd<T>(s.Q + off * dq, s.K + q_seq * dkv, s.V + q_seq * dkv, s.O + off * dq, s.dO + off * dq,
+                               s.lse + off * Hq, m, a - q_seq, Hq, Hkv, dh, s.delta + off * Hq, s.fa + off * dq,
+                               s.dK + q_seq * dkv, s.dV + q_seq * dkv, st);
+        }));
 
         // ---- Q projection backward ----
         T *dq_s = s.Q;  // Q is dead after the attention backward
@@ -208,14 +241,14 @@ int layer_backward(const streambp_layer_cfg &c, const streambp_layer_weights &w,
 template size_t layer_workspace<float>(const streambp_layer_cfg &, int64_t, int64_t);
 template size_t layer_workspace<bf16>(const streambp_layer_cfg &, int64_t, int64_t);
 template int layer_forward<float>(const streambp_layer_cfg &, const streambp_layer_weights &, const float *, int64_t,
-                                  int64_t, int64_t, float *, void *, cudaStream_t);
+                                  int64_t, int64_t, float *, void *, cudaStream_t, const int64_t *, int);
 template int layer_forward<bf16>(const streambp_layer_cfg &, const streambp_layer_weights &, const bf16 *, int64_t,
-                                 int64_t, int64_t, bf16 *, void *, cudaStream_t);
+                                 int64_t, int64_t, bf16 *, void *, cudaStream_t, const int64_t *, int);
 template int layer_backward<float>(const streambp_layer_cfg &, const streambp_layer_weights &, const float *,
                                    const float *, int64_t, int64_t, int64_t, bool, const streambp_layer_grads &,
-                                   float *, void *, cudaStream_t);
+                                   float *, void *, cudaStream_t, const int64_t *, int);
 template int layer_backward<bf16>(const streambp_layer_cfg &, const streambp_layer_weights &, const bf16 *,
                                   const bf16 *, int64_t, int64_t, int64_t, bool, const streambp_layer_grads &, bf16 *,
-                                  void *, cudaStream_t);
+                                  void *, cudaStream_t, const int64_t *, int);
 
 }  // namespace sbp

@@ -99,3 +99,34 @@ def test_layer_bf16_long_prefix_small_width():
     assert torch.equal(dX, dX2)
     for k in grads:
         assert torch.equal(grads[k], grads2[k]), k
+
+
+@pytest.mark.parametrize("dtype,dh,cu", [
+    (torch.float32, 64, [0, 70, 71, 200, 333]),          # sequences shorter and longer than the chunk, one of length 1
+    (torch.bfloat16, 128, [0, 300, 1100, 1101, 1500]),   # tensor-core attention on per-sequence prefixes
+])
+def test_packed_batch_matches_sum_over_sequences(dtype, dh, cu):
+    """Packed batch (several sequences back to back): attention and rotary positions stay inside each
+    sequence; the result is the sum over the sequences of the single-sequence backward."""
+    shape = synth.LayerShape(256, 4, 2, dh, 344, True, 1e4)
+    T, chunk = cu[-1], 128
+    wstd, dystd = (0.05, 1.0) if dtype == torch.float32 else (0.02, 1e-3)
+    ocfg, bcfg, W, X, dY = layer_case(shape, 17, T, dtype, dy_std=dystd, wstd=wstd)
+    Wd = {k: to_dev(v, dtype) for k, v in W.items()}
+    Xd, dYd = to_dev(X, dtype), to_dev(dY, dtype)
+    grads = B.alloc_layer_grads(bcfg)
+    for g in grads.values():
+        g.fill_(float("nan"))
+    dX = torch.full_like(Xd, float("nan"))
+    ws = B.alloc_workspace(B.layer_workspace_bytes(bcfg, T, chunk))
+    B.layer_backward_packed(bcfg, Wd, Xd, dYd, chunk, cu, grads, dX, ws, pos0=3)
+    assert B.last_device_status(ws) == B.OK
+    dX_ref, G_ref = O.layer_backward_packed(ocfg, W, X, dY, cu, pos0=3)
+    tol = TOL[dtype]
+    assert_close("dX", dX, dX_ref, tol)
+    for k, v in G_ref.items():
+        assert_close(k, grads[k], v, tol)
+    # malformed boundaries are refused on the host
+    bad = B.layer_backward_packed(bcfg, Wd, Xd, dYd, chunk, [0, 50, 50, T], grads, dX, ws, check=False)
+    assert bad == B.E_SHAPE
+    assert B.layer_backward_packed(bcfg, Wd, Xd, dYd, chunk, [0, 50, T - 1], grads, dX, ws, check=False) == B.E_SHAPE

@@ -288,3 +288,18 @@ def test_error_metrics():
     assert abs(O.rel_frobenius(a * 1.01, a) - 0.01) < 1e-12
     ea, er = O.paper_errors(a + 0.5, a)
     assert abs(ea - 0.5) < 1e-12 and abs(er - (0.5 + 0.25 + 0.25) / 3) < 1e-9
+
+
+def test_packed_batch_is_a_set_of_independent_sequences():
+    cfg = small_layer(True)
+    W, X, dY = rand_layer(cfg, 9, 20)
+    one = O.layer_backward(cfg, W, X, dY)
+    packed_one = O.layer_backward_packed(cfg, W, X, dY, [0, 20])
+    assert np.array_equal(one[0], packed_one[0]) and all(np.array_equal(one[1][k], packed_one[1][k]) for k in one[1])
+    dXp, Gp = O.layer_backward_packed(cfg, W, X, dY, [0, 7, 20])
+    X2 = X.copy()
+    X2[7:] += 1.0                                       # changing the second sequence leaves the first one's dX alone
+    dXq, _ = O.layer_backward_packed(cfg, W, X2, dY, [0, 7, 20])
+    assert np.array_equal(dXp[:7], dXq[:7]) and not np.allclose(dXp[7:], dXq[7:])
+    # and differs from treating the rows as one sequence
+    assert O.rel_frobenius(dXp, one[0]) > 1e-3
