@@ -241,6 +241,36 @@ int streambp_gemm(int op, int64_t M, int64_t N, int64_t K, const void *A, int64_
                   int32_t out_dtype, int accumulate, int engine, void *cuda_stream);
 
 /*
+ * Building block exposed for tests and profiling: several independent products in ONE launch of the
+ * tensor-core kernel (bf16 operands).  The per-chunk gradients of Eq. (1) that become ready together
+ * (e.g. dWg += dg^T h2, dWu += du^T h2 and dh2 = dg Wg + du Wu after the partitioned MLP of
+ * Sec. 3.2.2) share a launch so that their tiles fill the GPU together.  Problem i computes
+ * C_i (+)= sum over its n_segments K segments of op(A_s, B_s), `op` and layouts as in streambp_gemm;
+ * all segments of a problem share M, N and C.  n <= 4 problems, 8 segments in total, 1..3 per problem.
+ * out_dtype STREAMBP_F32 (accumulate allowed) or STREAMBP_BF16 (the sum over segments is formed in fp32
+ * and rounded once; accumulate not allowed).
+ * sched: NULL, or two int32 of device memory that are zero when the launch starts; the kernel then
+ * hands tiles to CTAs dynamically (longest first) and leaves the two ints zero again.  The result does
+ * not depend on the schedule.  Returns STREAMBP_E_SHAPE if a problem does not meet the tensor-core
+ * kernel's alignment rules (leading dimensions multiples of 8 elements, 16-byte aligned pointers).
+ */
+typedef struct {
+    int32_t op;
+    int32_t n_segments;
+    int64_t M, N;
+    const void *A[3];
+    int64_t lda[3];
+    const void *B[3];
+    int64_t ldb[3];
+    int64_t K[3];
+    void *C;
+    int64_t ldc;
+    int32_t out_dtype;
+    int32_t accumulate;
+} streambp_gemm_problem;
+int streambp_gemm_grouped(const streambp_gemm_problem *problems, int32_t n, int32_t *sched, void *cuda_stream);
+
+/*
  * Building blocks exposed for tests and profiling: the partitioned attention of Sec. 3.2.2
  * (S^(i) = Q^(i) K^(:i)T, causal softmax, O^(i) = P^(i) V^(:i)) for one chunk of n query rows that
  * sit at absolute rows q0 .. q0+n-1 and attend to keys 0 .. q0+n-1, and its backward.

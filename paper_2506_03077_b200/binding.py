@@ -29,7 +29,7 @@ EXPORTS = (
     "streambp_lmhead_workspace_bytes", "streambp_lmhead_ce_backward",
     "streambp_model_workspace_bytes", "streambp_model_backward",
     "streambp_last_device_status", "streambp_status_string",
-    "streambp_last_cuda_error", "streambp_last_launch_count", "streambp_gemm",
+    "streambp_last_cuda_error", "streambp_last_launch_count", "streambp_gemm", "streambp_gemm_grouped",
     "streambp_profile_enable", "streambp_profile_read",
     "streambp_attention_forward", "streambp_attention_backward", "streambp_attention_backward_static",
     "streambp_lmhead_rl_backward", "streambp_layer_backward_packed",
@@ -53,6 +53,13 @@ class HeadCfgC(C.Structure):
 
 class RlCfgC(C.Structure):
     _fields_ = [("objective", C.c_int32), ("beta", C.c_float), ("clip_eps", C.c_float)]
+
+
+class GemmProblemC(C.Structure):
+    _fields_ = [("op", C.c_int32), ("n_segments", C.c_int32), ("M", C.c_int64), ("N", C.c_int64),
+                ("A", C.c_void_p * 3), ("lda", C.c_int64 * 3), ("B", C.c_void_p * 3), ("ldb", C.c_int64 * 3),
+                ("K", C.c_int64 * 3), ("C", C.c_void_p), ("ldc", C.c_int64), ("out_dtype", C.c_int32),
+                ("accumulate", C.c_int32)]
 
 
 class ModelCfgC(C.Structure):
@@ -108,6 +115,8 @@ def lib() -> C.CDLL:
     L.streambp_last_cuda_error.argtypes = []
     L.streambp_last_launch_count.restype = i64
     L.streambp_last_launch_count.argtypes = []
+    L.streambp_gemm_grouped.restype = C.c_int
+    L.streambp_gemm_grouped.argtypes = [C.POINTER(GemmProblemC), i32, vp, vp]
     L.streambp_gemm.restype = C.c_int
     L.streambp_gemm.argtypes = [C.c_int, i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, i32, C.c_int, C.c_int, vp]
     L.streambp_attention_forward.restype = C.c_int
@@ -313,6 +322,31 @@ def gemm(op: int, A: torch.Tensor, B: torch.Tensor, C_out: torch.Tensor, accumul
                              engine, _stream_ptr(stream))
     if check:
         _check(st, "streambp_gemm")
+    return st
+
+
+def gemm_grouped(problems, sched: Optional[torch.Tensor] = None, stream=None, check: bool = True) -> int:
+    """streambp_gemm_grouped.  problems: list of (op, [(A, B), ...], C_out, accumulate) with 2-D row-major bf16
+    operands; each problem sums its (A, B) segments.  sched: None or an int32 CUDA tensor of two zeros."""
+    arr = (GemmProblemC * len(problems))()
+    for i, (op, segs, C_out, acc) in enumerate(problems):
+        g = arr[i]
+        g.op, g.n_segments = op, len(segs)
+        for s, (A, B) in enumerate(segs):
+            assert A.stride(1) == 1 and B.stride(1) == 1
+            if op == OP_NT:
+                M, K, N = A.shape[0], A.shape[1], B.shape[0]
+            elif op == OP_NN:
+                M, K, N = A.shape[0], A.shape[1], B.shape[1]
+            else:
+                K, M, N = A.shape[0], A.shape[1], B.shape[1]
+            g.A[s], g.lda[s], g.B[s], g.ldb[s], g.K[s] = A.data_ptr(), A.stride(0), B.data_ptr(), B.stride(0), K
+        g.M, g.N = M, N
+        assert C_out.stride(1) == 1 and tuple(C_out.shape) == (M, N)
+        g.C, g.ldc, g.out_dtype, g.accumulate = C_out.data_ptr(), C_out.stride(0), _dtype_code(C_out.dtype), 1 if acc else 0
+    st = lib().streambp_gemm_grouped(arr, len(problems), _ptr(sched), _stream_ptr(stream))
+    if check:
+        _check(st, "streambp_gemm_grouped")
     return st
 
 

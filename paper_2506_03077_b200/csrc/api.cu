@@ -78,6 +78,67 @@ int mm<bf16, bf16>(GemmOp op, int64_t M, int64_t N, int64_t K, const bf16 *A, in
     if (e == 2) return STREAMBP_E_SHAPE;
     return gemm<bf16, bf16>(op, M, N, K, A, lda, B, ldb, C, ldc, bias, accumulate, st);
 }
+namespace {
+bool grouping_enabled() {
+    static int on = -1;
+    if (on < 0) {
+        const char *e = std::getenv("STREAMBP_NO_GROUP");
+        on = (e && e[0] == '1') ? 0 : 1;
+    }
+    return on == 1;
+}
+}  // namespace
+
+template <>
+int mm_group<float>(const MmProb<float> *probs, int n, cudaStream_t st) {
+    for (int i = 0; i < n; i++) {
+        const MmProb<float> &g = probs[i];
+        for (int s = 0; s < g.nseg; s++)
+            SBP_TRY((mm<float, float>(g.op, g.M, g.N, g.seg[s].K, g.seg[s].A, g.seg[s].lda, g.seg[s].B, g.seg[s].ldb,
+                                      (float *)g.C, g.ldc, s == 0 ? g.bias : nullptr, g.accumulate || s > 0, st)));
+    }
+    return STREAMBP_OK;
+}
+template <>
+int mm_group<bf16>(const MmProb<bf16> *probs, int n, cudaStream_t st) {
+    GemmProb gp[4];
+    bool grouped = grouping_enabled() && gemm_engine() != 1 && n <= 4;
+    if (grouped) {
+        for (int i = 0; i < n; i++) {
+            const MmProb<bf16> &g = probs[i];
+            gp[i].op = g.op; gp[i].M = g.M; gp[i].N = g.N; gp[i].nseg = g.nseg;
+            for (int s = 0; s < g.nseg; s++) gp[i].seg[s] = GemmSeg{g.seg[s].A, g.seg[s].lda, g.seg[s].B, g.seg[s].ldb, g.seg[s].K};
+            gp[i].C = g.C; gp[i].ldc = g.ldc; gp[i].c_is_f32 = g.c_is_f32; gp[i].bias = g.bias; gp[i].accumulate = g.accumulate;
+        }
+        grouped = gemm_tc_group_supported(gp, n);
+    }
+    if (grouped) {
+        double flops = 0.0;
+        for (int i = 0; i < n; i++)
+            for (int s = 0; s < probs[i].nseg; s++) flops += 2.0 * (double)probs[i].M * (double)probs[i].N * (double)probs[i].seg[s].K;
+        ProfScope prof(KC_GEMM, flops, st);
+        CallState &cs = call_state();
+        int *sched = cs.sched ? cs.sched + 2 * (cs.sched_slot++ % kSchedSlots) : nullptr;
+        return gemm_tc_group(gp, n, sched, st);
+    }
+    for (int i = 0; i < n; i++) {
+        const MmProb<bf16> &g = probs[i];
+        // a bf16 output cannot be accumulated into: several segments need an fp32 C
+        if (!g.c_is_f32 && g.nseg > 1) return STREAMBP_E_SHAPE;
+        for (int s = 0; s < g.nseg; s++) {
+            const bf16 *b = s == 0 ? g.bias : nullptr;
+            const bool acc = g.accumulate || s > 0;
+            if (g.c_is_f32)
+                SBP_TRY((mm<bf16, float>(g.op, g.M, g.N, g.seg[s].K, g.seg[s].A, g.seg[s].lda, g.seg[s].B, g.seg[s].ldb,
+                                         (float *)g.C, g.ldc, b, acc, st)));
+            else
+                SBP_TRY((mm<bf16, bf16>(g.op, g.M, g.N, g.seg[s].K, g.seg[s].A, g.seg[s].lda, g.seg[s].B, g.seg[s].ldb,
+                                        (bf16 *)g.C, g.ldc, b, acc, st)));
+        }
+    }
+    return STREAMBP_OK;
+}
+
 template <>
 int attn_fwd<float>(const float *q, const float *k, const float *v, int64_t n, int64_t q0, int Hq, int Hkv, int dh,
                     float *o, float *lse, cudaStream_t st) {
@@ -177,6 +238,8 @@ streambp_layer_weights effective(const streambp_layer_cfg *c, const streambp_lay
 int begin_call(void *ws, cudaStream_t st) {
     call_state().cuda_error = 0;
     call_state().launches = 0;
+    call_state().sched = nullptr;
+    call_state().sched_slot = 0;
     return fill_zero(ws, kHeaderBytes, st);
 }
 
@@ -479,6 +542,38 @@ int streambp_gemm(int op, int64_t M, int64_t N, int64_t K, const void *A, int64_
         return gemm<bf16, float>(g, M, N, K, (const bf16 *)A, lda, (const bf16 *)B, ldb, (float *)C, ldc, nullptr, acc,
                                  st);
     return gemm<bf16, bf16>(g, M, N, K, (const bf16 *)A, lda, (const bf16 *)B, ldb, (bf16 *)C, ldc, nullptr, false, st);
+}
+
+int streambp_gemm_grouped(const streambp_gemm_problem *problems, int32_t n, int32_t *sched, void *cuda_stream) {
+    if (!problems) return STREAMBP_E_NULL;
+    if (n < 1 || n > 4) return STREAMBP_E_SHAPE;
+    if (sched && !aligned(sched, 8)) return STREAMBP_E_ALIGN;
+    GemmProb gp[4];
+    for (int i = 0; i < n; i++) {
+        const streambp_gemm_problem &q = problems[i];
+        if (q.op < 0 || q.op > 2 || q.n_segments < 1 || q.n_segments > 3 || q.M < 1 || q.N < 1) return STREAMBP_E_SHAPE;
+        if (q.out_dtype != STREAMBP_F32 && q.out_dtype != STREAMBP_BF16) return STREAMBP_E_DTYPE;
+        if (q.out_dtype == STREAMBP_BF16 && q.accumulate) return STREAMBP_E_DTYPE;
+        if (!q.C) return STREAMBP_E_NULL;
+        gp[i].op = static_cast<GemmOp>(q.op);
+        gp[i].M = q.M;
+        gp[i].N = q.N;
+        gp[i].nseg = q.n_segments;
+        for (int s = 0; s < q.n_segments; s++) {
+            if (!q.A[s] || !q.B[s]) return STREAMBP_E_NULL;
+            if (q.K[s] < 1) return STREAMBP_E_SHAPE;
+            gp[i].seg[s] = GemmSeg{(const bf16 *)q.A[s], q.lda[s], (const bf16 *)q.B[s], q.ldb[s], q.K[s]};
+        }
+        gp[i].C = q.C;
+        gp[i].ldc = q.ldc;
+        gp[i].c_is_f32 = q.out_dtype == STREAMBP_F32;
+        gp[i].bias = nullptr;
+        gp[i].accumulate = q.accumulate != 0;
+    }
+    call_state().cuda_error = 0;
+    call_state().launches = 0;
+    if (!gemm_tc_group_supported(gp, n)) return STREAMBP_E_SHAPE;
+    return gemm_tc_group(gp, n, sched, static_cast<cudaStream_t>(cuda_stream));
 }
 
 }  // extern "C"

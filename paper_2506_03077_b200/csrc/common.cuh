@@ -19,6 +19,10 @@ struct CallState {
     // (or write exact zeros, where an output must still be defined) when *gate == 0.  Used by the LM
     // head to skip chunks whose labels are all ignored without a host round trip.
     const int *gate = nullptr;
+    // Device memory for the dynamic tile schedule of grouped products: kSchedSlots pairs of ints inside the
+    // current call's workspace header (zero between launches), used in rotation; nullptr = static schedule.
+    int *sched = nullptr;
+    int sched_slot = 0;
 };
 CallState &call_state();
 
@@ -151,8 +155,21 @@ struct WsHeader {
     unsigned long long n_valid;
     double loss_sum;
     float factor;       // DPO: sigmoid(beta * ell) - 1, the in-place correction applied after the chunk loop
+    int32_t pad_[9];
+    int32_t sched[16];  // tile counters of grouped products (see CallState::sched), at byte 64
 };
 static constexpr size_t kHeaderBytes = 256;
+static constexpr int kSchedSlots = 8;
+static_assert(sizeof(WsHeader) <= kHeaderBytes, "workspace header too large");
+
+// Points the grouped products of the enclosed launches at the counters of this workspace header.
+struct SchedScope {
+    int *saved;
+    explicit SchedScope(WsHeader *hdr) : saved(call_state().sched) {
+        call_state().sched = reinterpret_cast<int *>(reinterpret_cast<char *>(hdr) + 64);
+    }
+    ~SchedScope() { call_state().sched = saved; }
+};
 
 __device__ __forceinline__ void set_status(WsHeader *h, int st, int detail) {
     if (atomicCAS(&h->status, 0, st) == 0) h->detail = detail;
@@ -188,6 +205,31 @@ bool gemm_tc_supported(GemmOp op, int64_t M, int64_t N, int64_t K, int64_t lda, 
                        const void *A, const void *B, const void *C, bool c_is_f32);
 int gemm_tc(GemmOp op, int64_t M, int64_t N, int64_t K, const bf16 *A, int64_t lda, const bf16 *B, int64_t ldb,
             void *C, int64_t ldc, bool c_is_f32, const bf16 *bias, bool accumulate, cudaStream_t st);
+
+// Several independent products in one launch.  A problem is C (+)= sum_s op(A_s, B_s) (+ bias) over
+// up to three K segments that share M, N, the operand layout and C.
+struct GemmSeg {
+    const bf16 *A;
+    int64_t lda;
+    const bf16 *B;
+    int64_t ldb;
+    int64_t K;
+};
+struct GemmProb {
+    GemmOp op;
+    int64_t M, N;
+    int nseg;
+    GemmSeg seg[3];
+    void *C;
+    int64_t ldc;
+    bool c_is_f32;
+    const bf16 *bias;
+    bool accumulate;
+};
+bool gemm_tc_group_supported(const GemmProb *probs, int n);
+// sched: two ints of device memory that are zero when the launch starts (the kernel leaves them zero),
+// enabling the dynamic tile schedule; nullptr selects the static one.
+int gemm_tc_group(const GemmProb *probs, int n, int *sched, cudaStream_t st);
 
 // Reads and clears the flag a tensor-core kernel raises when one of its bounded waits expires.
 int gemm_tc_take_fault();
@@ -306,6 +348,44 @@ int embedding_gather(const T *embed, const int64_t *ids, int64_t rows, int d, in
 template <typename T>
 int embedding_scatter_add(const T *dx, const int64_t *ids, int64_t rows, int d, int64_t vocab, float *d_embed,
                           cudaStream_t st);
+
+// Grouped products used by the schedulers: independent problems that become ready together go out as one
+// launch (tensor cores) or one after the other (CUDA cores); a problem may sum several K segments.
+template <typename T>
+struct MmSeg {
+    const T *A;
+    int64_t lda;
+    const T *B;
+    int64_t ldb;
+    int64_t K;
+};
+template <typename T>
+struct MmProb {
+    GemmOp op;
+    int64_t M, N;
+    int nseg;
+    MmSeg<T> seg[3];
+    void *C;            // fp32 if c_is_f32, else T
+    int64_t ldc;
+    bool c_is_f32;
+    const T *bias;
+    bool accumulate;
+};
+template <typename T>
+MmProb<T> mm_prob(GemmOp op, int64_t M, int64_t N, int64_t K, const T *A, int64_t lda, const T *B, int64_t ldb, void *C,
+                  int64_t ldc, bool c_is_f32, const T *bias, bool accumulate) {
+    MmProb<T> g{};
+    g.op = op; g.M = M; g.N = N; g.nseg = 1;
+    g.seg[0] = MmSeg<T>{A, lda, B, ldb, K};
+    g.C = C; g.ldc = ldc; g.c_is_f32 = c_is_f32; g.bias = bias; g.accumulate = accumulate;
+    return g;
+}
+template <typename T>
+void mm_add_seg(MmProb<T> &g, int64_t K, const T *A, int64_t lda, const T *B, int64_t ldb) {
+    g.seg[g.nseg++] = MmSeg<T>{A, lda, B, ldb, K};
+}
+template <typename T>
+int mm_group(const MmProb<T> *probs, int n, cudaStream_t st);
 
 // ---- schedulers (T = storage dtype) --------------------------------------------------
 template <typename T>

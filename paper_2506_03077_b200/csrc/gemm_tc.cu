@@ -1,8 +1,9 @@
 // tcgen05 tensor-core GEMM for sm_100a: bf16 operands staged in shared memory by TMA
-// (128-byte swizzle), fp32 accumulation in tensor memory, three operand layouts.
+// (128-byte swizzle), fp32 accumulation in tensor memory, three operand layouts, several
+// independent products (each possibly a sum over K segments) per launch.
 //
 //   persistent grid, one CTA per SM, output tile 128 x 256, K slices of 64
-//   warp 0      : TMA producer (one elected lane)
+//   warp 0      : tile scheduler and TMA producer (one elected lane)
 //   warp 1      : allocates tensor memory, issues tcgen05.mma (one elected lane)
 //   warps 2..5  : epilogue -- tcgen05.ld of a 32-lane quarter, bias, then
 //                 fp32 output: 32x32 blocks staged in shared memory (128-byte swizzle) and written
@@ -20,6 +21,8 @@
 // Every mbarrier wait is bounded (2 s of %globaltimer): on expiry the CTA raises a fault flag that
 // streambp_last_device_status() reports as STREAMBP_E_DEVICE_TIMEOUT, all roles leave their loops,
 // tensor memory is released and the kernel returns.
+#include <cstring>
+
 #include "sm100.cuh"
 
 namespace sbp {
@@ -31,7 +34,7 @@ constexpr int B_BYTES = BN * BK * 2;   // 32 KiB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int EPI_BUF_BYTES = 32 * 128;                  // one 32 x 32 fp32 block
 constexpr int EPI_BYTES = 4 * 2 * EPI_BUF_BYTES;          // 4 epilogue warps, double-buffered
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 /* alignment slack */ + 256 /* barriers, tile ring */;
 constexpr int NUM_THREADS = 192;
 constexpr uint32_t TMEM_COLS = 512;
 
@@ -92,19 +95,126 @@ int sm_count() {
 
 namespace {
 
-struct TcParams {
-    int M, N, K;
-    void *C;
-    long long ldc;
-    const bf16 *bias;
-    int accumulate;
-    const int *gate;      // optional: the kernel returns at once when *gate == 0
+// ---------------------------------------------------------------------------------------------
+// One launch, several products.  A launch carries up to MAX_PROBS independent problems; a problem
+// is C (+)= sum over its K segments of op(A_s, B_s), so that e.g. dh2 = dg Wg + du Wu is ONE
+// accumulation in tensor memory and not a product followed by a read-modify-write of C.  The tiles
+// of all problems form one list, longest tiles first; CTAs take tiles from it either statically
+// (tile = blockIdx.x + i * gridDim.x) or, when the caller provides a counter, dynamically with one
+// atomicAdd per tile.  Either way an output tile is produced by exactly one CTA in a fixed order of
+// K, so results do not depend on the schedule.  Grouping the products that become ready together
+// removes most of the part-empty last wave each of them would have on its own.
+// Operand layouts, output type and accumulation are per-problem run-time flags.
+// ---------------------------------------------------------------------------------------------
+constexpr int MAX_PROBS = 4, MAX_SEGS = 8, RING = 4;
+constexpr uint32_t F_A_MN = 1u, F_B_MN = 2u, F_OUT_F32 = 4u, F_ACC = 8u;
+
+struct GroupParams {
+    CUtensorMap map_a[MAX_SEGS];
+    CUtensorMap map_b[MAX_SEGS];
+    CUtensorMap map_c[MAX_PROBS];
+    int seg_kb[MAX_SEGS];              // K blocks of each segment
+    int seg_begin[MAX_PROBS + 1];      // segments of problem q: seg_begin[q] .. seg_begin[q+1]-1
+    int tile_begin[MAX_PROBS + 1];     // tiles of problem q: tile_begin[q] .. tile_begin[q+1]-1
+    int tiles_m[MAX_PROBS];
+    int M[MAX_PROBS], N[MAX_PROBS];
+    void *C[MAX_PROBS];
+    long long ldc[MAX_PROBS];
+    const bf16 *bias[MAX_PROBS];
+    uint32_t flags[MAX_PROBS];
+    int nprob;
+    int *sched;                        // {next tile, CTAs finished}, both zero at launch; or nullptr: static schedule
+    const int *gate;                   // optional: the kernel returns at once when *gate == 0
 };
 
-template <bool A_MN, bool B_MN, bool OUT_F32>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
-    gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                   const __grid_constant__ CUtensorMap map_c, const TcParams p) {
+template <typename T>
+__device__ __forceinline__ T pick(const T (&a)[MAX_PROBS], int q) {
+    T v = a[0];
+#pragma unroll
+    for (int i = 1; i < MAX_PROBS; i++) v = (q == i) ? a[i] : v;
+    return v;
+}
+
+struct TileRef { int q, m0, n0, seg0, seg1; };
+__device__ __forceinline__ TileRef locate(const GroupParams &p, int tile) {
+    int q = 0;
+#pragma unroll
+    for (int i = 1; i < MAX_PROBS; i++) q = (i < p.nprob && tile >= p.tile_begin[i]) ? i : q;
+    int tb = p.tile_begin[0], s0 = p.seg_begin[0], s1 = p.seg_begin[1];
+#pragma unroll
+    for (int i = 1; i < MAX_PROBS; i++) {
+        tb = (q == i) ? p.tile_begin[i] : tb;
+        s0 = (q == i) ? p.seg_begin[i] : s0;
+        s1 = (q == i) ? p.seg_begin[i + 1] : s1;
+    }
+    const int local = tile - tb, tm = pick(p.tiles_m, q);
+    return {q, (local % tm) * BM, (local / tm) * BN, s0, s1};
+}
+
+// The K loops of one tile, specialised on the operand layouts so that descriptor strides and the choice of
+// TMA boxes are compile-time constants (a run-time layout costs ~10 % on MN-major operands: the two
+// single-thread issue paths are the critical ones).
+struct Pipe {
+    uint32_t tiles, bar_full, bar_empty;
+    volatile int *abort_flag;
+};
+
+template <bool A_MN, bool B_MN>
+__device__ __forceinline__ bool produce_tile(const GroupParams &p, const TileRef &t, const Pipe &pp, uint32_t &stage,
+                                             uint32_t &phase) {
+    for (int s = t.seg0; s < t.seg1; s++) {
+        const CUtensorMap *ma = &p.map_a[s], *mb = &p.map_b[s];
+        const int nkb = p.seg_kb[s];
+        for (int kb = 0; kb < nkb; kb++) {
+            if (!mbar_wait(pp.bar_empty + 8 * stage, phase ^ 1u, pp.abort_flag)) return false;
+            const uint32_t full = pp.bar_full + 8 * stage;
+            const uint32_t sa = pp.tiles + stage * STAGE_BYTES, sb = sa + A_BYTES;
+            mbar_expect_tx(full, STAGE_BYTES);
+            const int k0 = kb * BK;
+            if (A_MN) {
+#pragma unroll
+                for (int j = 0; j < BM / 64; j++) tma_load_2d(sa + j * 8192, ma, full, t.m0 + 64 * j, k0);
+            } else {
+                tma_load_2d(sa, ma, full, k0, t.m0);
+            }
+            if (B_MN) {
+#pragma unroll
+                for (int j = 0; j < BN / 64; j++) tma_load_2d(sb + j * 8192, mb, full, t.n0 + 64 * j, k0);
+            } else {
+                tma_load_2d(sb, mb, full, k0, t.n0);
+            }
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+    }
+    return true;
+}
+
+template <bool A_MN, bool B_MN>
+__device__ __forceinline__ bool mma_tile(const GroupParams &p, const TileRef &t, const Pipe &pp, uint32_t d_tmem,
+                                         uint32_t &stage, uint32_t &phase) {
+    constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) |
+                               ((B_MN ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+    constexpr uint32_t a_step = A_MN ? 2048u : 32u, b_step = B_MN ? 2048u : 32u;   // bytes per 16 k
+    uint32_t first = 0;
+    for (int s = t.seg0; s < t.seg1; s++) {
+        const int nkb = p.seg_kb[s];
+        for (int kb = 0; kb < nkb; kb++) {
+            if (!mbar_wait(pp.bar_full + 8 * stage, phase, pp.abort_flag)) return false;
+            tc_fence_after();
+            const uint32_t sa = pp.tiles + stage * STAGE_BYTES, sb = sa + A_BYTES;
+            const uint32_t a_lo = desc_lo(sa, A_MN ? 8192u : 16u), b_lo = desc_lo(sb, B_MN ? 8192u : 16u);
+#pragma unroll
+            for (int kk = 0; kk < BK / 16; kk++)
+                umma_ss(d_tmem, a_lo + kk * (a_step >> 4), b_lo + kk * (b_step >> 4), idesc, first | (uint32_t)kk);
+            first = 1u;
+            umma_commit(pp.bar_empty + 8 * stage);   // frees the stage once these MMAs have read it
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+    }
+    return true;
+}
+
+__global__ void __launch_bounds__(NUM_THREADS, 1) gemm_group_kernel(const __grid_constant__ GroupParams p) {
     extern __shared__ uint8_t smem_raw[];
     if (gated_off(p.gate)) return;
     const uint32_t raw = smem_u32(smem_raw);
@@ -115,13 +225,15 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
     const uint32_t bar_empty = bar_full + 8 * STAGES;        // STAGES x 8 B
     const uint32_t bar_tfull = bar_empty + 8 * STAGES;       // 2 x 8 B
     const uint32_t bar_tempty = bar_tfull + 16;              // 2 x 8 B
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux + 8 * STAGES * 2 + 32);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(aux + 8 * STAGES * 2 + 40);
+    const uint32_t bar_rfull = bar_tempty + 16;              // RING x 8 B: a tile index has been published
+    const uint32_t bar_rempty = bar_rfull + 8 * RING;        // RING x 8 B: all five readers have taken it
+    uint8_t *aux2 = aux + 8 * STAGES * 2 + 32 + 16 * RING;
+    volatile int *ring = reinterpret_cast<volatile int *>(aux2);              // RING tile indices
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux2 + 4 * RING);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(aux2 + 4 * RING + 8);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + BN - 1) / BN;
-    const int num_tiles = tiles_m * tiles_n;
-    const int num_kb = (p.K + BK - 1) / BK;
+    const int num_tiles = p.tile_begin[p.nprob < MAX_PROBS ? p.nprob : MAX_PROBS];
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; s++) {
@@ -132,97 +244,112 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
             mbar_init(bar_tfull + 8 * b, 1);
             mbar_init(bar_tempty + 8 * b, 4);
         }
+        for (int s = 0; s < RING; s++) {
+            mbar_init(bar_rfull + 8 * s, 1);
+            mbar_init(bar_rempty + 8 * s, 5);       // MMA thread + four epilogue warps
+        }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                     "r"(TMEM_COLS)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
-        // ------------------------------ TMA producer ------------------------------
+        // ------------------------------ tile scheduler + TMA producer ------------------------------
         if (lane == 0) {
-            uint32_t stage = 0, phase = 0;
+            uint32_t stage = 0, phase = 0, slot = 0, rphase = 0;
+            const bool dynamic = p.sched != nullptr;
+            int tile = dynamic ? atomicAdd(p.sched, 1) : (int)blockIdx.x;
             bool alive = true;
-            for (int tile = blockIdx.x; tile < num_tiles && alive; tile += gridDim.x) {
-                const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
-                for (int kb = 0; kb < num_kb; kb++) {
-                    if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { alive = false; break; }
-                    const uint32_t full = bar_full + 8 * stage;
-                    const uint32_t sa = tiles + stage * STAGE_BYTES, sb = sa + A_BYTES;
-                    mbar_expect_tx(full, STAGE_BYTES);
-                    const int k0 = kb * BK;
-                    if (A_MN) {
-#pragma unroll
-                        for (int j = 0; j < BM / 64; j++) tma_load_2d(sa + j * 8192, &map_a, full, m0 + 64 * j, k0);
-                    } else {
-                        tma_load_2d(sa, &map_a, full, k0, m0);
-                    }
-                    if (B_MN) {
-#pragma unroll
-                        for (int j = 0; j < BN / 64; j++) tma_load_2d(sb + j * 8192, &map_b, full, n0 + 64 * j, k0);
-                    } else {
-                        tma_load_2d(sb, &map_b, full, k0, n0);
-                    }
-                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            while (alive) {
+                if (tile >= num_tiles) tile = -1;
+                if (!mbar_wait(bar_rempty + 8 * slot, rphase ^ 1u, abort_flag)) break;
+                ring[slot] = tile;
+                mbar_arrive(bar_rfull + 8 * slot);
+                if (++slot == RING) { slot = 0; rphase ^= 1u; }
+                if (tile < 0) break;
+                // the next index is requested now and first looked at after this tile's loads are issued
+                const int next = dynamic ? atomicAdd(p.sched, 1) : tile + (int)gridDim.x;
+                const TileRef t = locate(p, tile);
+                const uint32_t fl = pick(p.flags, t.q);
+                const Pipe pipe{tiles, bar_full, bar_empty, abort_flag};
+                switch (fl & (F_A_MN | F_B_MN)) {
+                    case 0: alive = produce_tile<false, false>(p, t, pipe, stage, phase); break;
+                    case F_B_MN: alive = produce_tile<false, true>(p, t, pipe, stage, phase); break;
+                    default: alive = produce_tile<true, true>(p, t, pipe, stage, phase); break;
+                }
+                tile = next;
+            }
+            if (dynamic) {
+                // every CTA takes exactly one index past the end; the last CTA to get there re-arms the counter
+                __threadfence();
+                if (atomicAdd(p.sched + 1, 1) == (int)gridDim.x - 1) {
+                    p.sched[0] = 0;
+                    p.sched[1] = 0;
+                    __threadfence();
                 }
             }
         }
     } else if (warp == 1) {
         // ------------------------------ MMA issuer ------------------------------
         if (lane == 0) {
-            constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) |
-                                       ((B_MN ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) |
-                                       ((uint32_t)(BM >> 4) << 24);
-            constexpr uint32_t a_step = A_MN ? 2048u : 32u, b_step = B_MN ? 2048u : 32u;  // bytes per 16 k
-            uint32_t stage = 0, phase = 0, local = 0;
+            uint32_t stage = 0, phase = 0, slot = 0, rphase = 0, local = 0;
             bool alive = true;
-            for (int tile = blockIdx.x; tile < num_tiles && alive; tile += gridDim.x, local++) {
+            while (alive) {
+                if (!mbar_wait(bar_rfull + 8 * slot, rphase, abort_flag)) break;
+                const int tile = ring[slot];
+                mbar_arrive(bar_rempty + 8 * slot);
+                if (++slot == RING) { slot = 0; rphase ^= 1u; }
+                if (tile < 0) break;
+                const TileRef t = locate(p, tile);
+                const uint32_t fl = pick(p.flags, t.q);
                 const uint32_t buf = local & 1u, use = local >> 1;
-                if (!mbar_wait(bar_tempty + 8 * buf, (use & 1u) ^ 1u, abort_flag)) { alive = false; break; }
+                if (!mbar_wait(bar_tempty + 8 * buf, (use & 1u) ^ 1u, abort_flag)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN;
-                for (int kb = 0; kb < num_kb; kb++) {
-                    if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { alive = false; break; }
-                    tc_fence_after();
-                    const uint32_t sa = tiles + stage * STAGE_BYTES, sb = sa + A_BYTES;
-                    const uint32_t a_lo = desc_lo(sa, A_MN ? 8192u : 16u), b_lo = desc_lo(sb, B_MN ? 8192u : 16u);
-#pragma unroll
-                    for (int kk = 0; kk < BK / 16; kk++)
-                        umma_ss(d_tmem, a_lo + kk * (a_step >> 4), b_lo + kk * (b_step >> 4), idesc,
-                                (kb | kk) != 0 ? 1u : 0u);
-                    umma_commit(bar_empty + 8 * stage);   // frees the stage once these MMAs have read it
-                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                const Pipe pipe{tiles, bar_full, bar_empty, abort_flag};
+                switch (fl & (F_A_MN | F_B_MN)) {
+                    case 0: alive = mma_tile<false, false>(p, t, pipe, d_tmem, stage, phase); break;
+                    case F_B_MN: alive = mma_tile<false, true>(p, t, pipe, d_tmem, stage, phase); break;
+                    default: alive = mma_tile<true, true>(p, t, pipe, d_tmem, stage, phase); break;
                 }
                 if (alive) umma_commit(bar_tfull + 8 * buf);   // accumulator complete
+                local++;
             }
         }
     } else {
         // ------------------------------ epilogue ------------------------------
         const int quarter = warp & 3;                 // TMEM lanes 32*quarter .. +31
-        uint32_t local = 0, staged = 0;               // staged: fp32 blocks this warp has sent so far
-        bool alive = true;
-        for (int tile = blockIdx.x; tile < num_tiles && alive; tile += gridDim.x, local++) {
-            const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
+        uint32_t local = 0, staged = 0, slot = 0, rphase = 0;   // staged: fp32 blocks this warp has sent so far
+        while (true) {
+            if (!mbar_wait(bar_rfull + 8 * slot, rphase, abort_flag)) break;
+            const int tile = ring[slot];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_rempty + 8 * slot);
+            if (++slot == RING) { slot = 0; rphase ^= 1u; }
+            if (tile < 0) break;
+            const TileRef t = locate(p, tile);
+            const uint32_t fl = pick(p.flags, t.q);
+            const int Mq = pick(p.M, t.q), Nq = pick(p.N, t.q);
+            const bf16 *bias = pick(p.bias, t.q);
+            const CUtensorMap *mc = &p.map_c[t.q];
             const uint32_t buf = local & 1u, use = local >> 1;
-            if (!mbar_wait(bar_tfull + 8 * buf, use & 1u, abort_flag)) { alive = false; break; }
+            local++;
+            if (!mbar_wait(bar_tfull + 8 * buf, use & 1u, abort_flag)) break;
             tc_fence_after();
-            const int row = m0 + quarter * 32 + lane;
+            const int row = t.m0 + quarter * 32 + lane;
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * BN;
+            bf16 *out_row = reinterpret_cast<bf16 *>(pick(p.C, t.q)) + (long long)row * pick(p.ldc, t.q);
 #pragma unroll 1
             for (int c = 0; c < BN / 32; c++) {
-                const int col0 = n0 + c * 32;
-                if (col0 >= p.N) break;               // uniform across the warp
+                const int col0 = t.n0 + c * 32;
+                if (col0 >= Nq) break;               // uniform across the warp
                 uint32_t r[32];
                 tmem_ld32(taddr + c * 32, r);
-                if (OUT_F32) {
+                if (fl & F_OUT_F32) {
                     // stage the warp's 32 x 32 block (row = lane) with the 128-byte swizzle the tensor map expects
                     const uint32_t buf_s = epi + (uint32_t)(quarter * 2 + (staged & 1u)) * EPI_BUF_BYTES;
                     staged++;
@@ -234,7 +361,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
 #pragma unroll
                         for (int e = 0; e < 4; e++) {
                             v[e] = __uint_as_float(r[4 * j + e]);
-                            if (p.bias && col0 + 4 * j + e < p.N) v[e] += __bfloat162float(p.bias[col0 + 4 * j + e]);
+                            if (bias && col0 + 4 * j + e < Nq) v[e] += __bfloat162float(bias[col0 + 4 * j + e]);
                         }
                         const uint32_t dst = buf_s + lane * 128 + ((j ^ (lane & 7)) << 4);
                         asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v[0]), "f"(v[1]),
@@ -244,33 +371,31 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
                     if (lane == 0) {
-                        if (p.accumulate) tma_reduce_add_2d(&map_c, buf_s, col0, m0 + quarter * 32);
-                        else tma_store_2d(&map_c, buf_s, col0, m0 + quarter * 32);
+                        if (fl & F_ACC) tma_reduce_add_2d(mc, buf_s, col0, t.m0 + quarter * 32);
+                        else tma_store_2d(mc, buf_s, col0, t.m0 + quarter * 32);
                         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                     }
-                } else if (row < p.M) {
-                    {
-                        bf16 *out = reinterpret_cast<bf16 *>(p.C) + (long long)row * p.ldc + col0;
+                } else if (row < Mq) {
+                    bf16 *out = out_row + col0;
 #pragma unroll
-                        for (int j = 0; j < 32; j += 8) {
-                            float v[8];
+                    for (int j = 0; j < 32; j += 8) {
+                        float v[8];
 #pragma unroll
-                            for (int e = 0; e < 8; e++) {
-                                v[e] = __uint_as_float(r[j + e]);
-                                if (p.bias && col0 + j + e < p.N) v[e] += __bfloat162float(p.bias[col0 + j + e]);
+                        for (int e = 0; e < 8; e++) {
+                            v[e] = __uint_as_float(r[j + e]);
+                            if (bias && col0 + j + e < Nq) v[e] += __bfloat162float(bias[col0 + j + e]);
+                        }
+                        if (col0 + j + 7 < Nq) {
+                            uint32_t w[4];
+#pragma unroll
+                            for (int e = 0; e < 4; e++) {
+                                __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]);
+                                w[e] = *reinterpret_cast<uint32_t *>(&h);
                             }
-                            if (col0 + j + 7 < p.N) {
-                                uint32_t w[4];
-#pragma unroll
-                                for (int e = 0; e < 4; e++) {
-                                    __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]);
-                                    w[e] = *reinterpret_cast<uint32_t *>(&h);
-                                }
-                                *reinterpret_cast<uint4 *>(out + j) = make_uint4(w[0], w[1], w[2], w[3]);
-                            } else {
-                                for (int e = 0; e < 8; e++)
-                                    if (col0 + j + e < p.N) out[j + e] = __float2bfloat16_rn(v[e]);
-                            }
+                            *reinterpret_cast<uint4 *>(out + j) = make_uint4(w[0], w[1], w[2], w[3]);
+                        } else {
+                            for (int e = 0; e < 8; e++)
+                                if (col0 + j + e < Nq) out[j + e] = __float2bfloat16_rn(v[e]);
                         }
                     }
                 }
@@ -281,7 +406,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
         }
     }
 
-    if (OUT_F32 && warp >= 2 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    if (warp >= 2 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     __syncwarp();
     if (*abort_flag) {
         // give copies that are still in flight time to land before shared memory is released
@@ -292,30 +417,15 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+        tmem_dealloc(tmem_base, TMEM_COLS);
     }
-}
-
-// ---------------------------------------------------------------------------------------------
-// host side
-// ---------------------------------------------------------------------------------------------
-template <bool A_MN, bool B_MN, bool OUT_F32>
-int launch(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &mc, const TcParams &p, cudaStream_t st) {
-    auto kernel = gemm_tc_kernel<A_MN, B_MN, OUT_F32>;
-    static bool configured = false;
-    if (!configured) {
-        if (!cuda_ok(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES)))
-            return STREAMBP_E_CUDA;
-        configured = true;
-    }
-    const int tiles = ((p.M + BM - 1) / BM) * ((p.N + BN - 1) / BN);
-    const int grid = tiles < sm_count() ? tiles : sm_count();
-    SBP_LAUNCH(kernel, grid, NUM_THREADS, SMEM_BYTES, st, ma, mb, mc, p);
-    return STREAMBP_OK;
 }
 
 }  // namespace
 
+// ---------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------
 bool gemm_tc_supported(GemmOp op, int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb, int64_t ldc,
                        const void *A, const void *B, const void *C, bool c_is_f32) {
     (void)op;
@@ -327,28 +437,97 @@ bool gemm_tc_supported(GemmOp op, int64_t M, int64_t N, int64_t K, int64_t lda, 
     return tensor_maps_available();
 }
 
+bool gemm_tc_group_supported(const GemmProb *probs, int n) {
+    if (n < 1 || n > MAX_PROBS) return false;
+    int segs = 0;
+    for (int i = 0; i < n; i++) {
+        const GemmProb &g = probs[i];
+        if (g.nseg < 1 || g.nseg > 3) return false;
+        if (!g.c_is_f32 && g.accumulate) return false;
+        segs += g.nseg;
+        for (int s = 0; s < g.nseg; s++)
+            if (!gemm_tc_supported(g.op, g.M, g.N, g.seg[s].K, g.seg[s].lda, g.seg[s].ldb, g.ldc, g.seg[s].A,
+                                   g.seg[s].B, g.C, g.c_is_f32))
+                return false;
+    }
+    return segs <= MAX_SEGS;
+}
+
+int gemm_tc_group(const GemmProb *probs, int n, int *sched, cudaStream_t st) {
+    if (!gemm_tc_group_supported(probs, n)) return STREAMBP_E_SHAPE;
+    // longest tiles first: with a dynamic schedule the short tiles then fill the gaps the long ones leave
+    int order[MAX_PROBS];
+    int64_t cost[MAX_PROBS];
+    for (int i = 0; i < n; i++) {
+        order[i] = i;
+        cost[i] = 0;
+        for (int s = 0; s < probs[i].nseg; s++) cost[i] += (probs[i].seg[s].K + BK - 1) / BK;
+    }
+    for (int i = 1; i < n; i++)
+        for (int j = i; j > 0 && cost[order[j]] > cost[order[j - 1]]; j--) {
+            const int t = order[j]; order[j] = order[j - 1]; order[j - 1] = t;
+        }
+    GroupParams p;
+    memset(&p, 0, sizeof(p));
+    p.nprob = n;
+    int seg = 0;
+    int64_t tiles = 0;
+    for (int i = 0; i < n; i++) {
+        const GemmProb &g = probs[order[i]];
+        p.seg_begin[i] = seg;
+        p.tile_begin[i] = (int)tiles;
+        const bool a_mn = g.op == OP_TN, b_mn = g.op != OP_NT;
+        for (int s = 0; s < g.nseg; s++, seg++) {
+            const GemmSeg &e = g.seg[s];
+            bool ok;
+            // K-major operands: [rows][64 k] boxes; MN-major operands: [64 k][64 mn] boxes
+            if (a_mn) ok = make_tensor_map(&p.map_a[seg], e.A, e.K, g.M, e.lda, 64, BK, false);
+            else ok = make_tensor_map(&p.map_a[seg], e.A, g.M, e.K, e.lda, BK, BM, false);
+            if (b_mn) ok = ok && make_tensor_map(&p.map_b[seg], e.B, e.K, g.N, e.ldb, 64, BK, false);
+            else ok = ok && make_tensor_map(&p.map_b[seg], e.B, g.N, e.K, e.ldb, BK, BN, false);
+            if (!ok) return STREAMBP_E_CUDA;
+            p.seg_kb[seg] = (int)((e.K + BK - 1) / BK);
+        }
+        if (g.c_is_f32) {
+            if (!make_tensor_map(&p.map_c[i], g.C, g.M, g.N, g.ldc, 32, 32, true)) return STREAMBP_E_CUDA;
+        } else {
+            p.map_c[i] = p.map_a[p.seg_begin[i]];   // unused by bf16 outputs
+        }
+        p.tiles_m[i] = (int)((g.M + BM - 1) / BM);
+        p.M[i] = (int)g.M;
+        p.N[i] = (int)g.N;
+        p.C[i] = g.C;
+        p.ldc[i] = g.ldc;
+        p.bias[i] = g.bias;
+        p.flags[i] = (a_mn ? F_A_MN : 0u) | (b_mn ? F_B_MN : 0u) | (g.c_is_f32 ? F_OUT_F32 : 0u) |
+                     (g.accumulate ? F_ACC : 0u);
+        tiles += (int64_t)p.tiles_m[i] * ((g.N + BN - 1) / BN);
+        if (tiles > (1ll << 30)) return STREAMBP_E_SHAPE;
+    }
+    for (int i = n; i <= MAX_PROBS; i++) {
+        p.seg_begin[i] = seg;
+        p.tile_begin[i] = (int)tiles;
+    }
+    p.sched = sched;
+    p.gate = call_state().gate;
+    static bool configured = false;
+    if (!configured) {
+        if (!cuda_ok(cudaFuncSetAttribute(gemm_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES)))
+            return STREAMBP_E_CUDA;
+        configured = true;
+    }
+    const int grid = tiles < sm_count() ? (int)tiles : sm_count();
+    SBP_LAUNCH(gemm_group_kernel, grid, NUM_THREADS, SMEM_BYTES, st, p);
+    return STREAMBP_OK;
+}
+
 int gemm_tc(GemmOp op, int64_t M, int64_t N, int64_t K, const bf16 *A, int64_t lda, const bf16 *B, int64_t ldb,
             void *C, int64_t ldc, bool c_is_f32, const bf16 *bias, bool accumulate, cudaStream_t st) {
-    CUtensorMap ma, mb;
-    bool ok = true;
-    switch (op) {
-        case OP_NT:   // A [M,K] K-major, B [N,K] K-major
-            ok = make_tensor_map(&ma, A, M, K, lda, BK, BM, false) && make_tensor_map(&mb, B, N, K, ldb, BK, BN, false);
-            break;
-        case OP_NN:   // A [M,K] K-major, B [K,N] N-major
-            ok = make_tensor_map(&ma, A, M, K, lda, BK, BM, false) && make_tensor_map(&mb, B, K, N, ldb, 64, BK, false);
-            break;
-        case OP_TN:   // A [K,M] M-major, B [K,N] N-major
-            ok = make_tensor_map(&ma, A, K, M, lda, 64, BK, false) && make_tensor_map(&mb, B, K, N, ldb, 64, BK, false);
-            break;
-    }
-    CUtensorMap mc = ma;   // unused by the bf16-output kernels
-    if (ok && c_is_f32) ok = make_tensor_map(&mc, C, M, N, ldc, 32, 32, true);
-    if (!ok) return STREAMBP_E_CUDA;
-    TcParams p{(int)M, (int)N, (int)K, C, (long long)ldc, bias, accumulate ? 1 : 0, call_state().gate};
-    if (op == OP_NT) return c_is_f32 ? launch<false, false, true>(ma, mb, mc, p, st) : launch<false, false, false>(ma, mb, mc, p, st);
-    if (op == OP_NN) return c_is_f32 ? launch<false, true, true>(ma, mb, mc, p, st) : launch<false, true, false>(ma, mb, mc, p, st);
-    return c_is_f32 ? launch<true, true, true>(ma, mb, mc, p, st) : launch<true, true, false>(ma, mb, mc, p, st);
+    GemmProb g;
+    g.op = op; g.M = M; g.N = N; g.nseg = 1;
+    g.seg[0] = GemmSeg{A, lda, B, ldb, K};
+    g.C = C; g.ldc = ldc; g.c_is_f32 = c_is_f32; g.bias = bias; g.accumulate = accumulate;
+    return gemm_tc_group(&g, 1, nullptr, st);
 }
 
 int gemm_tc_take_fault() { return take_fault_local(); }

@@ -94,9 +94,12 @@ int kv_prologue(const streambp_layer_cfg &c, const streambp_layer_weights &w, co
     for (int64_t r0 = 0; r0 < T_; r0 += cn) {
         const int64_t n = (T_ - r0 < cn) ? T_ - r0 : cn;
         SBP_TRY(rmsnorm_fwd<T>(X + r0 * d, nullptr, (const T *)w.g1, c.rms_eps, n, d, s.h1, s.rstd1, nullptr, st));
-        SBP_TRY((mm<T, float>(OP_NT, n, dkv, d, s.h1, d, (const T *)w.wk, d, s.fa, dkv, (const T *)w.bk, false, st)));
+        const MmProb<T> kv[2] = {
+            mm_prob<T>(OP_NT, n, dkv, d, s.h1, d, (const T *)w.wk, d, s.fa, dkv, true, (const T *)w.bk, false),
+            mm_prob<T>(OP_NT, n, dkv, d, s.h1, d, (const T *)w.wv, d, s.V + r0 * dkv, dkv, sizeof(T) == 4,
+                       (const T *)w.bv, false)};
+        SBP_TRY(mm_group<T>(kv, 2, st));
         SBP_TRY(rope_apply<T>(s.fa, s.cs + r0 * dh, n, Hkv, dh, false, s.K + r0 * dkv, st));
-        SBP_TRY((mm<T, T>(OP_NT, n, dkv, d, s.h1, d, (const T *)w.wv, d, s.V + r0 * dkv, dkv, (const T *)w.bv, false, st)));
     }
     return STREAMBP_OK;
 }
@@ -123,8 +126,10 @@ int chunk_forward(const streambp_layer_cfg &c, const streambp_layer_weights &w, 
     }));
     SBP_TRY((mm<T, float>(OP_NT, n, d, dq, s.O, dq, (const T *)w.wo, dq, s.fa, d, nullptr, false, st)));
     SBP_TRY(rmsnorm_fwd<T>(Xi, s.fa, (const T *)w.g2, c.rms_eps, n, d, s.h2, s.rstd2, s.r, st));
-    SBP_TRY((mm<T, T>(OP_NT, n, I, d, s.h2, d, (const T *)w.w_gate, d, s.g, I, nullptr, false, st)));
-    SBP_TRY((mm<T, T>(OP_NT, n, I, d, s.h2, d, (const T *)w.w_up, d, s.u, I, nullptr, false, st)));
+    const MmProb<T> gu[2] = {
+        mm_prob<T>(OP_NT, n, I, d, s.h2, d, (const T *)w.w_gate, d, s.g, I, sizeof(T) == 4, nullptr, false),
+        mm_prob<T>(OP_NT, n, I, d, s.h2, d, (const T *)w.w_up, d, s.u, I, sizeof(T) == 4, nullptr, false)};
+    SBP_TRY(mm_group<T>(gu, 2, st));
     SBP_TRY(swiglu_fwd<T>(s.g, s.u, n * I, s.m, st));
     return STREAMBP_OK;
 }
@@ -142,6 +147,7 @@ int layer_forward(const streambp_layer_cfg &c, const streambp_layer_weights &w, 
     const Segments seg(cu_seqlens, n_seqs, T_);
     const int64_t cn = chunk < T_ ? chunk : T_;
     LayerWs<T> s = plan<T>(c, T_, chunk, ws);
+    const SchedScope sched(s.hdr);
     const int d = c.d_model;
     const int64_t I = c.d_ff;
     SBP_TRY(kv_prologue<T>(c, w, X, T_, cn, pos0, seg, s, st));
@@ -161,6 +167,7 @@ int layer_backward(const streambp_layer_cfg &c, const streambp_layer_weights &w,
     const Segments seg(cu_seqlens, n_seqs, T_);
     const int64_t cn = chunk < T_ ? chunk : T_;
     LayerWs<T> s = plan<T>(c, T_, chunk, ws);
+    const SchedScope sched(s.hdr);
     const int d = c.d_model, dh = c.head_dim, Hq = c.n_q_heads, Hkv = c.n_kv_heads;
     const int64_t dq = (int64_t)Hq * dh, dkv = (int64_t)Hkv * dh, I = c.d_ff;
     constexpr bool kF32 = sizeof(T) == 4;
@@ -189,18 +196,26 @@ int layer_backward(const streambp_layer_cfg &c, const streambp_layer_weights &w,
         SBP_TRY((mm<T, float>(OP_TN, d, I, n, dYi, d, s.m, I, G.w_down, I, nullptr, acc, st)));       // dWd += dY^T m
         SBP_TRY((mm<T, T>(OP_NN, n, I, d, dYi, d, (const T *)w.w_down, I, s.m, I, nullptr, false, st)));  // dm = dY Wd
         SBP_TRY(swiglu_bwd<T>(s.m, s.g, s.u, n * I, st));                                             // g := dg, u := du
-        SBP_TRY((mm<T, float>(OP_TN, I, d, n, s.g, I, s.h2, d, G.w_gate, d, nullptr, acc, st)));
-        SBP_TRY((mm<T, float>(OP_TN, I, d, n, s.u, I, s.h2, d, G.w_up, d, nullptr, acc, st)));
-        SBP_TRY((mm<T, float>(OP_NN, n, d, I, s.g, I, (const T *)w.w_gate, d, s.fa, d, nullptr, false, st)));
-        SBP_TRY((mm<T, float>(OP_NN, n, d, I, s.u, I, (const T *)w.w_up, d, s.fa, d, nullptr, true, st)));   // dh2
+        {   // dWg += dg^T h2, dWu += du^T h2, dh2 = dg Wg + du Wu: all three need only dg, du, h2
+            MmProb<T> pr[3] = {
+                mm_prob<T>(OP_TN, I, d, n, s.g, I, s.h2, d, G.w_gate, d, true, nullptr, acc),
+                mm_prob<T>(OP_TN, I, d, n, s.u, I, s.h2, d, G.w_up, d, true, nullptr, acc),
+                mm_prob<T>(OP_NN, n, d, I, s.g, I, (const T *)w.w_gate, d, s.fa, d, true, nullptr, false)};
+            mm_add_seg<T>(pr[2], I, s.u, I, (const T *)w.w_up, d);
+            SBP_TRY(mm_group<T>(pr, 3, st));
+        }
         // dr = dY + norm2_bwd(dh2)
         SBP_TRY(rmsnorm_bwd<T>(s.fa, nullptr, s.r, s.rstd2, (const T *)w.g2, dYi, nullptr, n, d, s.dr,
                                kF32 ? nullptr : s.dr_s, G.g2, s.partials, st));
         const T *dr_op = kF32 ? reinterpret_cast<const T *>(s.dr) : s.dr_s;
 
         // ---- attention output projection backward ----
-        SBP_TRY((mm<T, float>(OP_TN, d, dq, n, dr_op, d, s.O, dq, G.wo, dq, nullptr, acc, st)));       // dWo += dr^T O
-        SBP_TRY((mm<T, T>(OP_NN, n, dq, d, dr_op, d, (const T *)w.wo, dq, s.dO, dq, nullptr, false, st)));  // dO = dr Wo
+        {   // dWo += dr^T O, dO = dr Wo
+            const MmProb<T> pr[2] = {
+                mm_prob<T>(OP_TN, d, dq, n, dr_op, d, s.O, dq, G.wo, dq, true, nullptr, acc),
+                mm_prob<T>(OP_NN, n, dq, d, dr_op, d, (const T *)w.wo, dq, s.dO, dq, sizeof(T) == 4, nullptr, false)};
+            SBP_TRY(mm_group<T>(pr, 2, st));
+        }
 
         // ---- partitioned attention backward: dQ (into fa), dK/dV prefix += ----
         SBP_TRY(seg.for_each(r0, r0 + n, [&](int64_t a, int64_t e, int64_t q_seq) {
@@ -212,24 +227,26 @@ int layer_backward(const streambp_layer_cfg &c, const streambp_layer_weights &w,
                                s.dK + q_seq * dkv, s.dV + q_seq * dkv, st);
         }));
 
-        // ---- Q projection backward ----
+        // ---- Q, K, V projection backward (this chunk's dK/dV rows are final now) ----
         T *dq_s = s.Q;  // Q is dead after the attention backward
         SBP_TRY(rope_apply<T>(s.fa, s.cs + r0 * dh, n, Hq, dh, true, dq_s, st));
-        SBP_TRY((mm<T, float>(OP_TN, dq, d, n, dq_s, dq, s.h1, d, G.wq, d, nullptr, acc, st)));
-        if (c.qkv_bias) SBP_TRY(colsum<T>(dq_s, n, (int)dq, G.bq, true, s.partials, st));
-        SBP_TRY((mm<T, float>(OP_NN, n, d, dq, dq_s, dq, (const T *)w.wq, d, s.fa, d, nullptr, false, st)));   // dh1
-
-        // ---- K/V projection backward of this chunk's rows (their dK/dV are final now) ----
         SBP_TRY(rope_apply<T>(s.dK + r0 * dkv, s.cs + r0 * dh, n, Hkv, dh, true, s.dk_s, st));
         SBP_TRY(cast_from_f32<T>(s.dV + r0 * dkv, n * dkv, s.dv_s, st));
-        SBP_TRY((mm<T, float>(OP_TN, dkv, d, n, s.dk_s, dkv, s.h1, d, G.wk, d, nullptr, acc, st)));
-        SBP_TRY((mm<T, float>(OP_TN, dkv, d, n, s.dv_s, dkv, s.h1, d, G.wv, d, nullptr, acc, st)));
+        {   // dWq, dWk, dWv and dh1 = dq Wq + dk Wk + dv Wv
+            MmProb<T> pr[4] = {
+                mm_prob<T>(OP_TN, dq, d, n, dq_s, dq, s.h1, d, G.wq, d, true, nullptr, acc),
+                mm_prob<T>(OP_TN, dkv, d, n, s.dk_s, dkv, s.h1, d, G.wk, d, true, nullptr, acc),
+                mm_prob<T>(OP_TN, dkv, d, n, s.dv_s, dkv, s.h1, d, G.wv, d, true, nullptr, acc),
+                mm_prob<T>(OP_NN, n, d, dq, dq_s, dq, (const T *)w.wq, d, s.fa, d, true, nullptr, false)};
+            mm_add_seg<T>(pr[3], dkv, s.dk_s, dkv, (const T *)w.wk, d);
+            mm_add_seg<T>(pr[3], dkv, s.dv_s, dkv, (const T *)w.wv, d);
+            SBP_TRY(mm_group<T>(pr, 4, st));
+        }
         if (c.qkv_bias) {
+            SBP_TRY(colsum<T>(dq_s, n, (int)dq, G.bq, true, s.partials, st));
             SBP_TRY(colsum<T>(s.dk_s, n, (int)dkv, G.bk, true, s.partials, st));
             SBP_TRY(colsum<T>(s.dv_s, n, (int)dkv, G.bv, true, s.partials, st));
         }
-        SBP_TRY((mm<T, float>(OP_NN, n, d, dkv, s.dk_s, dkv, (const T *)w.wk, d, s.fa, d, nullptr, true, st)));
-        SBP_TRY((mm<T, float>(OP_NN, n, d, dkv, s.dv_s, dkv, (const T *)w.wv, d, s.fa, d, nullptr, true, st)));
 
         // ---- dX = dr + norm1_bwd(dh1) ----
         SBP_TRY(rmsnorm_bwd<T>(s.fa, Xi, nullptr, s.rstd1, (const T *)w.g1, nullptr, s.dr, n, d, nullptr, dX + r0 * d,

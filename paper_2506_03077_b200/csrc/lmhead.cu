@@ -46,6 +46,7 @@ int lmhead_backward(const streambp_head_cfg &c, const T *g_final, const T *w_voc
                     float *d_g_final, void *ws, cudaStream_t st, const RlRows *rl, float *ell) {
     const int64_t cn = chunk < T_ ? chunk : T_;
     HeadWs<T> s = plan<T>(c, T_, chunk, ws);
+    const SchedScope sched(s.hdr);
     const int d = c.d_model;
     const int64_t V = c.vocab;
     // N is global: it is counted before the chunk loop so that every chunk scales by the same 1/N
@@ -77,8 +78,11 @@ int lmhead_backward(const streambp_head_cfg &c, const T *g_final, const T *w_voc
         else
             SBP_TRY(ce_rows<T>(s.z, labels + r0, n, V, c.ignore_index, s.hdr, s.dz, s.row_loss, st));
         SBP_TRY(loss_accumulate(s.row_loss, n, s.hdr, st));
-        SBP_TRY((mm<T, float>(OP_TN, V, d, n, s.dz, V, s.hn, d, d_w_vocab, d, nullptr, acc, st)));          // dW += dZ^T hn
-        SBP_TRY((mm<T, float>(OP_NN, n, d, V, s.dz, V, w_vocab, d, s.dhn, d, nullptr, false, st)));         // dhn = dZ W
+        {   // dW += dZ^T hn and dhn = dZ W need only dZ: one launch, the few long dhn tiles first
+            const MmProb<T> pr[2] = {mm_prob<T>(OP_TN, V, d, n, s.dz, V, s.hn, d, d_w_vocab, d, true, nullptr, acc),
+                                     mm_prob<T>(OP_NN, n, d, V, s.dz, V, w_vocab, d, s.dhn, d, true, nullptr, false)};
+            SBP_TRY(mm_group<T>(pr, 2, st));
+        }
         SBP_TRY(rmsnorm_bwd<T>(s.dhn, Hi, nullptr, s.rstd, g_final, nullptr, nullptr, n, d, nullptr, dH + r0 * d,
                                d_g_final, s.partials, st));
     }

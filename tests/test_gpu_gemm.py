@@ -88,3 +88,81 @@ def test_tensor_core_product_strided_views():
     ref = A.double().cpu() @ Bm.double().cpu().T
     assert ((C.double().cpu() - ref).norm() / ref.norm()) < 1e-5
     assert torch.count_nonzero(Cbuf[:, :8]) == 0 and torch.count_nonzero(Cbuf[:, 408:]) == 0
+
+
+def _operands(op, M, N, K, gen):
+    sa, sb = shapes(op, M, N, K)
+    return (torch.randn(sa, generator=gen).bfloat16().cuda(), torch.randn(sb, generator=gen).bfloat16().cuda())
+
+
+@pytest.mark.parametrize("dynamic", [False, True])
+def test_grouped_products_mixed_layouts(dynamic):
+    """Four problems of different layouts, output types and tile lengths in one launch: two weight-gradient
+    shaped accumulations, one input gradient summed over three K segments, one bf16 forward product; every
+    size ragged against the 128 x 256 x 64 tile.  Each output equals the fp64 product of the same bf16
+    operands, with either tile schedule, and the scheduler's counters are left at zero."""
+    gen = torch.Generator(device="cpu").manual_seed(11)
+    n = 328
+    a1, b1 = _operands(B.OP_TN, 520, 264, n, gen)
+    a2, b2 = _operands(B.OP_TN, 136, 264, n, gen)
+    segs = [_operands(B.OP_NN, n, 264, K, gen) for K in (520, 136, 72)]
+    a4, b4 = _operands(B.OP_NT, n, 1000, 264, gen)
+    base1 = torch.randn(520, 264, generator=gen).cuda()
+    C1, C2 = base1.clone(), torch.full((136, 264), float("nan"), device="cuda")
+    C3 = torch.full((n, 264), float("nan"), device="cuda")
+    C4 = torch.full((n, 1000), float("nan"), device="cuda", dtype=torch.bfloat16)
+    sched = torch.zeros(2, dtype=torch.int32, device="cuda") if dynamic else None
+    B.gemm_grouped([(B.OP_TN, [(a1, b1)], C1, True), (B.OP_TN, [(a2, b2)], C2, False),
+                    (B.OP_NN, segs, C3, False), (B.OP_NT, [(a4, b4)], C4, False)], sched)
+    torch.cuda.synchronize()
+    r1 = ref_product(B.OP_TN, a1, b1) + base1.double().cpu()
+    r2 = ref_product(B.OP_TN, a2, b2)
+    r3 = sum(ref_product(B.OP_NN, a, b) for a, b in segs)
+    r4 = ref_product(B.OP_NT, a4, b4)
+    for got, ref, tol in ((C1, r1, 2e-6), (C2, r2, 2e-6), (C3, r3, 2e-6), (C4, r4, 4e-3)):
+        assert torch.isfinite(got).all()
+        assert (got.double().cpu() - ref).norm() / ref.norm() < tol
+    if dynamic:
+        assert sched.tolist() == [0, 0]
+
+
+def test_grouped_products_schedule_invariance():
+    """More tiles than CTAs, long and short tiles mixed: the dynamic schedule gives bit-identical results to
+    the static one and to one launch per problem, twice in a row with the same counters."""
+    gen = torch.Generator(device="cpu").manual_seed(12)
+    n = 1024
+    dg, h2 = _operands(B.OP_TN, 4096, 1024, n, gen)          # dWg += dg^T h2
+    du = torch.randn(n, 4096, generator=gen).bfloat16().cuda()
+    wg = torch.randn(4096, 1024, generator=gen).bfloat16().cuda()
+    wu = torch.randn(4096, 1024, generator=gen).bfloat16().cuda()
+    sched = torch.zeros(2, dtype=torch.int32, device="cuda")
+    outs = []
+    for mode in ("static", "dynamic", "dynamic", "single"):
+        dWg = torch.ones(4096, 1024, device="cuda")
+        dWu = torch.ones(4096, 1024, device="cuda")
+        dh2 = torch.full((n, 1024), float("nan"), device="cuda")
+        if mode == "single":
+            B.gemm(B.OP_TN, dg, h2, dWg, accumulate=True, engine=2)
+            B.gemm(B.OP_TN, du, h2, dWu, accumulate=True, engine=2)
+            B.gemm_grouped([(B.OP_NN, [(dg, wg), (du, wu)], dh2, False)])
+        else:
+            B.gemm_grouped([(B.OP_TN, [(dg, h2)], dWg, True), (B.OP_TN, [(du, h2)], dWu, True),
+                            (B.OP_NN, [(dg, wg), (du, wu)], dh2, False)], sched if mode == "dynamic" else None)
+        torch.cuda.synchronize()
+        outs.append((dWg, dWu, dh2))
+    assert sched.tolist() == [0, 0]
+    ref = ref_product(B.OP_NN, dg, wg) + ref_product(B.OP_NN, du, wu)
+    assert (outs[0][2].double().cpu() - ref).norm() / ref.norm() < 1e-5     # fp32 sum over K = 8192
+    for o in outs[1:]:
+        for a, b in zip(outs[0], o):
+            assert torch.equal(a, b)
+
+
+def test_grouped_products_rejects_bad_arguments():
+    a = torch.zeros(64, 64, dtype=torch.bfloat16, device="cuda")
+    c16 = torch.zeros(64, 64, dtype=torch.bfloat16, device="cuda")
+    c32 = torch.zeros(64, 64, device="cuda")
+    assert B.gemm_grouped([(B.OP_NT, [(a, a)], c16, True)], check=False) == B.E_DTYPE       # bf16 C cannot accumulate
+    assert B.gemm_grouped([(B.OP_NT, [(a, a)], c32, False)] * 5, check=False) == B.E_SHAPE   # more than 4 problems
+    odd = torch.zeros(64, 68, dtype=torch.bfloat16, device="cuda")[:, :64]                   # pitch 68: not 16-byte rows
+    assert B.gemm_grouped([(B.OP_NT, [(odd, a)], c32, False)], check=False) == B.E_SHAPE
