@@ -132,6 +132,7 @@ __global__ void __launch_bounds__(FWD16_THREADS, 1)
             }
         }
     } else if (warp == 1) {
+        // softmax-bound kernel: a single issuing lane leaves the other warps more issue slots
         if (lane == 0) {
             constexpr uint32_t idesc_s = make_idesc(TILE, TILE, false, false);
             constexpr uint32_t idesc_pv = make_idesc(TILE, TILE, false, true);
@@ -294,6 +295,11 @@ __global__ void __launch_bounds__(FWD16_THREADS, 1)
 // product needs -- and only then combine it with dP into dS.  The MMA thread interleaves accordingly:
 // dV_i, then S_{i+1} (its buffer is free again), then dK_i, then dP_{i+1}; the tensor pipe therefore
 // always has the next tile's products queued while the softmax warps work.
+// Timelines taken with clock64 stamps inside the kernels showed what bounds them: not the exponential unit
+// (replacing half of the exp2 by a polynomial on the FMA pipe made both kernels slower) but (a) the latency
+// of refilling a shared-memory stage that is released late -- hence the three-stage K ring of the dQ kernel
+// and the separate release of Q and dO stages in the dK/dV kernel -- and (b) the rate at which one thread
+// can issue tcgen05.mma while arithmetic warps share its scheduler -- hence the warp-uniform issue loops.
 // ---------------------------------------------------------------------------------------------
 struct BwdParams {
     int n;
@@ -307,6 +313,8 @@ struct BwdParams {
 };
 
 constexpr int BWD_SMEM = 6 * TILE_BYTES + 4 * TILE * 4 /* lse, delta x 2 stages */ + 1024 + 256;
+constexpr int DQ_KSTAGES = 3;
+constexpr int DQ_SMEM = (4 + DQ_KSTAGES) * TILE_BYTES + 1024 + 256;   // Q, dO, K x 3, V x 2
 constexpr int BWD_THREADS = 64 + 512;
 constexpr int HALF = 64;
 
@@ -330,10 +338,10 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
     float *s_delta = s_lse + 2 * TILE;                        // [2][128]
     uint8_t *aux = tail + 4 * TILE * 4;
     const uint32_t bars = smem_u32(aux);
-    const uint32_t kv_full = bars, in_full = bars + 8, in_empty = bars + 24, s_full = bars + 40, dp_full = bars + 48,
-                   p1_full = bars + 56, p2_full = bars + 64, acc_full = bars + 72;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux + 80);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(aux + 88);
+    const uint32_t kv_full = bars, in_full = bars + 8, q_empty = bars + 24, s_full = bars + 40, dp_full = bars + 48,
+                   p1_full = bars + 56, p2_full = bars + 64, acc_full = bars + 72, do_empty = bars + 80;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux + 96);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(aux + 104);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = blockIdx.y, G = p.Hq / p.Hkv;
@@ -347,7 +355,8 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
         mbar_init(kv_full, 1);
         for (int s = 0; s < 2; s++) {
             mbar_init(in_full + 8 * s, 1);
-            mbar_init(in_empty + 8 * s, 1);
+            mbar_init(q_empty + 8 * s, 1);
+            mbar_init(do_empty + 8 * s, 1);
         }
         mbar_init(s_full, 1);
         mbar_init(dp_full, 1);
@@ -374,11 +383,26 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
             tma_load_2d(sV, &map_v, kv_full, g * TILE, (int)k_abs0);
             tma_load_2d(sV + HALF_BYTES, &map_v, kv_full, g * TILE + 64, (int)k_abs0);
         }
+        // A stage's dO tile is free once dV of its previous user is done, its Q tile (and the lse / delta rows)
+        // once dK is done; the copies are issued before the row loads so that their latencies overlap.
         for (int it = 0; it < iters; it++) {
             const int h = g * G + it / per_head, qt0 = (first_qt + it % per_head) * TILE;
             const uint32_t st = it & 1, ph = (it >> 1) & 1;
+            const uint32_t full = in_full + 8 * st;
             int ok = 1;
-            if (lane == 0) ok = mbar_wait(in_empty + 8 * st, ph ^ 1u, abort_flag) ? 1 : 0;
+            if (lane == 0) {
+                ok = mbar_wait(do_empty + 8 * st, ph ^ 1u, abort_flag) ? 1 : 0;
+                if (ok) {
+                    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(full), "r"(2 * TILE_BYTES) : "memory");
+                    tma_load_2d(sdO + st * TILE_BYTES, &map_do, full, h * TILE, qt0);
+                    tma_load_2d(sdO + st * TILE_BYTES + HALF_BYTES, &map_do, full, h * TILE + 64, qt0);
+                    ok = mbar_wait(q_empty + 8 * st, ph ^ 1u, abort_flag) ? 1 : 0;
+                }
+                if (ok) {
+                    tma_load_2d(sQ + st * TILE_BYTES, &map_q, full, h * TILE, qt0);
+                    tma_load_2d(sQ + st * TILE_BYTES + HALF_BYTES, &map_q, full, h * TILE + 64, qt0);
+                }
+            }
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
 #pragma unroll
@@ -388,65 +412,58 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
                 s_delta[st * TILE + col] = r < p.n ? p.delta[(long long)h * p.n + r] * p.scale : 0.f;
             }
             __syncwarp();
-            if (lane == 0) {
-                const uint32_t full = in_full + 8 * st;
-                mbar_expect_tx(full, 2 * TILE_BYTES);
-                tma_load_2d(sQ + st * TILE_BYTES, &map_q, full, h * TILE, qt0);
-                tma_load_2d(sQ + st * TILE_BYTES + HALF_BYTES, &map_q, full, h * TILE + 64, qt0);
-                tma_load_2d(sdO + st * TILE_BYTES, &map_do, full, h * TILE, qt0);
-                tma_load_2d(sdO + st * TILE_BYTES + HALF_BYTES, &map_do, full, h * TILE + 64, qt0);
-            }
+            if (lane == 0) mbar_arrive(full);      // publishes the rows; the phase completes when the tiles have landed too
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            constexpr uint32_t idesc_kk = make_idesc(TILE, TILE, false, false);     // both operands K-major
-            constexpr uint32_t idesc_acc = make_idesc(TILE, TILE, false, true);     // B MN-major (N = head dims)
-            bool alive = mbar_wait(kv_full, 0, abort_flag);
-            const uint32_t k_lo = klo(sK), v_lo = klo(sV);
-            auto issue_st = [&](int it) {      // S^T = K Q^T
-                const uint32_t q_lo = klo(sQ + (it & 1) * TILE_BYTES);
+        // the whole warp runs the issue loop; each MMA / commit executes in one elected lane
+        constexpr uint32_t idesc_kk = make_idesc(TILE, TILE, false, false);     // both operands K-major
+        constexpr uint32_t idesc_acc = make_idesc(TILE, TILE, false, true);     // B MN-major (N = head dims)
+        bool alive = mbar_wait_warp(kv_full, 0, abort_flag);
+        const uint32_t k_lo = klo(sK), v_lo = klo(sV);
+        auto issue_st = [&](int it) {      // S^T = K Q^T
+            const uint32_t q_lo = klo(sQ + (it & 1) * TILE_BYTES);
 #pragma unroll
-                for (int kk = 0; kk < 8; kk++) umma_ss(tST, k_lo + kstep(kk), q_lo + kstep(kk), idesc_kk, kk != 0);
-                umma_commit(s_full);
-            };
-            auto issue_dpt = [&](int it) {     // dP^T = V dO^T
-                const uint32_t do_lo = klo(sdO + (it & 1) * TILE_BYTES);
+            for (int kk = 0; kk < 8; kk++) umma_ss_w(tST, k_lo + kstep(kk), q_lo + kstep(kk), idesc_kk, kk != 0);
+            umma_commit_w(s_full);
+        };
+        auto issue_dpt = [&](int it) {     // dP^T = V dO^T
+            const uint32_t do_lo = klo(sdO + (it & 1) * TILE_BYTES);
 #pragma unroll
-                for (int kk = 0; kk < 8; kk++) umma_ss(tDPT, v_lo + kstep(kk), do_lo + kstep(kk), idesc_kk, kk != 0);
-                umma_commit(dp_full);
-            };
-            if (alive) alive = mbar_wait(in_full, 0, abort_flag);
-            if (alive) {
-                tc_fence_after();
-                issue_st(0);
-                issue_dpt(0);
-            }
-            for (int it = 0; it < iters && alive; it++) {
-                const uint32_t st = it & 1;
-                const uint32_t q_mn = mnlo(sQ + st * TILE_BYTES), do_mn = mnlo(sdO + st * TILE_BYTES);
-                // dV += P^T dO as soon as P^T is packed
-                if (!mbar_wait(p1_full, it & 1, abort_flag)) { alive = false; break; }
-                tc_fence_after();
-#pragma unroll
-                for (int kk = 0; kk < 8; kk++)
-                    umma_ts(tDV, tST + (kk >> 1) * 32 + (kk & 1) * 8, do_mn + mnstep(kk), idesc_acc, (it | kk) != 0);
-                // the S^T columns are free again once dV has read them (in order): next tile's S^T
-                if (it + 1 < iters) {
-                    if (!mbar_wait(in_full + 8 * ((it + 1) & 1), ((it + 1) >> 1) & 1, abort_flag)) { alive = false; break; }
-                    tc_fence_after();
-                    issue_st(it + 1);
-                }
-                // dK += dS^T Q
-                if (!mbar_wait(p2_full, it & 1, abort_flag)) { alive = false; break; }
-                tc_fence_after();
-#pragma unroll
-                for (int kk = 0; kk < 8; kk++)
-                    umma_ts(tDK, tDPT + (kk >> 1) * 32 + (kk & 1) * 8, q_mn + mnstep(kk), idesc_acc, (it | kk) != 0);
-                umma_commit(in_empty + 8 * st);            // Q and dO of this stage are consumed
-                if (it + 1 < iters) issue_dpt(it + 1);
-            }
-            if (alive) umma_commit(acc_full);
+            for (int kk = 0; kk < 8; kk++) umma_ss_w(tDPT, v_lo + kstep(kk), do_lo + kstep(kk), idesc_kk, kk != 0);
+            umma_commit_w(dp_full);
+        };
+        if (alive) alive = mbar_wait_warp(in_full, 0, abort_flag);
+        if (alive) {
+            tc_fence_after();
+            issue_st(0);
+            issue_dpt(0);
         }
+        for (int it = 0; it < iters && alive; it++) {
+            const uint32_t st = it & 1;
+            const uint32_t q_mn = mnlo(sQ + st * TILE_BYTES), do_mn = mnlo(sdO + st * TILE_BYTES);
+            // dV += P^T dO as soon as P^T is packed
+            if (!mbar_wait_warp(p1_full, it & 1, abort_flag)) { alive = false; break; }
+            tc_fence_after();
+#pragma unroll
+            for (int kk = 0; kk < 8; kk++)
+                umma_ts_w(tDV, tST + (kk >> 1) * 32 + (kk & 1) * 8, do_mn + mnstep(kk), idesc_acc, (it | kk) != 0);
+            umma_commit_w(do_empty + 8 * st);            // dO of this stage is consumed (dP^T was issued earlier)
+            // the S^T columns are free again once dV has read them (in order): next tile's S^T
+            if (it + 1 < iters) {
+                if (!mbar_wait_warp(in_full + 8 * ((it + 1) & 1), ((it + 1) >> 1) & 1, abort_flag)) { alive = false; break; }
+                tc_fence_after();
+                issue_st(it + 1);
+            }
+            // dK += dS^T Q
+            if (!mbar_wait_warp(p2_full, it & 1, abort_flag)) { alive = false; break; }
+            tc_fence_after();
+#pragma unroll
+            for (int kk = 0; kk < 8; kk++)
+                umma_ts_w(tDK, tDPT + (kk >> 1) * 32 + (kk & 1) * 8, q_mn + mnstep(kk), idesc_acc, (it | kk) != 0);
+            umma_commit_w(q_empty + 8 * st);             // Q of this stage is consumed
+            if (it + 1 < iters) issue_dpt(it + 1);
+        }
+        if (alive) umma_commit_w(acc_full);
     } else {
         const int quarter = warp & 3;
         const int wg = (warp - 2) >> 2;                           // 0..3: 32-query group of the tile
@@ -559,13 +576,16 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
-    const uint32_t sQ = base, sdO = sQ + TILE_BYTES, sK = sdO + TILE_BYTES, sV = sK + 2 * TILE_BYTES;
-    uint8_t *aux = smem_raw + (base - raw) + 6 * TILE_BYTES + 4 * TILE * 4;
+    // K tiles live from S_j to dQ_j, so their ring has three stages: the copy of tile j+2 then starts when dQ of
+    // tile j-1 is done and its latency hides behind a whole tile of work.  V tiles are released right after dP_j.
+    const uint32_t sQ = base, sdO = sQ + TILE_BYTES, sK = sdO + TILE_BYTES, sV = sK + DQ_KSTAGES * TILE_BYTES;
+    uint8_t *aux = smem_raw + (base - raw) + (4 + DQ_KSTAGES) * TILE_BYTES;
     const uint32_t bars = smem_u32(aux);
-    const uint32_t q_full = bars, kv_full = bars + 8, kv_empty = bars + 24, s_full = bars + 40, dp_full = bars + 48,
-                   s_free = bars + 56, p2_full = bars + 64, acc_full = bars + 72;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux + 80);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(aux + 88);
+    const uint32_t q_full = bars, k_full = bars + 8, k_empty = bars + 32, v_full = bars + 56, v_empty = bars + 72,
+                   s_full = bars + 88, dp_full = bars + 96, s_free = bars + 104, p2_full = bars + 112,
+                   acc_full = bars + 120;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux + 128);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(aux + 136);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int h = blockIdx.y, g = h / (p.Hq / p.Hkv);
@@ -577,9 +597,13 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
 
     if (threadIdx.x == 0) {
         mbar_init(q_full, 1);
+        for (int s = 0; s < DQ_KSTAGES; s++) {
+            mbar_init(k_full + 8 * s, 1);
+            mbar_init(k_empty + 8 * s, 1);
+        }
         for (int s = 0; s < 2; s++) {
-            mbar_init(kv_full + 8 * s, 1);
-            mbar_init(kv_empty + 8 * s, 1);
+            mbar_init(v_full + 8 * s, 1);
+            mbar_init(v_empty + 8 * s, 1);
         }
         mbar_init(s_full, 1);
         mbar_init(dp_full, 1);
@@ -604,61 +628,70 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
             tma_load_2d(sQ + HALF_BYTES, &map_q, q_full, h * TILE + 64, qt0);
             tma_load_2d(sdO, &map_do, q_full, h * TILE, qt0);
             tma_load_2d(sdO + HALF_BYTES, &map_do, q_full, h * TILE + 64, qt0);
+            uint32_t ks = 0, kph = 0;
             for (int j = 0; j < nkv; j++) {
-                const uint32_t st = j & 1, ph = (j >> 1) & 1;
-                if (!mbar_wait(kv_empty + 8 * st, ph ^ 1u, abort_flag)) break;
-                const uint32_t full = kv_full + 8 * st;
-                mbar_expect_tx(full, 2 * TILE_BYTES);
-                tma_load_2d(sK + st * TILE_BYTES, &map_k, full, g * TILE, j * TILE);
-                tma_load_2d(sK + st * TILE_BYTES + HALF_BYTES, &map_k, full, g * TILE + 64, j * TILE);
-                tma_load_2d(sV + st * TILE_BYTES, &map_v, full, g * TILE, j * TILE);
-                tma_load_2d(sV + st * TILE_BYTES + HALF_BYTES, &map_v, full, g * TILE + 64, j * TILE);
+                if (!mbar_wait(k_empty + 8 * ks, kph ^ 1u, abort_flag)) break;
+                mbar_expect_tx(k_full + 8 * ks, TILE_BYTES);
+                tma_load_2d(sK + ks * TILE_BYTES, &map_k, k_full + 8 * ks, g * TILE, j * TILE);
+                tma_load_2d(sK + ks * TILE_BYTES + HALF_BYTES, &map_k, k_full + 8 * ks, g * TILE + 64, j * TILE);
+                if (++ks == DQ_KSTAGES) { ks = 0; kph ^= 1u; }
+                const uint32_t vs = j & 1, vph = (j >> 1) & 1;
+                if (!mbar_wait(v_empty + 8 * vs, vph ^ 1u, abort_flag)) break;
+                mbar_expect_tx(v_full + 8 * vs, TILE_BYTES);
+                tma_load_2d(sV + vs * TILE_BYTES, &map_v, v_full + 8 * vs, g * TILE, j * TILE);
+                tma_load_2d(sV + vs * TILE_BYTES + HALF_BYTES, &map_v, v_full + 8 * vs, g * TILE + 64, j * TILE);
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            constexpr uint32_t idesc_kk = make_idesc(TILE, TILE, false, false);
-            constexpr uint32_t idesc_acc = make_idesc(TILE, TILE, false, true);
-            bool alive = mbar_wait(q_full, 0, abort_flag);
-            const uint32_t q_lo = klo(sQ), do_lo = klo(sdO);
-            auto issue_s = [&](int j) {        // S = Q K^T
-                const uint32_t k_lo = klo(sK + (j & 1) * TILE_BYTES);
+        // the whole warp runs the issue loop; each MMA / commit executes in one elected lane
+        constexpr uint32_t idesc_kk = make_idesc(TILE, TILE, false, false);
+        constexpr uint32_t idesc_acc = make_idesc(TILE, TILE, false, true);
+        bool alive = mbar_wait_warp(q_full, 0, abort_flag);
+        const uint32_t q_lo = klo(sQ), do_lo = klo(sdO);
+        // K stage and phase of the tile whose S is issued next / whose dQ is issued next
+        uint32_t ks_s = 0, kph_s = 0, ks_q = 0;
+        auto issue_s = [&](int j) -> bool {        // S = Q K^T
+            (void)j;
+            if (!mbar_wait_warp(k_full + 8 * ks_s, kph_s, abort_flag)) return false;
+            tc_fence_after();
+            const uint32_t k_lo = klo(sK + ks_s * TILE_BYTES);
 #pragma unroll
-                for (int kk = 0; kk < 8; kk++) umma_ss(tS, q_lo + kstep(kk), k_lo + kstep(kk), idesc_kk, kk != 0);
-                umma_commit(s_full);
-            };
-            auto issue_dp = [&](int j) {       // dP = dO V^T
-                const uint32_t v_lo = klo(sV + (j & 1) * TILE_BYTES);
+            for (int kk = 0; kk < 8; kk++) umma_ss_w(tS, q_lo + kstep(kk), k_lo + kstep(kk), idesc_kk, kk != 0);
+            umma_commit_w(s_full);
+            if (++ks_s == DQ_KSTAGES) { ks_s = 0; kph_s ^= 1u; }
+            return true;
+        };
+        auto issue_dp = [&](int j) -> bool {       // dP = dO V^T
+            const uint32_t vs = j & 1;
+            if (!mbar_wait_warp(v_full + 8 * vs, (j >> 1) & 1, abort_flag)) return false;
+            tc_fence_after();
+            const uint32_t v_lo = klo(sV + vs * TILE_BYTES);
 #pragma unroll
-                for (int kk = 0; kk < 8; kk++) umma_ss(tDP, do_lo + kstep(kk), v_lo + kstep(kk), idesc_kk, kk != 0);
-                umma_commit(dp_full);
-            };
-            if (alive) alive = mbar_wait(kv_full, 0, abort_flag);
-            if (alive) {
+            for (int kk = 0; kk < 8; kk++) umma_ss_w(tDP, do_lo + kstep(kk), v_lo + kstep(kk), idesc_kk, kk != 0);
+            umma_commit_w(v_empty + 8 * vs);             // V of this stage is consumed
+            umma_commit_w(dp_full);
+            return true;
+        };
+        if (alive) alive = issue_s(0) && issue_dp(0);
+        for (int j = 0; j < nkv && alive; j++) {
+            if (j + 1 < nkv) {
+                // next tile's S as soon as the softmax warps have read this tile's S into registers
+                if (!mbar_wait_warp(s_free, j & 1, abort_flag)) { alive = false; break; }
                 tc_fence_after();
-                issue_s(0);
-                issue_dp(0);
+                if (!issue_s(j + 1)) { alive = false; break; }
             }
-            for (int j = 0; j < nkv && alive; j++) {
-                const uint32_t st = j & 1;
-                if (j + 1 < nkv) {
-                    // next tile's S as soon as the softmax warps have read this tile's S into registers
-                    if (!mbar_wait(kv_full + 8 * ((j + 1) & 1), ((j + 1) >> 1) & 1, abort_flag)) { alive = false; break; }
-                    if (!mbar_wait(s_free, j & 1, abort_flag)) { alive = false; break; }
-                    tc_fence_after();
-                    issue_s(j + 1);
-                }
-                if (!mbar_wait(p2_full, j & 1, abort_flag)) { alive = false; break; }
-                tc_fence_after();
-                const uint32_t k_mn = mnlo(sK + st * TILE_BYTES);
+            if (!mbar_wait_warp(p2_full, j & 1, abort_flag)) { alive = false; break; }
+            tc_fence_after();
+            const uint32_t k_mn = mnlo(sK + ks_q * TILE_BYTES);
 #pragma unroll
-                for (int kk = 0; kk < 8; kk++)
-                    umma_ts(tDQ, tDP + (kk >> 1) * 32 + (kk & 1) * 8, k_mn + mnstep(kk), idesc_acc, (j | kk) != 0);
-                umma_commit(kv_empty + 8 * st);            // K and V of this stage are consumed
-                if (j + 1 < nkv) issue_dp(j + 1);          // the dP columns are free once dQ has read dS (in order)
-            }
-            if (alive) umma_commit(acc_full);
+            for (int kk = 0; kk < 8; kk++)
+                umma_ts_w(tDQ, tDP + (kk >> 1) * 32 + (kk & 1) * 8, k_mn + mnstep(kk), idesc_acc, (j | kk) != 0);
+            umma_commit_w(k_empty + 8 * ks_q);           // K of this stage is consumed
+            if (++ks_q == DQ_KSTAGES) ks_q = 0;
+            // the dP columns are free once dQ has read dS (in order)
+            if (j + 1 < nkv && !issue_dp(j + 1)) { alive = false; break; }
         }
+        if (alive) umma_commit_w(acc_full);
     } else {
         const int quarter = warp & 3;
         const int wg = (warp - 2) >> 2;                           // 0..3: 32-key group of the tile
@@ -782,7 +815,7 @@ int attention_bwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, const bf16 *do
         return STREAMBP_E_CUDA;
     static bool configured = false;
     if (!configured) {
-        if (!opt_in_smem(attn_bwd_dkdv_tc_kernel, BWD_SMEM) || !opt_in_smem(attn_bwd_dq_tc_kernel, BWD_SMEM))
+        if (!opt_in_smem(attn_bwd_dkdv_tc_kernel, BWD_SMEM) || !opt_in_smem(attn_bwd_dq_tc_kernel, DQ_SMEM))
             return STREAMBP_E_CUDA;
         configured = true;
     }
@@ -791,7 +824,7 @@ int attention_bwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, const bf16 *do
     dim3 gkv((unsigned)((kv_len + TILE - 1) / TILE), Hkv);
     dim3 gq((unsigned)((n + TILE - 1) / TILE), Hq);
     SBP_LAUNCH(attn_bwd_dkdv_tc_kernel, gkv, BWD_THREADS, BWD_SMEM, st, mq, mk, mv, mdo, p);
-    SBP_LAUNCH(attn_bwd_dq_tc_kernel, gq, BWD_THREADS, BWD_SMEM, st, mq, mk, mv, mdo, p);
+    SBP_LAUNCH(attn_bwd_dq_tc_kernel, gq, BWD_THREADS, DQ_SMEM, st, mq, mk, mv, mdo, p);
     return STREAMBP_OK;
 }
 
