@@ -236,6 +236,59 @@ def layer_backward(cfg: LayerConfig, weights: Dict[str, torch.Tensor], X: torch.
     return st
 
 
+class HostFedLayerBackward:
+    """streambp_layer_backward for activations that live in pinned host memory (plumbing only: streams, events and
+    copies; every step of the path still runs in the library's kernels).  Two sets of device buffers alternate:
+    while the kernels of step k run on the compute stream, a copy stream brings in the X, dY of step k+1 and
+    takes out the dX of step k-1, so a sequence's 3 T d storage-dtype values cross PCIe behind the compute of
+    its neighbours instead of in front of its own."""
+
+    def __init__(self, cfg: LayerConfig, weights, grads, T: int, chunk: int, workspace: torch.Tensor):
+        self.cfg, self.weights, self.grads, self.chunk, self.ws = cfg, weights, grads, chunk, workspace
+        dev = workspace.device
+        mk = lambda: torch.empty(T, cfg.d_model, dtype=cfg.dtype, device=dev)
+        self.X, self.dY, self.dX = [mk(), mk()], [mk(), mk()], [mk(), mk()]
+        self.copy_stream = torch.cuda.Stream(device=dev)
+        self.loaded = [torch.cuda.Event(), torch.cuda.Event()]      # inputs of buffer i are on the device
+        self.computed = [torch.cuda.Event(), torch.cuda.Event()]    # the call on buffer i has finished
+        self.n_prefetched = 0       # prefetch() calls so far; call k fills buffer pair k % 2
+        self.n_run = 0              # step() calls so far; call k consumes buffer pair k % 2
+
+    def prefetch(self, X_host: torch.Tensor, dY_host: torch.Tensor) -> None:
+        """Starts the host-to-device copy of the inputs of the next step that has none yet (at most two ahead)."""
+        assert self.n_prefetched - self.n_run < 2, "both buffer pairs hold inputs that have not been consumed"
+        i = self.n_prefetched & 1
+        cs = self.copy_stream
+        if self.n_prefetched >= 2:
+            cs.wait_event(self.computed[i])     # the previous user of these buffers is done with them
+        with torch.cuda.stream(cs):
+            self.X[i].copy_(X_host, non_blocking=True)
+            self.dY[i].copy_(dY_host, non_blocking=True)
+            self.loaded[i].record(cs)
+        self.n_prefetched += 1
+
+    def step(self, dX_host: torch.Tensor, accumulate: bool = False, stream=None) -> None:
+        """Runs the backward on the oldest prefetched inputs and starts the copy of its dX to dX_host.  The copy
+        stream is in order, so that copy also precedes the next prefetch into the same buffer pair."""
+        assert self.n_run < self.n_prefetched, "prefetch() the inputs first"
+        i = self.n_run & 1
+        st = stream if stream is not None else torch.cuda.current_stream()
+        st.wait_event(self.loaded[i])
+        layer_backward(self.cfg, self.weights, self.X[i], self.dY[i], self.chunk, self.grads, self.dX[i], self.ws,
+                       accumulate=accumulate, stream=st)
+        self.computed[i].record(st)
+        cs = self.copy_stream
+        cs.wait_event(self.computed[i])
+        with torch.cuda.stream(cs):
+            dX_host.copy_(self.dX[i], non_blocking=True)
+        self.n_run += 1
+
+    def drain(self, stream=None) -> None:
+        """Makes `stream` wait for the copies that are still in flight."""
+        st = stream if stream is not None else torch.cuda.current_stream()
+        st.wait_stream(self.copy_stream)
+
+
 def layer_backward_packed(cfg: LayerConfig, weights, X, dY, chunk: int, cu_seqlens: Sequence[int], grads, dX, workspace,
                           pos0: int = 0, accumulate: bool = False, stream=None, check: bool = True) -> int:
     """streambp_layer_backward_packed: X, dY hold the sequences back to back; cu_seqlens = [0, ..., T] on the host."""

@@ -130,3 +130,40 @@ def test_packed_batch_matches_sum_over_sequences(dtype, dh, cu):
     bad = B.layer_backward_packed(bcfg, Wd, Xd, dYd, chunk, [0, 50, 50, T], grads, dX, ws, check=False)
     assert bad == B.E_SHAPE
     assert B.layer_backward_packed(bcfg, Wd, Xd, dYd, chunk, [0, 50, T - 1], grads, dX, ws, check=False) == B.E_SHAPE
+
+
+def test_host_fed_runner_matches_direct_calls():
+    """Three sequences fed from pinned host memory through the two-buffer runner (copies on a second stream,
+    overlapping the kernels of the neighbouring steps) give, bit for bit, the dX and the accumulated weight
+    gradients of three direct calls on device-resident inputs."""
+    shape = synth.LayerShape(256, 4, 2, 128, 512, True, 1e6)
+    T, chunk, dt = 384, 128, torch.bfloat16
+    _, bcfg, W, _, _ = layer_case(shape, 5, T, dt)
+    Wd = {k: to_dev(v, dt) for k, v in W.items()}
+    ios = [synth.make_layer_io(shape, 50 + i, T, True) for i in range(3)]
+    ws = B.alloc_workspace(B.layer_workspace_bytes(bcfg, T, chunk))
+    # direct calls
+    g_ref = B.alloc_layer_grads(bcfg)
+    dX_ref = []
+    for i, (X, dY) in enumerate(ios):
+        dX = torch.empty(T, shape.d_model, dtype=dt, device="cuda")
+        B.layer_backward(bcfg, Wd, to_dev(X, dt), to_dev(dY, dt), chunk, g_ref, dX, ws, accumulate=i > 0)
+        dX_ref.append(dX.cpu())
+    assert B.last_device_status(ws) == B.OK
+    # host-fed
+    g = B.alloc_layer_grads(bcfg)
+    fed = B.HostFedLayerBackward(bcfg, Wd, g, T, chunk, ws)
+    host = [(torch.from_numpy(X).to(dt).pin_memory(), torch.from_numpy(dY).to(dt).pin_memory()) for X, dY in ios]
+    out = [torch.empty(T, shape.d_model, dtype=dt).pin_memory() for _ in ios]
+    fed.prefetch(*host[0])
+    for i in range(3):
+        if i + 1 < 3:
+            fed.prefetch(*host[i + 1])
+        fed.step(out[i], accumulate=i > 0)
+    fed.drain()
+    torch.cuda.synchronize()
+    assert B.last_device_status(ws) == B.OK
+    for i in range(3):
+        assert torch.equal(out[i], dX_ref[i])
+    for k in g:
+        assert torch.equal(g[k], g_ref[k])
