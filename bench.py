@@ -35,10 +35,10 @@ def layer_flops(s, T):
     return fwd + bwd + att
 
 
-# DRAM bytes (read + write) of one representative launch of the dominant kernel, from the ncu capture
-# summarised in profiles/gemm_tc_kernel_chunk_products.md (the per-chunk product dh2 += du Wu:
-# M 1024, N 3584, K 18944; algorithmic bytes 189.3e6).  Launch shapes depend on the chunk, not on T.
-NCU_TRAFFIC_BYTES = {("qwen7b_layer", 1024): 192.9e6}
+# DRAM bytes (read + write) of the dominant launch of a chunk -- the {dWg += dg^T h2, dWu += du^T h2,
+# dh2 = dg Wg + du Wu} group -- from the ncu capture summarised in profiles/gemm_group_kernel_chunk_products.md
+# (qwen7b, chunk 1024: algorithmic bytes 1457e6).  Launch shapes depend on the chunk, not on T.
+NCU_TRAFFIC_BYTES = {("qwen7b_layer", 1024): 1680.8e6, ("llama8b_layer", 2048): 1927.5e6}
 
 
 def max_over_ranks(ms: float, world: int, device) -> float:
@@ -241,17 +241,28 @@ def run_head_or_model(args, cfg):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(0)
     sampler.start()
-    B.profile_enable(True)
     e0.record()
     for _ in range(args.steps):
         step()
     e1.record()
     torch.cuda.synchronize()
+    clocks = sampler.stop()
+    # class timing: the same steps again with CUDA events around every product launch
+    p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    B.profile_enable(True)
+    p0.record()
+    for _ in range(args.steps):
+        step()
+    p1.record()
+    torch.cuda.synchronize()
     prof = {k: B.profile_read(k) for k in B.KERNEL_CLASSES}
     B.profile_enable(False)
-    clocks = sampler.stop()
+    profiled_ms = p0.elapsed_time(p1)
     ms = e0.elapsed_time(e1) / args.steps
     gemm_ms, gemm_calls, gemm_flops = prof["gemm"]
+    # launches of chunks that are skipped on the device return at once but are still bracketed: count only the
+    # executed share of their FLOPs
+    gemm_flops *= executed_flops / flops
     achieved = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
     print(json.dumps({
         "metric": name, "value": T / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
@@ -266,7 +277,8 @@ def run_head_or_model(args, cfg):
         "frac_of_measured_sustained_bf16_executed": executed_flops / (ms * 1e-3) / 1e12 / peaks["sustained"],
         "peak_activation_gb": ws_bytes / 1e9, "peak_activation_gb_unchunked": ws_full / 1e9,
         "gpu_launches": int(launches * args.steps),
-        "roofline": {"bound": "tensor", "kernel": "linear products", "achieved": achieved, "peak": peaks["sustained"],
+        "roofline": {"bound": "tensor", "kernel": "linear products (executed FLOPs)", "achieved": achieved,
+                     "peak": peaks["sustained"],
                      "unit": "TFLOP/s", "frac": achieved / peaks["sustained"], "traffic": None,
                      "launches": int(gemm_calls), "ms_per_step": gemm_ms / args.steps,
                      "timed": "a second run of the same K steps with CUDA events around every launch of the class",
@@ -293,6 +305,9 @@ def main():
     ap.add_argument("--cpu-baseline-tokens", type=int, default=1024)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--dp", action="store_true",
+                    help="data parallel instead of independent replicas: every step ends with one reduce-scatter of "
+                         "the layer's fp32 gradient bucket over all ranks (Sec. 3.3 / App. A.3 of the paper)")
     args = ap.parse_args()
 
     from paper_2506_03077_b200 import synth
@@ -345,8 +360,18 @@ def main():
     ws = B.alloc_workspace(ws_bytes)
     stream = torch.cuda.current_stream()
 
+    dpr = None
+    if args.dp:
+        from paper_2506_03077_b200 import dp as DP
+        dpr = DP.DataParallelLayerBackward(bcfg, W, T, chunk)
+        grads, ws = dpr.bucket.views, dpr.ws
+
     def step():
-        B.layer_backward(bcfg, W, X, dY, chunk, grads, dX, ws)
+        if dpr is not None:
+            dpr.step(X, dY, dX)     # backward, then the gradient exchange on the communication stream
+            dpr.wait()
+        else:
+            B.layer_backward(bcfg, W, X, dY, chunk, grads, dX, ws)
 
     fed = B.HostFedLayerBackward(bcfg, W, grads, T, chunk, ws)
 
@@ -419,7 +444,8 @@ def main():
         "config": {"workload": cfg.name, "T": T, "chunk": chunk, "d_model": s.d_model, "n_q_heads": s.n_q_heads,
                    "n_kv_heads": s.n_kv_heads, "head_dim": s.head_dim, "d_ff": s.d_ff, "qkv_bias": s.qkv_bias,
                    "l2": "inputs larger than L2 (weights + gradients > 1 GB per step)",
-                   "multi_gpu": "replicas only"},
+                   "multi_gpu": ("data parallel: one NCCL reduce-scatter of the layer's fp32 gradient bucket per step"
+                                 if args.dp else "replicas only")},
         "algorithmic_tflop_per_step": flops / 1e12,
         "tflops": flops / (ms_per_step * 1e-3) / 1e12,
         "frac_of_measured_sustained_bf16": flops / (ms_per_step * 1e-3) / 1e12 / peaks["sustained"],
@@ -431,7 +457,7 @@ def main():
                      "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                      "peak_source": peaks["source"] + " sustained bf16",
                      "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, chunk)),
-                     "traffic_note": "dram bytes of one representative product launch under ncu (see profiles/)",
+                     "traffic_note": "dram bytes of the dominant product launch of a chunk under ncu (see profiles/)",
                      "launches": int(gemm_calls), "ms_per_step": gemm_ms / args.steps,
                      "timed": "a second run of the same K steps with CUDA events around every launch of the class",
                      "step_ms_with_events": profiled_ms / args.steps},

@@ -213,6 +213,17 @@ int streambp_model_backward(const streambp_model_cfg *cfg, const void *embed,
                             float *d_g_final, float *d_w_vocab, void *dX0,
                             void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/*
+ * Partition size for a memory budget (Sec. 4.3, "Effect of partition size": a partition that is too small
+ * pays for re-loading the weights and for the fp32 read-modify-write of every weight gradient once per
+ * partition, while a larger one costs only marginally more memory).  Returns the largest chunk, a multiple
+ * of 128 rows (or T itself when T fits), whose workspace as reported by streambp_layer_workspace_bytes /
+ * streambp_lmhead_workspace_bytes does not exceed budget_bytes; 0 if even one 128-row chunk does not fit or
+ * an argument is invalid.  Host-only: no GPU work, no allocation.
+ */
+int64_t streambp_layer_suggest_chunk(const streambp_layer_cfg *cfg, int64_t T, size_t budget_bytes);
+int64_t streambp_lmhead_suggest_chunk(const streambp_head_cfg *cfg, int64_t T, size_t budget_bytes);
+
 /* Synchronises `cuda_stream` and returns the status the kernels of the last call using
  * this workspace recorded (STREAMBP_OK, E_BAD_LABEL, E_NO_VALID_LABELS, E_DEVICE_TIMEOUT),
  * or STREAMBP_E_CUDA if the stream reports an error. */

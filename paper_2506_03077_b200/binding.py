@@ -30,6 +30,7 @@ EXPORTS = (
     "streambp_model_workspace_bytes", "streambp_model_backward",
     "streambp_last_device_status", "streambp_status_string",
     "streambp_last_cuda_error", "streambp_last_launch_count", "streambp_gemm", "streambp_gemm_grouped",
+    "streambp_layer_suggest_chunk", "streambp_lmhead_suggest_chunk",
     "streambp_profile_enable", "streambp_profile_read",
     "streambp_attention_forward", "streambp_attention_backward", "streambp_attention_backward_static",
     "streambp_lmhead_rl_backward", "streambp_layer_backward_packed",
@@ -115,6 +116,10 @@ def lib() -> C.CDLL:
     L.streambp_last_cuda_error.argtypes = []
     L.streambp_last_launch_count.restype = i64
     L.streambp_last_launch_count.argtypes = []
+    L.streambp_layer_suggest_chunk.restype = i64
+    L.streambp_layer_suggest_chunk.argtypes = [C.POINTER(LayerCfgC), i64, sz]
+    L.streambp_lmhead_suggest_chunk.restype = i64
+    L.streambp_lmhead_suggest_chunk.argtypes = [C.POINTER(HeadCfgC), i64, sz]
     L.streambp_gemm_grouped.restype = C.c_int
     L.streambp_gemm_grouped.argtypes = [C.POINTER(GemmProblemC), i32, vp, vp]
     L.streambp_gemm.restype = C.c_int
@@ -216,6 +221,17 @@ def alloc_layer_grads(cfg: LayerConfig, device="cuda") -> Dict[str, torch.Tensor
 def layer_workspace_bytes(cfg: LayerConfig, T: int, chunk: int) -> int:
     c = cfg.c()
     return int(lib().streambp_layer_workspace_bytes(C.byref(c), T, chunk))
+
+
+def layer_suggest_chunk(cfg: LayerConfig, T: int, budget_bytes: int) -> int:
+    """Largest chunk (multiple of 128 rows, or T) whose layer workspace fits budget_bytes; 0 if none does."""
+    c = cfg.c()
+    return int(lib().streambp_layer_suggest_chunk(C.byref(c), T, budget_bytes))
+
+
+def lmhead_suggest_chunk(cfg: HeadConfig, T: int, budget_bytes: int) -> int:
+    c = cfg.c()
+    return int(lib().streambp_lmhead_suggest_chunk(C.byref(c), T, budget_bytes))
 
 
 def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:

@@ -248,6 +248,24 @@ int begin_call(void *ws, cudaStream_t st) {
 
 using namespace sbp;
 
+namespace {
+// largest chunk in {128, 256, ..., } U {T} with bytes(chunk) <= budget; bytes() is non-decreasing in chunk
+template <typename F>
+int64_t suggest_chunk(int64_t T, size_t budget, F bytes) {
+    if (T < 1) return 0;
+    const size_t full = bytes(T);
+    if (full == 0) return 0;
+    if (full <= budget) return T;
+    int64_t lo = 0, hi = (T - 1) / 128;          // chunk = 128 * k for k in [1, hi] is < T
+    while (lo < hi) {
+        const int64_t mid = (lo + hi + 1) / 2;
+        if (bytes(128 * mid) <= budget) lo = mid;
+        else hi = mid - 1;
+    }
+    return 128 * lo;
+}
+}  // namespace
+
 extern "C" {
 
 size_t streambp_layer_workspace_bytes(const streambp_layer_cfg *cfg, int64_t T, int64_t chunk) {
@@ -406,6 +424,16 @@ int streambp_model_backward(const streambp_model_cfg *cfg, const void *embed, co
     return model_backward<bf16>(*cfg, (const bf16 *)embed, eff.data(), (const bf16 *)g_final, (const bf16 *)w_vocab,
                                 ids, (const bf16 *)X0, labels, T, chunk_layer, chunk_head, accumulate != 0, loss,
                                 d_embed, layer_grads, d_g_final, d_w_vocab, (bf16 *)dX0, workspace, st);
+}
+
+int64_t streambp_layer_suggest_chunk(const streambp_layer_cfg *cfg, int64_t T, size_t budget_bytes) {
+    if (check_layer_cfg(cfg) != STREAMBP_OK) return 0;
+    return suggest_chunk(T, budget_bytes, [&](int64_t c) { return streambp_layer_workspace_bytes(cfg, T, c); });
+}
+
+int64_t streambp_lmhead_suggest_chunk(const streambp_head_cfg *cfg, int64_t T, size_t budget_bytes) {
+    if (check_head_cfg(cfg) != STREAMBP_OK) return 0;
+    return suggest_chunk(T, budget_bytes, [&](int64_t c) { return streambp_lmhead_workspace_bytes(cfg, T, c); });
 }
 
 int streambp_last_device_status(void *workspace, void *cuda_stream) {

@@ -108,3 +108,23 @@ def test_host_side_errors(lib):
     assert st == B.E_NULL
     assert lib.streambp_gemm(5, 8, 8, 8, 4096, 8, 4096, 8, 4096, 8, 1, 0, 0, 0, None) == B.E_SHAPE
     assert lib.streambp_last_device_status(None, None) == B.E_NULL
+
+
+def test_suggested_chunk_is_the_largest_that_fits(lib):
+    """Sec. 4.3: partition size is the memory / time knob.  The suggestion is the largest multiple of 128 (or T)
+    whose exact workspace fits the budget, checked against a scan of the planner."""
+    import torch
+    c = B.LayerConfig(4096, 32, 8, 128, 14336, False, 5e5, dtype=torch.bfloat16)
+    T = 32768
+    assert B.layer_suggest_chunk(c, T, 1 << 62) == T
+    assert B.layer_suggest_chunk(c, T, B.layer_workspace_bytes(c, T, 128) - 1) == 0
+    for budget in (int(0.81e9), int(1.5e9), B.layer_workspace_bytes(c, T, 2048), B.layer_workspace_bytes(c, T, 2048) - 1):
+        got = B.layer_suggest_chunk(c, T, budget)
+        assert got % 128 == 0 and 0 < got < T
+        assert B.layer_workspace_bytes(c, T, got) <= budget < B.layer_workspace_bytes(c, T, got + 128)
+    assert B.layer_suggest_chunk(c, T, B.layer_workspace_bytes(c, T, 2048)) == 2048
+    assert B.layer_suggest_chunk(c, 100, B.layer_workspace_bytes(c, 100, 100)) == 100      # T itself when it fits
+    h = B.HeadConfig(3584, 152064, dtype=torch.bfloat16)
+    got = B.lmhead_suggest_chunk(h, 32768, int(1e9))
+    assert got % 128 == 0 and B.lmhead_workspace_bytes(h, 32768, got) <= 1e9 < B.lmhead_workspace_bytes(h, 32768, got + 128)
+    assert B.lmhead_suggest_chunk(h, 0, int(1e9)) == 0

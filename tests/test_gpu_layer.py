@@ -167,3 +167,27 @@ def test_host_fed_runner_matches_direct_calls():
         assert torch.equal(out[i], dX_ref[i])
     for k in g:
         assert torch.equal(g[k], g_ref[k])
+
+
+def test_data_parallel_runner_single_rank_matches_direct_call():
+    """World size 1: the data-parallel runner (gradients accumulated into views of one flat bucket, exchange on a
+    second stream) returns the gradients of the direct call, bit for bit, and its shard is the whole bucket."""
+    from paper_2506_03077_b200 import dp
+    shape = synth.LayerShape(256, 4, 2, 128, 512, True, 1e6)
+    T, chunk, dt = 320, 128, torch.bfloat16
+    _, bcfg, W, X, dY = layer_case(shape, 11, T, dt)
+    dX_ref, g_ref = run_layer(bcfg, W, X, dY, chunk)
+    Wd = {k: to_dev(v, dt) for k, v in W.items()}
+    r = dp.DataParallelLayerBackward(bcfg, Wd, T, chunk)
+    dX = torch.empty(T, shape.d_model, dtype=dt, device="cuda")
+    for v in r.bucket.views.values():
+        v.fill_(float("nan"))            # the call must overwrite
+    r.step(to_dev(X, dt), to_dev(dY, dt), dX)
+    r.wait()
+    torch.cuda.synchronize()
+    assert B.last_device_status(r.ws) == B.OK
+    assert torch.equal(dX, dX_ref)
+    full = dp.gather_full_gradients(r.bucket, r.shard)
+    for k in g_ref:
+        assert torch.equal(full[k], g_ref[k])
+    assert r.shard.numel() == r.bucket.total
