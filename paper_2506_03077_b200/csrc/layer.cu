@@ -40,7 +40,7 @@ struct LayerWs {
     T *K, *V;             // [T, dkv]
     float *dK, *dV;       // [T, dkv]
     // one chunk
-    T *h1, *Q, *O, *h2, *g, *u, *m, *dr_s, *dO, *dk_s, *dv_s;
+    T *h1, *Q, *O, *h2, *g, *u, *m, *dr_s, *dO, *dk_s, *dv_s, *dm;
     float *fa, *r, *dr, *rstd1, *rstd2, *lse, *delta, *partials;
     size_t bytes;
 };
@@ -65,13 +65,20 @@ LayerWs<T> plan(const streambp_layer_cfg &c, int64_t T_, int64_t chunk, void *ba
     w.g = a.take<T>(cn * I);
     w.u = a.take<T>(cn * I);
     w.m = a.take<T>(cn * I);
+    const size_t dead_begin = align_up(a.off, 256);
     w.dr_s = a.take<T>(cn * d);
     w.dO = a.take<T>(cn * dq);
     w.dk_s = a.take<T>(cn * dkv);
     w.dv_s = a.take<T>(cn * dkv);
     w.fa = a.take<float>(cn * wide);
-    w.r = a.take<float>(cn * d);
     w.dr = a.take<float>(cn * d);
+    // dm = dY Wd lives only from its product to the SwiGLU backward, while dr_s, dO, dk_s, dv_s, fa and dr are all
+    // dead: it is laid over that span when it fits (it does for every LLM-shaped layer), else it gets its own block
+    if (a.off - dead_begin >= (size_t)(cn * I) * sizeof(T))
+        w.dm = a.base ? reinterpret_cast<T *>(a.base + dead_begin) : nullptr;
+    else
+        w.dm = a.take<T>(cn * I);
+    w.r = a.take<float>(cn * d);
     w.rstd1 = a.take<float>(cn);
     w.rstd2 = a.take<float>(cn);
     w.lse = a.take<float>(cn * c.n_q_heads);
@@ -193,16 +200,17 @@ int layer_backward(const streambp_layer_cfg &c, const streambp_layer_weights &w,
         SBP_TRY(chunk_forward<T>(c, w, X, r0, n, seg, s, st));
 
         // ---- MLP backward ----
-        SBP_TRY((mm<T, float>(OP_TN, d, I, n, dYi, d, s.m, I, G.w_down, I, nullptr, acc, st)));       // dWd += dY^T m
-        SBP_TRY((mm<T, T>(OP_NN, n, I, d, dYi, d, (const T *)w.w_down, I, s.m, I, nullptr, false, st)));  // dm = dY Wd
-        SBP_TRY(swiglu_bwd<T>(s.m, s.g, s.u, n * I, st));                                             // g := dg, u := du
-        {   // dWg += dg^T h2, dWu += du^T h2, dh2 = dg Wg + du Wu: all three need only dg, du, h2
-            MmProb<T> pr[3] = {
+        SBP_TRY((mm<T, T>(OP_NN, n, I, d, dYi, d, (const T *)w.w_down, I, s.dm, I, nullptr, false, st)));  // dm = dY Wd
+        SBP_TRY(swiglu_bwd<T>(s.dm, s.g, s.u, n * I, st));                                            // g := dg, u := du
+        {   // dWd += dY^T m, dWg += dg^T h2, dWu += du^T h2, dh2 = dg Wg + du Wu in one launch: the weight
+            // gradients are bound by the fp32 add into C at L2, the input gradient by the tensor pipe
+            MmProb<T> pr[4] = {
+                mm_prob<T>(OP_TN, d, I, n, dYi, d, s.m, I, G.w_down, I, true, nullptr, acc),
                 mm_prob<T>(OP_TN, I, d, n, s.g, I, s.h2, d, G.w_gate, d, true, nullptr, acc),
                 mm_prob<T>(OP_TN, I, d, n, s.u, I, s.h2, d, G.w_up, d, true, nullptr, acc),
                 mm_prob<T>(OP_NN, n, d, I, s.g, I, (const T *)w.w_gate, d, s.fa, d, true, nullptr, false)};
-            mm_add_seg<T>(pr[2], I, s.u, I, (const T *)w.w_up, d);
-            SBP_TRY(mm_group<T>(pr, 3, st));
+            mm_add_seg<T>(pr[3], I, s.u, I, (const T *)w.w_up, d);
+            SBP_TRY(mm_group<T>(pr, 4, st));
         }
         // dr = dY + norm2_bwd(dh2)
         SBP_TRY(rmsnorm_bwd<T>(s.fa, nullptr, s.r, s.rstd2, (const T *)w.g2, dYi, nullptr, n, d, s.dr,
