@@ -272,6 +272,10 @@ int swiglu_bwd(const T *dm, T *g, T *u, int64_t n, cudaStream_t st);
 template <typename T>
 int colsum(const T *a, int64_t rows, int cols, float *out, bool accumulate, float *partials, cudaStream_t st);
 int colsum_partial_rows(int64_t rows);
+// o_i += column sums of a_i [rows, c_i], i = 0..2, in one pair of launches; partials: [colsum_partial_rows(rows), c0+c1+c2]
+template <typename T>
+int colsum3_add(const T *a0, int c0, float *o0, const T *a1, int c1, float *o1, const T *a2, int c2, float *o2,
+                int64_t rows, float *partials, cudaStream_t st);
 template <typename T>
 int cast_from_f32(const float *in, int64_t n, T *out, cudaStream_t st);
 // out = a + b (fp32 inputs)

@@ -83,7 +83,7 @@ LayerWs<T> plan(const streambp_layer_cfg &c, int64_t T_, int64_t chunk, void *ba
     w.rstd2 = a.take<float>(cn);
     w.lse = a.take<float>(cn * c.n_q_heads);
     w.delta = a.take<float>(cn * c.n_q_heads);
-    w.partials = a.take<float>(64 * wide);
+    w.partials = a.take<float>(256 * wide);      // per-block partial rows of the gain / bias gradient reductions
     w.bytes = a.size();
     return w;
 }
@@ -250,11 +250,8 @@ int layer_backward(const streambp_layer_cfg &c, const streambp_layer_weights &w,
             mm_add_seg<T>(pr[3], dkv, s.dv_s, dkv, (const T *)w.wv, d);
             SBP_TRY(mm_group<T>(pr, 4, st));
         }
-        if (c.qkv_bias) {
-            SBP_TRY(colsum<T>(dq_s, n, (int)dq, G.bq, true, s.partials, st));
-            SBP_TRY(colsum<T>(s.dk_s, n, (int)dkv, G.bk, true, s.partials, st));
-            SBP_TRY(colsum<T>(s.dv_s, n, (int)dkv, G.bv, true, s.partials, st));
-        }
+        if (c.qkv_bias)
+            SBP_TRY(colsum3_add<T>(dq_s, (int)dq, G.bq, s.dk_s, (int)dkv, G.bk, s.dv_s, (int)dkv, G.bv, n, s.partials, st));
 
         // ---- dX = dr + norm1_bwd(dh1) ----
         SBP_TRY(rmsnorm_bwd<T>(s.fa, Xi, nullptr, s.rstd1, (const T *)w.g1, nullptr, s.dr, n, d, nullptr, dX + r0 * d,
