@@ -78,17 +78,6 @@ int mm<bf16, bf16>(GemmOp op, int64_t M, int64_t N, int64_t K, const bf16 *A, in
     if (e == 2) return STREAMBP_E_SHAPE;
     return gemm<bf16, bf16>(op, M, N, K, A, lda, B, ldb, C, ldc, bias, accumulate, st);
 }
-namespace {
-bool grouping_enabled() {
-    static int on = -1;
-    if (on < 0) {
-        const char *e = std::getenv("STREAMBP_NO_GROUP");
-        on = (e && e[0] == '1') ? 0 : 1;
-    }
-    return on == 1;
-}
-}  // namespace
-
 template <>
 int mm_group<float>(const MmProb<float> *probs, int n, cudaStream_t st) {
     for (int i = 0; i < n; i++) {
@@ -102,7 +91,7 @@ int mm_group<float>(const MmProb<float> *probs, int n, cudaStream_t st) {
 template <>
 int mm_group<bf16>(const MmProb<bf16> *probs, int n, cudaStream_t st) {
     GemmProb gp[4];
-    bool grouped = grouping_enabled() && gemm_engine() != 1 && n <= 4;
+    bool grouped = gemm_engine() != 1 && n <= 4;
     if (grouped) {
         for (int i = 0; i < n; i++) {
             const MmProb<bf16> &g = probs[i];
