@@ -148,129 +148,18 @@ __global__ void __launch_bounds__(256)
     out[col] = accumulate ? out[col] + acc : acc;
 }
 
-// RMSNorm backward in one pass: a block walks rows blockIdx.x, blockIdx.x + gridDim.x, ...; a thread owns the same
-// 4-column groups in every row, keeps the row's dh and x in registers between the dot product and the output,
-// and sums dh * xhat over its rows for the gain gradient (one partial row per block, reduced afterwards).
-// Every input is read exactly once.  NG = ceil(d / 1024) column groups per thread.
-constexpr int kNormBlocks = 256;
-template <typename T, int NG>
-__global__ void __launch_bounds__(256)
-    rmsnorm_bwd_fused_kernel(const float *__restrict__ dh, const T *__restrict__ xT, const float *__restrict__ xF,
-                             const float *__restrict__ rstd_in, const T *__restrict__ gain,
-                             const T *__restrict__ addT, const float *__restrict__ addF, int64_t rows, int d,
-                             float *__restrict__ outF, T *__restrict__ outT, float *__restrict__ partial,
-                             const int *gate) {
-    __shared__ float red[33];
-    const bool off = gated_off(gate);       // the upstream gradient of this block of rows is exactly zero
-    float gn[NG][4], acc[NG][4];
-#pragma unroll
-    for (int i = 0; i < NG; i++) {
-        const int c = (threadIdx.x + i * 256) * 4;
-#pragma unroll
-        for (int k = 0; k < 4; k++) {
-            gn[i][k] = (c + k < d) ? to_f32(gain[c + k]) : 0.f;
-            acc[i][k] = 0.f;
-        }
-    }
-    for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
-        if (off) {
-            for (int c = threadIdx.x; c < d; c += blockDim.x) {
-                if (outF) outF[row * d + c] = 0.f;
-                if (outT) outT[row * d + c] = from_f32<T>(0.f);
-            }
-            continue;
-        }
-        const float rstd = rstd_in[row];
-        float g[NG][4], xh[NG][4];
-        float dot = 0.f;
-#pragma unroll
-        for (int i = 0; i < NG; i++) {
-            const int c = (threadIdx.x + i * 256) * 4;
-            if (c < d) {       // d is a multiple of 4: a group is inside the row or outside it
-                const float4 g4 = *reinterpret_cast<const float4 *>(dh + row * d + c);
-                g[i][0] = g4.x; g[i][1] = g4.y; g[i][2] = g4.z; g[i][3] = g4.w;
-                if (xF) {
-                    const float4 x4 = *reinterpret_cast<const float4 *>(xF + row * d + c);
-                    xh[i][0] = x4.x * rstd; xh[i][1] = x4.y * rstd; xh[i][2] = x4.z * rstd; xh[i][3] = x4.w * rstd;
-                } else {
-#pragma unroll
-                    for (int k = 0; k < 4; k++) xh[i][k] = to_f32(xT[row * d + c + k]) * rstd;
-                }
-#pragma unroll
-                for (int k = 0; k < 4; k++) {
-                    dot += g[i][k] * gn[i][k] * xh[i][k];
-                    acc[i][k] += g[i][k] * xh[i][k];
-                }
-            }
-        }
-        dot = block_sum(dot, red);
-        const float mean = dot / (float)d;
-#pragma unroll
-        for (int i = 0; i < NG; i++) {
-            const int c = (threadIdx.x + i * 256) * 4;
-            if (c < d) {
-                float o[4];
-#pragma unroll
-                for (int k = 0; k < 4; k++) {
-                    float v = (g[i][k] * gn[i][k] - xh[i][k] * mean) * rstd;
-                    if (addF) v += addF[row * d + c + k];
-                    if (addT) v += to_f32(addT[row * d + c + k]);
-                    o[k] = v;
-                }
-                if (outF) *reinterpret_cast<float4 *>(outF + row * d + c) = make_float4(o[0], o[1], o[2], o[3]);
-                if (outT) {
-#pragma unroll
-                    for (int k = 0; k < 4; k++) outT[row * d + c + k] = from_f32<T>(o[k]);
-                }
-            }
-        }
-    }
-    if (partial && !off) {
-#pragma unroll
-        for (int i = 0; i < NG; i++) {
-            const int c = (threadIdx.x + i * 256) * 4;
-            if (c < d)
-                *reinterpret_cast<float4 *>(partial + (int64_t)blockIdx.x * d + c) =
-                    make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
-        }
-    }
-}
-
 static inline int split_count(int64_t rows) {
     int64_t n = (rows + 31) / 32;
     return (int)(n < 1 ? 1 : (n > 64 ? 64 : n));
 }
+int rmsnorm_bwd_partials_rows(int64_t rows) { return split_count(rows); }
 int colsum_partial_rows(int64_t rows) { return split_count(rows); }
-
-int rmsnorm_bwd_partials_rows(int64_t rows) { return (int)(rows < kNormBlocks ? (rows < 1 ? 1 : rows) : kNormBlocks); }
-
-template <typename T, int NG>
-static int rmsnorm_bwd_launch(const float *dh, const T *xT, const float *xF, const float *rstd, const T *gain,
-                              const T *addT, const float *addF, int64_t rows, int d, float *outF, T *outT,
-                              float *dgain, float *partials, cudaStream_t st) {
-    const int *gate = call_state().gate;
-    const int nb = rmsnorm_bwd_partials_rows(rows);
-    SBP_LAUNCH((rmsnorm_bwd_fused_kernel<T, NG>), nb, 256, 0, st, dh, xT, xF, rstd, gain, addT, addF, rows, d, outF,
-               outT, dgain ? partials : (float *)nullptr, gate);
-    if (dgain) SBP_LAUNCH(partial_reduce_kernel, (d + 255) / 256, 256, 0, st, partials, nb, d, dgain, 1, gate);
-    return STREAMBP_OK;
-}
 
 template <typename T>
 int rmsnorm_bwd(const float *dh, const T *xT, const float *xF, const float *rstd, const T *gain, const T *addT,
                 const float *addF, int64_t rows, int d, float *outF, T *outT, float *dgain, float *partials,
                 cudaStream_t st) {
     if (rows <= 0) return STREAMBP_OK;
-    const int ng = (d + 1023) / 1024;
-    if (d % 4 == 0 && ng <= 8) {
-#define SBP_NORM_CASE(N) case N: return rmsnorm_bwd_launch<T, N>(dh, xT, xF, rstd, gain, addT, addF, rows, d, outF, outT, dgain, partials, st)
-        switch (ng) {
-            SBP_NORM_CASE(1); SBP_NORM_CASE(2); SBP_NORM_CASE(3); SBP_NORM_CASE(4);
-            SBP_NORM_CASE(5); SBP_NORM_CASE(6); SBP_NORM_CASE(7); SBP_NORM_CASE(8);
-        }
-#undef SBP_NORM_CASE
-    }
-    // very wide rows: row kernel, then the gain gradient from a second pass over the inputs
     const int *gate = call_state().gate;
     SBP_LAUNCH(rmsnorm_bwd_rows_kernel<T>, (unsigned)rows, 256, 0, st, dh, xT, xF, rstd, gain, addT, addF, d, outF,
                outT, gate);

@@ -83,7 +83,7 @@ LayerWs<T> plan(const streambp_layer_cfg &c, int64_t T_, int64_t chunk, void *ba
     w.rstd2 = a.take<float>(cn);
     w.lse = a.take<float>(cn * c.n_q_heads);
     w.delta = a.take<float>(cn * c.n_q_heads);
-    w.partials = a.take<float>(256 * wide);      // per-block partial rows of the gain / bias gradient reductions
+    w.partials = a.take<float>(64 * wide);
     w.bytes = a.size();
     return w;
 }

@@ -28,7 +28,7 @@ HeadWs<T> plan(const streambp_head_cfg &c, int64_t T_, int64_t chunk, void *base
     w.dhn = a.take<float>(cn * d);
     w.rstd = a.take<float>(cn);
     w.row_loss = a.take<float>(cn);
-    w.partials = a.take<float>(256 * d);
+    w.partials = a.take<float>(64 * d);
     w.chunk_valid = a.take<int>((T_ + cn - 1) / cn);
     w.bytes = a.size();
     return w;

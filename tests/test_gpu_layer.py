@@ -191,3 +191,4 @@ def test_data_parallel_runner_single_rank_matches_direct_call():
     for k in g_ref:
         assert torch.equal(full[k], g_ref[k])
     assert r.shard.numel() == r.bucket.total
+
