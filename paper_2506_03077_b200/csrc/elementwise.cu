@@ -489,6 +489,15 @@ int count_valid_per_chunk(const int64_t *labels, int64_t T_, int64_t chunk, int6
     return STREAMBP_OK;
 }
 
+// four consecutive values of a row in one store (the row base and the column are multiples of 4 elements)
+__device__ __forceinline__ void store4(float *p, const float (&o)[4]) {
+    *reinterpret_cast<float4 *>(p) = make_float4(o[0], o[1], o[2], o[3]);
+}
+__device__ __forceinline__ void store4(bf16 *p, const float (&o)[4]) {
+    __nv_bfloat162 a = __floats2bfloat162_rn(o[0], o[1]), b = __floats2bfloat162_rn(o[2], o[3]);
+    *reinterpret_cast<uint2 *>(p) = make_uint2(*reinterpret_cast<uint32_t *>(&a), *reinterpret_cast<uint32_t *>(&b));
+}
+
 // one block per logits row: online (max, sum-exp), then dz = (softmax - onehot) / N
 template <typename T>
 __global__ void __launch_bounds__(1024)
@@ -548,13 +557,18 @@ __global__ void __launch_bounds__(1024)
         } else {
             for (int k = 0; k < 4; k++) v[k] = (c + k < V) ? zr[c + k] : -INFINITY;
         }
+        float o[4];
 #pragma unroll
         for (int k = 0; k < 4; k++) {
-            if (c + k < V) {
-                float p = __expf(v[k] - lse);
-                if (c + k == y) p -= 1.f;
-                dr[c + k] = from_f32<T>(p * invN);
-            }
+            float p = __expf(v[k] - lse);
+            if (c + k == y) p -= 1.f;
+            o[k] = p * invN;
+        }
+        if (vec && c + 3 < V) {
+            store4(dr + c, o);       // one 8- or 16-byte store per thread
+        } else {
+            for (int k = 0; k < 4; k++)
+                if (c + k < V) dr[c + k] = from_f32<T>(o[k]);
         }
     }
 }
@@ -644,13 +658,18 @@ __global__ void __launch_bounds__(1024)
         } else {
             for (int k = 0; k < 4; k++) v[k] = (c + k < V) ? zr[c + k] : -INFINITY;
         }
+        float o[4];
 #pragma unroll
         for (int k = 0; k < 4; k++) {
-            if (c + k < V) {
-                float pr = -__expf(v[k] - lse);
-                if (c + k == y) pr += 1.f;
-                dr[c + k] = from_f32<T>(coef * pr);
-            }
+            float pr = -__expf(v[k] - lse);
+            if (c + k == y) pr += 1.f;
+            o[k] = coef * pr;
+        }
+        if (vec && c + 3 < V) {
+            store4(dr + c, o);
+        } else {
+            for (int k = 0; k < 4; k++)
+                if (c + k < V) dr[c + k] = from_f32<T>(o[k]);
         }
     }
 }
