@@ -68,6 +68,25 @@ template int rmsnorm_fwd<float>(const float *, const float *, const float *, flo
 template int rmsnorm_fwd<bf16>(const bf16 *, const float *, const bf16 *, float, int64_t, int, bf16 *, float *,
                                float *, cudaStream_t);
 
+// four consecutive values of a row in one store (the row base and the column are multiples of 4 elements)
+__device__ __forceinline__ void store4(float *p, const float (&o)[4]) {
+    *reinterpret_cast<float4 *>(p) = make_float4(o[0], o[1], o[2], o[3]);
+}
+__device__ __forceinline__ void store4(bf16 *p, const float (&o)[4]) {
+    __nv_bfloat162 a = __floats2bfloat162_rn(o[0], o[1]), b = __floats2bfloat162_rn(o[2], o[3]);
+    *reinterpret_cast<uint2 *>(p) = make_uint2(*reinterpret_cast<uint32_t *>(&a), *reinterpret_cast<uint32_t *>(&b));
+}
+
+__device__ __forceinline__ void load4(const float *p, float (&o)[4]) {
+    const float4 t = *reinterpret_cast<const float4 *>(p);
+    o[0] = t.x; o[1] = t.y; o[2] = t.z; o[3] = t.w;
+}
+__device__ __forceinline__ void load4(const bf16 *p, float (&o)[4]) {
+    const uint2 t = *reinterpret_cast<const uint2 *>(p);
+    o[0] = __uint_as_float(t.x << 16); o[1] = __uint_as_float(t.x & 0xFFFF0000u);
+    o[2] = __uint_as_float(t.y << 16); o[3] = __uint_as_float(t.y & 0xFFFF0000u);
+}
+
 // ---------------------------------------------------------------------------------
 // RMSNorm backward, row part: out = add + ((dh*g) - xhat * mean((dh*g)*xhat)) * rstd
 // ---------------------------------------------------------------------------------
@@ -88,35 +107,39 @@ __global__ void __launch_bounds__(256)
     }
     const float rstd = rstd_in[row];
     float dot = 0.f;
-    for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
-        float4 g4 = *reinterpret_cast<const float4 *>(dh + row * d + c);
-        const float gh[4] = {g4.x, g4.y, g4.z, g4.w};
+    for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {     // d is a multiple of 4 (of 8 at the C ABI)
+        float gh[4], xv[4], gn[4];
+        load4(dh + row * d + c, gh);
+        if (xF) load4(xF + row * d + c, xv);
+        else load4(xT + row * d + c, xv);
+        load4(gain + c, gn);
 #pragma unroll
-        for (int i = 0; i < 4; i++) {
-            const float xv = xF ? xF[row * d + c + i] : to_f32(xT[row * d + c + i]);
-            dot += gh[i] * to_f32(gain[c + i]) * xv * rstd;
-        }
+        for (int i = 0; i < 4; i++) dot += gh[i] * gn[i] * xv[i] * rstd;
     }
     dot = block_sum(dot, red);
     const float mean = dot / (float)d;
     for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
-        float4 g4 = *reinterpret_cast<const float4 *>(dh + row * d + c);
-        const float gh[4] = {g4.x, g4.y, g4.z, g4.w};
-        float o[4];
+        float gh[4], xv[4], gn[4], o[4];
+        load4(dh + row * d + c, gh);
+        if (xF) load4(xF + row * d + c, xv);
+        else load4(xT + row * d + c, xv);
+        load4(gain + c, gn);
 #pragma unroll
-        for (int i = 0; i < 4; i++) {
-            const float xv = xF ? xF[row * d + c + i] : to_f32(xT[row * d + c + i]);
-            const float xhat = xv * rstd;
-            float v = (gh[i] * to_f32(gain[c + i]) - xhat * mean) * rstd;
-            if (addF) v += addF[row * d + c + i];
-            if (addT) v += to_f32(addT[row * d + c + i]);
-            o[i] = v;
-        }
-        if (outF) *reinterpret_cast<float4 *>(outF + row * d + c) = make_float4(o[0], o[1], o[2], o[3]);
-        if (outT) {
+        for (int i = 0; i < 4; i++) o[i] = (gh[i] * gn[i] - xv[i] * rstd * mean) * rstd;
+        if (addF) {
+            float t[4];
+            load4(addF + row * d + c, t);
 #pragma unroll
-            for (int i = 0; i < 4; i++) outT[row * d + c + i] = from_f32<T>(o[i]);
+            for (int i = 0; i < 4; i++) o[i] += t[i];
         }
+        if (addT) {
+            float t[4];
+            load4(addT + row * d + c, t);
+#pragma unroll
+            for (int i = 0; i < 4; i++) o[i] += t[i];
+        }
+        if (outF) store4(outF + row * d + c, o);
+        if (outT) store4(outT + row * d + c, o);
     }
 }
 
@@ -487,15 +510,6 @@ int count_valid_per_chunk(const int64_t *labels, int64_t T_, int64_t chunk, int6
     const int64_t D = (T_ + chunk - 1) / chunk;
     SBP_LAUNCH(count_chunk_labels_kernel, (unsigned)D, 256, 0, st, labels, T_, chunk, ignore, counts);
     return STREAMBP_OK;
-}
-
-// four consecutive values of a row in one store (the row base and the column are multiples of 4 elements)
-__device__ __forceinline__ void store4(float *p, const float (&o)[4]) {
-    *reinterpret_cast<float4 *>(p) = make_float4(o[0], o[1], o[2], o[3]);
-}
-__device__ __forceinline__ void store4(bf16 *p, const float (&o)[4]) {
-    __nv_bfloat162 a = __floats2bfloat162_rn(o[0], o[1]), b = __floats2bfloat162_rn(o[2], o[3]);
-    *reinterpret_cast<uint2 *>(p) = make_uint2(*reinterpret_cast<uint32_t *>(&a), *reinterpret_cast<uint32_t *>(&b));
 }
 
 // one block per logits row: online (max, sum-exp), then dz = (softmax - onehot) / N
