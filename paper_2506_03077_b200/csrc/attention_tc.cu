@@ -325,11 +325,9 @@ __device__ __forceinline__ void abort_drain(volatile int *abort_flag) {
     }
 }
 
-__global__ void __launch_bounds__(BWD_THREADS, 1)
-    attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                            const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
-                            const BwdParams p) {
-    extern __shared__ uint8_t smem_raw[];
+__device__ __forceinline__ void attn_bwd_dkdv_body(const CUtensorMap &map_q, const CUtensorMap &map_k,
+                                                   const CUtensorMap &map_v, const CUtensorMap &map_do,
+                                                   const BwdParams &p, uint8_t *smem_raw, int block_x, int block_y) {
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     const uint32_t sK = base, sV = sK + TILE_BYTES, sQ = sV + TILE_BYTES, sdO = sQ + 2 * TILE_BYTES;
@@ -344,8 +342,8 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
     volatile int *abort_flag = reinterpret_cast<volatile int *>(aux + 104);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int g = blockIdx.y, G = p.Hq / p.Hkv;
-    const long long k_abs0 = (long long)blockIdx.x * TILE;
+    const int g = block_y, G = p.Hq / p.Hkv;
+    const long long k_abs0 = (long long)block_x * TILE;
     const int nqt = (p.n + TILE - 1) / TILE;
     const int first_qt = k_abs0 > p.q0 ? (int)((k_abs0 - p.q0) / TILE) : 0;
     const int per_head = nqt - first_qt;
@@ -569,11 +567,9 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
     }
 }
 
-__global__ void __launch_bounds__(BWD_THREADS, 1)
-    attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                          const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
-                          const BwdParams p) {
-    extern __shared__ uint8_t smem_raw[];
+__device__ __forceinline__ void attn_bwd_dq_body(const CUtensorMap &map_q, const CUtensorMap &map_k,
+                                                 const CUtensorMap &map_v, const CUtensorMap &map_do,
+                                                 const BwdParams &p, uint8_t *smem_raw, int block_x, int block_y) {
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     // K tiles live from S_j to dQ_j, so their ring has three stages: the copy of tile j+2 then starts when dQ of
@@ -588,8 +584,8 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
     volatile int *abort_flag = reinterpret_cast<volatile int *>(aux + 136);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int h = blockIdx.y, g = h / (p.Hq / p.Hkv);
-    const int qt0 = blockIdx.x * TILE;
+    const int h = block_y, g = h / (p.Hq / p.Hkv);
+    const int qt0 = block_x * TILE;
     const long long q_abs0 = p.q0 + qt0;
     const int rows_here = (p.n - qt0) < TILE ? (p.n - qt0) : TILE;
     const long long kv_end = q_abs0 + rows_here;
@@ -769,6 +765,25 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
     }
 }
 
+// One launch for both backward kernels.  They are independent (both read Q, K, V, dO, lse, delta; one owns dK / dV
+// tiles, the other dQ tiles), and at short prefixes or small chunks neither fills the GPU on its own (e.g. 32 to
+// 256 key-tile CTAs and 224 query-tile CTAs per chunk of the 7B layer at chunk 1024): as one grid their CTAs pack
+// onto the SMs together.  The dK / dV CTAs come first (they run longest), lowest key tiles (most query tiles) first.
+constexpr int BWD_FUSED_SMEM = BWD_SMEM > DQ_SMEM ? BWD_SMEM : DQ_SMEM;
+__global__ void __launch_bounds__(BWD_THREADS, 1)
+    attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                       const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
+                       const BwdParams p, int kv_tiles, int n_dkdv, int q_tiles) {
+    extern __shared__ uint8_t smem_raw[];
+    const int b = (int)blockIdx.x;
+    if (b < n_dkdv) {
+        attn_bwd_dkdv_body(map_q, map_k, map_v, map_do, p, smem_raw, b % kv_tiles, b / kv_tiles);
+    } else {
+        const int c = b - n_dkdv;
+        attn_bwd_dq_body(map_q, map_k, map_v, map_do, p, smem_raw, q_tiles - 1 - c % q_tiles, c / q_tiles);
+    }
+}
+
 template <typename K>
 bool opt_in_smem(K kernel, int bytes) {
     return cuda_ok(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
@@ -815,16 +830,16 @@ int attention_bwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, const bf16 *do
         return STREAMBP_E_CUDA;
     static bool configured = false;
     if (!configured) {
-        if (!opt_in_smem(attn_bwd_dkdv_tc_kernel, BWD_SMEM) || !opt_in_smem(attn_bwd_dq_tc_kernel, DQ_SMEM))
-            return STREAMBP_E_CUDA;
+        if (!opt_in_smem(attn_bwd_tc_kernel, BWD_FUSED_SMEM)) return STREAMBP_E_CUDA;
         configured = true;
     }
     const float scale = 1.f / sqrtf((float)TILE);
     BwdParams p{(int)n, (long long)q0, Hq, Hkv, lse, delta, dq, dk, dv, scale, scale * kLog2e};
-    dim3 gkv((unsigned)((kv_len + TILE - 1) / TILE), Hkv);
-    dim3 gq((unsigned)((n + TILE - 1) / TILE), Hq);
-    SBP_LAUNCH(attn_bwd_dkdv_tc_kernel, gkv, BWD_THREADS, BWD_SMEM, st, mq, mk, mv, mdo, p);
-    SBP_LAUNCH(attn_bwd_dq_tc_kernel, gq, BWD_THREADS, DQ_SMEM, st, mq, mk, mv, mdo, p);
+    const int kv_tiles = (int)((kv_len + TILE - 1) / TILE), q_tiles = (int)((n + TILE - 1) / TILE);
+    const int64_t n_dkdv = (int64_t)kv_tiles * Hkv, n_dq = (int64_t)q_tiles * Hq;
+    if (n_dkdv + n_dq > 0x7fffffff) return STREAMBP_E_SHAPE;
+    SBP_LAUNCH(attn_bwd_tc_kernel, (unsigned)(n_dkdv + n_dq), BWD_THREADS, BWD_FUSED_SMEM, st, mq, mk, mv, mdo, p,
+               kv_tiles, (int)n_dkdv, q_tiles);
     return STREAMBP_OK;
 }
 
