@@ -280,7 +280,7 @@ __global__ void __launch_bounds__(FWD16_THREADS, 1)
 }
 
 // ---------------------------------------------------------------------------------------------
-// Backward.  Two kernels, both deterministic (no floating-point atomics):
+// Backward.  Two CTA roles in one grid (attn_bwd_tc_kernel), both deterministic (no floating-point atomics):
 //   dK/dV: one CTA per (128-key tile, KV head); K and V tiles stay in shared memory; loops over the
 //          G query heads of the group and over the query tiles that can see the key tile.
 //          S^T = K Q^T and dP^T = V dO^T land in tensor memory with keys on the lanes, so a thread owns
