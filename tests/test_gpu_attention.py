@@ -118,3 +118,46 @@ def test_attention_cuda_core_variants(dh, dtype):
     assert O.rel_frobenius(dq.cpu().numpy(), dq_ref) < tol
     assert O.rel_frobenius(dk.cpu().numpy(), dk_ref) < tol
     assert O.rel_frobenius(dv.cpu().numpy(), dv_ref) < tol
+
+
+def test_attention_growing_maxima_tensor_core():
+    """Scores that grow with the key index: the running row maximum rises by more than the lazy-rescale threshold
+    (2^8) from one 128-key tile to the next, so the forward kernel has to rescale its output accumulator at every
+    tile and the backward sees probabilities concentrated at the end of each row.  Pins the exactness of the lazy
+    rescale (output and log-sum-exp) against the oracle's plain softmax."""
+    n, q0, Hq, Hkv, dh, dt = 256, 768, 2, 1, 128, torch.bfloat16
+    kv = q0 + n
+    q, k, v, do = make_qkv(31, n, q0, Hq, Hkv, dh, dt, scale=0.25)
+    # a common direction e: q gets +4 e, key j gets +(j / 128) * 3.5 e  ->  score += 14 * (tile index) / sqrt(128) * ...
+    e = np.zeros(dh); e[:8] = 1.0
+    q = synth.round_bf16(q + 4.0 * e)
+    k = synth.round_bf16(k + (np.arange(kv)[:, None, None] / 128.0) * 3.5 * e)
+    tile_step = 4.0 * 3.5 * 8 / np.sqrt(dh) * 1.4426950408889634      # rise of the score per tile, in log2 units
+    assert tile_step > 8.0
+    o_ref, dq_ref, dk_ref, dv_ref = oracle_chunk(q, k, v, do, q0)
+    qd = torch.from_numpy(q[q0:]).to("cuda", dt).contiguous()
+    dod = torch.from_numpy(do[q0:]).to("cuda", dt).contiguous()
+    kd, vd = torch.from_numpy(k).to("cuda", dt), torch.from_numpy(v).to("cuda", dt)
+    o = torch.full((n, Hq, dh), float("nan"), device="cuda", dtype=dt)
+    lse = torch.full((Hq, n), float("nan"), device="cuda")
+    B.attention_forward(qd, kd, vd, q0, o, lse, engine=2)
+    got = o.float().cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    assert O.rel_frobenius(got, o_ref) < 6e-3
+    lse_ref = oracle_lse(q, k, q0, dh)
+    assert np.abs(lse.cpu().numpy() - lse_ref).max() < 2e-3 * max(1.0, np.abs(lse_ref).max() / 10)
+    # backward: dK and dV are well conditioned.  dQ = sum_j dS_j K_j is not, here: the rows of dS sum to zero, which
+    # cancels the large common component of these keys only as exactly as delta = rowsum(dO * O) is known, and O is
+    # stored in bf16.  The fp32 CUDA-core engine, fed the same bf16 O, shows the same loss; the tensor-core engine
+    # must stay within a small factor of it.
+    errs = {}
+    for engine in (1, 2):
+        dq = torch.full((n, Hq, dh), float("nan"), device="cuda")
+        dk = torch.zeros((kv, Hkv, dh), device="cuda")
+        dv = torch.zeros((kv, Hkv, dh), device="cuda")
+        B.attention_backward(qd, kd, vd, o, dod, lse, q0, dq, dk, dv, engine=engine)
+        torch.cuda.synchronize()
+        errs[engine] = (O.rel_frobenius(dq.cpu().numpy(), dq_ref), O.rel_frobenius(dk.cpu().numpy(), dk_ref),
+                        O.rel_frobenius(dv.cpu().numpy(), dv_ref))
+    assert errs[2][1] < 1e-2 and errs[2][2] < 1e-2
+    assert errs[2][0] < 2.5 * errs[1][0] + 1e-2
