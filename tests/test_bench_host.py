@@ -17,7 +17,7 @@ from paper_2506_03077_b200 import synth  # noqa: E402
 
 
 def test_layer_flops_match_the_published_totals():
-    # qwen7b layer T 8192 -> 12.03 TFLOP, llama8b layer T 32768 -> 69.82 TFLOP
+    # algorithmic totals of the two layer workloads: qwen7b layer T 8192 -> 12.03 TFLOP, llama8b layer T 32768 -> 69.82 TFLOP
     assert abs(bench.layer_flops(synth.QWEN7B_LAYER, 8192) / 1e12 - 12.03) < 0.01
     assert abs(bench.layer_flops(synth.LLAMA8B_LAYER, 32768) / 1e12 - 69.82) < 0.01
 
