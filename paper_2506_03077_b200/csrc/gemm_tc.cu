@@ -21,6 +21,9 @@
 // Every mbarrier wait is bounded (2 s of %globaltimer): on expiry the CTA raises a fault flag that
 // streambp_last_device_status() reports as STREAMBP_E_DEVICE_TIMEOUT, all roles leave their loops,
 // tensor memory is released and the kernel returns.
+#include <algorithm>
+#include <cstdio>
+#include <cstdlib>
 #include <cstring>
 
 #include "sm100.cuh"
@@ -37,6 +40,11 @@ constexpr int EPI_BYTES = 4 * 2 * EPI_BUF_BYTES;          // 4 epilogue warps, d
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 /* alignment slack */ + 256 /* barriers, tile ring */;
 constexpr int NUM_THREADS = 192;
 constexpr uint32_t TMEM_COLS = 512;
+// CTA-pair kernel: a pair works on a 256 x 256 tile, each CTA holding its 128 rows of A and its half of B
+constexpr int PAIR_BM = 2 * BM, PAIR_STAGES = 6;
+constexpr int PAIR_B_BYTES = (BN / 2) * BK * 2;             // 16 KiB
+constexpr int PAIR_STAGE_BYTES = A_BYTES + PAIR_B_BYTES;    // 32 KiB
+constexpr int PAIR_SMEM_BYTES = PAIR_STAGES * PAIR_STAGE_BYTES + EPI_BYTES + 1024 + 256;
 
 }  // namespace
 
@@ -136,6 +144,7 @@ __device__ __forceinline__ T pick(const T (&a)[MAX_PROBS], int q) {
 }
 
 struct TileRef { int q, m0, n0, seg0, seg1; };
+template <int TILE_M>
 __device__ __forceinline__ TileRef locate(const GroupParams &p, int tile) {
     int q = 0;
 #pragma unroll
@@ -148,7 +157,7 @@ __device__ __forceinline__ TileRef locate(const GroupParams &p, int tile) {
         s1 = (q == i) ? p.seg_begin[i + 1] : s1;
     }
     const int local = tile - tb, tm = pick(p.tiles_m, q);
-    return {q, (local % tm) * BM, (local / tm) * BN, s0, s1};
+    return {q, (local % tm) * TILE_M, (local / tm) * BN, s0, s1};
 }
 
 // The K loops of one tile, specialised on the operand layouts so that descriptor strides and the choice of
@@ -214,6 +223,77 @@ __device__ __forceinline__ bool mma_tile(const GroupParams &p, const TileRef &t,
     return true;
 }
 
+// One epilogue warp: rows m_base + 32 * quarter .. + 31 of tile t, all BN columns, from the accumulator at `acc`
+// (lane = row).  fp32 output: 32 x 32 blocks staged in shared memory with the 128-byte swizzle the tensor map expects,
+// then a TMA store, or a TMA reduce-add when accumulating; bf16 output: 16-byte stores from registers.
+__device__ __forceinline__ void epilogue_rows(const GroupParams &p, const TileRef &t, int m_base, int quarter, int lane,
+                                              uint32_t acc, uint32_t epi, uint32_t &staged) {
+    const uint32_t fl = pick(p.flags, t.q);
+    const int Mq = pick(p.M, t.q), Nq = pick(p.N, t.q);
+    const bf16 *bias = pick(p.bias, t.q);
+    const CUtensorMap *mc = &p.map_c[t.q];
+    const int row = m_base + quarter * 32 + lane;
+    const uint32_t taddr = acc + ((uint32_t)(quarter * 32) << 16);
+    bf16 *out_row = reinterpret_cast<bf16 *>(pick(p.C, t.q)) + (long long)row * pick(p.ldc, t.q);
+#pragma unroll 1
+    for (int c = 0; c < BN / 32; c++) {
+        const int col0 = t.n0 + c * 32;
+        if (col0 >= Nq) break;               // uniform across the warp
+        uint32_t r[32];
+        tmem_ld32(taddr + c * 32, r);
+        if (fl & F_OUT_F32) {
+            // stage the warp's 32 x 32 block (row = lane) with the 128-byte swizzle the tensor map expects
+            const uint32_t buf_s = epi + (uint32_t)(quarter * 2 + (staged & 1u)) * EPI_BUF_BYTES;
+            staged++;
+            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+            __syncwarp();
+#pragma unroll
+            for (int j = 0; j < 8; j++) {
+                float v[4];
+#pragma unroll
+                for (int e = 0; e < 4; e++) {
+                    v[e] = __uint_as_float(r[4 * j + e]);
+                    if (bias && col0 + 4 * j + e < Nq) v[e] += __bfloat162float(bias[col0 + 4 * j + e]);
+                }
+                const uint32_t dst = buf_s + lane * 128 + ((j ^ (lane & 7)) << 4);
+                asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v[0]), "f"(v[1]),
+                             "f"(v[2]), "f"(v[3])
+                             : "memory");
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) {
+                if (fl & F_ACC) tma_reduce_add_2d(mc, buf_s, col0, m_base + quarter * 32);
+                else tma_store_2d(mc, buf_s, col0, m_base + quarter * 32);
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            }
+        } else if (row < Mq) {
+            bf16 *out = out_row + col0;
+#pragma unroll
+            for (int j = 0; j < 32; j += 8) {
+                float v[8];
+#pragma unroll
+                for (int e = 0; e < 8; e++) {
+                    v[e] = __uint_as_float(r[j + e]);
+                    if (bias && col0 + j + e < Nq) v[e] += __bfloat162float(bias[col0 + j + e]);
+                }
+                if (col0 + j + 7 < Nq) {
+                    uint32_t w[4];
+#pragma unroll
+                    for (int e = 0; e < 4; e++) {
+                        __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]);
+                        w[e] = *reinterpret_cast<uint32_t *>(&h);
+                    }
+                    *reinterpret_cast<uint4 *>(out + j) = make_uint4(w[0], w[1], w[2], w[3]);
+                } else {
+                    for (int e = 0; e < 8; e++)
+                        if (col0 + j + e < Nq) out[j + e] = __float2bfloat16_rn(v[e]);
+                }
+            }
+        }
+    }
+}
+
 __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_group_kernel(const __grid_constant__ GroupParams p) {
     extern __shared__ uint8_t smem_raw[];
     if (gated_off(p.gate)) return;
@@ -273,7 +353,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_group_kernel(const __grid
                 if (tile < 0) break;
                 // the next index is requested now and first looked at after this tile's loads are issued
                 const int next = dynamic ? atomicAdd(p.sched, 1) : tile + (int)gridDim.x;
-                const TileRef t = locate(p, tile);
+                const TileRef t = locate<BM>(p, tile);
                 const uint32_t fl = pick(p.flags, t.q);
                 const Pipe pipe{tiles, bar_full, bar_empty, abort_flag};
                 switch (fl & (F_A_MN | F_B_MN)) {
@@ -304,7 +384,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_group_kernel(const __grid
                 mbar_arrive(bar_rempty + 8 * slot);
                 if (++slot == RING) { slot = 0; rphase ^= 1u; }
                 if (tile < 0) break;
-                const TileRef t = locate(p, tile);
+                const TileRef t = locate<BM>(p, tile);
                 const uint32_t fl = pick(p.flags, t.q);
                 const uint32_t buf = local & 1u, use = local >> 1;
                 if (!mbar_wait(bar_tempty + 8 * buf, (use & 1u) ^ 1u, abort_flag)) break;
@@ -331,75 +411,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_group_kernel(const __grid
             if (lane == 0) mbar_arrive(bar_rempty + 8 * slot);
             if (++slot == RING) { slot = 0; rphase ^= 1u; }
             if (tile < 0) break;
-            const TileRef t = locate(p, tile);
-            const uint32_t fl = pick(p.flags, t.q);
-            const int Mq = pick(p.M, t.q), Nq = pick(p.N, t.q);
-            const bf16 *bias = pick(p.bias, t.q);
-            const CUtensorMap *mc = &p.map_c[t.q];
+            const TileRef t = locate<BM>(p, tile);
             const uint32_t buf = local & 1u, use = local >> 1;
             local++;
             if (!mbar_wait(bar_tfull + 8 * buf, use & 1u, abort_flag)) break;
             tc_fence_after();
-            const int row = t.m0 + quarter * 32 + lane;
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * BN;
-            bf16 *out_row = reinterpret_cast<bf16 *>(pick(p.C, t.q)) + (long long)row * pick(p.ldc, t.q);
-#pragma unroll 1
-            for (int c = 0; c < BN / 32; c++) {
-                const int col0 = t.n0 + c * 32;
-                if (col0 >= Nq) break;               // uniform across the warp
-                uint32_t r[32];
-                tmem_ld32(taddr + c * 32, r);
-                if (fl & F_OUT_F32) {
-                    // stage the warp's 32 x 32 block (row = lane) with the 128-byte swizzle the tensor map expects
-                    const uint32_t buf_s = epi + (uint32_t)(quarter * 2 + (staged & 1u)) * EPI_BUF_BYTES;
-                    staged++;
-                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-                    __syncwarp();
-#pragma unroll
-                    for (int j = 0; j < 8; j++) {
-                        float v[4];
-#pragma unroll
-                        for (int e = 0; e < 4; e++) {
-                            v[e] = __uint_as_float(r[4 * j + e]);
-                            if (bias && col0 + 4 * j + e < Nq) v[e] += __bfloat162float(bias[col0 + 4 * j + e]);
-                        }
-                        const uint32_t dst = buf_s + lane * 128 + ((j ^ (lane & 7)) << 4);
-                        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v[0]), "f"(v[1]),
-                                     "f"(v[2]), "f"(v[3])
-                                     : "memory");
-                    }
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    __syncwarp();
-                    if (lane == 0) {
-                        if (fl & F_ACC) tma_reduce_add_2d(mc, buf_s, col0, t.m0 + quarter * 32);
-                        else tma_store_2d(mc, buf_s, col0, t.m0 + quarter * 32);
-                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                    }
-                } else if (row < Mq) {
-                    bf16 *out = out_row + col0;
-#pragma unroll
-                    for (int j = 0; j < 32; j += 8) {
-                        float v[8];
-#pragma unroll
-                        for (int e = 0; e < 8; e++) {
-                            v[e] = __uint_as_float(r[j + e]);
-                            if (bias && col0 + j + e < Nq) v[e] += __bfloat162float(bias[col0 + j + e]);
-                        }
-                        if (col0 + j + 7 < Nq) {
-                            uint32_t w[4];
-#pragma unroll
-                            for (int e = 0; e < 4; e++) {
-                                __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]);
-                                w[e] = *reinterpret_cast<uint32_t *>(&h);
-                            }
-                            *reinterpret_cast<uint4 *>(out + j) = make_uint4(w[0], w[1], w[2], w[3]);
-                        } else {
-                            for (int e = 0; e < 8; e++)
-                                if (col0 + j + e < Nq) out[j + e] = __float2bfloat16_rn(v[e]);
-                        }
-                    }
-                }
-            }
+            epilogue_rows(p, t, t.m0, quarter, lane, tmem_base + buf * BN, epi, staged);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
@@ -418,6 +435,243 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_group_kernel(const __grid
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// CTA-pair variant (tcgen05 cta_group::2).  The two CTAs of a cluster sit on the two SMs of one TPC and
+// share every MMA: a 256 x 256 x 64 step is issued by the even CTA, reads 128 rows of A and 128 rows of B
+// from the shared memory of EACH CTA and leaves 128 rows of the accumulator in the tensor memory of each.
+// Per CTA a K slice is then 32 KiB instead of 48, so the same shared memory holds six stages instead of
+// four -- the main loop of the single-CTA kernel spends about half of its time waiting for operand copies
+// (their latency under load is ~3000 cycles, four 512-cycle slices do not cover it) -- and a third less
+// data crosses L2 -> SM per FLOP.  Roles per CTA as in gemm_group_kernel; in addition
+//   * the even CTA's scheduler thread publishes each tile index in both CTAs' rings,
+//   * operand copies of both CTAs report to the even CTA's `full` barrier (armed there with the bytes of
+//     both); the MMA thread's commits arrive at `empty` / `tfull` in both CTAs,
+//   * the odd CTA's ring readers and epilogue warps arrive at the even CTA's `rempty` / `tempty`.
+// No copy is multicast: each CTA fetches its own operand rows.
+// ---------------------------------------------------------------------------------------------
+template <bool A_MN, bool B_MN>
+__device__ __forceinline__ bool produce_tile_pair(const GroupParams &p, const TileRef &t, const Pipe &pp, uint32_t rank,
+                                                  uint32_t &stage, uint32_t &phase) {
+    const int m = t.m0 + BM * (int)rank, n = t.n0 + (BN / 2) * (int)rank;
+    for (int s = t.seg0; s < t.seg1; s++) {
+        const CUtensorMap *ma = &p.map_a[s], *mb = &p.map_b[s];
+        const int nkb = p.seg_kb[s];
+        for (int kb = 0; kb < nkb; kb++) {
+            if (!mbar_wait(pp.bar_empty + 8 * stage, phase ^ 1u, pp.abort_flag)) return false;
+            if (rank == 0) mbar_expect_tx(pp.bar_full + 8 * stage, 2 * PAIR_STAGE_BYTES);
+            const uint32_t full = map_to_cta(pp.bar_full + 8 * stage, 0);
+            const uint32_t sa = pp.tiles + stage * PAIR_STAGE_BYTES, sb = sa + A_BYTES;
+            const int k0 = kb * BK;
+            if (A_MN) {
+#pragma unroll
+                for (int j = 0; j < BM / 64; j++) tma_load_2d_pair(sa + j * 8192, ma, full, m + 64 * j, k0);
+            } else {
+                tma_load_2d_pair(sa, ma, full, k0, m);
+            }
+            if (B_MN) {
+#pragma unroll
+                for (int j = 0; j < BN / 128; j++) tma_load_2d_pair(sb + j * 8192, mb, full, n + 64 * j, k0);
+            } else {
+                tma_load_2d_pair(sb, mb, full, k0, n);
+            }
+            if (++stage == PAIR_STAGES) { stage = 0; phase ^= 1u; }
+        }
+    }
+    return true;
+}
+
+template <bool A_MN, bool B_MN>
+__device__ __forceinline__ bool mma_tile_pair(const GroupParams &p, const TileRef &t, const Pipe &pp, uint32_t d_tmem,
+                                              uint32_t &stage, uint32_t &phase) {
+    constexpr uint32_t idesc = make_idesc(PAIR_BM, BN, A_MN, B_MN);
+    constexpr uint32_t a_step = A_MN ? 2048u : 32u, b_step = B_MN ? 2048u : 32u;   // bytes per 16 k
+    uint32_t first = 0;
+    for (int s = t.seg0; s < t.seg1; s++) {
+        const int nkb = p.seg_kb[s];
+        for (int kb = 0; kb < nkb; kb++) {
+            if (!mbar_wait_cluster(pp.bar_full + 8 * stage, phase, pp.abort_flag)) return false;
+            tc_fence_after();
+            const uint32_t sa = pp.tiles + stage * PAIR_STAGE_BYTES, sb = sa + A_BYTES;
+            const uint32_t a_lo = desc_lo(sa, A_MN ? 8192u : 16u), b_lo = desc_lo(sb, B_MN ? 8192u : 16u);
+#pragma unroll
+            for (int kk = 0; kk < BK / 16; kk++)
+                umma_ss_pair(d_tmem, a_lo + kk * (a_step >> 4), b_lo + kk * (b_step >> 4), idesc, first | (uint32_t)kk);
+            first = 1u;
+            umma_commit_pair(pp.bar_empty + 8 * stage);   // frees the stage in both CTAs
+            if (++stage == PAIR_STAGES) { stage = 0; phase ^= 1u; }
+        }
+    }
+    return true;
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
+    gemm_pair_kernel(const __grid_constant__ GroupParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    if (gated_off(p.gate)) return;
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;
+    const uint32_t epi = tiles + PAIR_STAGES * PAIR_STAGE_BYTES;
+    uint8_t *aux = smem_raw + (tiles - raw) + PAIR_STAGES * PAIR_STAGE_BYTES + EPI_BYTES;
+    const uint32_t bar_full = smem_u32(aux);                  // PAIR_STAGES x 8 B, used in the even CTA
+    const uint32_t bar_empty = bar_full + 8 * PAIR_STAGES;    // PAIR_STAGES x 8 B, in both
+    const uint32_t bar_tfull = bar_empty + 8 * PAIR_STAGES;   // 2 x 8 B, in both
+    const uint32_t bar_tempty = bar_tfull + 16;               // 2 x 8 B, even CTA: eight epilogue warps arrive
+    const uint32_t bar_rfull = bar_tempty + 16;               // RING x 8 B, in both
+    const uint32_t bar_rempty = bar_rfull + 8 * RING;         // RING x 8 B, even CTA: ten readers arrive
+    uint8_t *aux2 = aux + 8 * PAIR_STAGES * 2 + 32 + 16 * RING;
+    volatile int *ring = reinterpret_cast<volatile int *>(aux2);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux2 + 4 * RING);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(aux2 + 4 * RING + 8);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_cta_rank();
+    const int num_tiles = p.tile_begin[p.nprob < MAX_PROBS ? p.nprob : MAX_PROBS];
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < PAIR_STAGES; s++) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int b = 0; b < 2; b++) {
+            mbar_init(bar_tfull + 8 * b, 1);
+            mbar_init(bar_tempty + 8 * b, 8);
+        }
+        for (int s = 0; s < RING; s++) {
+            mbar_init(bar_rfull + 8 * s, 1);
+            mbar_init(bar_rempty + 8 * s, 10);      // even CTA: MMA thread + 4 epilogue warps; odd CTA: producer + 4
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc_pair(smem_u32(tmem_slot), TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();            // both CTAs' barriers exist before anything arrives at them
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const Pipe pipe{tiles, bar_full, bar_empty, abort_flag};
+
+    if (warp == 0) {
+        // ------------------------------ tile scheduler (even CTA) + TMA producer ------------------------------
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0, slot = 0, rphase = 0;
+            bool alive = true;
+            if (rank == 0) {
+                const bool dynamic = p.sched != nullptr;
+                const int npairs = (int)(gridDim.x >> 1);
+                int tile = dynamic ? atomicAdd(p.sched, 1) : (int)(blockIdx.x >> 1);
+                while (alive) {
+                    if (tile >= num_tiles) tile = -1;
+                    if (!mbar_wait_cluster(bar_rempty + 8 * slot, rphase ^ 1u, abort_flag)) break;
+                    ring[slot] = tile;
+                    st_remote_u32(map_to_cta(smem_u32(const_cast<int *>(ring + slot)), 1), (uint32_t)tile);
+                    mbar_arrive(bar_rfull + 8 * slot);
+                    mbar_arrive_remote(map_to_cta(bar_rfull + 8 * slot, 1));
+                    if (++slot == RING) { slot = 0; rphase ^= 1u; }
+                    if (tile < 0) break;
+                    const int next = dynamic ? atomicAdd(p.sched, 1) : tile + npairs;
+                    const TileRef t = locate<PAIR_BM>(p, tile);
+                    switch (pick(p.flags, t.q) & (F_A_MN | F_B_MN)) {
+                        case 0: alive = produce_tile_pair<false, false>(p, t, pipe, 0u, stage, phase); break;
+                        case F_B_MN: alive = produce_tile_pair<false, true>(p, t, pipe, 0u, stage, phase); break;
+                        default: alive = produce_tile_pair<true, true>(p, t, pipe, 0u, stage, phase); break;
+                    }
+                    tile = next;
+                }
+                if (dynamic) {
+                    // every pair takes exactly one index past the end; the last one to get there re-arms the counter
+                    __threadfence();
+                    if (atomicAdd(p.sched + 1, 1) == npairs - 1) {
+                        p.sched[0] = 0;
+                        p.sched[1] = 0;
+                        __threadfence();
+                    }
+                }
+            } else {
+                while (alive) {
+                    if (!mbar_wait_cluster(bar_rfull + 8 * slot, rphase, abort_flag)) break;
+                    const int tile = ring[slot];
+                    mbar_arrive_remote(map_to_cta(bar_rempty + 8 * slot, 0));
+                    if (++slot == RING) { slot = 0; rphase ^= 1u; }
+                    if (tile < 0) break;
+                    const TileRef t = locate<PAIR_BM>(p, tile);
+                    switch (pick(p.flags, t.q) & (F_A_MN | F_B_MN)) {
+                        case 0: alive = produce_tile_pair<false, false>(p, t, pipe, 1u, stage, phase); break;
+                        case F_B_MN: alive = produce_tile_pair<false, true>(p, t, pipe, 1u, stage, phase); break;
+                        default: alive = produce_tile_pair<true, true>(p, t, pipe, 1u, stage, phase); break;
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer (even CTA only) ------------------------------
+        if (lane == 0 && rank == 0) {
+            uint32_t stage = 0, phase = 0, slot = 0, rphase = 0, local = 0;
+            bool alive = true;
+            while (alive) {
+                if (!mbar_wait(bar_rfull + 8 * slot, rphase, abort_flag)) break;
+                const int tile = ring[slot];
+                mbar_arrive(bar_rempty + 8 * slot);
+                if (++slot == RING) { slot = 0; rphase ^= 1u; }
+                if (tile < 0) break;
+                const TileRef t = locate<PAIR_BM>(p, tile);
+                const uint32_t buf = local & 1u, use = local >> 1;
+                if (!mbar_wait_cluster(bar_tempty + 8 * buf, (use & 1u) ^ 1u, abort_flag)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * BN;
+                switch (pick(p.flags, t.q) & (F_A_MN | F_B_MN)) {
+                    case 0: alive = mma_tile_pair<false, false>(p, t, pipe, d_tmem, stage, phase); break;
+                    case F_B_MN: alive = mma_tile_pair<false, true>(p, t, pipe, d_tmem, stage, phase); break;
+                    default: alive = mma_tile_pair<true, true>(p, t, pipe, d_tmem, stage, phase); break;
+                }
+                if (alive) umma_commit_pair(bar_tfull + 8 * buf);   // accumulator complete, in both CTAs
+                local++;
+            }
+        }
+    } else {
+        // ------------------------------ epilogue: this CTA's 128 rows of the tile ------------------------------
+        const int quarter = warp & 3;
+        uint32_t local = 0, staged = 0, slot = 0, rphase = 0;
+        while (true) {
+            if (!mbar_wait_cluster(bar_rfull + 8 * slot, rphase, abort_flag)) break;
+            const int tile = ring[slot];
+            __syncwarp();
+            if (lane == 0) {
+                if (rank == 0) mbar_arrive(bar_rempty + 8 * slot);
+                else mbar_arrive_remote(map_to_cta(bar_rempty + 8 * slot, 0));
+            }
+            if (++slot == RING) { slot = 0; rphase ^= 1u; }
+            if (tile < 0) break;
+            const TileRef t = locate<PAIR_BM>(p, tile);
+            const uint32_t buf = local & 1u, use = local >> 1;
+            local++;
+            if (!mbar_wait(bar_tfull + 8 * buf, use & 1u, abort_flag)) break;
+            tc_fence_after();
+            epilogue_rows(p, t, t.m0 + BM * (int)rank, quarter, lane, tmem_base + buf * BN, epi, staged);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+                if (rank == 0) mbar_arrive(bar_tempty + 8 * buf);
+                else mbar_arrive_remote(map_to_cta(bar_tempty + 8 * buf, 0));
+            }
+        }
+    }
+
+    if (warp >= 2 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    __syncwarp();
+    if (*abort_flag) {
+        const unsigned long long t0 = global_timer();
+        while (global_timer() - t0 < 200000ull) { }
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();            // neither CTA's shared or tensor memory goes away while the other may still reach it
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, TMEM_COLS);
     }
 }
 
@@ -453,8 +707,36 @@ bool gemm_tc_group_supported(const GemmProb *probs, int n) {
     return segs <= MAX_SEGS;
 }
 
+namespace {
+// The CTA-pair kernel needs clusters of two CTAs with the full shared-memory carve-out; where the device cannot
+// co-schedule even one such cluster the single-CTA kernel runs instead.
+bool pair_kernel_available() {
+    static int state = -1;
+    if (state < 0) {
+        state = 0;
+        if (cudaFuncSetAttribute(gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PAIR_SMEM_BYTES) ==
+            cudaSuccess) {
+            cudaLaunchConfig_t cfg;
+            memset(&cfg, 0, sizeof(cfg));
+            cfg.gridDim = dim3(2, 1, 1);
+            cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+            cfg.dynamicSmemBytes = PAIR_SMEM_BYTES;
+            int clusters = 0;
+            if (cudaOccupancyMaxActiveClusters(&clusters, gemm_pair_kernel, &cfg) == cudaSuccess && clusters >= 1)
+                state = 1;
+        }
+        cudaGetLastError();
+        if (getenv("STREAMBP_GEMM_SINGLE_CTA")) state = 0;
+        if (getenv("STREAMBP_VERBOSE")) fprintf(stderr, "streambp: tcgen05 product kernel: %s\n", state ? "CTA pairs" : "single CTA");
+    }
+    return state == 1;
+}
+}  // namespace
+
 int gemm_tc_group(const GemmProb *probs, int n, int *sched, cudaStream_t st) {
     if (!gemm_tc_group_supported(probs, n)) return STREAMBP_E_SHAPE;
+    const bool pair = pair_kernel_available();
+    const int tile_m = pair ? PAIR_BM : BM;
     // longest tiles first: with a dynamic schedule the short tiles then fill the gaps the long ones leave
     int order[MAX_PROBS];
     int64_t cost[MAX_PROBS];
@@ -484,7 +766,7 @@ int gemm_tc_group(const GemmProb *probs, int n, int *sched, cudaStream_t st) {
             if (a_mn) ok = make_tensor_map(&p.map_a[seg], e.A, e.K, g.M, e.lda, 64, BK, false);
             else ok = make_tensor_map(&p.map_a[seg], e.A, g.M, e.K, e.lda, BK, BM, false);
             if (b_mn) ok = ok && make_tensor_map(&p.map_b[seg], e.B, e.K, g.N, e.ldb, 64, BK, false);
-            else ok = ok && make_tensor_map(&p.map_b[seg], e.B, g.N, e.K, e.ldb, BK, BN, false);
+            else ok = ok && make_tensor_map(&p.map_b[seg], e.B, g.N, e.K, e.ldb, BK, pair ? BN / 2 : BN, false);
             if (!ok) return STREAMBP_E_CUDA;
             p.seg_kb[seg] = (int)((e.K + BK - 1) / BK);
         }
@@ -493,7 +775,7 @@ int gemm_tc_group(const GemmProb *probs, int n, int *sched, cudaStream_t st) {
         } else {
             p.map_c[i] = p.map_a[p.seg_begin[i]];   // unused by bf16 outputs
         }
-        p.tiles_m[i] = (int)((g.M + BM - 1) / BM);
+        p.tiles_m[i] = (int)((g.M + tile_m - 1) / tile_m);
         p.M[i] = (int)g.M;
         p.N[i] = (int)g.N;
         p.C[i] = g.C;
@@ -515,6 +797,12 @@ int gemm_tc_group(const GemmProb *probs, int n, int *sched, cudaStream_t st) {
         if (!cuda_ok(cudaFuncSetAttribute(gemm_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES)))
             return STREAMBP_E_CUDA;
         configured = true;
+    }
+    if (pair) {
+        const int pairs = std::max(1, sm_count() / 2);
+        const int grid = 2 * (tiles < pairs ? (int)tiles : pairs);
+        SBP_LAUNCH(gemm_pair_kernel, grid, NUM_THREADS, PAIR_SMEM_BYTES, st, p);
+        return STREAMBP_OK;
     }
     const int grid = tiles < sm_count() ? (int)tiles : sm_count();
     SBP_LAUNCH(gemm_group_kernel, grid, NUM_THREADS, SMEM_BYTES, st, p);
