@@ -29,6 +29,13 @@
  *     back with streambp_last_device_status().  Nothing aborts, traps or throws.
  *   - `accumulate` = 0 overwrites the weight-gradient outputs ("initialised from
  *     zero", text after Eq. (3)); 1 adds to what they hold.
+ *   - Environment, read once per process: STREAMBP_GEMM_ENGINE = "simt" | "tc"
+ *     forces the CUDA-core or the tcgen05 product kernels (default: tcgen05 for bf16,
+ *     CUDA cores for fp32); STREAMBP_GEMM_SINGLE_CTA (any value) selects the
+ *     single-CTA tcgen05 product kernel instead of the CTA-pair one, which is also
+ *     what runs where a two-CTA cluster cannot be scheduled; STREAMBP_VERBOSE (any
+ *     value) reports that choice on stderr.  None of them changes a result beyond
+ *     floating-point summation order.
  */
 #ifndef STREAMBP_H_
 #define STREAMBP_H_

@@ -53,6 +53,7 @@ def test_cuda_core_product(op, M, N, K, dtype, out):
     (200, 264, 136),      # ragged in all three dimensions (multiples of 8 for the 16-byte pitch)
     (1000, 688, 256),     # the tiny configuration's d_ff
     (2048, 3584, 1024),   # more tiles than SMs: persistent loop, both accumulator buffers reused
+    (384, 512, 448),      # CTA pairs: the odd CTA of the last row tile has no rows; 7 K slices over 6 stages
 ])
 @pytest.mark.parametrize("out", [torch.float32, torch.bfloat16])
 def test_tensor_core_product(op, M, N, K, out):
@@ -166,3 +167,32 @@ def test_grouped_products_rejects_bad_arguments():
     assert B.gemm_grouped([(B.OP_NT, [(a, a)], c32, False)] * 5, check=False) == B.E_SHAPE   # more than 4 problems
     odd = torch.zeros(64, 68, dtype=torch.bfloat16, device="cuda")[:, :64]                   # pitch 68: not 16-byte rows
     assert B.gemm_grouped([(B.OP_NT, [(odd, a)], c32, False)], check=False) == B.E_SHAPE
+
+
+def test_single_cta_fallback_kernel():
+    """The single-CTA product kernel (used where a two-CTA cluster cannot be scheduled) is selected by an environment
+    variable read when the library first runs a product: exercised in a fresh interpreter, all three layouts."""
+    import os
+    import subprocess
+    import sys
+    code = r"""
+import torch
+from paper_2506_03077_b200 import binding as B
+gen = torch.Generator(device="cpu").manual_seed(3)
+for op in (B.OP_NT, B.OP_NN, B.OP_TN):
+    M, N, K = 392, 520, 456
+    sa, sb = {B.OP_NT: ((M, K), (N, K)), B.OP_NN: ((M, K), (K, N)), B.OP_TN: ((K, M), (K, N))}[op]
+    A = torch.randn(sa, generator=gen).bfloat16().cuda(); Bm = torch.randn(sb, generator=gen).bfloat16().cuda()
+    a, b = A.double().cpu(), Bm.double().cpu()
+    ref = a @ b.T if op == B.OP_NT else (a @ b if op == B.OP_NN else a.T @ b)
+    C = torch.full((M, N), float("nan"), device="cuda")
+    B.gemm(op, A, Bm, C, engine=2); B.gemm(op, A, Bm, C, accumulate=True, engine=2)
+    torch.cuda.synchronize()
+    assert ((C.double().cpu() - 2 * ref).norm() / ref.norm()) < 2e-5
+print("fallback ok")
+"""
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, STREAMBP_GEMM_SINGLE_CTA="1", STREAMBP_VERBOSE="1", PYTHONPATH=root)
+    out = subprocess.run([sys.executable, "-c", code], env=env, cwd=root, capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    assert "fallback ok" in out.stdout and "single CTA" in out.stderr
