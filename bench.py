@@ -35,10 +35,10 @@ def layer_flops(s, T):
     return fwd + bwd + att
 
 
-# DRAM bytes (read + write) of the dominant launch of a chunk -- the {dWg += dg^T h2, dWu += du^T h2,
-# dh2 = dg Wg + du Wu} group -- from the ncu capture summarised in profiles/gemm_group_kernel_chunk_products.md
-# (qwen7b, chunk 1024: algorithmic bytes 1457e6).  Launch shapes depend on the chunk, not on T.
-NCU_TRAFFIC_BYTES = {("qwen7b_layer", 1024): 1680.8e6, ("llama8b_layer", 2048): 1927.5e6}
+# DRAM bytes (read + write) of the dominant launch of a chunk -- the {dWd += dY^T m, dWg += dg^T h2, dWu += du^T h2,
+# dh2 = dg Wg + du Wu} group -- from the ncu capture summarised in profiles/gemm_pair_kernel_chunk_products.md
+# (qwen7b, chunk 1024: algorithmic bytes 2046e6).  Launch shapes depend on the chunk, not on T.
+NCU_TRAFFIC_BYTES = {("qwen7b_layer", 1024): 2142.5e6, ("llama8b_layer", 2048): 2421.9e6}
 
 
 def max_over_ranks(ms: float, world: int, device) -> float:
