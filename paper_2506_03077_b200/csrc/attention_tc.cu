@@ -15,6 +15,8 @@
 //
 // All mbarrier waits are bounded (see sm100.cuh); on expiry the CTA leaves its loops, frees its
 // tensor memory and returns, and the host sees STREAMBP_E_DEVICE_TIMEOUT.
+#include <cstdlib>
+
 #include "sm100.cuh"
 
 namespace sbp {
@@ -263,6 +265,246 @@ __global__ void __launch_bounds__(FWD16_THREADS, 1)
                     if (wg == 0) p.lse[(long long)h * p.n + qr] = (m_used + log2f(lt)) * kLn2;
                 }
             }
+        }
+    }
+
+    __syncwarp();
+    if (*abort_flag) {
+        const unsigned long long t0 = global_timer();
+        while (global_timer() - t0 < 200000ull) { }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem, 512);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Forward with two query tiles per CTA.  The single-tile kernel above spends ~1100 of the ~2300 cycles of a
+// key tile in latencies its sixteen softmax warps all sit through together (tensor-memory load, exchange of
+// partial row maxima, store of P, barrier hand-offs), with the exp2 unit idle.  Here a CTA owns two adjacent
+// 128-query tiles of one head, each with its own S / P and O in tensor memory and its own team of four softmax
+// warps; the two teams are independent of each other, so one team's latencies fall into the other's
+// exponential phase, and each K / V tile is fetched once for 256 query rows.
+//   warp 0     : TMA producer -- both Q tiles once, then K and V tiles through two-stage rings
+//   warp 1     : MMA issuer (warp-uniform issue) -- per key tile j and team X: S_X = Q_X K_j^T when the team has
+//                finished with its previous P (P is packed into the columns of S, so the product that reads P is
+//                queued before the one that overwrites S: the tensor pipe executes one thread's MMAs in order),
+//                O_X += P_X V_j when the team has stored P_X
+//   warps 2..9 : softmax, team (warp - 2) / 4 -- a thread owns a whole query row: 128 scores in registers, no
+//                exchange between threads, row maximum and row sum private; lazy exact rescale as above
+// ---------------------------------------------------------------------------------------------
+constexpr int FWD2Q_THREADS = 64 + 256;
+constexpr int FWD2Q_SMEM = 6 * TILE_BYTES + 1024 + 256;
+
+__global__ void __launch_bounds__(FWD2Q_THREADS, 1)
+    attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                       const __grid_constant__ CUtensorMap map_v, const FwdParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    const uint32_t sQ = base, sK = sQ + 2 * TILE_BYTES, sV = sK + 2 * TILE_BYTES;
+    uint8_t *aux = smem_raw + (base - raw) + 6 * TILE_BYTES;
+    const uint32_t bars = smem_u32(aux);
+    const uint32_t q_full = bars, k_full = bars + 8, k_empty = bars + 24, v_full = bars + 40, v_empty = bars + 56,
+                   s_full = bars + 72, p_full = bars + 88, o_done = bars + 104;   // the last three: one per team
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux + 120);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(aux + 128);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int h = blockIdx.y, g = h / (p.Hq / p.Hkv);
+    const int qt0 = blockIdx.x * 2 * TILE;
+    // team X: query rows qt0 + X * TILE .. ; its key tiles 0 .. nkv[X] - 1 (0 tiles: team absent)
+    int nkv[2];
+#pragma unroll
+    for (int x = 0; x < 2; x++) {
+        const int first = qt0 + x * TILE;
+        const int rows = (p.n - first) < TILE ? (p.n - first) : TILE;
+        nkv[x] = rows > 0 ? (int)((p.q0 + first + rows + TILE - 1) / TILE) : 0;
+    }
+    const int nkv_all = nkv[1] > nkv[0] ? nkv[1] : nkv[0];
+
+    if (threadIdx.x == 0) {
+        mbar_init(q_full, 1);
+        for (int s = 0; s < 2; s++) {
+            mbar_init(k_full + 8 * s, 1);
+            mbar_init(k_empty + 8 * s, 1);
+            mbar_init(v_full + 8 * s, 1);
+            mbar_init(v_empty + 8 * s, 1);
+            mbar_init(s_full + 8 * s, 1);
+            mbar_init(p_full + 8 * s, 4);
+            mbar_init(o_done + 8 * s, 1);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;      // columns: S_A 0..127, S_B 128..255, O_A 256..383, O_B 384..511
+
+    if (warp == 0) {
+        if (lane == 0) {
+            mbar_expect_tx(q_full, (nkv[1] > 0 ? 2 : 1) * TILE_BYTES);
+            for (int x = 0; x < 2; x++) {
+                if (nkv[x] == 0) continue;
+                tma_load_2d(sQ + x * TILE_BYTES, &map_q, q_full, h * TILE, qt0 + x * TILE);
+                tma_load_2d(sQ + x * TILE_BYTES + HALF_BYTES, &map_q, q_full, h * TILE + 64, qt0 + x * TILE);
+            }
+            for (int j = 0; j < nkv_all; j++) {
+                const uint32_t st = j & 1, ph = (j >> 1) & 1;
+                if (!mbar_wait(k_empty + 8 * st, ph ^ 1u, abort_flag)) break;
+                mbar_expect_tx(k_full + 8 * st, TILE_BYTES);
+                tma_load_2d(sK + st * TILE_BYTES, &map_k, k_full + 8 * st, g * TILE, j * TILE);
+                tma_load_2d(sK + st * TILE_BYTES + HALF_BYTES, &map_k, k_full + 8 * st, g * TILE + 64, j * TILE);
+                if (!mbar_wait(v_empty + 8 * st, ph ^ 1u, abort_flag)) break;
+                mbar_expect_tx(v_full + 8 * st, TILE_BYTES);
+                tma_load_2d(sV + st * TILE_BYTES, &map_v, v_full + 8 * st, g * TILE, j * TILE);
+                tma_load_2d(sV + st * TILE_BYTES + HALF_BYTES, &map_v, v_full + 8 * st, g * TILE + 64, j * TILE);
+            }
+        }
+    } else if (warp == 1) {
+        constexpr uint32_t idesc_s = make_idesc(TILE, TILE, false, false);
+        constexpr uint32_t idesc_pv = make_idesc(TILE, TILE, false, true);
+        bool alive = mbar_wait_warp(q_full, 0, abort_flag);
+        auto issue_s = [&](int x, int j) {          // S_x = Q_x K_j^T (K_j is in shared memory)
+            const uint32_t q_lo = klo(sQ + x * TILE_BYTES), k_lo = klo(sK + (j & 1) * TILE_BYTES);
+#pragma unroll
+            for (int kk = 0; kk < 8; kk++) umma_ss_w(tmem + x * TILE, q_lo + kstep(kk), k_lo + kstep(kk), idesc_s, kk != 0);
+            umma_commit_w(s_full + 8 * x);
+        };
+        auto issue_pv = [&](int x, int j) -> bool {  // O_x += P_x V_j once the team has stored P_x
+            if (!mbar_wait_warp(p_full + 8 * x, j & 1, abort_flag)) return false;
+            tc_fence_after();
+            const uint32_t v_lo = mnlo(sV + (j & 1) * TILE_BYTES);
+#pragma unroll
+            for (int kk = 0; kk < 8; kk++)
+                umma_ts_w(tmem + 256 + x * TILE, tmem + x * TILE + kk * 8, v_lo + mnstep(kk), idesc_pv, (j | kk) != 0);
+            if (j == nkv[x] - 1) umma_commit_w(o_done + 8 * x);
+            return true;
+        };
+        if (alive) alive = mbar_wait_warp(k_full, 0, abort_flag);
+        if (alive) {
+            tc_fence_after();
+            for (int x = 0; x < 2; x++)
+                if (nkv[x] > 0) issue_s(x, 0);
+            umma_commit_w(k_empty);
+        }
+        for (int j = 0; j < nkv_all && alive; j++) {
+            const uint32_t st = j & 1, ph = (j >> 1) & 1;
+            if (!mbar_wait_warp(v_full + 8 * st, ph, abort_flag)) { alive = false; break; }
+            if (j + 1 < nkv_all && !mbar_wait_warp(k_full + 8 * ((j + 1) & 1), ((j + 1) >> 1) & 1, abort_flag)) { alive = false; break; }
+            tc_fence_after();
+            for (int x = 0; x < 2 && alive; x++) {
+                if (j < nkv[x]) alive = issue_pv(x, j);
+                if (alive && j + 1 < nkv[x]) issue_s(x, j + 1);
+            }
+            if (!alive) break;
+            umma_commit_w(v_empty + 8 * st);
+            if (j + 1 < nkv_all) umma_commit_w(k_empty + 8 * ((j + 1) & 1));
+        }
+    } else {
+        const int x = (warp - 2) >> 2;                           // team
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;
+        const int first = qt0 + x * TILE;
+        const long long q_abs0 = p.q0 + first, q_abs = q_abs0 + row;
+        const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+        const uint32_t tS = tmem + x * TILE + lane_base, tO = tmem + 256 + x * TILE + lane_base;
+        float m_used = -INFINITY, l = 0.f;
+        bool alive = true;
+        for (int j = 0; j < nkv[x] && alive; j++) {
+            if (!mbar_wait(s_full + 8 * x, j & 1, abort_flag)) { alive = false; break; }
+            tc_fence_after();
+            uint32_t r[128];
+#pragma unroll
+            for (int c = 0; c < 4; c++) tmem_ld32_async(tS + c * 32, r + c * 32);
+            tmem_wait_ld();
+            const long long k_abs0 = (long long)j * TILE;
+            if (k_abs0 + TILE - 1 > q_abs0) {                    // the diagonal crosses this tile
+                const int lim = (int)(q_abs - k_abs0);            // keys 0..lim of the tile are visible
+#pragma unroll
+                for (int e = 0; e < 128; e++)
+                    if (e > lim) r[e] = 0xff800000u;              // -inf
+            }
+            float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int e = 0; e < 128; e += 4) {
+#pragma unroll
+                for (int t = 0; t < 4; t++) m4[t] = fmaxf(m4[t], __uint_as_float(r[e + t]));
+            }
+            const float mt = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * p.scale_log2;
+            float factor = 1.f;
+            const bool grow = mt > m_used + 8.f;                  // also true on the first tile (m_used = -inf)
+            if (grow) {
+                factor = fast_exp2(m_used - mt);
+                m_used = mt;
+                l *= factor;
+            }
+            // S_j complete implies P_{j-1} V_{j-1} complete (same issuing thread, earlier in its order): O is at rest
+            if (j > 0 && __any_sync(0xffffffffu, grow)) {
+#pragma unroll 1
+                for (int c = 0; c < 4; c++) {
+                    uint32_t o[32];
+                    tmem_ld32(tO + c * 32, o);
+#pragma unroll
+                    for (int e = 0; e < 32; e++) o[e] = __float_as_uint(__uint_as_float(o[e]) * factor);
+                    tmem_st32(tO + c * 32, o);
+                }
+            }
+            const float neg_m = -m_used;
+            float l4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int c = 0; c < 8; c++) {                        // 16 scores -> 8 packed words per step
+                uint32_t pk[8];
+#pragma unroll
+                for (int e = 0; e < 16; e += 2) {
+                    const float p0 = fast_exp2(fmaf(__uint_as_float(r[c * 16 + e]), p.scale_log2, neg_m));
+                    const float p1 = fast_exp2(fmaf(__uint_as_float(r[c * 16 + e + 1]), p.scale_log2, neg_m));
+                    l4[(e >> 1) & 3] += p0 + p1;
+                    pk[e >> 1] = pack_bf16(p0, p1);
+                }
+#pragma unroll
+                for (int e = 0; e < 8; e++) r[c * 8 + e] = pk[e];  // packed P reuses the registers of consumed scores
+            }
+            l += (l4[0] + l4[1]) + (l4[2] + l4[3]);
+            // P overwrites the first 64 columns of S (this thread's own lane)
+#pragma unroll
+            for (int c = 0; c < 4; c++) {
+                uint32_t w[16];
+#pragma unroll
+                for (int e = 0; e < 16; e++) w[e] = r[c * 16 + e];
+                tmem_st16(tS + c * 16, w);
+            }
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(p_full + 8 * x);
+        }
+        if (alive && nkv[x] > 0 && mbar_wait(o_done + 8 * x, 0, abort_flag)) {
+            tc_fence_after();
+            const float inv = 1.f / l;
+            const int qr = first + row;
+#pragma unroll 1
+            for (int c = 0; c < 4; c++) {
+                uint32_t o[32];
+                tmem_ld32(tO + c * 32, o);
+                if (qr < p.n) {
+                    bf16 *out = p.o + ((long long)qr * p.Hq + h) * TILE + c * 32;
+#pragma unroll
+                    for (int e = 0; e < 32; e += 8) {
+                        uint32_t w[4];
+#pragma unroll
+                        for (int t = 0; t < 4; t++)
+                            w[t] = pack_bf16(__uint_as_float(o[e + 2 * t]) * inv, __uint_as_float(o[e + 2 * t + 1]) * inv);
+                        *reinterpret_cast<uint4 *>(out + e) = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                }
+            }
+            if (qr < p.n) p.lse[(long long)h * p.n + qr] = (m_used + log2f(l)) * kLn2;
         }
     }
 
@@ -809,10 +1051,17 @@ int attention_fwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, int64_t n, int
         return STREAMBP_E_CUDA;
     static bool configured = false;
     if (!configured) {
-        if (!opt_in_smem(attn_fwd_tc16_kernel, FWD16_SMEM)) return STREAMBP_E_CUDA;
+        if (!opt_in_smem(attn_fwd_tc16_kernel, FWD16_SMEM) || !opt_in_smem(attn_fwd_2q_kernel, FWD2Q_SMEM))
+            return STREAMBP_E_CUDA;
         configured = true;
     }
     FwdParams p{(int)n, (long long)q0, Hq, Hkv, o, lse, kLog2e / sqrtf((float)TILE)};
+    static const bool one_tile = getenv("SBP_FWD1") != nullptr;
+    if (n > TILE && !one_tile) {
+        dim3 grid((unsigned)((n + 2 * TILE - 1) / (2 * TILE)), Hq);
+        SBP_LAUNCH(attn_fwd_2q_kernel, grid, FWD2Q_THREADS, FWD2Q_SMEM, st, mq, mk, mv, p);
+        return STREAMBP_OK;
+    }
     dim3 grid((unsigned)((n + TILE - 1) / TILE), Hq);
     SBP_LAUNCH(attn_fwd_tc16_kernel, grid, FWD16_THREADS, FWD16_SMEM, st, mq, mk, mv, p);
     return STREAMBP_OK;
