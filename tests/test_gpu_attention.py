@@ -52,6 +52,8 @@ CASES = [
     (200, 300, 4, 1),      # ragged chunk, offset not a tile multiple
     (77, 1000, 2, 1),      # short chunk against a long prefix
     (640, 0, 2, 1),        # un-partitioned
+    (384, 200, 2, 1),      # two-tile forward CTAs: the last CTA has one tile only; offset not a tile multiple
+    (130, 126, 4, 2),      # the second tile of the CTA has two rows
 ]
 
 
