@@ -1,17 +1,16 @@
 // Partitioned causal GQA attention on tcgen05 tensor cores (bf16 operands, head_dim 128):
 // the queries of one chunk against the key/value prefix that ends with the chunk.
 //
-// Forward, one CTA per (128-query tile, query head):
+// Forward, two kernels (attn_fwd_2q_kernel for chunks of more than 128 rows, attn_fwd_tc16_kernel otherwise):
 //   warp 0      : TMA producer -- Q once, then K and V tiles of 128 keys through two-stage rings
-//   warp 1      : MMA issuer   -- S_j = Q K_j^T into one of two tensor-memory buffers (so S_{j+1} is
-//                 computed while the softmax of S_j runs), then O += P_j V_j with P_j read from
+//   warp 1      : MMA issuer   -- S_j = Q K_j^T into tensor memory, then O += P_j V_j with P_j read from
 //                 tensor memory as the A operand
-//   warps 2..17 : softmax      -- a thread owns 32 key columns of one query row (see the kernel);
-//                 the running output in tensor memory is rescaled only when a row's maximum grows
-//                 by more than 2^8 (exact: the final division by the row sum uses the same
+//   other warps : softmax      -- row maxima, exponentials, row sums, P packed to bf16 back into tensor
+//                 memory; the running output in tensor memory is rescaled only when a row's maximum
+//                 grows by more than 2^8 (exact: the final division by the row sum uses the same
 //                 reference), which after the first tiles is rare
 //   Key tiles beyond the diagonal are never loaded; the causal predicate is evaluated only in
-//   tiles the diagonal crosses.
+//   tiles the diagonal crosses.  The two kernels differ in how the softmax work is laid out (see each).
 //
 // All mbarrier waits are bounded (see sm100.cuh); on expiry the CTA leaves its loops, frees its
 // tensor memory and returns, and the host sees STREAMBP_E_DEVICE_TIMEOUT.
