@@ -14,8 +14,6 @@
 //
 // All mbarrier waits are bounded (see sm100.cuh); on expiry the CTA leaves its loops, frees its
 // tensor memory and returns, and the host sees STREAMBP_E_DEVICE_TIMEOUT.
-#include <cstdlib>
-
 #include "sm100.cuh"
 
 namespace sbp {
@@ -1055,8 +1053,7 @@ int attention_fwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, int64_t n, int
         configured = true;
     }
     FwdParams p{(int)n, (long long)q0, Hq, Hkv, o, lse, kLog2e / sqrtf((float)TILE)};
-    static const bool one_tile = getenv("SBP_FWD1") != nullptr;
-    if (n > TILE && !one_tile) {
+    if (n > TILE) {
         dim3 grid((unsigned)((n + 2 * TILE - 1) / (2 * TILE)), Hq);
         SBP_LAUNCH(attn_fwd_2q_kernel, grid, FWD2Q_THREADS, FWD2Q_SMEM, st, mq, mk, mv, p);
         return STREAMBP_OK;
