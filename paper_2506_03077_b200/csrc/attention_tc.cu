@@ -1053,7 +1053,11 @@ int attention_fwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, int64_t n, int
         configured = true;
     }
     FwdParams p{(int)n, (long long)q0, Hq, Hkv, o, lse, kLog2e / sqrtf((float)TILE)};
-    if (n > TILE) {
+    // A key-tile step of a two-tile CTA takes ~1.5x that of a one-tile CTA: two tiles per CTA pay off unless they
+    // leave SMs empty that one-tile CTAs would fill (short chunks, few heads).
+    const int64_t ctas1 = (n + TILE - 1) / TILE * Hq, ctas2 = (n + 2 * TILE - 1) / (2 * TILE) * Hq;
+    const int64_t sms = sm_count();
+    if (n > TILE && 3 * ((ctas2 + sms - 1) / sms) <= 2 * ((ctas1 + sms - 1) / sms)) {
         dim3 grid((unsigned)((n + 2 * TILE - 1) / (2 * TILE)), Hq);
         SBP_LAUNCH(attn_fwd_2q_kernel, grid, FWD2Q_THREADS, FWD2Q_SMEM, st, mq, mk, mv, p);
         return STREAMBP_OK;
