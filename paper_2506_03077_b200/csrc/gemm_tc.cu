@@ -2,15 +2,20 @@
 // (128-byte swizzle), fp32 accumulation in tensor memory, three operand layouts, several
 // independent products (each possibly a sum over K segments) per launch.
 //
-//   persistent grid, one CTA per SM, output tile 128 x 256, K slices of 64
+// Two kernels with the same roles, epilogue and tile list:
+//   gemm_pair_kernel  : persistent grid of two-CTA clusters (one per TPC), output tile 256 x 256 per pair,
+//                       tcgen05.mma.cta_group::2, six 32 KiB operand stages per CTA -- the one that runs
+//   gemm_group_kernel : persistent grid, one CTA per SM, output tile 128 x 256, four 48 KiB stages -- the
+//                       fallback where a two-CTA cluster cannot be scheduled
+// Per CTA, K slices of 64:
 //   warp 0      : tile scheduler and TMA producer (one elected lane)
-//   warp 1      : allocates tensor memory, issues tcgen05.mma (one elected lane)
+//   warp 1      : allocates tensor memory, issues tcgen05.mma (one elected lane; even CTA of a pair)
 //   warps 2..5  : epilogue -- tcgen05.ld of a 32-lane quarter, bias, then
 //                 fp32 output: 32x32 blocks staged in shared memory (128-byte swizzle) and written
 //                 by TMA store, or added into C by TMA reduce-add when accumulating, so the
 //                 read-modify-write of a weight-gradient tile never passes through the SM;
 //                 bf16 output: 16-byte stores from registers
-//   tensor memory holds two 128 x 256 fp32 accumulators, so the epilogue of tile i overlaps
+//   tensor memory holds two 128 x 256 fp32 accumulators per CTA, so the epilogue of tile i overlaps
 //   the main loop of tile i+1.
 //
 // Operand layouts (GemmOp): K-major operands are loaded as [rows][64 k] boxes, MN-major operands
