@@ -269,7 +269,7 @@ def run_head_or_model(args, cfg):
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic", "loss": loss.item(),
         "config": {"workload": cfg.name, "T": T, "chunk": cfg.chunk, "n_layers": cfg.n_layers, "vocab": h.vocab,
-                   "l2": "inputs larger than L2"},
+                   "l2": "inputs larger than L2", "product_kernel": B.product_kernel()},
         "algorithmic_tflop_per_step": flops / 1e12, "tflops": flops / (ms * 1e-3) / 1e12,
         "frac_of_measured_sustained_bf16": flops / (ms * 1e-3) / 1e12 / peaks["sustained"],
         "executed_tflop_per_step": executed_flops / 1e12,
@@ -444,6 +444,7 @@ def main():
         "config": {"workload": cfg.name, "T": T, "chunk": chunk, "d_model": s.d_model, "n_q_heads": s.n_q_heads,
                    "n_kv_heads": s.n_kv_heads, "head_dim": s.head_dim, "d_ff": s.d_ff, "qkv_bias": s.qkv_bias,
                    "l2": "inputs larger than L2 (weights + gradients > 1 GB per step)",
+                   "product_kernel": B.product_kernel(),
                    "multi_gpu": ("data parallel: one NCCL reduce-scatter of the layer's fp32 gradient bucket per step"
                                  if args.dp else "replicas only")},
         "algorithmic_tflop_per_step": flops / 1e12,

@@ -340,6 +340,14 @@ int streambp_attention_backward_static(const void *q, const void *k, const void 
 void streambp_profile_enable(int on);
 int streambp_profile_read(int kernel_class, double *milliseconds, int64_t *calls, double *flops);
 
+/*
+ * Which tcgen05 product kernel bf16 products run on the current device: 2 = CTA pairs
+ * (cta_group::2, 256 x 256 tiles), 1 = single CTA (128 x 256 tiles; a two-CTA cluster cannot be
+ * scheduled, or STREAMBP_GEMM_SINGLE_CTA is set), 0 = none (no tensor-map support: bf16 products
+ * fall back to the CUDA-core kernels).  Host-only query; launches nothing.
+ */
+int streambp_product_kernel(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -31,7 +31,7 @@ EXPORTS = (
     "streambp_last_device_status", "streambp_status_string",
     "streambp_last_cuda_error", "streambp_last_launch_count", "streambp_gemm", "streambp_gemm_grouped",
     "streambp_layer_suggest_chunk", "streambp_lmhead_suggest_chunk",
-    "streambp_profile_enable", "streambp_profile_read",
+    "streambp_profile_enable", "streambp_profile_read", "streambp_product_kernel",
     "streambp_attention_forward", "streambp_attention_backward", "streambp_attention_backward_static",
     "streambp_lmhead_rl_backward", "streambp_layer_backward_packed",
 )
@@ -132,6 +132,8 @@ def lib() -> C.CDLL:
     L.streambp_attention_backward_static.restype = C.c_int
     L.streambp_attention_backward_static.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i32, i32, i32, i32, vp, vp, vp,
                                                      C.c_int, vp]
+    L.streambp_product_kernel.restype = C.c_int
+    L.streambp_product_kernel.argtypes = []
     L.streambp_profile_enable.restype = None
     L.streambp_profile_enable.argtypes = [C.c_int]
     L.streambp_profile_read.restype = C.c_int
@@ -420,6 +422,11 @@ def gemm_grouped(problems, sched: Optional[torch.Tensor] = None, stream=None, ch
 
 
 KERNEL_CLASSES = {"gemm": 0, "attention_fwd": 1, "attention_bwd": 2}
+
+
+def product_kernel() -> str:
+    """Which tcgen05 product kernel runs bf16 products on the current device."""
+    return {2: "cta_pair", 1: "single_cta", 0: "none"}[lib().streambp_product_kernel()]
 
 
 def profile_enable(on: bool) -> None:

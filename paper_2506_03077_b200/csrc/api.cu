@@ -507,6 +507,8 @@ int streambp_attention_backward(const void *q, const void *k, const void *v, con
     return rc;
 }
 
+int streambp_product_kernel(void) { return gemm_tc_variant(); }
+
 void streambp_profile_enable(int on) {
     g_prof_on = on != 0;
     g_prof_used = 0;

@@ -233,6 +233,7 @@ int gemm_tc_group(const GemmProb *probs, int n, int *sched, cudaStream_t st);
 
 // Reads and clears the flag a tensor-core kernel raises when one of its bounded waits expires.
 int gemm_tc_take_fault();
+int gemm_tc_variant();   // 2: CTA-pair kernel, 1: single-CTA kernel, 0: tensor maps unavailable
 
 // Engine choice for the dispatching product below: 0 automatic, 1 CUDA cores only, 2 tensor cores required.
 int gemm_engine();

@@ -825,4 +825,6 @@ int gemm_tc(GemmOp op, int64_t M, int64_t N, int64_t K, const bf16 *A, int64_t l
 
 int gemm_tc_take_fault() { return take_fault_local(); }
 
+int gemm_tc_variant() { return !tensor_maps_available() ? 0 : (pair_kernel_available() ? 2 : 1); }
+
 }  // namespace sbp
