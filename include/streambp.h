@@ -289,6 +289,17 @@ typedef struct {
 int streambp_gemm_grouped(const streambp_gemm_problem *problems, int32_t n, int32_t *sched, void *cuda_stream);
 
 /*
+ * The MLP's first half as the layer runs it (Sec. 3.2.2, the partitioned MLP): g = A W_gate^T, u = A W_up^T and
+ * m = silu(g) * u, with silu taken of the values ROUNDED to the storage type (the ones the backward reads).
+ * A: [M, K] (lda), W_gate, W_up: [N, K] (ldb), g, u, m: [M, N] dense; all of `dtype` (float or bf16), device.
+ * bf16 on the CTA-pair product kernel is ONE launch (the even CTA of a pair fetches W_gate rows, the odd one
+ * W_up rows, so g and u of the same columns meet in one accumulator row); otherwise two products and an
+ * element-wise kernel.  Same results either way up to the summation order of the products.
+ */
+int streambp_gemm_swiglu(const void *A, int64_t lda, const void *w_gate, const void *w_up, int64_t ldb, int64_t M,
+                         int64_t N, int64_t K, void *g, void *u, void *m, int32_t dtype, void *cuda_stream);
+
+/*
  * Building blocks exposed for tests and profiling: the partitioned attention of Sec. 3.2.2
  * (S^(i) = Q^(i) K^(:i)T, causal softmax, O^(i) = P^(i) V^(:i)) for one chunk of n query rows that
  * sit at absolute rows q0 .. q0+n-1 and attend to keys 0 .. q0+n-1, and its backward.

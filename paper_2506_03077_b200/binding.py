@@ -29,7 +29,7 @@ EXPORTS = (
     "streambp_lmhead_workspace_bytes", "streambp_lmhead_ce_backward",
     "streambp_model_workspace_bytes", "streambp_model_backward",
     "streambp_last_device_status", "streambp_status_string",
-    "streambp_last_cuda_error", "streambp_last_launch_count", "streambp_gemm", "streambp_gemm_grouped",
+    "streambp_last_cuda_error", "streambp_last_launch_count", "streambp_gemm", "streambp_gemm_grouped", "streambp_gemm_swiglu",
     "streambp_layer_suggest_chunk", "streambp_lmhead_suggest_chunk",
     "streambp_profile_enable", "streambp_profile_read", "streambp_product_kernel",
     "streambp_attention_forward", "streambp_attention_backward", "streambp_attention_backward_static",
@@ -122,6 +122,8 @@ def lib() -> C.CDLL:
     L.streambp_lmhead_suggest_chunk.argtypes = [C.POINTER(HeadCfgC), i64, sz]
     L.streambp_gemm_grouped.restype = C.c_int
     L.streambp_gemm_grouped.argtypes = [C.POINTER(GemmProblemC), i32, vp, vp]
+    L.streambp_gemm_swiglu.restype = C.c_int
+    L.streambp_gemm_swiglu.argtypes = [vp, i64, vp, vp, i64, i64, i64, i64, vp, vp, vp, i32, vp]
     L.streambp_gemm.restype = C.c_int
     L.streambp_gemm.argtypes = [C.c_int, i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, i32, C.c_int, C.c_int, vp]
     L.streambp_attention_forward.restype = C.c_int
@@ -418,6 +420,20 @@ def gemm_grouped(problems, sched: Optional[torch.Tensor] = None, stream=None, ch
     st = lib().streambp_gemm_grouped(arr, len(problems), _ptr(sched), _stream_ptr(stream))
     if check:
         _check(st, "streambp_gemm_grouped")
+    return st
+
+
+def gemm_swiglu(A, w_gate, w_up, g, u, m, stream=None, check: bool = True) -> int:
+    """streambp_gemm_swiglu: g = A w_gate^T, u = A w_up^T, m = silu(g) * u; A [M, K], weights [N, K], outputs [M, N] dense."""
+    M, K = A.shape
+    N = w_gate.shape[0]
+    assert A.stride(1) == 1 and w_gate.stride(1) == 1 and w_up.stride(1) == 1 and w_gate.stride(0) == w_up.stride(0)
+    for t in (g, u, m):
+        assert t.is_contiguous() and tuple(t.shape) == (M, N)
+    st = lib().streambp_gemm_swiglu(_ptr(A), A.stride(0), _ptr(w_gate), _ptr(w_up), w_gate.stride(0), M, N, K, _ptr(g),
+                                    _ptr(u), _ptr(m), _dtype_code(A.dtype), _stream_ptr(stream))
+    if check:
+        _check(st, "streambp_gemm_swiglu")
     return st
 
 

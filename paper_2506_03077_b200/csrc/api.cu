@@ -128,6 +128,38 @@ int mm_group<bf16>(const MmProb<bf16> *probs, int n, cudaStream_t st) {
     return STREAMBP_OK;
 }
 
+template <typename T>
+static int mm_swiglu_unfused(int64_t M, int64_t N, int64_t K, const T *A, int64_t lda, const T *Wg, const T *Wu, int64_t ldb,
+                             T *g, T *u, T *m, int64_t ldc, cudaStream_t st) {
+    if (ldc != N) return STREAMBP_E_SHAPE;      // the element-wise kernel walks dense [M, N] buffers
+    const MmProb<T> gu[2] = {mm_prob<T>(OP_NT, M, N, K, A, lda, Wg, ldb, g, ldc, sizeof(T) == 4, nullptr, false),
+                             mm_prob<T>(OP_NT, M, N, K, A, lda, Wu, ldb, u, ldc, sizeof(T) == 4, nullptr, false)};
+    SBP_TRY(mm_group<T>(gu, 2, st));
+    return swiglu_fwd<T>(g, u, M * N, m, st);
+}
+template <>
+int mm_swiglu<float>(int64_t M, int64_t N, int64_t K, const float *A, int64_t lda, const float *Wg, const float *Wu,
+                     int64_t ldb, float *g, float *u, float *m, int64_t ldc, cudaStream_t st) {
+    return mm_swiglu_unfused<float>(M, N, K, A, lda, Wg, Wu, ldb, g, u, m, ldc, st);
+}
+template <>
+int mm_swiglu<bf16>(int64_t M, int64_t N, int64_t K, const bf16 *A, int64_t lda, const bf16 *Wg, const bf16 *Wu,
+                    int64_t ldb, bf16 *g, bf16 *u, bf16 *m, int64_t ldc, cudaStream_t st) {
+    GemmProb gp;
+    gp.op = OP_NT; gp.M = M; gp.N = N; gp.nseg = 2;
+    gp.seg[0] = GemmSeg{A, lda, Wg, ldb, K};
+    gp.seg[1] = GemmSeg{A, lda, Wu, ldb, K};
+    gp.C = g; gp.ldc = ldc; gp.c_is_f32 = false; gp.bias = nullptr; gp.accumulate = false;
+    gp.swiglu = true; gp.C_up = u; gp.C_act = m;
+    if (gemm_engine() != 1 && gemm_tc_group_supported(&gp, 1)) {
+        ProfScope prof(KC_GEMM, 2.0 * 2.0 * (double)M * (double)N * (double)K, st);
+        CallState &cs = call_state();
+        int *sched = cs.sched ? cs.sched + 2 * (cs.sched_slot++ % kSchedSlots) : nullptr;
+        return gemm_tc_group(&gp, 1, sched, st);
+    }
+    return mm_swiglu_unfused<bf16>(M, N, K, A, lda, Wg, Wu, ldb, g, u, m, ldc, st);
+}
+
 template <>
 int attn_fwd<float>(const float *q, const float *k, const float *v, int64_t n, int64_t q0, int Hq, int Hkv, int dh,
                     float *o, float *lse, cudaStream_t st) {
@@ -593,6 +625,23 @@ int streambp_gemm_grouped(const streambp_gemm_problem *problems, int32_t n, int3
     call_state().launches = 0;
     if (!gemm_tc_group_supported(gp, n)) return STREAMBP_E_SHAPE;
     return gemm_tc_group(gp, n, sched, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int streambp_gemm_swiglu(const void *A, int64_t lda, const void *w_gate, const void *w_up, int64_t ldb, int64_t M,
+                         int64_t N, int64_t K, void *g, void *u, void *m, int32_t dtype, void *cuda_stream) {
+    if (!A || !w_gate || !w_up || !g || !u || !m) return STREAMBP_E_NULL;
+    if (M < 1 || N < 1 || K < 1 || lda < K || ldb < K) return STREAMBP_E_SHAPE;
+    if (dtype != STREAMBP_F32 && dtype != STREAMBP_BF16) return STREAMBP_E_DTYPE;
+    if (!aligned(A, 16) || !aligned(w_gate, 16) || !aligned(w_up, 16) || !aligned(g, 16) || !aligned(u, 16) || !aligned(m, 16))
+        return STREAMBP_E_ALIGN;
+    call_state().cuda_error = 0;
+    call_state().launches = 0;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (dtype == STREAMBP_F32)
+        return mm_swiglu<float>(M, N, K, (const float *)A, lda, (const float *)w_gate, (const float *)w_up, ldb, (float *)g,
+                                (float *)u, (float *)m, N, st);
+    return mm_swiglu<bf16>(M, N, K, (const bf16 *)A, lda, (const bf16 *)w_gate, (const bf16 *)w_up, ldb, (bf16 *)g, (bf16 *)u,
+                           (bf16 *)m, N, st);
 }
 
 }  // extern "C"

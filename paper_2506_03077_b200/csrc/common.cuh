@@ -225,6 +225,10 @@ struct GemmProb {
     bool c_is_f32;
     const bf16 *bias;
     bool accumulate;
+    // SwiGLU pair (CTA-pair kernel only): op NT, seg[0].B = W_gate, seg[1].B = W_up (same A, K); the three bf16
+    // outputs C = g = A W_gate^T, C_up = u = A W_up^T and C_act = silu(g) * u share ldc.  N counts the columns of each.
+    bool swiglu = false;
+    void *C_up = nullptr, *C_act = nullptr;
 };
 bool gemm_tc_group_supported(const GemmProb *probs, int n);
 // sched: two ints of device memory that are zero when the launch starts (the kernel leaves them zero),
@@ -391,6 +395,13 @@ void mm_add_seg(MmProb<T> &g, int64_t K, const T *A, int64_t lda, const T *B, in
 }
 template <typename T>
 int mm_group(const MmProb<T> *probs, int n, cudaStream_t st);
+// g = A Wg^T, u = A Wu^T, m = silu(g) * u  (A [M, K], Wg / Wu [N, K], outputs [M, N], all row-major of type T).
+// bf16 on the CTA-pair product kernel: ONE launch -- the even CTA of a pair fetches Wg rows, the odd one Wu rows, so
+// g and u of the same output columns land in one accumulator row and the epilogue writes all three.  Otherwise two
+// products and the element-wise kernel.
+template <typename T>
+int mm_swiglu(int64_t M, int64_t N, int64_t K, const T *A, int64_t lda, const T *Wg, const T *Wu, int64_t ldb, T *g, T *u,
+              T *m, int64_t ldc, cudaStream_t st);
 
 // ---- schedulers (T = storage dtype) --------------------------------------------------
 template <typename T>

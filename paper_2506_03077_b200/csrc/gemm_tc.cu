@@ -120,7 +120,7 @@ namespace {
 // Operand layouts, output type and accumulation are per-problem run-time flags.
 // ---------------------------------------------------------------------------------------------
 constexpr int MAX_PROBS = 4, MAX_SEGS = 8, RING = 4;
-constexpr uint32_t F_A_MN = 1u, F_B_MN = 2u, F_OUT_F32 = 4u, F_ACC = 8u;
+constexpr uint32_t F_A_MN = 1u, F_B_MN = 2u, F_OUT_F32 = 4u, F_ACC = 8u, F_SWIGLU = 16u;
 
 struct GroupParams {
     CUtensorMap map_a[MAX_SEGS];
@@ -132,6 +132,7 @@ struct GroupParams {
     int tiles_m[MAX_PROBS];
     int M[MAX_PROBS], N[MAX_PROBS];
     void *C[MAX_PROBS];
+    void *C_up[MAX_PROBS], *C_act[MAX_PROBS];   // SwiGLU pairs: u and silu(g) * u beside g in C
     long long ldc[MAX_PROBS];
     const bf16 *bias[MAX_PROBS];
     uint32_t flags[MAX_PROBS];
@@ -162,6 +163,8 @@ __device__ __forceinline__ TileRef locate(const GroupParams &p, int tile) {
         s1 = (q == i) ? p.seg_begin[i + 1] : s1;
     }
     const int local = tile - tb, tm = pick(p.tiles_m, q);
+    // a SwiGLU pair has two B operands (W_gate, W_up: segments s0, s0 + 1) but ONE pass over K
+    if (pick(p.flags, q) & F_SWIGLU) s1 = s0 + 1;
     return {q, (local % tm) * TILE_M, (local / tm) * BN, s0, s1};
 }
 
@@ -239,6 +242,53 @@ __device__ __forceinline__ void epilogue_rows(const GroupParams &p, const TileRe
     const CUtensorMap *mc = &p.map_c[t.q];
     const int row = m_base + quarter * 32 + lane;
     const uint32_t taddr = acc + ((uint32_t)(quarter * 32) << 16);
+    if (fl & F_SWIGLU) {
+        // accumulator columns c and 128 + c are g and u of output column n0 / 2 + c: round both to bf16 (what the
+        // backward will read), m = silu(g) * u from the rounded values, three 16-byte stores per 8 columns
+        const long long off = (long long)row * pick(p.ldc, t.q);
+        bf16 *og = reinterpret_cast<bf16 *>(pick(p.C, t.q)) + off, *ou = reinterpret_cast<bf16 *>(pick(p.C_up, t.q)) + off,
+             *om = reinterpret_cast<bf16 *>(pick(p.C_act, t.q)) + off;
+#pragma unroll 1
+        for (int c = 0; c < BN / 64; c++) {
+            const int col0 = t.n0 / 2 + c * 32;
+            if (col0 >= Nq) break;               // uniform across the warp
+            uint32_t rg[32], ru[32];
+            tmem_ld32(taddr + c * 32, rg);
+            tmem_ld32(taddr + BN / 2 + c * 32, ru);
+            if (row >= Mq) continue;
+#pragma unroll
+            for (int j = 0; j < 32; j += 8) {
+                uint32_t wg[4], wu[4], wm[4];
+#pragma unroll
+                for (int e = 0; e < 4; e++) {
+                    const __nv_bfloat162 hg = __floats2bfloat162_rn(__uint_as_float(rg[j + 2 * e]), __uint_as_float(rg[j + 2 * e + 1]));
+                    const __nv_bfloat162 hu = __floats2bfloat162_rn(__uint_as_float(ru[j + 2 * e]), __uint_as_float(ru[j + 2 * e + 1]));
+                    const float2 fg = __bfloat1622float2(hg), fu = __bfloat1622float2(hu);
+                    const float m0 = fg.x * (1.f / (1.f + __expf(-fg.x))) * fu.x;
+                    const float m1 = fg.y * (1.f / (1.f + __expf(-fg.y))) * fu.y;
+                    const __nv_bfloat162 hm = __floats2bfloat162_rn(m0, m1);
+                    wg[e] = *reinterpret_cast<const uint32_t *>(&hg);
+                    wu[e] = *reinterpret_cast<const uint32_t *>(&hu);
+                    wm[e] = *reinterpret_cast<const uint32_t *>(&hm);
+                }
+                if (col0 + j + 7 < Nq) {
+                    *reinterpret_cast<uint4 *>(og + col0 + j) = make_uint4(wg[0], wg[1], wg[2], wg[3]);
+                    *reinterpret_cast<uint4 *>(ou + col0 + j) = make_uint4(wu[0], wu[1], wu[2], wu[3]);
+                    *reinterpret_cast<uint4 *>(om + col0 + j) = make_uint4(wm[0], wm[1], wm[2], wm[3]);
+                } else {
+                    const bf16 *sg = reinterpret_cast<const bf16 *>(wg), *su = reinterpret_cast<const bf16 *>(wu),
+                               *sm = reinterpret_cast<const bf16 *>(wm);
+                    for (int e = 0; e < 8; e++)
+                        if (col0 + j + e < Nq) {
+                            og[col0 + j + e] = sg[e];
+                            ou[col0 + j + e] = su[e];
+                            om[col0 + j + e] = sm[e];
+                        }
+                }
+            }
+        }
+        return;
+    }
     bf16 *out_row = reinterpret_cast<bf16 *>(pick(p.C, t.q)) + (long long)row * pick(p.ldc, t.q);
 #pragma unroll 1
     for (int c = 0; c < BN / 32; c++) {
@@ -460,9 +510,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_group_kernel(const __grid
 template <bool A_MN, bool B_MN>
 __device__ __forceinline__ bool produce_tile_pair(const GroupParams &p, const TileRef &t, const Pipe &pp, uint32_t rank,
                                                   uint32_t &stage, uint32_t &phase) {
-    const int m = t.m0 + BM * (int)rank, n = t.n0 + (BN / 2) * (int)rank;
+    // SwiGLU pair: both CTAs fetch the SAME 128 weight rows, the even one of W_gate, the odd one of W_up, so that
+    // accumulator columns 0..127 hold g and 128..255 hold u of output columns n0 / 2 ..
+    const bool swiglu = (pick(p.flags, t.q) & F_SWIGLU) != 0;
+    const int m = t.m0 + BM * (int)rank, n = swiglu ? t.n0 / 2 : t.n0 + (BN / 2) * (int)rank;
     for (int s = t.seg0; s < t.seg1; s++) {
-        const CUtensorMap *ma = &p.map_a[s], *mb = &p.map_b[s];
+        const CUtensorMap *ma = &p.map_a[s], *mb = &p.map_b[s + ((swiglu && rank) ? 1 : 0)];
         const int nkb = p.seg_kb[s];
         for (int kb = 0; kb < nkb; kb++) {
             if (!mbar_wait(pp.bar_empty + 8 * stage, phase ^ 1u, pp.abort_flag)) return false;
@@ -696,22 +749,6 @@ bool gemm_tc_supported(GemmOp op, int64_t M, int64_t N, int64_t K, int64_t lda, 
     return tensor_maps_available();
 }
 
-bool gemm_tc_group_supported(const GemmProb *probs, int n) {
-    if (n < 1 || n > MAX_PROBS) return false;
-    int segs = 0;
-    for (int i = 0; i < n; i++) {
-        const GemmProb &g = probs[i];
-        if (g.nseg < 1 || g.nseg > 3) return false;
-        if (!g.c_is_f32 && g.accumulate) return false;
-        segs += g.nseg;
-        for (int s = 0; s < g.nseg; s++)
-            if (!gemm_tc_supported(g.op, g.M, g.N, g.seg[s].K, g.seg[s].lda, g.seg[s].ldb, g.ldc, g.seg[s].A,
-                                   g.seg[s].B, g.C, g.c_is_f32))
-                return false;
-    }
-    return segs <= MAX_SEGS;
-}
-
 namespace {
 // The CTA-pair kernel needs clusters of two CTAs with the full shared-memory carve-out; where the device cannot
 // co-schedule even one such cluster the single-CTA kernel runs instead.
@@ -738,6 +775,29 @@ bool pair_kernel_available() {
 }
 }  // namespace
 
+bool gemm_tc_group_supported(const GemmProb *probs, int n) {
+    if (n < 1 || n > MAX_PROBS) return false;
+    int segs = 0;
+    for (int i = 0; i < n; i++) {
+        const GemmProb &g = probs[i];
+        if (g.nseg < 1 || g.nseg > 3) return false;
+        if (!g.c_is_f32 && g.accumulate) return false;
+        if (g.swiglu) {
+            auto al16 = [](const void *q) { return q != nullptr && (reinterpret_cast<uintptr_t>(q) & 15u) == 0; };
+            if (g.op != OP_NT || g.nseg != 2 || g.c_is_f32 || g.accumulate || g.bias || g.seg[0].K != g.seg[1].K ||
+                !al16(g.C_up) || !al16(g.C_act) || !pair_kernel_available())
+                return false;
+        }
+        segs += g.nseg;
+        for (int s = 0; s < g.nseg; s++)
+            if (!gemm_tc_supported(g.op, g.M, g.N, g.seg[s].K, g.seg[s].lda, g.seg[s].ldb, g.ldc, g.seg[s].A,
+                                   g.seg[s].B, g.C, g.c_is_f32))
+                return false;
+    }
+    return segs <= MAX_SEGS;
+}
+
+
 int gemm_tc_group(const GemmProb *probs, int n, int *sched, cudaStream_t st) {
     if (!gemm_tc_group_supported(probs, n)) return STREAMBP_E_SHAPE;
     const bool pair = pair_kernel_available();
@@ -748,7 +808,7 @@ int gemm_tc_group(const GemmProb *probs, int n, int *sched, cudaStream_t st) {
     for (int i = 0; i < n; i++) {
         order[i] = i;
         cost[i] = 0;
-        for (int s = 0; s < probs[i].nseg; s++) cost[i] += (probs[i].seg[s].K + BK - 1) / BK;
+        for (int s = 0; s < (probs[i].swiglu ? 1 : probs[i].nseg); s++) cost[i] += (probs[i].seg[s].K + BK - 1) / BK;
     }
     for (int i = 1; i < n; i++)
         for (int j = i; j > 0 && cost[order[j]] > cost[order[j - 1]]; j--) {
@@ -786,9 +846,13 @@ int gemm_tc_group(const GemmProb *probs, int n, int *sched, cudaStream_t st) {
         p.C[i] = g.C;
         p.ldc[i] = g.ldc;
         p.bias[i] = g.bias;
+        p.C_up[i] = g.C_up;
+        p.C_act[i] = g.C_act;
         p.flags[i] = (a_mn ? F_A_MN : 0u) | (b_mn ? F_B_MN : 0u) | (g.c_is_f32 ? F_OUT_F32 : 0u) |
-                     (g.accumulate ? F_ACC : 0u);
-        tiles += (int64_t)p.tiles_m[i] * ((g.N + BN - 1) / BN);
+                     (g.accumulate ? F_ACC : 0u) | (g.swiglu ? F_SWIGLU : 0u);
+        // a SwiGLU tile covers BN / 2 output columns (g and u of the same columns side by side in the accumulator)
+        const int64_t tile_n = g.swiglu ? BN / 2 : BN;
+        tiles += (int64_t)p.tiles_m[i] * ((g.N + tile_n - 1) / tile_n);
         if (tiles > (1ll << 30)) return STREAMBP_E_SHAPE;
     }
     for (int i = n; i <= MAX_PROBS; i++) {

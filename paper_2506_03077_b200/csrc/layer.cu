@@ -133,11 +133,7 @@ int chunk_forward(const streambp_layer_cfg &c, const streambp_layer_weights &w, 
     }));
     SBP_TRY((mm<T, float>(OP_NT, n, d, dq, s.O, dq, (const T *)w.wo, dq, s.fa, d, nullptr, false, st)));
     SBP_TRY(rmsnorm_fwd<T>(Xi, s.fa, (const T *)w.g2, c.rms_eps, n, d, s.h2, s.rstd2, s.r, st));
-    const MmProb<T> gu[2] = {
-        mm_prob<T>(OP_NT, n, I, d, s.h2, d, (const T *)w.w_gate, d, s.g, I, sizeof(T) == 4, nullptr, false),
-        mm_prob<T>(OP_NT, n, I, d, s.h2, d, (const T *)w.w_up, d, s.u, I, sizeof(T) == 4, nullptr, false)};
-    SBP_TRY(mm_group<T>(gu, 2, st));
-    SBP_TRY(swiglu_fwd<T>(s.g, s.u, n * I, s.m, st));
+    SBP_TRY(mm_swiglu<T>(n, I, d, s.h2, d, (const T *)w.w_gate, (const T *)w.w_up, d, s.g, s.u, s.m, I, st));
     return STREAMBP_OK;
 }
 

@@ -169,6 +169,30 @@ def test_grouped_products_rejects_bad_arguments():
     assert B.gemm_grouped([(B.OP_NT, [(odd, a)], c32, False)], check=False) == B.E_SHAPE
 
 
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("M,N,K", [(256, 128, 64), (1000, 1376, 512), (300, 200, 136), (2048, 2816, 1024)])
+def test_swiglu_product(M, N, K, dtype):
+    """g = A Wg^T, u = A Wu^T, m = silu(g) * u in one call (one launch on CTA pairs in bf16): ragged rows and columns,
+    several tiles per pair, the odd CTA of the last row tile without rows."""
+    gen = torch.Generator(device="cpu").manual_seed(M + N + K)
+    A = (torch.randn(M, K, generator=gen) * 0.5).to(dtype).cuda()
+    Wg = (torch.randn(N, K, generator=gen) * 0.1).to(dtype).cuda()
+    Wu = (torch.randn(N, K, generator=gen) * 0.1).to(dtype).cuda()
+    g, u, m = (torch.full((M, N), float("nan"), dtype=dtype, device="cuda") for _ in range(3))
+    B.gemm_swiglu(A, Wg, Wu, g, u, m)
+    torch.cuda.synchronize()
+    a = A.double().cpu()
+    g_ref, u_ref = a @ Wg.double().cpu().T, a @ Wu.double().cpu().T
+    tol = 4e-3 if dtype == torch.bfloat16 else 1e-5
+    for got, ref in ((g, g_ref), (u, u_ref)):
+        assert torch.isfinite(got).all()
+        assert (got.double().cpu() - ref).norm() / ref.norm() < tol
+    # m is a function of the STORED g and u: exact up to the last rounding and the fast exponential
+    gs, us = g.double().cpu(), u.double().cpu()
+    m_ref = gs * torch.sigmoid(gs) * us
+    assert (m.double().cpu() - m_ref).norm() / m_ref.norm() < (3e-3 if dtype == torch.bfloat16 else 1e-6)
+
+
 def test_single_cta_fallback_kernel():
     """The single-CTA product kernel (used where a two-CTA cluster cannot be scheduled) is selected by an environment
     variable read when the library first runs a product: exercised in a fresh interpreter, all three layouts."""
@@ -189,6 +213,14 @@ for op in (B.OP_NT, B.OP_NN, B.OP_TN):
     B.gemm(op, A, Bm, C, engine=2); B.gemm(op, A, Bm, C, accumulate=True, engine=2)
     torch.cuda.synchronize()
     assert ((C.double().cpu() - 2 * ref).norm() / ref.norm()) < 2e-5
+A = torch.randn(300, 136, generator=gen).bfloat16().cuda(); Wg = torch.randn(200, 136, generator=gen).bfloat16().cuda()
+Wu = torch.randn(200, 136, generator=gen).bfloat16().cuda()
+g, u, m = (torch.empty(300, 200, dtype=torch.bfloat16, device="cuda") for _ in range(3))
+B.gemm_swiglu(A, Wg, Wu, g, u, m); torch.cuda.synchronize()
+ref = A.double().cpu() @ Wg.double().cpu().T
+assert ((g.double().cpu() - ref).norm() / ref.norm()) < 4e-3
+gs, us = g.double().cpu(), u.double().cpu()
+assert ((m.double().cpu() - gs * torch.sigmoid(gs) * us).norm() / (gs * torch.sigmoid(gs) * us).norm()) < 3e-3
 print("fallback ok")
 """
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
