@@ -307,7 +307,8 @@ int streambp_gemm_swiglu(const void *A, int64_t lda, const void *w_gate, const v
  * lse: [n_q_heads, n] fp32 (natural log of the row sums of exp(score / sqrt(head_dim)));
  * delta: scratch [n_q_heads, n] fp32; dq: [n, n_q_heads, head_dim] fp32, overwritten;
  * dk, dv: [q0+n, n_kv_heads, head_dim] fp32, ADDED to (the key-prefix accumulators).
- * engine: 0 automatic, 1 CUDA cores, 2 tensor cores (bf16, head_dim 128 only).
+ * engine: 0 automatic, 1 CUDA cores, 2 tensor cores (bf16, head_dim 128 only); the forward also takes 3 / 4 =
+ * tensor cores with one / two 128-query tiles per CTA (2 picks between them from the grid size).
  */
 int streambp_attention_forward(const void *q, const void *k, const void *v, int64_t n, int64_t q0,
                                int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, int32_t dtype,

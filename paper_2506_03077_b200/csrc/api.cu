@@ -499,16 +499,16 @@ int streambp_attention_forward(const void *q, const void *k, const void *v, int6
     call_state().cuda_error = 0;
     call_state().launches = 0;
     if (dtype == STREAMBP_F32) {
-        if (engine == 2) return STREAMBP_E_DTYPE;
+        if (engine >= 2) return STREAMBP_E_DTYPE;
         return attention_fwd<float>((const float *)q, (const float *)k, (const float *)v, n, q0, n_q_heads, n_kv_heads,
                                     head_dim, (float *)o, lse, st);
     }
     if (dtype != STREAMBP_BF16) return STREAMBP_E_DTYPE;
     const bool tc_ok = attention_tc_supported(n, q0, n_q_heads, n_kv_heads, head_dim, q, k, v);
-    if (engine == 2 && !tc_ok) return STREAMBP_E_SHAPE;
+    if (engine >= 2 && !tc_ok) return STREAMBP_E_SHAPE;
     if (engine != 1 && tc_ok)
         return attention_fwd_tc((const bf16 *)q, (const bf16 *)k, (const bf16 *)v, n, q0, n_q_heads, n_kv_heads,
-                                (bf16 *)o, lse, st);
+                                (bf16 *)o, lse, st, engine == 3 ? 1 : (engine == 4 ? 2 : 0));
     return attention_fwd<bf16>((const bf16 *)q, (const bf16 *)k, (const bf16 *)v, n, q0, n_q_heads, n_kv_heads,
                                head_dim, (bf16 *)o, lse, st);
 }

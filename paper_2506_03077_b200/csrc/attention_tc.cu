@@ -1039,7 +1039,7 @@ bool attention_tc_supported(int64_t n, int64_t q0, int Hq, int Hkv, int dh, cons
 }
 
 int attention_fwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, int64_t n, int64_t q0, int Hq, int Hkv, bf16 *o,
-                     float *lse, cudaStream_t st) {
+                     float *lse, cudaStream_t st, int tiles_per_cta) {
     CUtensorMap mq, mk, mv;
     const int64_t kv_len = q0 + n;
     if (!make_tensor_map(&mq, q, n, (int64_t)Hq * TILE, (int64_t)Hq * TILE, 64, TILE, false) ||
@@ -1057,7 +1057,8 @@ int attention_fwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, int64_t n, int
     // leave SMs empty that one-tile CTAs would fill (short chunks, few heads).
     const int64_t ctas1 = (n + TILE - 1) / TILE * Hq, ctas2 = (n + 2 * TILE - 1) / (2 * TILE) * Hq;
     const int64_t sms = sm_count();
-    if (n > TILE && 3 * ((ctas2 + sms - 1) / sms) <= 2 * ((ctas1 + sms - 1) / sms)) {
+    const bool two = tiles_per_cta == 2 || (tiles_per_cta == 0 && n > TILE && 3 * ((ctas2 + sms - 1) / sms) <= 2 * ((ctas1 + sms - 1) / sms));
+    if (two) {
         dim3 grid((unsigned)((n + 2 * TILE - 1) / (2 * TILE)), Hq);
         SBP_LAUNCH(attn_fwd_2q_kernel, grid, FWD2Q_THREADS, FWD2Q_SMEM, st, mq, mk, mv, p);
         return STREAMBP_OK;

@@ -303,8 +303,9 @@ int attention_bwd(const T *q, const T *k, const T *v, const T *o, const T *dout,
 // tcgen05 attention (bf16, head_dim 128)
 bool attention_tc_supported(int64_t n, int64_t q0, int Hq, int Hkv, int dh, const void *q, const void *k,
                             const void *v);
+// tiles_per_cta: 0 = chosen from the grid size, 1 / 2 = one / two 128-query tiles per CTA (tests, profiling)
 int attention_fwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, int64_t n, int64_t q0, int Hq, int Hkv, bf16 *o,
-                     float *lse, cudaStream_t st);
+                     float *lse, cudaStream_t st, int tiles_per_cta = 0);
 // delta [Hq, n] must already hold rowsum(dO * O) (attention_delta below).
 int attention_bwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, const bf16 *dout, const float *lse,
                      const float *delta, int64_t n, int64_t q0, int Hq, int Hkv, float *dq, float *dk, float *dv,
