@@ -193,6 +193,11 @@ def test_swiglu_product(M, N, K, dtype):
     assert (m.double().cpu() - m_ref).norm() / m_ref.norm() < (3e-3 if dtype == torch.bfloat16 else 1e-6)
 
 
+def test_product_kernel_query():
+    """On a B200 a two-CTA cluster with the full shared-memory carve-out can be scheduled, so bf16 products run on CTA pairs."""
+    assert B.product_kernel() == "cta_pair"
+
+
 def test_single_cta_fallback_kernel():
     """The single-CTA product kernel (used where a two-CTA cluster cannot be scheduled) is selected by an environment
     variable read when the library first runs a product: exercised in a fresh interpreter, all three layouts."""
