@@ -41,6 +41,17 @@ def layer_flops(s, T):
 NCU_TRAFFIC_BYTES = {("qwen7b_layer", 1024): 2142.5e6, ("llama8b_layer", 2048): 2421.9e6}
 
 
+def check_outputs(tensors) -> str:
+    """After the warm-up steps, outside any timed region: every output tensor is finite and not identically zero, so a
+    step that skipped its work cannot produce a number.  (Values are checked against the oracle by the tests.)"""
+    import torch
+    for name, t in tensors.items():
+        f = t.float()
+        assert bool(torch.isfinite(f).all()), f"bench: output {name} is not finite"
+        assert float(f.abs().max()) > 0.0, f"bench: output {name} is identically zero"
+    return "finite and non-zero: " + ", ".join(tensors)
+
+
 def max_over_ranks(ms: float, world: int, device) -> float:
     """Timing rule for N > 1: every rank reports the slowest rank's device time."""
     import torch
@@ -238,6 +249,7 @@ def run_head_or_model(args, cfg):
     assert B.last_device_status(ws) == B.OK
     launches = B.last_launch_count()
     torch.cuda.synchronize()
+    checked = check_outputs({"loss": loss, "d_w_vocab": dW if cfg.layer is None else dWv, "d_g_final": dg})
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(0)
     sampler.start()
@@ -276,7 +288,7 @@ def run_head_or_model(args, cfg):
         "tflops_executed": executed_flops / (ms * 1e-3) / 1e12,
         "frac_of_measured_sustained_bf16_executed": executed_flops / (ms * 1e-3) / 1e12 / peaks["sustained"],
         "peak_activation_gb": ws_bytes / 1e9, "peak_activation_gb_unchunked": ws_full / 1e9,
-        "gpu_launches": int(launches * args.steps),
+        "gpu_launches": int(launches * args.steps), "outputs_checked": checked,
         "roofline": {"bound": "tensor", "kernel": "linear products (executed FLOPs)", "achieved": achieved,
                      "peak": peaks["sustained"],
                      "unit": "TFLOP/s", "frac": achieved / peaks["sustained"], "traffic": None,
@@ -408,6 +420,7 @@ def main():
         step()
     assert B.last_device_status(ws) == B.OK
     launches_per_step = B.last_launch_count()
+    checked = check_outputs({"dX": dX, **{"d_" + k: v for k, v in grads.items()}})
 
     sampler = ClockSampler(local)
     if rank == 0:
@@ -453,7 +466,7 @@ def main():
         "frac_of_measured_burst_bf16": flops / (ms_per_step * 1e-3) / 1e12 / peaks["burst"],
         "frac_of_nominal_bf16": flops / (ms_per_step * 1e-3) / 1e12 / 2250.0,
         "peak_activation_gb": ws_bytes / 1e9, "peak_activation_gb_unchunked": ws_full / 1e9,
-        "gpu_launches": int(launches_per_step * args.steps),
+        "gpu_launches": int(launches_per_step * args.steps), "outputs_checked": checked,
         "roofline": {"bound": "tensor", "kernel": "linear products (all GEMM launches of the step)",
                      "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                      "peak_source": peaks["source"] + " sustained bf16",

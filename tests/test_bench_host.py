@@ -63,3 +63,13 @@ def test_reference_arm_prints_one_json_line():
     j = json.loads(lines[0])
     assert j["impl"] == "reference" and j["cpu_baseline"]["kind"] == "oracle"
     assert j["e2e"]["h2d_bytes_per_step"] == 0 and j["value"] > 0
+
+
+def test_output_check_rejects_skipped_work():
+    import torch
+    ok = {"a": torch.ones(4), "b": torch.tensor([0.0, -2.0])}
+    assert "a, b" in bench.check_outputs(ok)
+    with pytest.raises(AssertionError):
+        bench.check_outputs({"a": torch.zeros(4)})                       # a step that never wrote its output
+    with pytest.raises(AssertionError):
+        bench.check_outputs({"a": torch.tensor([1.0, float("nan")])})
