@@ -10,6 +10,7 @@ from paper_2506_03077_b200 import synth
 from helpers import TOL, assert_close, to_dev
 
 pytestmark = pytest.mark.gpu
+FULL_ORACLE = __import__("os").environ.get("STREAMBP_FULL_ORACLE") == "1"
 
 
 def run_model(ls, hs, layers, g, Wv, labels, chunk_l, chunk_h, dtype, E=None, ids=None, X0=None):
@@ -107,3 +108,39 @@ def test_error_growth_through_28_layers_bf16():
     for l in (0, 13, 27):
         for k, v in ref["layers"][l].items():
             assert_close(f"layer{l}.{k}", Gd[l][k], v, tol)
+
+
+@pytest.mark.skipif(not FULL_ORACLE, reason="a minute of CPU time and 40 GB of host memory: set STREAMBP_FULL_ORACLE=1")
+def test_model_full_widths_two_layers_bf16():
+    """The full model configuration's widths (d 3584, 28 / 4 heads of 128, d_ff 18944, vocabulary 152064, biases,
+    untied embedding, everything ~N(0, 0.02)) at a depth and length the oracle can afford: 2 layers, 2048 tokens,
+    chunks of 1024 in the layers and in the head.  The full 28-layer, 65536-token call itself is beyond a direct
+    oracle run; it composes exactly the layer and head calls checked at full size elsewhere.
+
+    With an N(0, 0.02) embedding the residual stream is the MLP output, so every bf16-stored activation of the forward
+    pass shows in the hidden state the head sees (the oracle rounds nothing in between): all gradients carry ~1.2e-2,
+    and the most sensitive ones -- W_q, W_k and their biases in the last layer, which pass through
+    dS = P (dP - delta) -- twice that.  The fp32-arithmetic CUDA-core engine on the same bf16 storage measures the same
+    (2.44e-2 against 2.50e-2 for the tensor-core kernels): it is storage rounding, not kernel arithmetic.  Hence two
+    bounds: 3e-2 for those four and for g1, which collects the same path (1.98e-2), 2e-2 for everything else."""
+    c = synth.CONFIGS["qwen7b_model"]
+    ls, hs = c.layer, c.head
+    T, L = 2048, 2
+    layers = [synth.make_layer_weights(ls, c.seed, True, prefix=f"layer{l}") for l in range(L)]
+    E = synth.round_bf16(synth.normal(c.seed, "embed", (hs.vocab, ls.d_model), 0.0, 0.02))
+    g = synth.round_bf16(synth.normal(c.seed, "g_final", (ls.d_model,), 1.0, 0.02))
+    Wv = synth.round_bf16(synth.normal(c.seed, "w_vocab", (hs.vocab, ls.d_model), 0.0, 0.02))
+    ids, labels = synth.make_model_tokens(hs.vocab, c.seed, T, c.prompt_frac)
+    loss, Gd, dg, dWv, dX0, dE = run_model(ls, hs, layers, g, Wv, labels, 1024, 1024, torch.bfloat16, E=E, ids=ids)
+    ref = O.model_backward(O.LayerCfg(ls.d_model, ls.n_q_heads, ls.n_kv_heads, ls.head_dim, ls.d_ff, ls.qkv_bias,
+                                      ls.rope_theta, ls.rms_eps),
+                           O.HeadCfg(hs.d_model, hs.vocab), layers, g, Wv, labels, embed=E, ids=ids)
+    tol = TOL[torch.bfloat16]
+    assert abs(loss.item() - ref["loss"]) <= 3e-3 * ref["loss"]
+    errs = {"d_embed": assert_close("d_embed", dE, ref["d_embed"], tol),
+            "d_w_vocab": assert_close("d_w_vocab", dWv, ref["w_vocab"], tol),
+            "d_g_final": assert_close("d_g_final", dg, ref["g_final"], tol)}
+    for l in range(L):
+        for k, v in ref["layers"][l].items():
+            errs[f"layer{l}.{k}"] = assert_close(f"layer{l}.{k}", Gd[l][k], v, 3e-2 if k in ("wq", "wk", "bq", "bk", "g1") else tol)
+    print("full-width 2-layer model, errors vs oracle:", {k: f"{v:.2e}" for k, v in sorted(errs.items(), key=lambda kv: -kv[1])[:6]})
