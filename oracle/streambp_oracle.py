@@ -129,41 +129,46 @@ def _causal_probs(q_rows, k_all, t0, scale):
     return e / np.sum(e, axis=-1, keepdims=True)
 
 
-def attention_forward(q, k, v, row_block=1024):
-    """q: [T, Hq, dh]; k, v: [T, Hkv, dh]; query head h reads KV head h // (Hq/Hkv)."""
-    T, Hq, dh = q.shape
+def attention_forward(q, k, v, row_block=1024, q_start=0):
+    """q: [T - q_start, Hq, dh], the query rows q_start .. T-1; k, v: [T, Hkv, dh]; query head h reads KV head
+    h // (Hq/Hkv).  q_start > 0 only restricts which rows are evaluated (rows are independent)."""
+    n, Hq, dh = q.shape
+    T = q_start + n
     G = Hq // k.shape[1]
     scale = 1.0 / np.sqrt(F64(dh))
     o = np.empty_like(q)
     for h in range(Hq):
         kh, vh = k[:, h // G, :], v[:, h // G, :]
-        for t0 in range(0, T, row_block):
+        for t0 in range(q_start, T, row_block):
             t1 = min(T, t0 + row_block)
-            p = _causal_probs(q[t0:t1, h, :], kh, t0, scale)
-            o[t0:t1, h, :] = p @ vh[:t1]
+            p = _causal_probs(q[t0 - q_start:t1 - q_start, h, :], kh, t0, scale)
+            o[t0 - q_start:t1 - q_start, h, :] = p @ vh[:t1]
     return o
 
 
-def attention_backward(q, k, v, do, row_block=1024):
-    """Returns (dq, dk, dv). dk, dv are summed over the query heads of each KV group."""
-    T, Hq, dh = q.shape
+def attention_backward(q, k, v, do, row_block=1024, q_start=0):
+    """Returns (dq, dk, dv). dk, dv are summed over the query heads of each KV group.  q, do: the query rows
+    q_start .. T-1 (as in attention_forward); dk, dv: [T, Hkv, dh], the contribution of those rows."""
+    n, Hq, dh = q.shape
+    T = q_start + n
     G = Hq // k.shape[1]
     scale = 1.0 / np.sqrt(F64(dh))
     dq = np.empty_like(q)
-    dk = np.zeros_like(k)
-    dv = np.zeros_like(v)
+    dk = np.zeros_like(k[:T])
+    dv = np.zeros_like(v[:T])
     for h in range(Hq):
         g = h // G
         kh, vh = k[:, g, :], v[:, g, :]
-        for t0 in range(0, T, row_block):
+        for t0 in range(q_start, T, row_block):
             t1 = min(T, t0 + row_block)
-            p = _causal_probs(q[t0:t1, h, :], kh, t0, scale)
-            doh = do[t0:t1, h, :]
+            a, b = t0 - q_start, t1 - q_start
+            p = _causal_probs(q[a:b, h, :], kh, t0, scale)
+            doh = do[a:b, h, :]
             dv[:t1, g, :] += p.T @ doh
             dp = doh @ vh[:t1].T
             ds = p * (dp - np.sum(p * dp, axis=-1, keepdims=True))
-            dq[t0:t1, h, :] = (ds @ kh[:t1]) * scale
-            dk[:t1, g, :] += (ds.T @ q[t0:t1, h, :]) * scale
+            dq[a:b, h, :] = (ds @ kh[:t1]) * scale
+            dk[:t1, g, :] += (ds.T @ q[a:b, h, :]) * scale
     return dq, dk, dv
 
 
@@ -379,32 +384,32 @@ def _backprop_token_coefficients(cfg: HeadCfg, g_final, w_vocab, H, tokens, coef
     return dH, dW, dg
 
 
-def grpo_token_terms(logp, logp_old, logp_ref, advantage, beta, clip_eps, branch_logp=None):
+def grpo_token_terms(logp, logp_old, logp_ref, advantage, beta, clip_eps):
     """f(t) of Eq. (4) and df/dlog pi_theta(t):
     f = min(r A, clip(r, 1-eps, 1+eps) A) - beta (log pi_theta - log pi_ref), r = pi_theta / pi_old.
 
-    The min / clip is a branch decided by a floating-point comparison.  `branch_logp` (float32 log pi_theta
-    values, e.g. those a lower-precision implementation reports) lets a comparison take that decision from
-    the same numbers, in float32, as the implementation under test; the values of f and df are always
-    computed from `logp` in float64."""
+    The min / clip is a branch; it is decided here, in float64, from this function's own arguments only.
+    A comparison with a lower-precision implementation is meaningful for tokens whose ratio keeps a margin
+    from 1 +- eps (see `grpo_branch_margin`): the caller builds its inputs that way."""
     r = np.exp(logp - logp_old)
     unclipped = r * advantage
     clipped = np.clip(r, 1.0 - clip_eps, 1.0 + clip_eps) * advantage
-    if branch_logp is None:
-        inside = (r > 1.0 - clip_eps) & (r < 1.0 + clip_eps)
-        takes_unclipped = unclipped <= clipped
-    else:
-        f32 = np.float32
-        rb = np.exp(np.asarray(branch_logp, f32) - np.asarray(logp_old, f32))
-        adv32 = np.asarray(advantage, f32)
-        lo, hi = f32(1.0) - f32(clip_eps), f32(1.0) + f32(clip_eps)
-        inside = (rb > lo) & (rb < hi)
-        takes_unclipped = rb * adv32 <= np.minimum(np.maximum(rb, lo), hi) * adv32
+    inside = (r > 1.0 - clip_eps) & (r < 1.0 + clip_eps)
+    takes_unclipped = unclipped <= clipped
     # d(r A)/dlog pi = r A; the clipped branch is constant in log pi wherever the clip is active
     keeps = takes_unclipped | inside
     f = np.where(keeps, unclipped, clipped) - beta * (logp - logp_ref)
     df = np.where(keeps, unclipped, 0.0) - beta
     return f, df
+
+
+def grpo_branch_margin(logp, logp_old, clip_eps):
+    """Per token, the distance in log pi_theta to the nearest point where the min / clip branch of Eq. (4)
+    changes: |log r - log(1 - eps)| and |log r - log(1 + eps)| (the only places where the derivative of
+    min(r A, clip(r) A) jumps for A != 0).  An implementation whose log-probabilities are within less than
+    this margin of the exact ones takes the same branch."""
+    x = _f64(logp) - _f64(logp_old)
+    return np.minimum(np.abs(x - np.log1p(-clip_eps)), np.abs(x - np.log1p(clip_eps)))
 
 
 def lmhead_grpo_forward(cfg: HeadCfg, g_final, w_vocab, H, tokens, logp_old, logp_ref, advantage, weight,
@@ -419,13 +424,13 @@ def lmhead_grpo_forward(cfg: HeadCfg, g_final, w_vocab, H, tokens, logp_old, log
 
 
 def lmhead_grpo_backward(cfg: HeadCfg, g_final, w_vocab, H, tokens, logp_old, logp_ref, advantage, weight,
-                         beta, clip_eps, row_block=512, branch_logp=None):
+                         beta, clip_eps, row_block=512):
     """Returns (loss, logp, dH, dW_vocab, dg_final) for the GRPO objective."""
     g_final, w_vocab, H = _f64(g_final), _f64(w_vocab), _f64(H)
     tokens = np.asarray(tokens, dtype=np.int64)
     part = tokens != cfg.ignore_index
     logp = _token_logprobs(cfg, g_final, w_vocab, H, tokens, row_block)
-    f, df = grpo_token_terms(logp, _f64(logp_old), _f64(logp_ref), _f64(advantage), beta, clip_eps, branch_logp)
+    f, df = grpo_token_terms(logp, _f64(logp_old), _f64(logp_ref), _f64(advantage), beta, clip_eps)
     w = _f64(weight)
     loss = float(-np.sum(np.where(part, w * f, 0.0)))
     dH, dW, dg = _backprop_token_coefficients(cfg, g_final, w_vocab, H, tokens, -w * df, row_block)

@@ -256,6 +256,19 @@ streambp_layer_weights effective(const streambp_layer_cfg *c, const streambp_lay
     if (!c->qkv_bias) e.bq = e.bk = e.bv = nullptr;
     return e;
 }
+}  // namespace
+
+// Alignment the attention backward needs of its arguments (16-byte vector accesses and TMA tiles on the tensors,
+// 4 bytes on the per-row vectors); `delta` may be nullptr where the caller does not pass one.
+bool attention_bwd_aligned(const void *q, const void *k, const void *v, const void *o, const void *d_o,
+                           const void *lse, const void *delta, const void *dq, const void *dk, const void *dv) {
+    const void *t16[] = {q, k, v, o, d_o, dq, dk, dv};
+    for (const void *p : t16)
+        if (!aligned(p, 16)) return false;
+    return aligned(lse, 4) && (delta == nullptr || aligned(delta, 4));
+}
+
+namespace {
 int begin_call(void *ws, cudaStream_t st) {
     call_state().cuda_error = 0;
     call_state().launches = 0;
@@ -495,6 +508,9 @@ int streambp_attention_forward(const void *q, const void *k, const void *v, int6
     if (n < 1 || q0 < 0 || n_q_heads < 1 || n_kv_heads < 1 || n_q_heads % n_kv_heads ||
         (head_dim != 64 && head_dim != 128))
         return STREAMBP_E_SHAPE;
+    // the kernels use 16-byte vector accesses and TMA tiles on every tensor: refused here, never faulted on the device
+    if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(o, 16) || !aligned(lse, 4))
+        return STREAMBP_E_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     call_state().cuda_error = 0;
     call_state().launches = 0;
@@ -521,6 +537,7 @@ int streambp_attention_backward(const void *q, const void *k, const void *v, con
     if (n < 1 || q0 < 0 || n_q_heads < 1 || n_kv_heads < 1 || n_q_heads % n_kv_heads ||
         (head_dim != 64 && head_dim != 128))
         return STREAMBP_E_SHAPE;
+    if (!attention_bwd_aligned(q, k, v, o, d_o, lse, delta, dq, dk, dv)) return STREAMBP_E_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     call_state().cuda_error = 0;
     call_state().launches = 0;

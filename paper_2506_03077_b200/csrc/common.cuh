@@ -313,6 +313,9 @@ int attention_bwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, const bf16 *do
 template <typename T>
 int attention_delta(const T *o, const T *dout, int64_t n, int Hq, int dh, float *delta, cudaStream_t st);
 int attention_tc_take_fault();
+// Pointer alignment the attention backward entry points require (delta may be nullptr: not checked then).
+bool attention_bwd_aligned(const void *q, const void *k, const void *v, const void *o, const void *d_o,
+                           const void *lse, const void *delta, const void *dq, const void *dk, const void *dv);
 // Dispatching attention used by the schedulers (tensor cores when supported, else CUDA cores).
 template <typename T>
 int attn_fwd(const T *q, const T *k, const T *v, int64_t n, int64_t q0, int Hq, int Hkv, int dh, T *o, float *lse,

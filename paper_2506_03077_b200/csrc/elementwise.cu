@@ -528,13 +528,11 @@ __global__ void __launch_bounds__(1024)
     const unsigned long long N = hdr->n_valid;
     const bool vec = (V & 3) == 0;
     if (!valid || N == 0) {
-        for (int64_t c = threadIdx.x * 4; c < V; c += blockDim.x * 4) {
-            if (vec && c + 3 < V) {
-                dr[c] = from_f32<T>(0.f); dr[c + 1] = from_f32<T>(0.f);
-                dr[c + 2] = from_f32<T>(0.f); dr[c + 3] = from_f32<T>(0.f);
-            } else {
-                for (int64_t k = c; k < V; k++) dr[k] = from_f32<T>(0.f);
-            }
+        if (vec) {
+            const float zero4[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int64_t c = threadIdx.x * 4; c < V; c += blockDim.x * 4) store4(dr + c, zero4);
+        } else {
+            for (int64_t c = threadIdx.x; c < V; c += blockDim.x) dr[c] = from_f32<T>(0.f);
         }
         if (threadIdx.x == 0) row_loss[row] = 0.f;
         return;

@@ -59,6 +59,8 @@ extern "C" int streambp_attention_backward_static(const void *q, const void *k, 
     if (n > kMaxDeltaFloats / n_q_heads) return STREAMBP_E_WORKSPACE;
     if (dtype != STREAMBP_F32 && dtype != STREAMBP_BF16) return STREAMBP_E_DTYPE;
     if (dtype == STREAMBP_F32 && engine == 2) return STREAMBP_E_DTYPE;
+    // misaligned tensors are refused on the host: on the device they would fault and poison the context
+    if (!attention_bwd_aligned(q, k, v, o, d_o, lse, nullptr, dq, dk, dv)) return STREAMBP_E_ALIGN;
     float *delta = nullptr;
     SBP_TRY(static_delta(&delta));
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);

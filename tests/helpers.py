@@ -44,11 +44,39 @@ def run_layer(bcfg, W, X, dY, chunk, pos0=0, accumulate=False, grads=None):
     return dX, grads
 
 
-def assert_close(name, got: torch.Tensor, ref: np.ndarray, tol: float):
+# A relative Frobenius norm over a whole tensor cannot see a fault confined to a few rows: at 2e-2 three wrong rows
+# of an [8192, d] tensor, or one mis-addressed 128-row tile of a 32k-row one, still pass.  So every comparison also
+# bounds the error of each block of BLOCK_ROWS rows (and, for [rows, heads, head_dim] tensors, of each head's
+# columns) by BLOCK_FACTOR x the tensor's tolerance, relative to that block's own reference norm -- or to a
+# quarter of the mean block norm where the block itself is small (masked rows, keys few queries attend to).
+BLOCK_ROWS = 128
+BLOCK_FACTOR = 4.0
+
+
+def block_errors(g: np.ndarray, ref: np.ndarray, heads: int = 1) -> np.ndarray:
+    """[row blocks, heads] relative errors as described above; g, ref: float64, same shape, >= 1 dimension."""
+    rows = ref.shape[0]
+    g2 = g.reshape(rows, heads, -1)
+    r2 = ref.reshape(rows, heads, -1)
+    edges = list(range(0, rows, BLOCK_ROWS))
+    num = np.add.reduceat(((g2 - r2) ** 2).sum(-1), edges, axis=0)
+    den = np.add.reduceat((r2 ** 2).sum(-1), edges, axis=0)
+    floor = den.mean() / 16.0
+    return np.sqrt(num / np.maximum(np.maximum(den, floor), 1e-300))
+
+
+def assert_close(name, got: torch.Tensor, ref: np.ndarray, tol: float, heads: int = 1):
     g = got.detach().float().cpu().numpy().astype(np.float64)
     assert np.isfinite(g).all(), f"{name}: non-finite values"
+    ref = np.asarray(ref, dtype=np.float64)
+    assert g.shape == ref.shape, f"{name}: shape {g.shape} vs {ref.shape}"
     err = O.rel_frobenius(g, ref)
     assert err <= tol, f"{name}: relative Frobenius error {err:.3e} > {tol:.1e}"
+    if ref.ndim >= 1 and ref.size and np.linalg.norm(ref) > 0.0:
+        be = block_errors(g, ref, heads)
+        worst = np.unravel_index(np.argmax(be), be.shape)
+        assert be[worst] <= BLOCK_FACTOR * tol, \
+            f"{name}: rows {worst[0] * BLOCK_ROWS}.., head {worst[1]}: block error {be[worst]:.3e} > {BLOCK_FACTOR * tol:.1e}"
     return err
 
 

@@ -110,6 +110,31 @@ def test_host_side_errors(lib):
     assert lib.streambp_last_device_status(None, None) == B.E_NULL
 
 
+def test_attention_entry_points_refuse_misaligned_pointers(lib):
+    """A tensor that is only 4-byte aligned (an offset view) would fault on the device, where the kernels use 16-byte
+    vector accesses and TMA tiles; the three attention entry points return E_ALIGN before anything is enqueued."""
+    a = 4096                                  # never dereferenced: validation precedes every CUDA call
+    fwd = lambda **kw: lib.streambp_attention_forward(kw.get("q", a), kw.get("k", a), kw.get("v", a), 128, 0, 4, 2, 128,
+                                                      1, kw.get("o", a), kw.get("lse", a), 0, None)
+    for name in ("q", "k", "v", "o"):
+        assert fwd(**{name: a + 4}) == B.E_ALIGN, name
+    assert fwd(lse=a + 2) == B.E_ALIGN
+    names = ("q", "k", "v", "o", "d_o", "lse", "delta", "dq", "dk", "dv")
+
+    def bwd(static, **kw):
+        p = {n: kw.get(n, a) for n in names}
+        if static:
+            return lib.streambp_attention_backward_static(p["q"], p["k"], p["v"], p["o"], p["d_o"], p["lse"], 128, 0, 4,
+                                                          2, 128, 1, p["dq"], p["dk"], p["dv"], 0, None)
+        return lib.streambp_attention_backward(p["q"], p["k"], p["v"], p["o"], p["d_o"], p["lse"], 128, 0, 4, 2, 128, 1,
+                                               p["delta"], p["dq"], p["dk"], p["dv"], 0, None)
+    for static in (False, True):
+        for name in ("q", "k", "v", "o", "d_o", "dq", "dk", "dv"):
+            assert bwd(static, **{name: a + 4}) == B.E_ALIGN, (static, name)
+        assert bwd(static, lse=a + 2) == B.E_ALIGN
+    assert bwd(False, delta=a + 2) == B.E_ALIGN
+
+
 def test_suggested_chunk_is_the_largest_that_fits(lib):
     """Sec. 4.3: partition size is the memory / time knob.  The suggestion is the largest multiple of 128 (or T)
     whose exact workspace fits the budget, checked against a scan of the planner."""

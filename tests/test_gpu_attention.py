@@ -7,6 +7,7 @@ import torch
 from oracle import streambp_oracle as O
 from paper_2506_03077_b200 import binding as B
 from paper_2506_03077_b200 import synth
+from helpers import assert_close
 
 pytestmark = pytest.mark.gpu
 
@@ -30,6 +31,14 @@ def oracle_chunk(q, k, v, do, q0):
     do_chunk[:q0] = 0.0
     dq, dk, dv = O.attention_backward(q.astype(np.float64), k.astype(np.float64), v.astype(np.float64), do_chunk)
     return o[q0:], dq[q0:], dk, dv
+
+
+def oracle_window(q, k, v, do, q0):
+    """The same for a long prefix: only the chunk's query rows are evaluated (q, do hold rows q0.. only)."""
+    f = lambda a: a.astype(np.float64)
+    o = O.attention_forward(f(q), f(k), f(v), q_start=q0)
+    dq, dk, dv = O.attention_backward(f(q), f(k), f(v), f(do), q_start=q0)
+    return o, dq, dk, dv
 
 
 def oracle_lse(q, k, q0, dh):
@@ -94,9 +103,41 @@ def test_attention_backward_bf16(engine, n, q0, Hq, Hkv):
     dv = torch.ones((q0 + n, Hkv, dh), device="cuda")
     B.attention_backward(qd, kd, vd, o, dod, lse, q0, dq, dk, dv, engine=engine)
     torch.cuda.synchronize()
-    assert O.rel_frobenius(dq.cpu().numpy(), dq_ref) < 1.5e-2
-    assert O.rel_frobenius(dk.cpu().numpy() - 1.0, dk_ref) < 1.5e-2
-    assert O.rel_frobenius(dv.cpu().numpy() - 1.0, dv_ref) < 1.5e-2
+    assert_close("dq", dq, dq_ref, 1.5e-2, heads=Hq)
+    assert_close("dk", dk - 1.0, dk_ref, 1.5e-2, heads=Hkv)
+    assert_close("dv", dv - 1.0, dv_ref, 1.5e-2, heads=Hkv)
+
+
+# The prefix lengths of the T = 32768 layer configuration: the last chunk (2048 queries against 32768 keys, 256 key
+# tiles per CTA: lazy rescale, the K/V rings and the merged dK/dV + dQ grid all in their long-run regime) and a ragged
+# 200-row chunk that ends at the same row.  Four query heads on one KV head keep the oracle (numpy, float64) at a few
+# seconds.  Every (128-row block, head) of every output is bounded, not only the whole tensor.
+@pytest.mark.parametrize("n,q0", [(2048, 30720), (200, 32768 - 200)])
+def test_attention_full_prefix_bf16(n, q0):
+    Hq, Hkv, dh, dt = 4, 1, 128, torch.bfloat16
+    kv = q0 + n
+    f = lambda name, shape, s=1.0: synth.round_bf16(synth.normal(900 + n, name, shape, 0.0, s))
+    q, do = f("q", (n, Hq, dh), 1.5), f("do", (n, Hq, dh))
+    k, v = f("k", (kv, Hkv, dh), 1.5), f("v", (kv, Hkv, dh))
+    o_ref, dq_ref, dk_ref, dv_ref = oracle_window(q, k, v, do, q0)
+    qd, dod = (torch.from_numpy(a).to("cuda", dt).contiguous() for a in (q, do))
+    kd, vd = torch.from_numpy(k).to("cuda", dt), torch.from_numpy(v).to("cuda", dt)
+    o = torch.empty((n, Hq, dh), device="cuda", dtype=dt)
+    lse = torch.empty((Hq, n), device="cuda")
+    for engine in (3, 4):                  # one and two query tiles per CTA
+        o.fill_(float("nan")); lse.fill_(float("nan"))
+        B.attention_forward(qd, kd, vd, q0, o, lse, engine=engine)
+        torch.cuda.synchronize()
+        assert_close(f"o (engine {engine})", o, o_ref, 6e-3, heads=Hq)
+        assert torch.isfinite(lse).all()
+    dq = torch.full((n, Hq, dh), float("nan"), device="cuda")
+    dk = torch.zeros((kv, Hkv, dh), device="cuda")
+    dv = torch.zeros((kv, Hkv, dh), device="cuda")
+    B.attention_backward(qd, kd, vd, o, dod, lse, q0, dq, dk, dv, engine=2)
+    torch.cuda.synchronize()
+    assert_close("dq", dq, dq_ref, 1.5e-2, heads=Hq)
+    assert_close("dk", dk, dk_ref, 1.5e-2, heads=Hkv)
+    assert_close("dv", dv, dv_ref, 1.5e-2, heads=Hkv)
 
 
 @pytest.mark.parametrize("dh,dtype", [(64, torch.float32), (128, torch.float32), (64, torch.bfloat16)])
@@ -165,3 +206,9 @@ def test_attention_growing_maxima_tensor_core():
                         O.rel_frobenius(dv.cpu().numpy(), dv_ref))
     assert errs[2][1] < 1e-2 and errs[2][2] < 1e-2
     assert errs[2][0] < 2.5 * errs[1][0] + 1e-2
+    assert errs[2][0] < DQ_GROWING_MAXIMA_TOL, errs
+
+
+# dQ against the oracle in the ill-conditioned case above, as measured for both engines on the same bf16 O
+# (the bound is the conditioning of the case, see the comment in the test, not a property of either engine)
+DQ_GROWING_MAXIMA_TOL = 0.25

@@ -11,6 +11,14 @@ from helpers import TOL, assert_close, to_dev
 pytestmark = pytest.mark.gpu
 
 
+# Every GRPO token keeps this distance (in log pi_theta) from the points where the min / clip branch of Eq. (4)
+# changes, so the oracle (float64) and the kernel (float32 from bf16 products) take the same branch without
+# either side seeing the other's numbers; the kernel's own log-probabilities are checked to be closer than that.
+CLIP_EPS = 0.2
+BRANCH_MARGIN = 0.08
+LOGP_TOL = {torch.float32: 2e-5, torch.bfloat16: 3e-2}
+
+
 def make_case(seed, T, d, V, dtype, masked):
     bf = dtype == torch.bfloat16
     hs = synth.HeadShape(d, V)
@@ -20,7 +28,11 @@ def make_case(seed, T, d, V, dtype, masked):
         W = synth.round_bf16(W)
     cfg = O.HeadCfg(d, V)
     lp = O._token_logprobs(cfg, g.astype(np.float64), W.astype(np.float64), H.astype(np.float64), tok, 256)
-    old = (lp + synth.normal(seed, "old", (T,), 0.0, 0.3)).astype(np.float32)
+    x = -synth.normal(seed, "old", (T,), 0.0, 0.3)              # log r = log pi_theta - log pi_old
+    for edge in (np.log1p(-CLIP_EPS), np.log1p(CLIP_EPS)):         # push ratios near a clip edge away from it
+        near = np.abs(x - edge) < BRANCH_MARGIN
+        x = np.where(near, edge + np.where(x >= edge, 1.0, -1.0) * BRANCH_MARGIN * 1.25, x)
+    old = (lp - x).astype(np.float32)
     ref = (lp + synth.normal(seed, "ref", (T,), 0.0, 0.3)).astype(np.float32)
     adv = synth.normal(seed, "adv", (T,)).astype(np.float32)
     return hs, cfg, g, W, H, tok, old, ref, adv
@@ -53,16 +65,18 @@ def test_grpo_matches_oracle(dtype, T, V, chunk):
     hs, cfg, g, W, H, tok, old, ref, adv = make_case(40 + T, T, 128, V, dtype, masked)
     tok[T // 2] = -100
     wt = np.full(T, 1.0 / (T - masked - 1), dtype=np.float32)
-    beta, eps = 0.04, 0.2
+    beta, eps = 0.04, CLIP_EPS
+    # the oracle decides alone; its own float64 log-probabilities confirm the margin the inputs were built with
+    ref_out = O.lmhead_grpo_backward(cfg, g, W, H, tok, old, ref, adv, wt, beta, eps)
+    part = tok != -100
+    margin = O.grpo_branch_margin(ref_out[1], old, eps)[part]
+    assert margin.min() >= BRANCH_MARGIN and LOGP_TOL[dtype] < 0.5 * BRANCH_MARGIN
+    r = np.exp(ref_out[1] - old)[part]
+    assert (r > 1 + eps).any() and (r < 1 - eps).any() and ((r > 1 - eps) & (r < 1 + eps)).any()
+    assert np.abs(adv[part]).min() > 0.0
     for ch in (chunk, 23):                         # chunk invariance, ragged
         loss, _, logp, dH, dW, dg = run_rl(hs, B.OBJ_GRPO, beta, eps, g, W, H, tok, old, ref, adv, wt, ch, dtype)
-        # the clip / min branch is a floating-point decision: the oracle takes it from the log-probabilities the
-        # kernel reports, in float32, and computes every value itself in float64
-        ref_out = O.lmhead_grpo_backward(cfg, g, W, H, tok, old, ref, adv, wt, beta, eps,
-                                         branch_logp=logp.cpu().numpy())
-        part = tok != -100
-        lp_tol = 2e-5 if dtype == torch.float32 else 3e-2
-        assert np.abs(logp.cpu().numpy()[part] - ref_out[1][part]).max() < lp_tol
+        assert np.abs(logp.cpu().numpy()[part] - ref_out[1][part]).max() < LOGP_TOL[dtype]
         assert torch.count_nonzero(logp[torch.from_numpy(~part).cuda()]) == 0
         assert abs(loss - ref_out[0]) <= (2e-5 if dtype == torch.float32 else 2e-2) * max(1.0, abs(ref_out[0]))
         assert_close("dH", dH, ref_out[2], TOL[dtype])

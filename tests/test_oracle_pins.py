@@ -252,6 +252,26 @@ def test_attention_uniform_when_keys_are_equal():
         assert np.allclose(o[:, h, :], expect, rtol=1e-13, atol=1e-15)
 
 
+def test_attention_query_window_selects_rows_only():
+    # evaluating the rows q_start.. alone gives those rows of the full result; their dk / dv contribution is what
+    # the full backward gives when the upstream gradient of the other rows is zero (linearity in do)
+    T, Hq, Hkv, dh, q0 = 19, 4, 2, 8, 11
+    q = synth.normal(2, "q", (T, Hq, dh)).astype(np.float64)
+    k = synth.normal(2, "k", (T, Hkv, dh)).astype(np.float64)
+    v = synth.normal(2, "v", (T, Hkv, dh)).astype(np.float64)
+    do = synth.normal(2, "do", (T, Hq, dh)).astype(np.float64)
+    o = O.attention_forward(q, k, v, row_block=5)
+    ow = O.attention_forward(q[q0:], k, v, row_block=3, q_start=q0)
+    assert np.allclose(ow, o[q0:], rtol=1e-13, atol=1e-15)
+    do0 = do.copy()
+    do0[:q0] = 0.0
+    dq, dk, dv = O.attention_backward(q, k, v, do0, row_block=5)
+    dqw, dkw, dvw = O.attention_backward(q[q0:], k, v, do[q0:], row_block=4, q_start=q0)
+    assert np.allclose(dqw, dq[q0:], rtol=1e-12, atol=1e-15)
+    assert np.allclose(dkw, dk, rtol=1e-12, atol=1e-15) and np.allclose(dvw, dv, rtol=1e-12, atol=1e-15)
+    assert np.abs(dq[:q0]).max() == 0.0
+
+
 def test_row_block_is_only_a_memory_knob():
     cfg = small_layer(True)
     W, X, dY = rand_layer(cfg, 6, 21)

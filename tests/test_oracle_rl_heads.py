@@ -122,16 +122,25 @@ def test_special_cases_reduce_to_cross_entropy():
         assert O.rel_frobenius(a, b) < 1e-12
 
 
-def test_branch_logp_only_moves_the_decision():
+def test_branch_margin_is_the_distance_to_a_change_of_branch():
+    # moving one token's log-probability by less than its margin leaves its (f, df) branch unchanged; moving it
+    # by more than the margin towards the nearest boundary changes df for a token whose advantage makes the clip bind
     cfg, g, W, H, tok, old, ref, adv, wt = setup(7)
-    base = O.lmhead_grpo_backward(cfg, g, W, H, tok, old, ref, adv, wt, 0.04, 0.2)
-    same = O.lmhead_grpo_backward(cfg, g, W, H, tok, old, ref, adv, wt, 0.04, 0.2, branch_logp=base[1].astype(np.float32))
-    assert same[0] == base[0] and np.array_equal(same[3], base[3])
-    # a perturbed log-probability that pushes one token across the clip boundary changes that token's term only
-    r = np.exp(base[1] - old)
+    lp = O._token_logprobs(cfg, g, W, H, tok, 7)
+    margin = O.grpo_branch_margin(lp, old, 0.2)
+    _, df0 = O.grpo_token_terms(lp, old, ref, adv, 0.04, 0.2)
+    r = np.exp(lp - old)
+    for t in np.nonzero(tok != -100)[0]:
+        for sgn in (-1.0, 1.0):
+            near = lp.copy()
+            near[t] += sgn * 0.9 * margin[t]
+            _, df1 = O.grpo_token_terms(near, old, ref, adv, 0.04, 0.2)
+            # same branch: df is either r A - beta on both sides or -beta on both sides
+            assert (df1[t] == -0.04) == (df0[t] == -0.04)
+    # a token inside the range with positive advantage: crossing 1 + eps switches the policy-gradient term off
     t = int(np.argmax((tok != -100) & (r > 1.0) & (r < 1.2) & (adv > 0)))
-    bl = base[1].astype(np.float32).copy()
-    bl[t] = old[t] + np.log(1.3)
-    moved = O.lmhead_grpo_backward(cfg, g, W, H, tok, old, ref, adv, wt, 0.04, 0.2, branch_logp=bl)
-    diff_rows = np.nonzero(np.abs(moved[2] - base[2]).sum(-1) > 0)[0]
-    assert list(diff_rows) == [t]
+    far = lp.copy()
+    far[t] = old[t] + np.log(1.2) + 1e-9
+    _, df2 = O.grpo_token_terms(far, old, ref, adv, 0.04, 0.2)
+    assert df0[t] != -0.04 and df2[t] == -0.04
+    assert abs(margin[t] - (np.log(1.2) - (lp[t] - old[t]))) < 1e-12

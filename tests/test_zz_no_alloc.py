@@ -31,9 +31,16 @@ def test_static_scratch_variant_matches_ordinary_entry_point(dtype, dh, engine):
         got = [torch.full_like(ref[0], float("nan")), torch.zeros_like(ref[1]), torch.zeros_like(ref[2])]
         B.attention_backward(q, k, v, o, do, lse, q0, *ref, engine=engine)
         before = torch.cuda.memory_allocated()
-        B.attention_backward_static(q, k, v, o, do, lse, q0, *got, engine=engine)
-        assert torch.cuda.memory_allocated() == before
         torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
+        B.attention_backward_static(q, k, v, o, do, lse, q0, *got, engine=engine)
+        torch.cuda.synchronize()
+        assert torch.cuda.memory_allocated() == before
+        # the driver's own count of free device memory sees an allocation made behind PyTorch's back; the first
+        # call may still load kernels and look up the array's address, so the second call is the one that must
+        # leave it unchanged
+        if call == 1:
+            assert torch.cuda.mem_get_info()[0] == free_before
         for name, a, b in zip(("dq", "dk", "dv"), got, ref):
             err = (a.double() - b.double()).norm() / b.double().norm()
             assert err <= (2e-2 if dtype == torch.bfloat16 else 1e-4), (call, name, float(err))
