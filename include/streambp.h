@@ -18,10 +18,15 @@
  *     dH, every weight): float or bf16.  Weight gradients, the loss and all
  *     accumulators are always float (fp32).  bf16 runs multiply bf16 operands and
  *     accumulate in fp32.
- *   - The library allocates no device memory and keeps no state between calls;
- *     it writes only to the outputs and the workspace.  Work is enqueued on
- *     `cuda_stream` (a cudaStream_t passed as void*, NULL = default stream) and
- *     the call returns without synchronising.
+ *   - The library allocates no device memory and writes only to the outputs and the
+ *     workspace; nothing a call computes survives it.  What the process does keep:
+ *     per-device facts looked up once (SM count, kernel attributes, the address of
+ *     the fixed scratch array of streambp_attention_backward_static), the per-thread
+ *     record behind streambp_last_cuda_error / streambp_last_launch_count, a device
+ *     flag a kernel raises when a bounded wait expires, and the event records of the
+ *     optional profiling below.  Work is enqueued on `cuda_stream` (a cudaStream_t
+ *     passed as void*, NULL = default stream) and the call returns without
+ *     synchronising.
  *   - Return value: STREAMBP_OK (0) or a negative streambp_status.  Errors found
  *     on the host are returned before anything is enqueued.  Conditions only the
  *     device can see (a label outside [0, vocab), no unmasked label, an expired
@@ -359,6 +364,22 @@ int streambp_profile_read(int kernel_class, double *milliseconds, int64_t *calls
  * fall back to the CUDA-core kernels).  Host-only query; launches nothing.
  */
 int streambp_product_kernel(void);
+
+/*
+ * Test hooks (no counterpart in the paper; not part of the method).
+ *
+ * streambp_test_expire_wait: launches a one-CTA kernel that runs the library's bounded mbarrier wait -- the
+ * same device function every tensor-core kernel waits in -- on a barrier nothing arrives at, with `limit_ns`
+ * (1 us .. 100 ms) in place of the kernels' two seconds, and then winds down as those kernels do (abort flag,
+ * drain, tensor memory freed).  The GPU is not hung and the context stays usable; afterwards
+ * streambp_last_device_status() on that stream returns STREAMBP_E_DEVICE_TIMEOUT once and clears the flag.
+ *
+ * streambp_test_per_device_value: the library caches per-device facts (SM count, shared-memory opt-in, product
+ * kernel choice) by device ordinal.  This runs that cache with `ordinal` in place of the current device and a
+ * value to remember on first use: it returns the value cached for that ordinal.  Host-only.
+ */
+int streambp_test_expire_wait(uint64_t limit_ns, void *cuda_stream);
+int streambp_test_per_device_value(int ordinal, int value);
 
 #ifdef __cplusplus
 }

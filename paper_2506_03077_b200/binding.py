@@ -34,6 +34,7 @@ EXPORTS = (
     "streambp_profile_enable", "streambp_profile_read", "streambp_product_kernel",
     "streambp_attention_forward", "streambp_attention_backward", "streambp_attention_backward_static",
     "streambp_lmhead_rl_backward", "streambp_layer_backward_packed",
+    "streambp_test_expire_wait", "streambp_test_per_device_value",
 )
 
 
@@ -140,6 +141,10 @@ def lib() -> C.CDLL:
     L.streambp_profile_enable.argtypes = [C.c_int]
     L.streambp_profile_read.restype = C.c_int
     L.streambp_profile_read.argtypes = [C.c_int, C.POINTER(C.c_double), C.POINTER(i64), C.POINTER(C.c_double)]
+    L.streambp_test_expire_wait.restype = C.c_int
+    L.streambp_test_expire_wait.argtypes = [C.c_uint64, vp]
+    L.streambp_test_per_device_value.restype = C.c_int
+    L.streambp_test_per_device_value.argtypes = [C.c_int, C.c_int]
     _lib = L
     return L
 
@@ -438,6 +443,14 @@ def gemm_swiglu(A, w_gate, w_up, g, u, m, stream=None, check: bool = True) -> in
 
 
 KERNEL_CLASSES = {"gemm": 0, "attention_fwd": 1, "attention_bwd": 2}
+
+
+def test_expire_wait(limit_ns: int, stream=None) -> int:
+    """Test hook: one tiny kernel whose bounded wait runs out after `limit_ns` (see streambp.h)."""
+    return lib().streambp_test_expire_wait(int(limit_ns), _stream_ptr(stream))
+
+
+test_expire_wait.__test__ = False     # a library call, not a pytest test
 
 
 def product_kernel() -> str:

@@ -1,4 +1,5 @@
 // extern "C" boundary: argument validation, dtype dispatch, status handling.
+#include <atomic>
 #include <cstdlib>
 #include <cstring>
 #include <vector>
@@ -13,7 +14,7 @@ CallState &call_state() {
 }
 
 namespace {
-int g_engine = -1;
+std::atomic<int> g_device_override{-1};
 
 struct ProfRec {
     cudaEvent_t a, b;
@@ -42,15 +43,21 @@ ProfScope::~ProfScope() {
 }
 
 int gemm_engine() {
-    if (g_engine < 0) {
+    static const int engine = [] {
         const char *e = std::getenv("STREAMBP_GEMM_ENGINE");
-        g_engine = 0;
-        if (e && !std::strcmp(e, "simt")) g_engine = 1;
-        if (e && !std::strcmp(e, "tc")) g_engine = 2;
-    }
-    return g_engine;
+        if (e && !std::strcmp(e, "simt")) return 1;
+        if (e && !std::strcmp(e, "tc")) return 2;
+        return 0;
+    }();
+    return engine;
 }
-void set_gemm_engine(int e) { g_engine = e; }
+
+int current_device_ordinal() {
+    const int fake = g_device_override.load();
+    if (fake >= 0) return fake;
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess ? dev : -1;
+}
 
 template <typename TI, typename TC>
 int mm(GemmOp op, int64_t M, int64_t N, int64_t K, const TI *A, int64_t lda, const TI *B, int64_t ldb, TC *C,
@@ -177,14 +184,14 @@ int attn_fwd<bf16>(const bf16 *q, const bf16 *k, const bf16 *v, int64_t n, int64
 template <>
 int attn_bwd<float>(const float *q, const float *k, const float *v, const float *o, const float *dout,
                     const float *lse, int64_t n, int64_t q0, int Hq, int Hkv, int dh, float *delta, float *dq,
-                    float *dk, float *dv, cudaStream_t st) {
+                    float *dk, float *dv, cudaStream_t st, int) {
     return attention_bwd<float>(q, k, v, o, dout, lse, n, q0, Hq, Hkv, dh, delta, dq, dk, dv, st);
 }
 template <>
 int attn_bwd<bf16>(const bf16 *q, const bf16 *k, const bf16 *v, const bf16 *o, const bf16 *dout, const float *lse,
                    int64_t n, int64_t q0, int Hq, int Hkv, int dh, float *delta, float *dq, float *dk, float *dv,
-                   cudaStream_t st) {
-    const int e = gemm_engine();
+                   cudaStream_t st, int engine) {
+    const int e = engine < 0 ? gemm_engine() : engine;
     if (e != 1 && attention_tc_supported(n, q0, Hq, Hkv, dh, q, k, v)) {
         SBP_TRY(attention_delta<bf16>(o, dout, n, Hq, dh, delta, st));
         return attention_bwd_tc(q, k, v, dout, lse, delta, n, q0, Hq, Hkv, dq, dk, dv, st);
@@ -476,9 +483,9 @@ int streambp_last_device_status(void *workspace, void *cuda_stream) {
     WsHeader h;
     if (!cuda_ok(cudaMemcpyAsync(&h, workspace, sizeof(h), cudaMemcpyDeviceToHost, st))) return STREAMBP_E_CUDA;
     if (!cuda_ok(cudaStreamSynchronize(st))) return STREAMBP_E_CUDA;
-    const int f1 = gemm_tc_take_fault(), f2 = attention_tc_take_fault();
-    if (f1 < 0 || f2 < 0) return STREAMBP_E_CUDA;
-    if (f1 > 0 || f2 > 0) return STREAMBP_E_DEVICE_TIMEOUT;
+    const int f1 = gemm_tc_take_fault(), f2 = attention_tc_take_fault(), f3 = wait_probe_take_fault();
+    if (f1 < 0 || f2 < 0 || f3 < 0) return STREAMBP_E_CUDA;
+    if (f1 > 0 || f2 > 0 || f3 > 0) return STREAMBP_E_DEVICE_TIMEOUT;
     return h.status;
 }
 
@@ -548,15 +555,28 @@ int streambp_attention_backward(const void *q, const void *k, const void *v, con
                                     st);
     }
     if (dtype != STREAMBP_BF16) return STREAMBP_E_DTYPE;
-    const int saved = gemm_engine();
-    set_gemm_engine(engine);
-    const int rc = attn_bwd<bf16>((const bf16 *)q, (const bf16 *)k, (const bf16 *)v, (const bf16 *)o,
-                                  (const bf16 *)d_o, lse, n, q0, n_q_heads, n_kv_heads, head_dim, delta, dq, dk, dv, st);
-    set_gemm_engine(saved);
-    return rc;
+    if (engine < 0 || engine > 2) return STREAMBP_E_SHAPE;
+    return attn_bwd<bf16>((const bf16 *)q, (const bf16 *)k, (const bf16 *)v, (const bf16 *)o, (const bf16 *)d_o, lse, n,
+                          q0, n_q_heads, n_kv_heads, head_dim, delta, dq, dk, dv, st, engine);
 }
 
 int streambp_product_kernel(void) { return gemm_tc_variant(); }
+
+int streambp_test_expire_wait(uint64_t limit_ns, void *cuda_stream) {
+    if (limit_ns < 1000 || limit_ns > 100000000ull) return STREAMBP_E_SHAPE;     // 1 us .. 100 ms
+    call_state().cuda_error = 0;
+    call_state().launches = 0;
+    return wait_probe_launch(limit_ns, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int streambp_test_per_device_value(int ordinal, int value) {
+    static PerDevice cache;
+    if (ordinal < 0) return STREAMBP_E_SHAPE;
+    g_device_override.store(ordinal);
+    const int got = cache.get([&] { return value; });
+    g_device_override.store(-1);
+    return got;
+}
 
 void streambp_profile_enable(int on) {
     g_prof_on = on != 0;

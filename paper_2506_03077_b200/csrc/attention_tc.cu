@@ -1046,12 +1046,9 @@ int attention_fwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, int64_t n, int
         !make_tensor_map(&mk, k, kv_len, (int64_t)Hkv * TILE, (int64_t)Hkv * TILE, 64, TILE, false) ||
         !make_tensor_map(&mv, v, kv_len, (int64_t)Hkv * TILE, (int64_t)Hkv * TILE, 64, TILE, false))
         return STREAMBP_E_CUDA;
-    static bool configured = false;
-    if (!configured) {
-        if (!opt_in_smem(attn_fwd_tc16_kernel, FWD16_SMEM) || !opt_in_smem(attn_fwd_2q_kernel, FWD2Q_SMEM))
-            return STREAMBP_E_CUDA;
-        configured = true;
-    }
+    static PerDevice configured;
+    if (!configured.get([] { return opt_in_smem(attn_fwd_tc16_kernel, FWD16_SMEM) && opt_in_smem(attn_fwd_2q_kernel, FWD2Q_SMEM) ? 1 : 0; }))
+        return STREAMBP_E_CUDA;
     FwdParams p{(int)n, (long long)q0, Hq, Hkv, o, lse, kLog2e / sqrtf((float)TILE)};
     // A key-tile step of a two-tile CTA takes ~1.5x that of a one-tile CTA: two tiles per CTA pay off unless they
     // leave SMs empty that one-tile CTAs would fill (short chunks, few heads).
@@ -1078,11 +1075,8 @@ int attention_bwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, const bf16 *do
         !make_tensor_map(&mk, k, kv_len, (int64_t)Hkv * TILE, (int64_t)Hkv * TILE, 64, TILE, false) ||
         !make_tensor_map(&mv, v, kv_len, (int64_t)Hkv * TILE, (int64_t)Hkv * TILE, 64, TILE, false))
         return STREAMBP_E_CUDA;
-    static bool configured = false;
-    if (!configured) {
-        if (!opt_in_smem(attn_bwd_tc_kernel, BWD_FUSED_SMEM)) return STREAMBP_E_CUDA;
-        configured = true;
-    }
+    static PerDevice configured;
+    if (!configured.get([] { return opt_in_smem(attn_bwd_tc_kernel, BWD_FUSED_SMEM) ? 1 : 0; })) return STREAMBP_E_CUDA;
     const float scale = 1.f / sqrtf((float)TILE);
     BwdParams p{(int)n, (long long)q0, Hq, Hkv, lse, delta, dq, dk, dv, scale, scale * kLog2e};
     const int kv_tiles = (int)((kv_len + TILE - 1) / TILE), q_tiles = (int)((n + TILE - 1) / TILE);

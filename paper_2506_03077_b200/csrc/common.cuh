@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "../../include/streambp.h"
 
 namespace sbp {
@@ -33,6 +35,31 @@ inline bool cuda_ok(cudaError_t e) {
     }
     return true;
 }
+
+// ---- per-device one-time state ------------------------------------------------------
+// The SM count, the opt-in to large dynamic shared memory (cudaFuncSetAttribute) and the choice of product kernel
+// are properties of a DEVICE, and one process may drive several: each is computed once per device ordinal (the
+// device current at the call), under a mutex, so host threads and devices never see each other's answer.
+constexpr int kMaxDevices = 64;
+int current_device_ordinal();             // cudaGetDevice, or the ordinal a test has put in its place; -1 on error
+class PerDevice {
+    std::mutex m_;
+    int value_[kMaxDevices];
+    bool have_[kMaxDevices] = {};
+public:
+    // the value for the current device; `init` runs once per device (again on every call where the ordinal
+    // cannot be read or is out of range: nothing is cached then)
+    template <typename F> int get(F init) {
+        const int dev = current_device_ordinal();
+        if (dev < 0 || dev >= kMaxDevices) return init();
+        std::lock_guard<std::mutex> lock(m_);
+        if (!have_[dev]) {
+            value_[dev] = init();
+            have_[dev] = true;
+        }
+        return value_[dev];
+    }
+};
 
 // Every kernel launch goes through this so launches are counted and launch errors
 // are caught without synchronising.
@@ -239,9 +266,9 @@ int gemm_tc_group(const GemmProb *probs, int n, int *sched, cudaStream_t st);
 int gemm_tc_take_fault();
 int gemm_tc_variant();   // 2: CTA-pair kernel, 1: single-CTA kernel, 0: tensor maps unavailable
 
-// Engine choice for the dispatching product below: 0 automatic, 1 CUDA cores only, 2 tensor cores required.
+// Engine choice for the dispatching product below: 0 automatic, 1 CUDA cores only, 2 tensor cores required
+// (STREAMBP_GEMM_ENGINE, read once per process).
 int gemm_engine();
-void set_gemm_engine(int e);
 
 // Dispatching product used by the schedulers.
 template <typename TI, typename TC>
@@ -313,6 +340,9 @@ int attention_bwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, const bf16 *do
 template <typename T>
 int attention_delta(const T *o, const T *dout, int64_t n, int Hq, int dh, float *delta, cudaStream_t st);
 int attention_tc_take_fault();
+// Test kernel whose bounded wait is made to run out (wait_probe.cu).
+int wait_probe_launch(unsigned long long limit_ns, cudaStream_t st);
+int wait_probe_take_fault();
 // Pointer alignment the attention backward entry points require (delta may be nullptr: not checked then).
 bool attention_bwd_aligned(const void *q, const void *k, const void *v, const void *o, const void *d_o,
                            const void *lse, const void *delta, const void *dq, const void *dk, const void *dv);
@@ -320,9 +350,10 @@ bool attention_bwd_aligned(const void *q, const void *k, const void *v, const vo
 template <typename T>
 int attn_fwd(const T *q, const T *k, const T *v, int64_t n, int64_t q0, int Hq, int Hkv, int dh, T *o, float *lse,
              cudaStream_t st);
+// engine: -1 = the process-wide choice (gemm_engine()), else 0 / 1 / 2 as above for this call only.
 template <typename T>
 int attn_bwd(const T *q, const T *k, const T *v, const T *o, const T *dout, const float *lse, int64_t n, int64_t q0,
-             int Hq, int Hkv, int dh, float *delta, float *dq, float *dk, float *dv, cudaStream_t st);
+             int Hq, int Hkv, int dh, float *delta, float *dq, float *dk, float *dv, cudaStream_t st, int engine = -1);
 
 // LM head pieces
 int count_valid_labels(const int64_t *labels, int64_t T, int64_t vocab, int64_t ignore, WsHeader *hdr,

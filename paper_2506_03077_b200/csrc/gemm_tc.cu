@@ -96,13 +96,13 @@ bool make_tensor_map(CUtensorMap *map, const void *base, int64_t rows, int64_t c
 }
 
 int sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
+    static PerDevice cache;
+    return cache.get([] {
+        int dev = 0, n = 0;
         if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
             n = 148;
-    }
-    return n;
+        return n;
+    });
 }
 
 
@@ -753,9 +753,9 @@ namespace {
 // The CTA-pair kernel needs clusters of two CTAs with the full shared-memory carve-out; where the device cannot
 // co-schedule even one such cluster the single-CTA kernel runs instead.
 bool pair_kernel_available() {
-    static int state = -1;
-    if (state < 0) {
-        state = 0;
+    static PerDevice cache;
+    return cache.get([] {
+        int state = 0;
         if (cudaFuncSetAttribute(gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PAIR_SMEM_BYTES) ==
             cudaSuccess) {
             cudaLaunchConfig_t cfg;
@@ -770,8 +770,8 @@ bool pair_kernel_available() {
         cudaGetLastError();
         if (getenv("STREAMBP_GEMM_SINGLE_CTA")) state = 0;
         if (getenv("STREAMBP_VERBOSE")) fprintf(stderr, "streambp: tcgen05 product kernel: %s\n", state ? "CTA pairs" : "single CTA");
-    }
-    return state == 1;
+        return state;
+    }) == 1;
 }
 }  // namespace
 
@@ -861,12 +861,11 @@ int gemm_tc_group(const GemmProb *probs, int n, int *sched, cudaStream_t st) {
     }
     p.sched = sched;
     p.gate = call_state().gate;
-    static bool configured = false;
-    if (!configured) {
-        if (!cuda_ok(cudaFuncSetAttribute(gemm_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES)))
-            return STREAMBP_E_CUDA;
-        configured = true;
-    }
+    static PerDevice configured;
+    if (!configured.get([] {
+            return cuda_ok(cudaFuncSetAttribute(gemm_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES)) ? 1 : 0;
+        }))
+        return STREAMBP_E_CUDA;
     if (pair) {
         const int pairs = std::max(1, sm_count() / 2);
         const int grid = 2 * (tiles < pairs ? (int)tiles : pairs);

@@ -11,15 +11,12 @@
 // The array's name is only a host-side handle; kernels need its device address, which is looked up
 // once per device with cudaGetSymbolAddress (with that device current) on the first call made on
 // that device.  Nothing here calls cudaMalloc, cudaFree or any allocating library routine.
-#include <mutex>
-
 #include "common.cuh"
 
 namespace sbp {
 namespace {
 
 constexpr int64_t kMaxDeltaFloats = STREAMBP_STATIC_DELTA_MAX_FLOATS;
-constexpr int kMaxDevices = 64;
 
 static __device__ __align__(256) float g_static_delta[kMaxDeltaFloats];
 

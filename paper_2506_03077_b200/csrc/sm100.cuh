@@ -50,15 +50,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait. Returns false if the CTA is aborting or the time limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+// Bounded wait. Returns false if the CTA is aborting or the time limit ran out.  The limit is a parameter so
+// that a test can make this very wait run out in a millisecond on a barrier nobody arrives at; every kernel of
+// the library passes the default.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          unsigned long long limit_ns = kWaitLimitNs) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_timer();
     for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 255u) == 0u) {
             if (*abort_flag) return false;
-            if (global_timer() - t0 > kWaitLimitNs) {
+            if (global_timer() - t0 > limit_ns) {
                 *abort_flag = 1;
                 atomicExch(&g_tc_fault, 1);
                 return false;
@@ -230,8 +233,9 @@ __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32
 // to 65-100 (busy arithmetic warps on the same scheduler) for a loop inside an `if (lane == 0)` branch.
 // The warp must be converged at every call: waits return a warp-uniform result (mbar_wait_warp).
 // (Polling from lane 0 only and broadcasting the result was measured slower: up to 2x in the dK/dV kernel.)
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
-    const bool ok = mbar_wait(bar, parity, abort_flag);
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                               unsigned long long limit_ns = kWaitLimitNs) {
+    const bool ok = mbar_wait(bar, parity, abort_flag, limit_ns);
     return __all_sync(0xffffffffu, ok);
 }
 __device__ __forceinline__ void umma_ss_w(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,

@@ -135,6 +135,17 @@ def test_attention_entry_points_refuse_misaligned_pointers(lib):
     assert bwd(False, delta=a + 2) == B.E_ALIGN
 
 
+def test_per_device_facts_are_keyed_by_device_ordinal(lib):
+    """SM count, shared-memory opt-in and product-kernel choice are cached per device: a second device must not get
+    the first one's answer.  The hook runs that cache with a stand-in ordinal."""
+    f = lib.streambp_test_per_device_value
+    assert f(0, 5) == 5 and f(0, 7) == 5          # first use on ordinal 0 decides; later calls see the cached value
+    assert f(1, 7) == 7 and f(1, 9) == 7          # ordinal 1 has its own entry
+    assert f(0, 11) == 5
+    assert f(63, 3) == 3 and f(64, 4) == 4 and f(64, 6) == 6      # beyond the table: computed every time, never cached
+    assert f(-1, 1) == B.E_SHAPE
+
+
 def test_suggested_chunk_is_the_largest_that_fits(lib):
     """Sec. 4.3: partition size is the memory / time knob.  The suggestion is the largest multiple of 128 (or T)
     whose exact workspace fits the budget, checked against a scan of the planner."""

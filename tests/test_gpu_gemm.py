@@ -234,3 +234,31 @@ print("fallback ok")
     out = subprocess.run([sys.executable, "-c", code], env=env, cwd=root, capture_output=True, text=True, timeout=300)
     assert out.returncode == 0, out.stderr[-2000:]
     assert "fallback ok" in out.stdout and "single CTA" in out.stderr
+
+
+def test_bounded_wait_runs_out_and_the_context_stays_usable():
+    """The tensor-core kernels wait on mbarriers with a time limit; when it runs out the CTA raises a flag, every
+    role leaves its loop, tensor memory is freed, the kernel returns and the host reads E_DEVICE_TIMEOUT.  The test
+    kernel runs that same wait on a barrier nothing arrives at, with a 1 ms limit: nothing hangs, the status is
+    reported once, and a product launched afterwards is correct."""
+    ws = B.alloc_workspace(4096)
+    ws.zero_()
+    assert B.last_device_status(ws) == B.OK
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    assert B.test_expire_wait(1_000_000) == B.OK
+    t1.record()
+    assert B.last_device_status(ws) == B.E_DEVICE_TIMEOUT
+    assert 0.9 < t0.elapsed_time(t1) < 50.0                  # gave up after the limit, not after the 2 s default
+    assert B.last_device_status(ws) == B.OK                  # reading the status clears the flag
+    assert B.lib().streambp_test_expire_wait(10, None) == B.E_SHAPE     # limits outside 1 us .. 100 ms are refused
+    M, N, K = 384, 512, 256
+    A = torch.randn(M, K, device="cuda").to(torch.bfloat16)
+    Bm = torch.randn(N, K, device="cuda").to(torch.bfloat16)
+    Cm = torch.empty(M, N, device="cuda")
+    B.gemm(B.OP_NT, A, Bm, Cm, engine=2)
+    torch.cuda.synchronize()
+    ref = A.double() @ Bm.double().T
+    assert float((Cm.double() - ref).norm() / ref.norm()) < 1e-5
+    assert B.last_device_status(ws) == B.OK
