@@ -35,10 +35,78 @@ def layer_flops(s, T):
     return fwd + bwd + att
 
 
-# DRAM bytes (read + write) of the dominant launch of a chunk -- the {dWd += dY^T m, dWg += dg^T h2, dWu += du^T h2,
-# dh2 = dg Wg + du Wu} group -- from the ncu capture summarised in profiles/gemm_pair_kernel_chunk_products.md
-# (qwen7b, chunk 1024: algorithmic bytes 2046e6).  Launch shapes depend on the chunk, not on T.
-NCU_TRAFFIC_BYTES = {("qwen7b_layer", 1024): 2142.5e6, ("llama8b_layer", 2048): 2421.9e6}
+def attn_bwd_bytes(s, kv_len, n):
+    """Algorithmic DRAM bytes of one attention-backward launch (n queries against kv_len keys): K, V read (storage
+    dtype), fp32 dK, dV read and written, Q, dO read, fp32 dQ written, lse / delta read."""
+    e = 2
+    return kv_len * s.dkv * (2 * e + 2 * 2 * 4) + n * s.dq * (2 * e + 4) + 2 * 4 * n * s.n_q_heads
+
+
+def attn_fwd_bytes(s, kv_len, n):
+    """K, V read, Q read, O written, lse written."""
+    e = 2
+    return kv_len * s.dkv * 2 * e + n * s.dq * 2 * e + 4 * n * s.n_q_heads
+
+
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of ONE captured launch per kernel class, from the ncu
+# captures summarised under profiles/ -- (config, chunk, class) -> (bytes, what was captured, algorithmic bytes of
+# that launch).  The step's average launch is this figure scaled by the ratio of algorithmic bytes (product launches
+# depend on the chunk only; attention launches grow with the key prefix, and their traffic in proportion).
+NCU_TRAFFIC = {
+    ("qwen7b_layer", 1024, "gemm"): (2142.5e6, "MLP-backward group of a chunk, profiles/gemm_pair_kernel_chunk_products.md", None),
+    ("llama8b_layer", 2048, "gemm"): (2421.9e6, "MLP-backward group of a chunk, profiles/gemm_pair_kernel_chunk_products.md", None),
+    ("llama8b_layer", 2048, "attention_bwd"): (483.8e6, "2048 queries against a 16384-key prefix, "
+                                               "profiles/attention_tc_kernels_llama8b_chunk2048.md", (16384, 2048)),
+    ("llama8b_layer", 2048, "attention_fwd"): (88.4e6, "2048 queries against a 16384-key prefix, "
+                                               "profiles/attention_tc_kernels_llama8b_chunk2048.md", (16384, 2048)),
+}
+
+
+def class_traffic(cfg, chunk, cls):
+    """(bytes per average launch or None, note).  Never silently None: the note says why a figure is absent."""
+    rec = NCU_TRAFFIC.get((cfg.name, chunk, cls))
+    if rec is None:
+        return None, f"no ncu capture of the {cls} class at ({cfg.name}, chunk {chunk}) under profiles/"
+    nbytes, what, at = rec
+    if at is None:
+        return nbytes, f"dram bytes under ncu of: {what}"
+    s, T = cfg.layer, cfg.T
+    fn = attn_bwd_bytes if cls == "attention_bwd" else attn_fwd_bytes
+    ends = [min(T, r0 + chunk) for r0 in range(0, T, chunk)]
+    avg = sum(fn(s, e, min(chunk, e)) for e in ends) / len(ends)
+    return nbytes * avg / fn(s, at[0], at[1]), (f"dram bytes under ncu of: {what}; scaled to the step's average launch "
+                                                 f"by algorithmic bytes ({avg / fn(s, at[0], at[1]):.3f}x)")
+
+
+CLASS_NAMES = {"gemm": "linear products (gemm_pair_kernel, all GEMM launches of the step)",
+               "attention_fwd": "partitioned attention forward (attn_fwd_2q_kernel / attn_fwd_tc16_kernel)",
+               "attention_bwd": "partitioned attention backward (attn_bwd_tc_kernel)"}
+
+
+def roofline_object(prof, steps, peaks, cfg, chunk, profiled_ms, flops_scale=1.0):
+    """The roofline entry is the kernel class that takes the largest share of the step that was actually run; the
+    other classes ride along with their own achieved rate and fraction.  All three are tensor-core bound (dense
+    contractions); the denominator is the measured sustained bf16 peak (kernels timed inside a long step)."""
+    peak = peaks["sustained"]
+    classes = {}
+    for k, (ms, calls, fl) in prof.items():
+        fl *= flops_scale
+        tf = fl / (ms * 1e-3) / 1e12 if ms > 0 else 0.0
+        classes[k] = {"ms_per_step": ms / steps, "launches_per_step": calls / steps, "tflops": tf, "frac": tf / peak,
+                      "frac_of_burst": tf / peaks["burst"], "frac_of_nominal_2250": tf / 2250.0}
+    dom = max(classes, key=lambda k: classes[k]["ms_per_step"])
+    traffic, note = class_traffic(cfg, chunk, dom) if cfg.layer is not None and not cfg.n_layers else \
+        (None, "no ncu capture of this workload's launches under profiles/ (captures are made on the layer workloads)")
+    return dom, classes, {
+        "bound": "tensor", "kernel": CLASS_NAMES[dom], "class": dom, "achieved": classes[dom]["tflops"], "peak": peak,
+        "unit": "TFLOP/s", "frac": classes[dom]["frac"], "peak_source": peaks["source"] + " sustained bf16",
+        "traffic": traffic, "traffic_note": note,
+        "launches": int(prof[dom][1]), "ms_per_step": classes[dom]["ms_per_step"],
+        "algorithmic_flops_per_launch": prof[dom][2] * flops_scale / max(1, prof[dom][1]),
+        "timed": "a second run of the same K steps with CUDA events around every launch of the class",
+        "step_ms_with_events": profiled_ms / steps,
+        "classes": {k: {"achieved": v["tflops"], "frac": v["frac"], "ms_per_step": v["ms_per_step"]} for k, v in classes.items()},
+    }
 
 
 def check_outputs(tensors) -> str:
@@ -155,7 +223,8 @@ def run_reference(args, cfg):
     total = sum(times)
     value = T_sample * args.steps / total
     cores = os.cpu_count()
-    sample = f"first {T_sample} tokens of {cfg.name} (full widths), fp64 numpy oracle, full-sequence backward"
+    sample = (f"first {T_sample} tokens of {cfg.name} (full widths), fp64 numpy oracle, full-sequence backward; a "
+              f"{T_sample}-token prefix under-counts the attention term, which is quadratic in T")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True, "scaling": "weak",
@@ -219,6 +288,9 @@ def run_head_or_model(args, cfg):
             step = lambda: B.lmhead_rl_backward(hc, obj, beta, eps, gd, Wd, Hd, ld, old, ref, adv, wt, cfg.chunk, loss,
                                                 dH, dW, dg, ws)
             name = f"streamed_lmhead_{args.objective}_backward_tokens_per_s"
+        H_host, l_host = torch.from_numpy(H).to(dt).pin_memory(), torch.from_numpy(labels).pin_memory()
+        dH_host, loss_host = torch.empty_like(H_host).pin_memory(), torch.zeros(1).pin_memory()
+        e2e_io = lambda: ([(Hd, H_host), (ld, l_host)], [(dH_host, dH), (loss_host, loss)])
         # chunks whose labels are all ignored are skipped on the device (their gradient is exactly zero)
         live_chunks = sum(1 for r0 in range(0, T, cfg.chunk) if (labels[r0:r0 + cfg.chunk] != h.ignore_index).any())
         executed_flops = head_flops(h, min(T, live_chunks * cfg.chunk))
@@ -239,6 +311,9 @@ def run_head_or_model(args, cfg):
         ws = B.alloc_workspace(ws_bytes)
         step = lambda: B.model_backward(lc, hc, layers, gf, Wv, ld, cfg.chunk, ch, loss, grads, dg, dWv, ws,
                                         embed=E, ids=idd, d_embed=dE)
+        id_host, l_host = torch.from_numpy(ids).pin_memory(), torch.from_numpy(labels).pin_memory()
+        loss_host = torch.zeros(1).pin_memory()
+        e2e_io = lambda: ([(idd, id_host), (ld, l_host)], [(loss_host, loss)])
         P = s.d_model * s.dq + 2 * s.d_model * s.dkv + s.dq * s.d_model + 3 * s.d_model * s.d_ff
         fwd_extra = 2 * T * P + 4 * s.head_dim * s.n_q_heads * T * (T + 1) / 2      # checkpointing forward
         flops = L * (layer_flops(s, T) + fwd_extra) + head_flops(h, T)
@@ -271,12 +346,11 @@ def run_head_or_model(args, cfg):
     B.profile_enable(False)
     profiled_ms = p0.elapsed_time(p1)
     ms = e0.elapsed_time(e1) / args.steps
-    gemm_ms, gemm_calls, gemm_flops = prof["gemm"]
     # launches of chunks that are skipped on the device return at once but are still bracketed: count only the
-    # executed share of their FLOPs
-    gemm_flops *= executed_flops / flops
-    achieved = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
-    print(json.dumps({
+    # executed share of their FLOPs (the head workload has product launches only)
+    _, classes, roofline = roofline_object(prof, args.steps, peaks, cfg, cfg.chunk, profiled_ms,
+                                           flops_scale=executed_flops / flops if cfg.n_layers == 0 else 1.0)
+    out = {
         "metric": name, "value": T / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic", "loss": loss.item(),
@@ -289,15 +363,59 @@ def run_head_or_model(args, cfg):
         "frac_of_measured_sustained_bf16_executed": executed_flops / (ms * 1e-3) / 1e12 / peaks["sustained"],
         "peak_activation_gb": ws_bytes / 1e9, "peak_activation_gb_unchunked": ws_full / 1e9,
         "gpu_launches": int(launches * args.steps), "outputs_checked": checked,
-        "roofline": {"bound": "tensor", "kernel": "linear products (executed FLOPs)", "achieved": achieved,
-                     "peak": peaks["sustained"],
-                     "unit": "TFLOP/s", "frac": achieved / peaks["sustained"], "traffic": None,
-                     "launches": int(gemm_calls), "ms_per_step": gemm_ms / args.steps,
-                     "timed": "a second run of the same K steps with CUDA events around every launch of the class",
-                     "step_ms_with_events": profiled_ms / args.steps},
-        "kernel_classes": {k: {"ms_per_step": v[0] / args.steps} for k, v in prof.items()},
-        "clocks": clocks,
-    }))
+        "roofline": roofline, "kernel_classes": classes, "clocks": clocks,
+    }
+    if not args.no_e2e:
+        # the same call fed from pinned host memory: every step copies its inputs in and its result out on the
+        # launching stream (serial: nothing overlaps), inside the timed region
+        h2d, d2h = e2e_io()
+        nb = lambda ts: sum(t.numel() * t.element_size() for _, t in ts)
+        def e2e_step():
+            for dev, host in h2d:
+                dev.copy_(host, non_blocking=True)
+            step()
+            for host, dev in d2h:
+                host.copy_(dev, non_blocking=True)
+        e2e_step()
+        torch.cuda.synchronize()
+        q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        q0.record()
+        for _ in range(args.steps):
+            e2e_step()
+        q1.record()
+        torch.cuda.synchronize()
+        out["e2e"] = {"value": T / (q0.elapsed_time(q1) / args.steps * 1e-3), "unit": UNIT,
+                      "h2d_bytes_per_step": nb(h2d), "d2h_bytes_per_step": nb(d2h),
+                      "mode": "serial: copies and kernels of a step on one stream, nothing overlapped"}
+    if not args.no_cpu_baseline:
+        out["cpu_baseline"] = head_model_cpu_baseline(cfg, args)
+    print(json.dumps(out))
+
+
+def head_model_cpu_baseline(cfg, args):
+    """The oracle, as it stands, on a bounded sample: rows of the head workload at the full widths; for the model
+    workload the per-token cost of one full-width layer (a token prefix) and of the head (rows), combined as
+    n_layers * layer + head.  A reported baseline, not the target."""
+    from oracle import streambp_oracle as O
+    from paper_2506_03077_b200 import synth
+    h = cfg.head
+    rows = min(cfg.T, args.cpu_baseline_head_rows)
+    g, Wv, H, labels = synth.make_head_inputs(h, cfg.seed, rows, True, rows // 4)
+    t0 = time.perf_counter()
+    O.lmhead_ce_backward(O.HeadCfg(h.d_model, h.vocab, h.rms_eps, h.ignore_index), g, Wv, H, labels)
+    head_s = (time.perf_counter() - t0) / rows
+    if cfg.n_layers == 0:
+        return {"value": 1.0 / head_s, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+                "sample": f"{rows} rows of {cfg.name} (d {h.d_model}, vocab {h.vocab}), fp64 numpy oracle, "
+                          f"{head_s * rows:.1f} s"}
+    Ts = min(args.cpu_baseline_tokens, cfg.T)
+    layer_s = oracle_sample(cfg, Ts) / Ts
+    per_token = cfg.n_layers * layer_s + head_s
+    return {"value": 1.0 / per_token, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+            "sample": f"per-token cost of one full-width layer backward on the first {Ts} tokens "
+                      f"({layer_s * Ts:.1f} s) x {cfg.n_layers} layers + of the head on {rows} rows ({head_s * rows:.1f} s); "
+                      f"the layers' forward pass is not counted and a {Ts}-token prefix under-counts the quadratic "
+                      f"attention term, both in the oracle's favour"}
 
 
 def main():
@@ -306,7 +424,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="qwen7b_layer",
+    ap.add_argument("--config", default="llama8b_layer",
                     choices=["qwen7b_layer", "llama8b_layer", "qwen7b_head", "qwen7b_model"])
     ap.add_argument("--layers", type=int, default=0, help="override the layer count of the model configuration")
     ap.add_argument("--objective", default="sft", choices=["sft", "grpo", "dpo"],
@@ -315,6 +433,7 @@ def main():
     ap.add_argument("--T", type=int, default=0, help="override the sequence length (profiling on small cases)")
     ap.add_argument("--ref-tokens", type=int, default=512)
     ap.add_argument("--cpu-baseline-tokens", type=int, default=1024)
+    ap.add_argument("--cpu-baseline-head-rows", type=int, default=256)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--dp", action="store_true",
@@ -444,12 +563,7 @@ def main():
     value = aggregate_tokens_per_s(T, world, ms_per_step)
     peaks = read_peaks()
     flops = layer_flops(s, T)
-    gemm_ms, gemm_calls, gemm_flops = prof["gemm"]
-    af_ms, af_calls, af_flops = prof["attention_fwd"]
-    ab_ms, ab_calls, ab_flops = prof["attention_bwd"]
-    achieved = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
-    # the bracketed kernels run inside a long step: compare with the sustained measured peak
-    peak = peaks["sustained"]
+    _, classes, roofline = roofline_object(prof, args.steps, peaks, cfg, chunk, profiled_ms)
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -467,33 +581,24 @@ def main():
         "frac_of_nominal_bf16": flops / (ms_per_step * 1e-3) / 1e12 / 2250.0,
         "peak_activation_gb": ws_bytes / 1e9, "peak_activation_gb_unchunked": ws_full / 1e9,
         "gpu_launches": int(launches_per_step * args.steps), "outputs_checked": checked,
-        "roofline": {"bound": "tensor", "kernel": "linear products (all GEMM launches of the step)",
-                     "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-                     "peak_source": peaks["source"] + " sustained bf16",
-                     "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, chunk)),
-                     "traffic_note": "dram bytes of the dominant product launch of a chunk under ncu (see profiles/)",
-                     "launches": int(gemm_calls), "ms_per_step": gemm_ms / args.steps,
-                     "timed": "a second run of the same K steps with CUDA events around every launch of the class",
-                     "step_ms_with_events": profiled_ms / args.steps},
-        "kernel_classes": {
-            "gemm": {"ms_per_step": gemm_ms / args.steps, "tflops": achieved},
-            "attention_fwd": {"ms_per_step": af_ms / args.steps,
-                              "tflops": af_flops / (af_ms * 1e-3) / 1e12 if af_ms > 0 else 0.0},
-            "attention_bwd": {"ms_per_step": ab_ms / args.steps,
-                              "tflops": ab_flops / (ab_ms * 1e-3) / 1e12 if ab_ms > 0 else 0.0},
-        },
+        "roofline": roofline,
+        "kernel_classes": classes,
         "clocks": clocks,
     }
     if e2e_ms is not None:
         nbytes = X_host.numel() * X_host.element_size()
         out["e2e"] = {"value": aggregate_tokens_per_s(T, world, e2e_ms / args.steps), "unit": UNIT,
-                      "h2d_bytes_per_step": 2 * nbytes, "d2h_bytes_per_step": nbytes}
+                      "h2d_bytes_per_step": 2 * nbytes, "d2h_bytes_per_step": nbytes,
+                      "mode": "pipelined: two buffer sets, a step's copies overlap the neighbouring steps' kernels "
+                              "(throughput, not the latency of one isolated step)"}
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         Ts = min(args.cpu_baseline_tokens, T)
         sec = oracle_sample(cfg, Ts)
         out["cpu_baseline"] = {"value": Ts / sec, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
                                "sample": f"first {Ts} tokens of {cfg.name} (full widths), fp64 numpy oracle, "
-                                         f"full-sequence backward, {sec:.1f} s"}
+                                         f"full-sequence backward, {sec:.1f} s; a {Ts}-token prefix under-counts the "
+                                         f"attention term, which is quadratic in T: at T = {T} the oracle's "
+                                         f"tokens/s would be lower"}
     if rank == 0:
         print(json.dumps(out))
     if world > 1:

@@ -209,6 +209,6 @@ def test_attention_growing_maxima_tensor_core():
     assert errs[2][0] < DQ_GROWING_MAXIMA_TOL, errs
 
 
-# dQ against the oracle in the ill-conditioned case above, as measured for both engines on the same bf16 O
-# (the bound is the conditioning of the case, see the comment in the test, not a property of either engine)
-DQ_GROWING_MAXIMA_TOL = 0.25
+# dQ against the oracle in the ill-conditioned case above: measured 5.7e-2 (CUDA-core engine) and 7.0e-2 (tensor-core
+# engine) on the same bf16 O -- the conditioning of the case (see the comment in the test), not a property of an engine
+DQ_GROWING_MAXIMA_TOL = 0.1

@@ -96,17 +96,13 @@ def test_dpo_matches_oracle(dtype):
     ref_out = O.lmhead_dpo_backward(cfg, g, W, H, tok, ref, sign, beta)
     for ch in (chunk, T, 50):
         loss, ell, logp, dH, dW, dg = run_rl(hs, B.OBJ_DPO, beta, 0.0, g, W, H, tok, None, ref, None, sign, ch, dtype)
-        assert abs(ell - ref_out[1]) <= (1e-4 if dtype == torch.float32 else 0.3)
-        assert abs(loss - ref_out[0]) <= (1e-5 if dtype == torch.float32 else 5e-2)
-        # the correction factor sigmoid(beta ell) - 1 inherits ell's error in bf16; compare directions and scale
-        assert_close("dH", dH, ref_out[2], TOL[dtype] if dtype == torch.float32 else 6e-2)
-        assert_close("dW", dW, ref_out[3], TOL[dtype] if dtype == torch.float32 else 6e-2)
-        assert_close("dg", dg, ref_out[4], TOL[dtype] if dtype == torch.float32 else 6e-2)
-        if dtype == torch.bfloat16:
-            # with the oracle's own factor the gradients agree to the usual tolerance
-            f_gpu = 1.0 / (1.0 + np.exp(-beta * ell)) - 1.0
-            f_ref = 1.0 / (1.0 + np.exp(-beta * ref_out[1])) - 1.0
-            assert_close("dW rescaled", dW * (f_ref / f_gpu), ref_out[3], TOL[dtype])
+        # bf16: ell sums 152 log-probabilities whose errors (up to 6e-3 each, from the bf16 operands of the logits
+        # product) add up to 0.04; the correction factor sigmoid(beta ell) - 1 moves by beta * 0.04 / 2 < 1e-2
+        assert abs(ell - ref_out[1]) <= (1e-4 if dtype == torch.float32 else 0.1)
+        assert abs(loss - ref_out[0]) <= (1e-5 if dtype == torch.float32 else 1.5e-2)
+        assert_close("dH", dH, ref_out[2], TOL[dtype])
+        assert_close("dW", dW, ref_out[3], TOL[dtype])
+        assert_close("dg", dg, ref_out[4], TOL[dtype])
         assert torch.count_nonzero(dH[64:128]) == 0
 
 
