@@ -523,22 +523,29 @@ __global__ void __launch_bounds__(FWD2Q_THREADS, 1)
 //   dK/dV: one CTA per (128-key tile, KV head); K and V tiles stay in shared memory; loops over the
 //          G query heads of the group and over the query tiles that can see the key tile.
 //          S^T = K Q^T and dP^T = V dO^T land in tensor memory with keys on the lanes, so a thread owns
-//          one key row; P^T and dS^T are packed to bf16 in place and feed dV += P^T dO and dK += dS^T Q
-//          as tensor-memory A operands.  The Q / dO tiles serve both as K-major B operands (first two
-//          products) and as MN-major B operands (last two) without being moved.
+//          one key row.  The softmax warps read S^T and dP^T into registers and write BOTH packed bf16
+//          operands -- P^T and dS^T -- over the columns of dP^T (first / second 16 columns of each 32-column
+//          group), from where they feed dV += P^T dO and dK += dS^T Q as tensor-memory A operands.  The
+//          columns of S^T are therefore free as soon as they have been read, and S^T of the next iteration is
+//          queued at once, a whole iteration ahead (the Q ring has three stages for that: Q_i is read by
+//          S^T_i and again, an iteration later, by dK_i); dP^T of the next iteration follows dK in the same
+//          thread's issue order.  The Q / dO tiles serve both as K-major B operands (first two products) and
+//          as MN-major B operands (last two) without being moved.
 //   dQ   : one CTA per (128-query tile, query head); Q and dO tiles stay resident, K / V tiles stream;
 //          S = Q K^T, dP = dO V^T, dS packed in place, dQ += dS K.
 // Work inside a tile pair is split in TIME, not in space, so every product is a full 128 x 128 x 128 one
 // (an N = 64 product is limited by shared-memory bandwidth to 2/3 of the tensor rate): the softmax
 // warps (16 per CTA, each thread owns 32 columns of one row) first turn S into P -- which is all the dV
-// product needs -- and only then combine it with dP into dS.  The MMA thread interleaves accordingly:
-// dV_i, then S_{i+1} (its buffer is free again), then dK_i, then dP_{i+1}; the tensor pipe therefore
-// always has the next tile's products queued while the softmax warps work.
-// Timelines taken with clock64 stamps inside the kernels showed what bounds them: not the exponential unit
-// (replacing half of the exp2 by a polynomial on the FMA pipe made both kernels slower) but (a) the latency
-// of refilling a shared-memory stage that is released late -- hence the three-stage K ring of the dQ kernel
-// and the separate release of Q and dO stages in the dK/dV kernel -- and (b) the rate at which one thread
-// can issue tcgen05.mma while arithmetic warps share its scheduler -- hence the warp-uniform issue loops.
+// product needs -- and only then combine it with dP into dS.
+// Tensor memory is full in both roles (four 128-column fp32 tiles), which leaves one dependency cycle per
+// iteration that cannot be cut: packed operands -> dK -> next dP^T -> softmax.  Timelines (clock64 stamps in
+// the kernel) put an iteration of the dK/dV role at ~3000 cycles for 2048 cycles of products.  More overlap
+// does not buy time on this part, though: run back to back for seconds, every variant of this kernel that was
+// built -- a second issuing warp, Q / dO of the dQ role as tensor-memory operands, the older S^T-in-place
+// scheme -- draws the board's full power limit and the clock settles so that the time per call is the same
+// within 1-2 % (fewer cycles per tile, lower clock).  At the limit the kernel is bound by energy per tile
+// pair, of which the seven products (five algorithmic + S and dP recomputed by the dQ role, the price of a
+// deterministic result) are the bulk.
 // ---------------------------------------------------------------------------------------------
 struct BwdParams {
     int n;
@@ -551,7 +558,10 @@ struct BwdParams {
     float scale, scale_log2;
 };
 
-constexpr int BWD_SMEM = 6 * TILE_BYTES + 4 * TILE * 4 /* lse, delta x 2 stages */ + 1024 + 256;
+constexpr int KV_QSTAGES = 3;
+constexpr int BWD_ALIGN_SLACK = 768;    // what the 227 KB carve-out leaves for aligning the tiles to 1024 bytes
+constexpr int BWD_SMEM = (4 + KV_QSTAGES) * TILE_BYTES + 4 * TILE * 4 /* lse, delta x 2 stages */ + 256 + BWD_ALIGN_SLACK;
+static_assert(BWD_SMEM <= 232448, "dK/dV role exceeds the shared memory of an SM");
 constexpr int DQ_KSTAGES = 3;
 constexpr int DQ_SMEM = (4 + DQ_KSTAGES) * TILE_BYTES + 1024 + 256;   // Q, dO, K x 3, V x 2
 constexpr int BWD_THREADS = 64 + 512;
@@ -569,16 +579,17 @@ __device__ __forceinline__ void attn_bwd_dkdv_body(const CUtensorMap &map_q, con
                                                    const BwdParams &p, uint8_t *smem_raw, int block_x, int block_y) {
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
-    const uint32_t sK = base, sV = sK + TILE_BYTES, sQ = sV + TILE_BYTES, sdO = sQ + 2 * TILE_BYTES;
-    uint8_t *tail = smem_raw + (base - raw) + 6 * TILE_BYTES;
+    const uint32_t sK = base, sV = sK + TILE_BYTES, sQ = sV + TILE_BYTES, sdO = sQ + KV_QSTAGES * TILE_BYTES;
+    uint8_t *tail = smem_raw + (base - raw) + (4 + KV_QSTAGES) * TILE_BYTES;
     float *s_lse = reinterpret_cast<float *>(tail);           // [2][128], pre-multiplied by log2(e)
-    float *s_delta = s_lse + 2 * TILE;                        // [2][128]
+    float *s_delta = s_lse + 2 * TILE;                        // [2][128], pre-multiplied by the score scale
     uint8_t *aux = tail + 4 * TILE * 4;
     const uint32_t bars = smem_u32(aux);
-    const uint32_t kv_full = bars, in_full = bars + 8, q_empty = bars + 24, s_full = bars + 40, dp_full = bars + 48,
-                   p1_full = bars + 56, p2_full = bars + 64, acc_full = bars + 72, do_empty = bars + 80;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux + 96);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(aux + 104);
+    const uint32_t kv_full = bars, q_full = bars + 8, q_empty = bars + 32, do_full = bars + 56, do_empty = bars + 72,
+                   rows_empty = bars + 88, s_full = bars + 104, dp_full = bars + 112, loaded = bars + 120,
+                   p1_full = bars + 128, p2_full = bars + 136, acc_full = bars + 144;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux + 152);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(aux + 160);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = block_y, G = p.Hq / p.Hkv;
@@ -590,17 +601,24 @@ __device__ __forceinline__ void attn_bwd_dkdv_body(const CUtensorMap &map_q, con
 
     if (threadIdx.x == 0) {
         mbar_init(kv_full, 1);
-        for (int s = 0; s < 2; s++) {
-            mbar_init(in_full + 8 * s, 1);
+        for (int s = 0; s < KV_QSTAGES; s++) {
+            mbar_init(q_full + 8 * s, 1);
             mbar_init(q_empty + 8 * s, 1);
+        }
+        for (int s = 0; s < 2; s++) {
+            mbar_init(do_full + 8 * s, 1);
             mbar_init(do_empty + 8 * s, 1);
+            mbar_init(rows_empty + 8 * s, 1);
         }
         mbar_init(s_full, 1);
         mbar_init(dp_full, 1);
+        mbar_init(loaded, 16);
         mbar_init(p1_full, 16);
         mbar_init(p2_full, 16);
         mbar_init(acc_full, 1);
-        *abort_flag = 0;
+        // the carve-out leaves at most 768 bytes for aligning the tiles to 1024: a base that needs more cannot be used
+        *abort_flag = (base - raw) > BWD_ALIGN_SLACK ? 1 : 0;
+        if (*abort_flag) atomicExch(&g_tc_fault, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 512);
@@ -608,11 +626,16 @@ __device__ __forceinline__ void attn_bwd_dkdv_body(const CUtensorMap &map_q, con
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    // columns: S^T at 0, dP^T at 128, dV at 256, dK at 384
+    // columns: S^T at 0; dP^T at 128, later P^T (packed) in the first and dS^T (packed) in the second 16 columns of
+    // every 32-column group; dV at 256, dK at 384
     const uint32_t tST = tmem, tDPT = tmem + 128, tDV = tmem + 256, tDK = tmem + 384;
+    const bool usable = *abort_flag == 0;
 
-    if (warp == 0) {
-        // ---- producer: K, V once; then per iteration lse / delta (plain loads) and the Q, dO tiles (TMA)
+    if (!usable) {
+        // nothing was issued: fall through to the common exit
+    } else if (warp == 0) {
+        // ---- producer: K, V once; per iteration the dO tile with the lse / delta rows (two stages) and the Q tile
+        // (three stages: Q_i is read by S^T_i, which is issued a whole iteration ahead, and again by dK_i at the end)
         if (lane == 0) {
             mbar_expect_tx(kv_full, 2 * TILE_BYTES);
             tma_load_2d(sK, &map_k, kv_full, g * TILE, (int)k_abs0);
@@ -620,24 +643,24 @@ __device__ __forceinline__ void attn_bwd_dkdv_body(const CUtensorMap &map_q, con
             tma_load_2d(sV, &map_v, kv_full, g * TILE, (int)k_abs0);
             tma_load_2d(sV + HALF_BYTES, &map_v, kv_full, g * TILE + 64, (int)k_abs0);
         }
-        // A stage's dO tile is free once dV of its previous user is done, its Q tile (and the lse / delta rows)
-        // once dK is done; the copies are issued before the row loads so that their latencies overlap.
+        uint32_t sq = 0, qph = 0;
         for (int it = 0; it < iters; it++) {
             const int h = g * G + it / per_head, qt0 = (first_qt + it % per_head) * TILE;
-            const uint32_t st = it & 1, ph = (it >> 1) & 1;
-            const uint32_t full = in_full + 8 * st;
+            const uint32_t sd = it & 1, dph = (it >> 1) & 1;
             int ok = 1;
             if (lane == 0) {
-                ok = mbar_wait(do_empty + 8 * st, ph ^ 1u, abort_flag) ? 1 : 0;
+                ok = mbar_wait(q_empty + 8 * sq, qph ^ 1u, abort_flag) ? 1 : 0;          // dK of the stage's last user
                 if (ok) {
-                    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(full), "r"(2 * TILE_BYTES) : "memory");
-                    tma_load_2d(sdO + st * TILE_BYTES, &map_do, full, h * TILE, qt0);
-                    tma_load_2d(sdO + st * TILE_BYTES + HALF_BYTES, &map_do, full, h * TILE + 64, qt0);
-                    ok = mbar_wait(q_empty + 8 * st, ph ^ 1u, abort_flag) ? 1 : 0;
+                    mbar_expect_tx(q_full + 8 * sq, TILE_BYTES);
+                    tma_load_2d(sQ + sq * TILE_BYTES, &map_q, q_full + 8 * sq, h * TILE, qt0);
+                    tma_load_2d(sQ + sq * TILE_BYTES + HALF_BYTES, &map_q, q_full + 8 * sq, h * TILE + 64, qt0);
+                    ok = mbar_wait(do_empty + 8 * sd, dph ^ 1u, abort_flag) ? 1 : 0;     // dV of the stage's last user
                 }
                 if (ok) {
-                    tma_load_2d(sQ + st * TILE_BYTES, &map_q, full, h * TILE, qt0);
-                    tma_load_2d(sQ + st * TILE_BYTES + HALF_BYTES, &map_q, full, h * TILE + 64, qt0);
+                    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(do_full + 8 * sd), "r"(TILE_BYTES) : "memory");
+                    tma_load_2d(sdO + sd * TILE_BYTES, &map_do, do_full + 8 * sd, h * TILE, qt0);
+                    tma_load_2d(sdO + sd * TILE_BYTES + HALF_BYTES, &map_do, do_full + 8 * sd, h * TILE + 64, qt0);
+                    ok = mbar_wait(rows_empty + 8 * sd, dph ^ 1u, abort_flag) ? 1 : 0;   // delta rows: read until dS^T is packed
                 }
             }
             ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -645,115 +668,134 @@ __device__ __forceinline__ void attn_bwd_dkdv_body(const CUtensorMap &map_q, con
 #pragma unroll
             for (int e = 0; e < 4; e++) {
                 const int col = lane * 4 + e, r = qt0 + col;
-                s_lse[st * TILE + col] = r < p.n ? p.lse[(long long)h * p.n + r] * kLog2e : 0.f;
-                s_delta[st * TILE + col] = r < p.n ? p.delta[(long long)h * p.n + r] * p.scale : 0.f;
+                s_lse[sd * TILE + col] = r < p.n ? p.lse[(long long)h * p.n + r] * kLog2e : 0.f;
+                s_delta[sd * TILE + col] = r < p.n ? p.delta[(long long)h * p.n + r] * p.scale : 0.f;
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(full);      // publishes the rows; the phase completes when the tiles have landed too
+            if (lane == 0) mbar_arrive(do_full + 8 * sd);   // publishes the rows; the phase completes when dO has landed too
+            if (++sq == KV_QSTAGES) { sq = 0; qph ^= 1u; }
         }
-    } else if (warp == 1) {
+    }
+    else if (warp == 1) {
         // the whole warp runs the issue loop; each MMA / commit executes in one elected lane
         constexpr uint32_t idesc_kk = make_idesc(TILE, TILE, false, false);     // both operands K-major
         constexpr uint32_t idesc_acc = make_idesc(TILE, TILE, false, true);     // B MN-major (N = head dims)
         bool alive = mbar_wait_warp(kv_full, 0, abort_flag);
         const uint32_t k_lo = klo(sK), v_lo = klo(sV);
-        auto issue_st = [&](int it) {      // S^T = K Q^T
-            const uint32_t q_lo = klo(sQ + (it & 1) * TILE_BYTES);
+        uint32_t sq_s = 0, qph_s = 0;      // Q stage / phase of the next S^T
+        uint32_t sq_k = 0;                 // Q stage of the next dK
+        auto issue_st = [&]() -> bool {    // S^T = K Q^T for the next iteration
+            if (!mbar_wait_warp(q_full + 8 * sq_s, qph_s, abort_flag)) return false;
+            tc_fence_after();
+            const uint32_t q_lo = klo(sQ + sq_s * TILE_BYTES);
 #pragma unroll
             for (int kk = 0; kk < 8; kk++) umma_ss_w(tST, k_lo + kstep(kk), q_lo + kstep(kk), idesc_kk, kk != 0);
             umma_commit_w(s_full);
+            if (++sq_s == KV_QSTAGES) { sq_s = 0; qph_s ^= 1u; }
+            return true;
         };
-        auto issue_dpt = [&](int it) {     // dP^T = V dO^T
+        auto issue_dpt = [&](int it) -> bool {     // dP^T = V dO^T of iteration `it`
+            if (!mbar_wait_warp(do_full + 8 * (it & 1), (it >> 1) & 1, abort_flag)) return false;
+            tc_fence_after();
             const uint32_t do_lo = klo(sdO + (it & 1) * TILE_BYTES);
 #pragma unroll
             for (int kk = 0; kk < 8; kk++) umma_ss_w(tDPT, v_lo + kstep(kk), do_lo + kstep(kk), idesc_kk, kk != 0);
             umma_commit_w(dp_full);
+            return true;
         };
-        if (alive) alive = mbar_wait_warp(in_full, 0, abort_flag);
-        if (alive) {
-            tc_fence_after();
-            issue_st(0);
-            issue_dpt(0);
-        }
+        if (alive && iters > 0) alive = issue_st() && issue_dpt(0);
         for (int it = 0; it < iters && alive; it++) {
-            const uint32_t st = it & 1;
-            const uint32_t q_mn = mnlo(sQ + st * TILE_BYTES), do_mn = mnlo(sdO + st * TILE_BYTES);
-            // dV += P^T dO as soon as P^T is packed
+            const uint32_t sd = it & 1;
+            // the softmax warps hold S^T_it in registers: its columns take S^T of the next iteration at once
+            if (it + 1 < iters) {
+                if (!mbar_wait_warp(loaded, it & 1, abort_flag)) { alive = false; break; }
+                tc_fence_after();
+                if (!issue_st()) { alive = false; break; }
+            }
+            // dV += P^T dO as soon as P^T is packed (first 16 columns of each group of the dP^T region)
             if (!mbar_wait_warp(p1_full, it & 1, abort_flag)) { alive = false; break; }
             tc_fence_after();
+            const uint32_t do_mn = mnlo(sdO + sd * TILE_BYTES);
 #pragma unroll
             for (int kk = 0; kk < 8; kk++)
-                umma_ts_w(tDV, tST + (kk >> 1) * 32 + (kk & 1) * 8, do_mn + mnstep(kk), idesc_acc, (it | kk) != 0);
-            umma_commit_w(do_empty + 8 * st);            // dO of this stage is consumed (dP^T was issued earlier)
-            // the S^T columns are free again once dV has read them (in order): next tile's S^T
-            if (it + 1 < iters) {
-                if (!mbar_wait_warp(in_full + 8 * ((it + 1) & 1), ((it + 1) >> 1) & 1, abort_flag)) { alive = false; break; }
-                tc_fence_after();
-                issue_st(it + 1);
-            }
-            // dK += dS^T Q
+                umma_ts_w(tDV, tDPT + (kk >> 1) * 32 + (kk & 1) * 8, do_mn + mnstep(kk), idesc_acc, (it | kk) != 0);
+            umma_commit_w(do_empty + 8 * sd);            // dO of this stage is consumed (dP^T was issued earlier)
+            // dK += dS^T Q (second 16 columns of each group)
             if (!mbar_wait_warp(p2_full, it & 1, abort_flag)) { alive = false; break; }
             tc_fence_after();
+            const uint32_t q_mn = mnlo(sQ + sq_k * TILE_BYTES);
 #pragma unroll
             for (int kk = 0; kk < 8; kk++)
-                umma_ts_w(tDK, tDPT + (kk >> 1) * 32 + (kk & 1) * 8, q_mn + mnstep(kk), idesc_acc, (it | kk) != 0);
-            umma_commit_w(q_empty + 8 * st);             // Q of this stage is consumed
-            if (it + 1 < iters) issue_dpt(it + 1);
+                umma_ts_w(tDK, tDPT + (kk >> 1) * 32 + 16 + (kk & 1) * 8, q_mn + mnstep(kk), idesc_acc, (it | kk) != 0);
+            umma_commit_w(q_empty + 8 * sq_k);           // Q of this stage is consumed
+            umma_commit_w(rows_empty + 8 * sd);          // and so are the lse / delta rows
+            if (++sq_k == KV_QSTAGES) sq_k = 0;
+            // the dP^T region is free once dV and dK have read it (in order): next iteration's dP^T
+            if (it + 1 < iters && !issue_dpt(it + 1)) { alive = false; break; }
         }
         if (alive) umma_commit_w(acc_full);
-    } else {
+    }
+    else {
         const int quarter = warp & 3;
         const int wg = (warp - 2) >> 2;                           // 0..3: 32-query group of the tile
         const int col_base = wg * 32;
         const int row = quarter * 32 + lane;                      // key row within the tile
         const long long k_abs = k_abs0 + row;
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-        // packed bf16 pairs overwrite the front of the group's OWN fp32 columns (already consumed);
-        // the MMA thread addresses each 16-query slice of the A operand separately
+        // The group reads its 32 fp32 columns of S^T and of dP^T into registers, then writes the packed bf16 pairs
+        // of P^T over the first and of dS^T over the second 16 of ITS OWN dP^T columns; the MMA thread addresses
+        // each 16-query slice of those A operands separately.  S^T's columns are never written by these warps, so
+        // the product of the next iteration can refill them while this iteration's exponentials are computed.
         const uint32_t tS_g = tST + col_base + lane_base, tP_g = tDPT + col_base + lane_base;
         bool alive = true;
         for (int it = 0; it < iters && alive; it++) {
             const int qt0 = (first_qt + it % per_head) * TILE;
-            const uint32_t st = it & 1;
-            // the producer's lse / delta rows of this stage are published together with the tiles
-            if (!mbar_wait(in_full + 8 * st, (it >> 1) & 1, abort_flag)) { alive = false; break; }
+            const uint32_t sd = it & 1;
             if (!mbar_wait(s_full, it & 1, abort_flag)) { alive = false; break; }
             tc_fence_after();
+            uint32_t rs[32];
+            tmem_ld32(tS_g, rs);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(loaded);
+            // the producer's lse / delta rows of this stage are published together with the dO tile
+            if (!mbar_wait(do_full + 8 * sd, (it >> 1) & 1, abort_flag)) { alive = false; break; }
             const long long q_abs0 = p.q0 + qt0;
             const bool diag = k_abs0 + TILE - 1 > q_abs0;          // the tile pair holds masked (query, key) pairs
             // query column c of the tile is visible to this key iff q_abs0 + c >= k_abs
             const int first_col = (k_abs > q_abs0) ? (int)((k_abs - q_abs0) > TILE ? TILE : (k_abs - q_abs0)) : 0;
-            const float *lse2 = s_lse + st * TILE + col_base, *dl = s_delta + st * TILE + col_base;
+            const float *lse2 = s_lse + sd * TILE + col_base, *dl = s_delta + sd * TILE + col_base;
             // phase 1: P^T = exp2(S^T * scale - lse), all the dV product needs
             float pv[32];
-            {
-                uint32_t rs[32], pp[16];
-                tmem_ld32(tS_g, rs);
 #pragma unroll
-                for (int e = 0; e < 32; e += 4) {
-                    const float4 l4 = *reinterpret_cast<const float4 *>(lse2 + e);
-                    const float lv[4] = {l4.x, l4.y, l4.z, l4.w};
+            for (int e = 0; e < 32; e += 4) {
+                const float4 l4 = *reinterpret_cast<const float4 *>(lse2 + e);
+                const float lv[4] = {l4.x, l4.y, l4.z, l4.w};
 #pragma unroll
-                    for (int t = 0; t < 4; t++) {
-                        float x = fmaf(__uint_as_float(rs[e + t]), p.scale_log2, -lv[t]);
-                        if (diag && col_base + e + t < first_col) x = -INFINITY;
-                        pv[e + t] = fast_exp2(x);
-                    }
-                    pp[e / 2] = pack_bf16(pv[e], pv[e + 1]);
-                    pp[e / 2 + 1] = pack_bf16(pv[e + 2], pv[e + 3]);
+                for (int t = 0; t < 4; t++) {
+                    float x = fmaf(__uint_as_float(rs[e + t]), p.scale_log2, -lv[t]);
+                    if (diag && col_base + e + t < first_col) x = -INFINITY;
+                    pv[e + t] = fast_exp2(x);
                 }
-                tmem_st16(tS_g, pp);
+            }
+            // dP^T of this iteration was queued a whole iteration ago; its columns become P^T and dS^T
+            uint32_t pp[16];
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) pp[e / 2] = pack_bf16(pv[e], pv[e + 1]);
+            if (!mbar_wait(dp_full, it & 1, abort_flag)) { alive = false; break; }
+            tc_fence_after();
+            uint32_t rp[32];
+            tmem_ld32(tP_g, rp);
+            {
+                tmem_st16(tP_g, pp);
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(p1_full);
             }
             // phase 2: dS^T = P^T * (dP^T * scale - delta * scale)
-            if (!mbar_wait(dp_full, it & 1, abort_flag)) { alive = false; break; }
-            tc_fence_after();
             {
-                uint32_t rp[32], ds[16];
-                tmem_ld32(tP_g, rp);
+                uint32_t ds[16];
 #pragma unroll
                 for (int e = 0; e < 32; e += 4) {
                     const float4 d4 = *reinterpret_cast<const float4 *>(dl + e);
@@ -764,7 +806,7 @@ __device__ __forceinline__ void attn_bwd_dkdv_body(const CUtensorMap &map_q, con
                     ds[e / 2] = pack_bf16(dsv[0], dsv[1]);
                     ds[e / 2 + 1] = pack_bf16(dsv[2], dsv[3]);
                 }
-                tmem_st16(tP_g, ds);
+                tmem_st16(tP_g + 16, ds);
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
@@ -1013,7 +1055,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
     attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                        const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
                        const BwdParams p, int kv_tiles, int n_dkdv, int q_tiles) {
-    extern __shared__ uint8_t smem_raw[];
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
     const int b = (int)blockIdx.x;
     if (b < n_dkdv) {
         attn_bwd_dkdv_body(map_q, map_k, map_v, map_do, p, smem_raw, b % kv_tiles, b / kv_tiles);
