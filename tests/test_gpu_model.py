@@ -117,6 +117,10 @@ def test_error_growth_through_28_layers_bf16():
             assert_close(f"layer{l}.{k}", Gd[l][k], v, tol)
 
 
+# measured 2.2-2.5e-2 (2.47e-2 in the emulation): see the docstring of the test below
+FULL_WIDTH_SOFTMAX_PATH_BOUND = 3e-2
+
+
 @pytest.mark.skipif(_host_memory_gb() < 48, reason="the oracle run peaks at 29 GB of host memory (and takes a minute)")
 def test_model_full_widths_two_layers_bf16():
     """The full model configuration's widths (d 3584, 28 / 4 heads of 128, d_ff 18944, vocabulary 152064, biases,
@@ -124,12 +128,16 @@ def test_model_full_widths_two_layers_bf16():
     chunks of 1024 in the layers and in the head.  The full 28-layer, 65536-token call itself is beyond a direct
     oracle run; it composes exactly the layer and head calls checked at full size elsewhere.
 
-    With an N(0, 0.02) embedding the residual stream is the MLP output, so every bf16-stored activation of the forward
-    pass shows in the hidden state the head sees (the oracle rounds nothing in between): all gradients carry ~1.2e-2,
-    and the most sensitive ones -- W_q, W_k and their biases in the last layer, which pass through
-    dS = P (dP - delta) -- twice that.  The fp32-arithmetic CUDA-core engine on the same bf16 storage measures the same
-    (2.44e-2 against 2.50e-2 for the tensor-core kernels): it is storage rounding, not kernel arithmetic.  Hence two
-    bounds: 3e-2 for those four and for g1, which collects the same path (1.98e-2), 2e-2 for everything else."""
+    With an N(0, 0.02) embedding the residual stream is the MLP output, so the bf16 rounding of every operand of the
+    forward products (normalised activations, Q, K, V, P, O, gate / up, their product) shows in the hidden state the
+    head sees, and the oracle rounds nothing: all gradients carry ~1.2e-2, and W_q, W_k, their biases and g1 of the
+    last layer -- the ones that pass through dS = P (dP - delta), which amplifies a perturbation of the scores about
+    tenfold at this initialisation -- 2.0 to 2.5e-2.  That exceeds the 2e-2 stated for bf16 runs.  It is a DOCUMENTED
+    DEPARTURE, not a tolerance: a site-by-site emulation of the model (every bf16 rounding switched on alone / left
+    out) reproduces 2.47e-2 and shows that only the rounding of tensor-core operands contributes (storage that is not
+    an operand -- checkpoints, inter-layer gradients -- moves it from 2.47e-2 to 2.43e-2), and the fp32-arithmetic
+    CUDA-core engine on the same bf16 operands measures 2.44e-2.  So those five tensors are bounded by
+    FULL_WIDTH_SOFTMAX_PATH_BOUND and everything else by the common 2e-2."""
     c = synth.CONFIGS["qwen7b_model"]
     ls, hs = c.layer, c.head
     T, L = 2048, 2
@@ -149,5 +157,6 @@ def test_model_full_widths_two_layers_bf16():
             "d_g_final": assert_close("d_g_final", dg, ref["g_final"], tol)}
     for l in range(L):
         for k, v in ref["layers"][l].items():
-            errs[f"layer{l}.{k}"] = assert_close(f"layer{l}.{k}", Gd[l][k], v, 3e-2 if k in ("wq", "wk", "bq", "bk", "g1") else tol)
+            errs[f"layer{l}.{k}"] = assert_close(f"layer{l}.{k}", Gd[l][k], v,
+                                                   FULL_WIDTH_SOFTMAX_PATH_BOUND if k in ("wq", "wk", "bq", "bk", "g1") else tol)
     print("full-width 2-layer model, errors vs oracle:", {k: f"{v:.2e}" for k, v in sorted(errs.items(), key=lambda kv: -kv[1])[:6]})
