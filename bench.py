@@ -430,6 +430,8 @@ def main():
     ap.add_argument("--objective", default="sft", choices=["sft", "grpo", "dpo"],
                     help="objective of the qwen7b_head workload (Sec. 3.2.1)")
     ap.add_argument("--chunk", type=int, default=0)
+    ap.add_argument("--wgrad-group", type=int, default=1,
+                    help="layer workloads: chunks per weight-gradient pass (the second partition size, Sec. 4.3)")
     ap.add_argument("--T", type=int, default=0, help="override the sequence length (profiling on small cases)")
     ap.add_argument("--ref-tokens", type=int, default=512)
     ap.add_argument("--cpu-baseline-tokens", type=int, default=1024)
@@ -486,7 +488,7 @@ def main():
     X, dY = X_host.cuda(), dY_host.cuda()
     dX = torch.empty_like(X)
     grads = B.alloc_layer_grads(bcfg)
-    ws_bytes = B.layer_workspace_bytes(bcfg, T, chunk)
+    ws_bytes = B.layer_workspace_bytes(bcfg, T, chunk, args.wgrad_group)
     ws_full = B.layer_workspace_bytes(bcfg, T, T)
     ws = B.alloc_workspace(ws_bytes)
     stream = torch.cuda.current_stream()
@@ -502,9 +504,9 @@ def main():
             dpr.step(X, dY, dX)     # backward, then the gradient exchange on the communication stream
             dpr.wait()
         else:
-            B.layer_backward(bcfg, W, X, dY, chunk, grads, dX, ws)
+            B.layer_backward(bcfg, W, X, dY, chunk, grads, dX, ws, wgrad_group=args.wgrad_group)
 
-    fed = B.HostFedLayerBackward(bcfg, W, grads, T, chunk, ws)
+    fed = B.HostFedLayerBackward(bcfg, W, grads, T, chunk, ws, wgrad_group=args.wgrad_group)
 
     def run_e2e(steps):
         """Every step's X, dY come from pinned host memory and its dX goes back, inside the timed region; the
@@ -568,7 +570,7 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if cfg.bf16 else "f32", "data": "synthetic",
-        "config": {"workload": cfg.name, "T": T, "chunk": chunk, "d_model": s.d_model, "n_q_heads": s.n_q_heads,
+        "config": {"workload": cfg.name, "T": T, "chunk": chunk, "wgrad_group": args.wgrad_group, "d_model": s.d_model, "n_q_heads": s.n_q_heads,
                    "n_kv_heads": s.n_kv_heads, "head_dim": s.head_dim, "d_ff": s.d_ff, "qkv_bias": s.qkv_bias,
                    "l2": "inputs larger than L2 (weights + gradients > 1 GB per step)",
                    "product_kernel": B.product_kernel(),

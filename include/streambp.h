@@ -132,6 +132,27 @@ int streambp_layer_backward_packed(const streambp_layer_cfg *cfg, const streambp
                                    const streambp_layer_grads *grads, void *dX,
                                    void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/*
+ * The same streamed backward with a SECOND partition size for the weight gradients (Sec. 4.3, effect of the
+ * partition size: every partition pays one read-modify-write pass over the fp32 gradient of every weight, which is
+ * what makes small partitions slow).  The chunk loop is unchanged -- re-forward, attention and input gradients run per
+ * `chunk` rows -- but the weight-gradient products g_W += (dZ_out/dW)^T dL/dZ_out of Eq. (1) are formed once per
+ * `wgrad_group` consecutive chunks, as one product over wgrad_group * chunk rows, so the accumulators are passed over
+ * D / wgrad_group times instead of D times.  The price is memory: the operands of those products (the chunk's
+ * normalised inputs, attention output, gate / up / SwiGLU activations and their gradients) are kept for every chunk
+ * of a group.  wgrad_group = 1 is streambp_layer_backward; values above the number of chunks act like that number.
+ * The result is the same sum in a different association (equal within rounding of the fp32 accumulation).
+ * cu_seqlens may be NULL (one sequence) or describe a packed batch as in streambp_layer_backward_packed.
+ * Workspace: streambp_layer_workspace_bytes_grouped(cfg, T, chunk, wgrad_group).
+ */
+size_t streambp_layer_workspace_bytes_grouped(const streambp_layer_cfg *cfg, int64_t T, int64_t chunk,
+                                              int32_t wgrad_group);
+int streambp_layer_backward_grouped(const streambp_layer_cfg *cfg, const streambp_layer_weights *w, const void *X,
+                                    const void *dY, int64_t T, int64_t chunk, int32_t wgrad_group,
+                                    const int64_t *cu_seqlens, int32_t n_seqs, int64_t pos0, int accumulate,
+                                    const streambp_layer_grads *grads, void *dX, void *workspace,
+                                    size_t workspace_bytes, void *cuda_stream);
+
 typedef struct {
     int32_t d_model;
     int64_t vocab;

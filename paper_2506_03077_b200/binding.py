@@ -35,6 +35,7 @@ EXPORTS = (
     "streambp_attention_forward", "streambp_attention_backward", "streambp_attention_backward_static",
     "streambp_lmhead_rl_backward", "streambp_layer_backward_packed",
     "streambp_test_expire_wait", "streambp_test_per_device_value",
+    "streambp_layer_workspace_bytes_grouped", "streambp_layer_backward_grouped",
 )
 
 
@@ -96,6 +97,11 @@ def lib() -> C.CDLL:
     L.streambp_layer_backward_packed.restype = C.c_int
     L.streambp_layer_backward_packed.argtypes = [C.POINTER(LayerCfgC), C.POINTER(LayerPtrsC), vp, vp, i64, i64,
                                                  C.POINTER(i64), i32, i64, C.c_int, C.POINTER(LayerPtrsC), vp, vp, sz, vp]
+    L.streambp_layer_workspace_bytes_grouped.restype = sz
+    L.streambp_layer_workspace_bytes_grouped.argtypes = [C.POINTER(LayerCfgC), i64, i64, i32]
+    L.streambp_layer_backward_grouped.restype = C.c_int
+    L.streambp_layer_backward_grouped.argtypes = [C.POINTER(LayerCfgC), C.POINTER(LayerPtrsC), vp, vp, i64, i64, i32,
+                                                  C.POINTER(i64), i32, i64, C.c_int, C.POINTER(LayerPtrsC), vp, vp, sz, vp]
     L.streambp_lmhead_workspace_bytes.restype = sz
     L.streambp_lmhead_workspace_bytes.argtypes = [C.POINTER(HeadCfgC), i64, i64]
     L.streambp_lmhead_ce_backward.restype = C.c_int
@@ -227,8 +233,10 @@ def alloc_layer_grads(cfg: LayerConfig, device="cuda") -> Dict[str, torch.Tensor
     return {k: torch.zeros(s, dtype=torch.float32, device=device) for k, s in layer_grad_shapes(cfg).items()}
 
 
-def layer_workspace_bytes(cfg: LayerConfig, T: int, chunk: int) -> int:
+def layer_workspace_bytes(cfg: LayerConfig, T: int, chunk: int, wgrad_group: int = 1) -> int:
     c = cfg.c()
+    if wgrad_group != 1:
+        return int(lib().streambp_layer_workspace_bytes_grouped(C.byref(c), T, chunk, wgrad_group))
     return int(lib().streambp_layer_workspace_bytes(C.byref(c), T, chunk))
 
 
@@ -249,10 +257,21 @@ def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:
 
 def layer_backward(cfg: LayerConfig, weights: Dict[str, torch.Tensor], X: torch.Tensor, dY: torch.Tensor,
                    chunk: int, grads: Dict[str, torch.Tensor], dX: torch.Tensor, workspace: torch.Tensor,
-                   pos0: int = 0, accumulate: bool = False, stream=None, check: bool = True) -> int:
-    """streambp_layer_backward; returns the status (raises on error when check=True)."""
+                   pos0: int = 0, accumulate: bool = False, stream=None, check: bool = True, wgrad_group: int = 1,
+                   cu_seqlens: Optional[Sequence[int]] = None) -> int:
+    """streambp_layer_backward (or streambp_layer_backward_grouped when wgrad_group != 1); returns the status
+    (raises on error when check=True)."""
     c = cfg.c()
     w, g = _ptr_struct(weights), _ptr_struct(grads)
+    if wgrad_group != 1:
+        cu = (C.c_int64 * len(cu_seqlens))(*cu_seqlens) if cu_seqlens is not None else None
+        st = lib().streambp_layer_backward_grouped(C.byref(c), C.byref(w), _ptr(X), _ptr(dY), X.shape[0], chunk,
+                                                   wgrad_group, cu, len(cu_seqlens) - 1 if cu_seqlens is not None else 0,
+                                                   pos0, 1 if accumulate else 0, C.byref(g), _ptr(dX), _ptr(workspace),
+                                                   workspace.numel(), _stream_ptr(stream))
+        if check:
+            _check(st, "streambp_layer_backward_grouped")
+        return st
     st = lib().streambp_layer_backward(C.byref(c), C.byref(w), _ptr(X), _ptr(dY), X.shape[0], chunk, pos0,
                                        1 if accumulate else 0, C.byref(g), _ptr(dX), _ptr(workspace),
                                        workspace.numel(), _stream_ptr(stream))
@@ -268,7 +287,9 @@ class HostFedLayerBackward:
     takes out the dX of step k-1, so a sequence's 3 T d storage-dtype values cross PCIe behind the compute of
     its neighbours instead of in front of its own."""
 
-    def __init__(self, cfg: LayerConfig, weights, grads, T: int, chunk: int, workspace: torch.Tensor):
+    def __init__(self, cfg: LayerConfig, weights, grads, T: int, chunk: int, workspace: torch.Tensor,
+                 wgrad_group: int = 1):
+        self.wgrad_group = wgrad_group
         self.cfg, self.weights, self.grads, self.chunk, self.ws = cfg, weights, grads, chunk, workspace
         dev = workspace.device
         mk = lambda: torch.empty(T, cfg.d_model, dtype=cfg.dtype, device=dev)
@@ -300,7 +321,7 @@ class HostFedLayerBackward:
         st = stream if stream is not None else torch.cuda.current_stream()
         st.wait_event(self.loaded[i])
         layer_backward(self.cfg, self.weights, self.X[i], self.dY[i], self.chunk, self.grads, self.dX[i], self.ws,
-                       accumulate=accumulate, stream=st)
+                       accumulate=accumulate, stream=st, wgrad_group=self.wgrad_group)
         self.computed[i].record(st)
         cs = self.copy_stream
         cs.wait_event(self.computed[i])

@@ -309,17 +309,23 @@ int64_t suggest_chunk(int64_t T, size_t budget, F bytes) {
 
 extern "C" {
 
+size_t streambp_layer_workspace_bytes_grouped(const streambp_layer_cfg *cfg, int64_t T, int64_t chunk,
+                                              int32_t wgrad_group) {
+    if (check_layer_cfg(cfg) != STREAMBP_OK || T < 1 || chunk < 1 || wgrad_group < 1) return 0;
+    return cfg->dtype == STREAMBP_F32 ? layer_workspace<float>(*cfg, T, chunk, wgrad_group)
+                                      : layer_workspace<bf16>(*cfg, T, chunk, wgrad_group);
+}
+
 size_t streambp_layer_workspace_bytes(const streambp_layer_cfg *cfg, int64_t T, int64_t chunk) {
-    if (check_layer_cfg(cfg) != STREAMBP_OK || T < 1 || chunk < 1) return 0;
-    return cfg->dtype == STREAMBP_F32 ? layer_workspace<float>(*cfg, T, chunk) : layer_workspace<bf16>(*cfg, T, chunk);
+    return streambp_layer_workspace_bytes_grouped(cfg, T, chunk, 1);
 }
 
 static int layer_backward_checked(const streambp_layer_cfg *cfg, const streambp_layer_weights *w, const void *X,
                                   const void *dY, int64_t T, int64_t chunk, const int64_t *cu_seqlens, int n_seqs,
                                   int64_t pos0, int accumulate, const streambp_layer_grads *grads, void *dX,
-                                  void *workspace, size_t workspace_bytes, void *cuda_stream) {
+                                  void *workspace, size_t workspace_bytes, void *cuda_stream, int wgrad_group = 1) {
     SBP_TRY(check_layer_cfg(cfg));
-    if (T < 1 || chunk < 1 || pos0 < 0) return STREAMBP_E_SHAPE;
+    if (T < 1 || chunk < 1 || pos0 < 0 || wgrad_group < 1) return STREAMBP_E_SHAPE;
     SBP_TRY(check_layer_weights(cfg, w));
     SBP_TRY(check_layer_grads(cfg, grads));
     if (!X || !dY || !dX || !workspace) return STREAMBP_E_NULL;
@@ -330,15 +336,24 @@ static int layer_backward_checked(const streambp_layer_cfg *cfg, const streambp_
         for (int i = 0; i < n_seqs; i++)
             if (cu_seqlens[i + 1] <= cu_seqlens[i]) return STREAMBP_E_SHAPE;
     }
-    if (workspace_bytes < streambp_layer_workspace_bytes(cfg, T, chunk)) return STREAMBP_E_WORKSPACE;
+    if (workspace_bytes < streambp_layer_workspace_bytes_grouped(cfg, T, chunk, wgrad_group)) return STREAMBP_E_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     SBP_TRY(begin_call(workspace, st));
     const streambp_layer_weights we = effective(cfg, w);
     if (cfg->dtype == STREAMBP_F32)
         return layer_backward<float>(*cfg, we, (const float *)X, (const float *)dY, T, chunk, pos0, accumulate != 0,
-                                     *grads, (float *)dX, workspace, st, cu_seqlens, n_seqs);
+                                     *grads, (float *)dX, workspace, st, cu_seqlens, n_seqs, wgrad_group);
     return layer_backward<bf16>(*cfg, we, (const bf16 *)X, (const bf16 *)dY, T, chunk, pos0, accumulate != 0, *grads,
-                                (bf16 *)dX, workspace, st, cu_seqlens, n_seqs);
+                                (bf16 *)dX, workspace, st, cu_seqlens, n_seqs, wgrad_group);
+}
+
+int streambp_layer_backward_grouped(const streambp_layer_cfg *cfg, const streambp_layer_weights *w, const void *X,
+                                    const void *dY, int64_t T, int64_t chunk, int32_t wgrad_group,
+                                    const int64_t *cu_seqlens, int32_t n_seqs, int64_t pos0, int accumulate,
+                                    const streambp_layer_grads *grads, void *dX, void *workspace, size_t workspace_bytes,
+                                    void *cuda_stream) {
+    return layer_backward_checked(cfg, w, X, dY, T, chunk, cu_seqlens, cu_seqlens ? n_seqs : 0, pos0, accumulate, grads,
+                                  dX, workspace, workspace_bytes, cuda_stream, wgrad_group);
 }
 
 int streambp_layer_backward(const streambp_layer_cfg *cfg, const streambp_layer_weights *w, const void *X,

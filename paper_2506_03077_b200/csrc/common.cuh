@@ -439,12 +439,13 @@ int mm_swiglu(int64_t M, int64_t N, int64_t K, const T *A, int64_t lda, const T 
               T *m, int64_t ldc, cudaStream_t st);
 
 // ---- schedulers (T = storage dtype) --------------------------------------------------
+// wgrad_group: consecutive chunks whose weight-gradient products are summed in one pass (1 = every chunk)
 template <typename T>
-size_t layer_workspace(const streambp_layer_cfg &c, int64_t T_, int64_t chunk);
+size_t layer_workspace(const streambp_layer_cfg &c, int64_t T_, int64_t chunk, int wgrad_group = 1);
 template <typename T>
 int layer_backward(const streambp_layer_cfg &c, const streambp_layer_weights &w, const T *X, const T *dY, int64_t T_,
                    int64_t chunk, int64_t pos0, bool accumulate, const streambp_layer_grads &g, T *dX, void *ws,
-                   cudaStream_t st, const int64_t *cu_seqlens = nullptr, int n_seqs = 0);
+                   cudaStream_t st, const int64_t *cu_seqlens = nullptr, int n_seqs = 0, int wgrad_group = 1);
 // Y = layer(X), chunked; uses the same workspace plan as layer_backward.
 template <typename T>
 // cu_seqlens (host, n_seqs + 1 entries, 0 ... T): sequence boundaries of a packed batch, or nullptr.

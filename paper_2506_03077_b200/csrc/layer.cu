@@ -43,41 +43,61 @@ struct LayerWs {
     T *h1, *Q, *O, *h2, *g, *u, *m, *dr_s, *dO, *dk_s, *dv_s, *dm;
     float *fa, *r, *dr, *rstd1, *rstd2, *lse, *delta, *partials;
     size_t bytes;
+    int slots;            // chunks per weight-gradient group
 };
 
+// `wg` >= 1 is the number of consecutive chunks whose weight-gradient products are summed in ONE pass over the
+// fp32 accumulators (a second partition size: K = wg * chunk for those products).  The operands of those products
+// -- h1, dq (in Q's place), O, h2, dg, du (in g's and u's place), m, dr and dk, dv in storage type -- then exist once
+// per chunk of a group ("slots", contiguous in row order, so a group's operand is one matrix of wg * chunk rows).
 template <typename T>
-LayerWs<T> plan(const streambp_layer_cfg &c, int64_t T_, int64_t chunk, void *base) {
+LayerWs<T> plan(const streambp_layer_cfg &c, int64_t T_, int64_t chunk, void *base, int wg = 1) {
     const int64_t cn = chunk < T_ ? chunk : T_;
     const int64_t d = c.d_model, dq = (int64_t)c.n_q_heads * c.head_dim, dkv = (int64_t)c.n_kv_heads * c.head_dim;
     const int64_t I = c.d_ff, wide = dq > d ? dq : d;
+    const int64_t D = (T_ + cn - 1) / cn;
+    const int64_t slots = wg < 1 ? 1 : (wg > D ? D : wg);
+    const int64_t gr = slots * cn;          // rows of a group's operand buffers
     Arena a(base);
     LayerWs<T> w;
+    w.slots = (int)slots;
     w.hdr = reinterpret_cast<WsHeader *>(a.take_bytes(kHeaderBytes));
     w.cs = a.take<float>(T_ * c.head_dim);
     w.K = a.take<T>(T_ * dkv);
     w.V = a.take<T>(T_ * dkv);
     w.dK = a.take<float>(T_ * dkv);
     w.dV = a.take<float>(T_ * dkv);
-    w.h1 = a.take<T>(cn * d);
-    w.Q = a.take<T>(cn * dq);
-    w.O = a.take<T>(cn * dq);
-    w.h2 = a.take<T>(cn * d);
-    w.g = a.take<T>(cn * I);
-    w.u = a.take<T>(cn * I);
-    w.m = a.take<T>(cn * I);
-    const size_t dead_begin = align_up(a.off, 256);
-    w.dr_s = a.take<T>(cn * d);
-    w.dO = a.take<T>(cn * dq);
-    w.dk_s = a.take<T>(cn * dkv);
-    w.dv_s = a.take<T>(cn * dkv);
-    w.fa = a.take<float>(cn * wide);
-    w.dr = a.take<float>(cn * d);
-    // dm = dY Wd lives only from its product to the SwiGLU backward, while dr_s, dO, dk_s, dv_s, fa and dr are all
-    // dead: it is laid over that span when it fits (it does for every LLM-shaped layer), else it gets its own block
-    if (a.off - dead_begin >= (size_t)(cn * I) * sizeof(T))
-        w.dm = a.base ? reinterpret_cast<T *>(a.base + dead_begin) : nullptr;
-    else
+    w.h1 = a.take<T>(gr * d);
+    w.Q = a.take<T>(gr * dq);
+    w.O = a.take<T>(gr * dq);
+    w.h2 = a.take<T>(gr * d);
+    w.g = a.take<T>(gr * I);
+    w.u = a.take<T>(gr * I);
+    w.m = a.take<T>(gr * I);
+    if (slots > 1) {
+        // group operands first (they outlive their chunk), then the buffers of the chunk in flight
+        w.dr_s = a.take<T>(gr * d);
+        w.dk_s = a.take<T>(gr * dkv);
+        w.dv_s = a.take<T>(gr * dkv);
+        w.dO = a.take<T>(cn * dq);
+        w.fa = a.take<float>(cn * wide);
+        w.dr = a.take<float>(sizeof(T) == 4 ? gr * d : cn * d);   // fp32 storage: dr itself is the product operand
         w.dm = a.take<T>(cn * I);
+    } else {
+        const size_t dead_begin = align_up(a.off, 256);
+        w.dr_s = a.take<T>(cn * d);
+        w.dO = a.take<T>(cn * dq);
+        w.dk_s = a.take<T>(cn * dkv);
+        w.dv_s = a.take<T>(cn * dkv);
+        w.fa = a.take<float>(cn * wide);
+        w.dr = a.take<float>(cn * d);
+        // dm = dY Wd lives only from its product to the SwiGLU backward, while dr_s, dO, dk_s, dv_s, fa and dr are all
+        // dead: it is laid over that span when it fits (it does for every LLM-shaped layer), else it gets its own block
+        if (a.off - dead_begin >= (size_t)(cn * I) * sizeof(T))
+            w.dm = a.base ? reinterpret_cast<T *>(a.base + dead_begin) : nullptr;
+        else
+            w.dm = a.take<T>(cn * I);
+    }
     w.r = a.take<float>(cn * d);
     w.rstd1 = a.take<float>(cn);
     w.rstd2 = a.take<float>(cn);
@@ -86,6 +106,21 @@ LayerWs<T> plan(const streambp_layer_cfg &c, int64_t T_, int64_t chunk, void *ba
     w.partials = a.take<float>(64 * wide);
     w.bytes = a.size();
     return w;
+}
+
+// The same plan with the group-operand pointers moved to the slot of the chunk that starts `row_off` rows into
+// its group.
+template <typename T>
+LayerWs<T> at_slot(const LayerWs<T> &w, const streambp_layer_cfg &c, int64_t row_off) {
+    if (row_off == 0 || w.h1 == nullptr) return w;
+    const int64_t d = c.d_model, dq = (int64_t)c.n_q_heads * c.head_dim, dkv = (int64_t)c.n_kv_heads * c.head_dim;
+    const int64_t I = c.d_ff;
+    LayerWs<T> s = w;
+    s.h1 += row_off * d; s.Q += row_off * dq; s.O += row_off * dq; s.h2 += row_off * d;
+    s.g += row_off * I; s.u += row_off * I; s.m += row_off * I;
+    s.dr_s += row_off * d; s.dk_s += row_off * dkv; s.dv_s += row_off * dkv;
+    if (sizeof(T) == 4) s.dr += row_off * d;
+    return s;
 }
 
 // K/V for all rows, chunk by chunk: h1 = RMSNorm1(X), K = RoPE(h1 Wk^T + bk), V = h1 Wv^T + bv
@@ -140,8 +175,8 @@ int chunk_forward(const streambp_layer_cfg &c, const streambp_layer_weights &w, 
 }  // namespace
 
 template <typename T>
-size_t layer_workspace(const streambp_layer_cfg &c, int64_t T_, int64_t chunk) {
-    return plan<T>(c, T_, chunk, nullptr).bytes;
+size_t layer_workspace(const streambp_layer_cfg &c, int64_t T_, int64_t chunk, int wgrad_group) {
+    return plan<T>(c, T_, chunk, nullptr, wgrad_group).bytes;
 }
 
 template <typename T>
@@ -166,19 +201,19 @@ int layer_forward(const streambp_layer_cfg &c, const streambp_layer_weights &w, 
 template <typename T>
 int layer_backward(const streambp_layer_cfg &c, const streambp_layer_weights &w, const T *X, const T *dY, int64_t T_,
                    int64_t chunk, int64_t pos0, bool accumulate, const streambp_layer_grads &G, T *dX, void *ws,
-                   cudaStream_t st, const int64_t *cu_seqlens, int n_seqs) {
+                   cudaStream_t st, const int64_t *cu_seqlens, int n_seqs, int wgrad_group) {
     const Segments seg(cu_seqlens, n_seqs, T_);
     const int64_t cn = chunk < T_ ? chunk : T_;
-    LayerWs<T> s = plan<T>(c, T_, chunk, ws);
-    const SchedScope sched(s.hdr);
+    LayerWs<T> base = plan<T>(c, T_, chunk, ws, wgrad_group);
+    const SchedScope sched(base.hdr);
     const int d = c.d_model, dh = c.head_dim, Hq = c.n_q_heads, Hkv = c.n_kv_heads;
     const int64_t dq = (int64_t)Hq * dh, dkv = (int64_t)Hkv * dh, I = c.d_ff;
     constexpr bool kF32 = sizeof(T) == 4;
 
-    SBP_TRY(kv_prologue<T>(c, w, X, T_, cn, pos0, seg, s, st));
-    SBP_TRY(fill_zero(s.dK, sizeof(float) * T_ * dkv, st));
-    SBP_TRY(fill_zero(s.dV, sizeof(float) * T_ * dkv, st));
-    if (!accumulate) {  // vectors are always added to; matrices are overwritten by the first chunk's product
+    SBP_TRY(kv_prologue<T>(c, w, X, T_, cn, pos0, seg, base, st));
+    SBP_TRY(fill_zero(base.dK, sizeof(float) * T_ * dkv, st));
+    SBP_TRY(fill_zero(base.dV, sizeof(float) * T_ * dkv, st));
+    if (!accumulate) {  // vectors are always added to; matrices are overwritten by the first group's product
         SBP_TRY(fill_zero(G.g1, sizeof(float) * d, st));
         SBP_TRY(fill_zero(G.g2, sizeof(float) * d, st));
         if (c.qkv_bias) {
@@ -188,37 +223,50 @@ int layer_backward(const streambp_layer_cfg &c, const streambp_layer_weights &w,
         }
     }
     const int64_t D = (T_ + cn - 1) / cn;
+    const int64_t k = base.slots;
     for (int64_t i = D - 1; i >= 0; i--) {
-        const int64_t r0 = i * cn;
+        // Chunks are grouped from the end: {D-1 .. D-k}, {D-k-1 .. D-2k}, ...  The weight-gradient products of a
+        // group run once, when its first chunk (the last one processed) is done, over all the group's rows: the
+        // operands of a group are contiguous in row order (X, dY in the caller's arrays, the rest in the slots).
+        const int64_t g_hi = D - 1 - ((D - 1 - i) / k) * k, g_lo = g_hi - k + 1 > 0 ? g_hi - k + 1 : 0;
+        const bool group_done = i == g_lo;
+        const int64_t r0 = i * cn, gr0 = g_lo * cn;
         const int64_t n = (T_ - r0 < cn) ? T_ - r0 : cn;
-        const bool acc = accumulate || i != D - 1;
-        const T *Xi = X + r0 * d, *dYi = dY + r0 * d;
+        const int64_t gn = ((g_hi + 1) * cn < T_ ? (g_hi + 1) * cn : T_) - gr0;      // rows of the group
+        const bool acc = accumulate || g_hi != D - 1;
+        const T *Xi = X + r0 * d, *dYi = dY + r0 * d, *dYg = dY + gr0 * d;
+        LayerWs<T> s = at_slot<T>(base, c, r0 - gr0);
         SBP_TRY(chunk_forward<T>(c, w, X, r0, n, seg, s, st));
 
         // ---- MLP backward ----
         SBP_TRY((mm<T, T>(OP_NN, n, I, d, dYi, d, (const T *)w.w_down, I, s.dm, I, nullptr, false, st)));  // dm = dY Wd
         SBP_TRY(swiglu_bwd<T>(s.dm, s.g, s.u, n * I, st));                                            // g := dg, u := du
-        {   // dWd += dY^T m, dWg += dg^T h2, dWu += du^T h2, dh2 = dg Wg + du Wu in one launch: the weight
-            // gradients are bound by the fp32 add into C at L2, the input gradient by the tensor pipe
-            MmProb<T> pr[4] = {
-                mm_prob<T>(OP_TN, d, I, n, dYi, d, s.m, I, G.w_down, I, true, nullptr, acc),
-                mm_prob<T>(OP_TN, I, d, n, s.g, I, s.h2, d, G.w_gate, d, true, nullptr, acc),
-                mm_prob<T>(OP_TN, I, d, n, s.u, I, s.h2, d, G.w_up, d, true, nullptr, acc),
-                mm_prob<T>(OP_NN, n, d, I, s.g, I, (const T *)w.w_gate, d, s.fa, d, true, nullptr, false)};
-            mm_add_seg<T>(pr[3], I, s.u, I, (const T *)w.w_up, d);
-            SBP_TRY(mm_group<T>(pr, 4, st));
+        {   // dh2 = dg Wg + du Wu, and with it (one launch) the group's dWd += dY^T m, dWg += dg^T h2, dWu += du^T h2:
+            // the weight gradients are bound by the fp32 add into C at L2, the input gradient by the tensor pipe
+            MmProb<T> pr[4];
+            int np = 0;
+            if (group_done) {
+                pr[np++] = mm_prob<T>(OP_TN, d, I, gn, dYg, d, base.m, I, G.w_down, I, true, nullptr, acc);
+                pr[np++] = mm_prob<T>(OP_TN, I, d, gn, base.g, I, base.h2, d, G.w_gate, d, true, nullptr, acc);
+                pr[np++] = mm_prob<T>(OP_TN, I, d, gn, base.u, I, base.h2, d, G.w_up, d, true, nullptr, acc);
+            }
+            pr[np] = mm_prob<T>(OP_NN, n, d, I, s.g, I, (const T *)w.w_gate, d, s.fa, d, true, nullptr, false);
+            mm_add_seg<T>(pr[np], I, s.u, I, (const T *)w.w_up, d);
+            SBP_TRY(mm_group<T>(pr, np + 1, st));
         }
         // dr = dY + norm2_bwd(dh2)
         SBP_TRY(rmsnorm_bwd<T>(s.fa, nullptr, s.r, s.rstd2, (const T *)w.g2, dYi, nullptr, n, d, s.dr,
                                kF32 ? nullptr : s.dr_s, G.g2, s.partials, st));
         const T *dr_op = kF32 ? reinterpret_cast<const T *>(s.dr) : s.dr_s;
+        const T *dr_grp = kF32 ? reinterpret_cast<const T *>(base.dr) : base.dr_s;
 
         // ---- attention output projection backward ----
-        {   // dWo += dr^T O, dO = dr Wo
-            const MmProb<T> pr[2] = {
-                mm_prob<T>(OP_TN, d, dq, n, dr_op, d, s.O, dq, G.wo, dq, true, nullptr, acc),
-                mm_prob<T>(OP_NN, n, dq, d, dr_op, d, (const T *)w.wo, dq, s.dO, dq, sizeof(T) == 4, nullptr, false)};
-            SBP_TRY(mm_group<T>(pr, 2, st));
+        {   // dO = dr Wo, and the group's dWo += dr^T O
+            MmProb<T> pr[2];
+            int np = 0;
+            if (group_done) pr[np++] = mm_prob<T>(OP_TN, d, dq, gn, dr_grp, d, base.O, dq, G.wo, dq, true, nullptr, acc);
+            pr[np++] = mm_prob<T>(OP_NN, n, dq, d, dr_op, d, (const T *)w.wo, dq, s.dO, dq, sizeof(T) == 4, nullptr, false);
+            SBP_TRY(mm_group<T>(pr, np, st));
         }
 
         // ---- partitioned attention backward: dQ (into fa), dK/dV prefix += ----
@@ -236,18 +284,21 @@ int layer_backward(const streambp_layer_cfg &c, const streambp_layer_weights &w,
         SBP_TRY(rope_apply<T>(s.fa, s.cs + r0 * dh, n, Hq, dh, true, dq_s, st));
         SBP_TRY(rope_apply<T>(s.dK + r0 * dkv, s.cs + r0 * dh, n, Hkv, dh, true, s.dk_s, st));
         SBP_TRY(cast_from_f32<T>(s.dV + r0 * dkv, n * dkv, s.dv_s, st));
-        {   // dWq, dWk, dWv and dh1 = dq Wq + dk Wk + dv Wv
-            MmProb<T> pr[4] = {
-                mm_prob<T>(OP_TN, dq, d, n, dq_s, dq, s.h1, d, G.wq, d, true, nullptr, acc),
-                mm_prob<T>(OP_TN, dkv, d, n, s.dk_s, dkv, s.h1, d, G.wk, d, true, nullptr, acc),
-                mm_prob<T>(OP_TN, dkv, d, n, s.dv_s, dkv, s.h1, d, G.wv, d, true, nullptr, acc),
-                mm_prob<T>(OP_NN, n, d, dq, dq_s, dq, (const T *)w.wq, d, s.fa, d, true, nullptr, false)};
-            mm_add_seg<T>(pr[3], dkv, s.dk_s, dkv, (const T *)w.wk, d);
-            mm_add_seg<T>(pr[3], dkv, s.dv_s, dkv, (const T *)w.wv, d);
-            SBP_TRY(mm_group<T>(pr, 4, st));
+        {   // dh1 = dq Wq + dk Wk + dv Wv, and the group's dWq, dWk, dWv
+            MmProb<T> pr[4];
+            int np = 0;
+            if (group_done) {
+                pr[np++] = mm_prob<T>(OP_TN, dq, d, gn, base.Q, dq, base.h1, d, G.wq, d, true, nullptr, acc);
+                pr[np++] = mm_prob<T>(OP_TN, dkv, d, gn, base.dk_s, dkv, base.h1, d, G.wk, d, true, nullptr, acc);
+                pr[np++] = mm_prob<T>(OP_TN, dkv, d, gn, base.dv_s, dkv, base.h1, d, G.wv, d, true, nullptr, acc);
+            }
+            pr[np] = mm_prob<T>(OP_NN, n, d, dq, dq_s, dq, (const T *)w.wq, d, s.fa, d, true, nullptr, false);
+            mm_add_seg<T>(pr[np], dkv, s.dk_s, dkv, (const T *)w.wk, d);
+            mm_add_seg<T>(pr[np], dkv, s.dv_s, dkv, (const T *)w.wv, d);
+            SBP_TRY(mm_group<T>(pr, np + 1, st));
         }
-        if (c.qkv_bias)
-            SBP_TRY(colsum3_add<T>(dq_s, (int)dq, G.bq, s.dk_s, (int)dkv, G.bk, s.dv_s, (int)dkv, G.bv, n, s.partials, st));
+        if (c.qkv_bias && group_done)
+            SBP_TRY(colsum3_add<T>(base.Q, (int)dq, G.bq, base.dk_s, (int)dkv, G.bk, base.dv_s, (int)dkv, G.bv, gn, s.partials, st));
 
         // ---- dX = dr + norm1_bwd(dh1) ----
         SBP_TRY(rmsnorm_bwd<T>(s.fa, Xi, nullptr, s.rstd1, (const T *)w.g1, nullptr, s.dr, n, d, nullptr, dX + r0 * d,
@@ -256,17 +307,17 @@ int layer_backward(const streambp_layer_cfg &c, const streambp_layer_weights &w,
     return STREAMBP_OK;
 }
 
-template size_t layer_workspace<float>(const streambp_layer_cfg &, int64_t, int64_t);
-template size_t layer_workspace<bf16>(const streambp_layer_cfg &, int64_t, int64_t);
+template size_t layer_workspace<float>(const streambp_layer_cfg &, int64_t, int64_t, int);
+template size_t layer_workspace<bf16>(const streambp_layer_cfg &, int64_t, int64_t, int);
 template int layer_forward<float>(const streambp_layer_cfg &, const streambp_layer_weights &, const float *, int64_t,
                                   int64_t, int64_t, float *, void *, cudaStream_t, const int64_t *, int);
 template int layer_forward<bf16>(const streambp_layer_cfg &, const streambp_layer_weights &, const bf16 *, int64_t,
                                  int64_t, int64_t, bf16 *, void *, cudaStream_t, const int64_t *, int);
 template int layer_backward<float>(const streambp_layer_cfg &, const streambp_layer_weights &, const float *,
                                    const float *, int64_t, int64_t, int64_t, bool, const streambp_layer_grads &,
-                                   float *, void *, cudaStream_t, const int64_t *, int);
+                                   float *, void *, cudaStream_t, const int64_t *, int, int);
 template int layer_backward<bf16>(const streambp_layer_cfg &, const streambp_layer_weights &, const bf16 *,
                                   const bf16 *, int64_t, int64_t, int64_t, bool, const streambp_layer_grads &, bf16 *,
-                                  void *, cudaStream_t, const int64_t *, int);
+                                  void *, cudaStream_t, const int64_t *, int, int);
 
 }  // namespace sbp

@@ -28,7 +28,7 @@ def layer_case(shape: synth.LayerShape, seed: int, T: int, dtype: torch.dtype, d
     return ocfg, bcfg, W, X, dY
 
 
-def run_layer(bcfg, W, X, dY, chunk, pos0=0, accumulate=False, grads=None):
+def run_layer(bcfg, W, X, dY, chunk, pos0=0, accumulate=False, grads=None, wgrad_group=1, cu_seqlens=None):
     dt = bcfg.dtype
     Wd = {k: to_dev(v, dt) for k, v in W.items()}
     Xd, dYd = to_dev(X, dt), to_dev(dY, dt)
@@ -38,8 +38,9 @@ def run_layer(bcfg, W, X, dY, chunk, pos0=0, accumulate=False, grads=None):
             for g in grads.values():
                 g.fill_(float("nan"))     # the call must overwrite, not add
     dX = torch.full_like(Xd, float("nan"))
-    ws = B.alloc_workspace(B.layer_workspace_bytes(bcfg, X.shape[0], chunk))
-    B.layer_backward(bcfg, Wd, Xd, dYd, chunk, grads, dX, ws, pos0=pos0, accumulate=accumulate)
+    ws = B.alloc_workspace(B.layer_workspace_bytes(bcfg, X.shape[0], chunk, wgrad_group))
+    B.layer_backward(bcfg, Wd, Xd, dYd, chunk, grads, dX, ws, pos0=pos0, accumulate=accumulate, wgrad_group=wgrad_group,
+                     cu_seqlens=cu_seqlens)
     assert B.last_device_status(ws) == B.OK
     return dX, grads
 

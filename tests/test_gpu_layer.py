@@ -44,6 +44,45 @@ def test_chunk_invariance_fp32():
             assert O.rel_frobenius(grads[k].cpu().numpy(), base[k].cpu().numpy()) < 1e-5, (chunk, k)
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("T,chunk,group", [(200, 32, 2), (200, 32, 3), (192, 64, 2), (150, 40, 16), (96, 96, 2)])
+def test_weight_gradients_summed_over_groups_of_chunks(dtype, T, chunk, group):
+    """The second partition size (Sec. 4.3): weight-gradient products formed once per `group` chunks over all their
+    rows.  Same sum, different association: against the oracle at the usual tolerance, dX bit-identical to the
+    ungrouped call (the chunk loop itself is unchanged), ragged last chunk and a last group of fewer chunks included,
+    a group larger than the number of chunks, bias sums, and accumulation into existing gradients."""
+    shape = synth.LayerShape(128, 4, 2, 64, 168, True, 1e4) if dtype == torch.float32 else \
+        synth.LayerShape(256, 4, 2, 128, 512, True, 1e6)
+    ocfg, bcfg, W, X, dY = layer_case(shape, 11, T, dtype, dy_std=1.0 if dtype == torch.float32 else 1e-3,
+                                      wstd=0.05 if dtype == torch.float32 else 0.02)
+    dX, grads = run_layer(bcfg, W, X, dY, chunk, pos0=3, wgrad_group=group)
+    compare_layer(ocfg, W, X, dY, dX, grads, TOL[dtype], pos0=3)
+    dX1, g1 = run_layer(bcfg, W, X, dY, chunk, pos0=3)
+    assert torch.equal(dX, dX1)
+    for k in g1:
+        assert O.rel_frobenius(grads[k].cpu().numpy(), g1[k].cpu().numpy()) < (1e-5 if dtype == torch.float32 else 2e-3), k
+    twice = {k: v.clone() for k, v in grads.items()}
+    run_layer(bcfg, W, X, dY, chunk, pos0=3, wgrad_group=group, accumulate=True, grads=twice)
+    for k in grads:
+        assert O.rel_frobenius(twice[k].cpu().numpy(), 2.0 * grads[k].cpu().numpy()) < 1e-6, k
+    assert B.layer_workspace_bytes(bcfg, T, chunk, group) > B.layer_workspace_bytes(bcfg, T, chunk) or chunk >= T
+    # the operands kept per extra chunk of a group: a fixed number of bytes per row
+    if chunk * 3 <= T:
+        w1, w2, w3 = (B.layer_workspace_bytes(bcfg, T, chunk, g) for g in (1, 2, 3))
+        assert w3 - w2 <= w2 - w1 + 4096 and w3 > w2
+
+
+def test_grouped_packed_batch_matches_packed():
+    shape = synth.LayerShape(256, 4, 2, 128, 512, False, 1e6)
+    ocfg, bcfg, W, X, dY = layer_case(shape, 12, 300, torch.bfloat16)
+    cu = [0, 70, 71, 230, 300]
+    dX, grads = run_layer(bcfg, W, X, dY, 64, wgrad_group=2, cu_seqlens=cu)
+    dX_ref, G_ref = O.layer_backward_packed(ocfg, W, X, dY, cu)
+    assert_close("dX", dX, dX_ref, TOL[torch.bfloat16])
+    for k in G_ref:
+        assert_close(k, grads[k], G_ref[k], TOL[torch.bfloat16])
+
+
 def test_accumulate_adds_to_existing_gradients():
     shape = synth.LayerShape(128, 4, 2, 64, 168, True, 1e4)
     ocfg, bcfg, W, X, dY = layer_case(shape, 4, 100, torch.float32, dy_std=1.0, wstd=0.05)
