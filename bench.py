@@ -55,7 +55,7 @@ def attn_fwd_bytes(s, kv_len, n):
 NCU_TRAFFIC = {
     ("qwen7b_layer", 1024, "gemm"): (2142.5e6, "MLP-backward group of a chunk, profiles/gemm_pair_kernel_chunk_products.md", None),
     ("llama8b_layer", 2048, "gemm"): (2421.9e6, "MLP-backward group of a chunk, profiles/gemm_pair_kernel_chunk_products.md", None),
-    ("llama8b_layer", 2048, "attention_bwd"): (483.8e6, "2048 queries against a 16384-key prefix, "
+    ("llama8b_layer", 2048, "attention_bwd"): (488.6e6, "2048 queries against a 16384-key prefix, "
                                                "profiles/attention_tc_kernels_llama8b_chunk2048.md", (16384, 2048)),
     ("llama8b_layer", 2048, "attention_fwd"): (88.4e6, "2048 queries against a 16384-key prefix, "
                                                "profiles/attention_tc_kernels_llama8b_chunk2048.md", (16384, 2048)),
