@@ -39,8 +39,12 @@
  *     CUDA cores for fp32); STREAMBP_GEMM_SINGLE_CTA (any value) selects the
  *     single-CTA tcgen05 product kernel instead of the CTA-pair one, which is also
  *     what runs where a two-CTA cluster cannot be scheduled; STREAMBP_VERBOSE (any
- *     value) reports that choice on stderr.  None of them changes a result beyond
- *     floating-point summation order.
+ *     value) reports that choice on stderr; STREAMBP_WS_GUARD (any value) is a debug mode
+ *     that puts a 256-byte guard after every sub-buffer of the workspaces (the size
+ *     queries grow accordingly), fills the guards before and checks them after each
+ *     call, and reports an overwritten guard as STREAMBP_E_WORKSPACE_GUARD through
+ *     streambp_last_device_status.  None of them changes a result beyond floating-point
+ *     summation order.
  */
 #ifndef STREAMBP_H_
 #define STREAMBP_H_
@@ -62,7 +66,8 @@ typedef enum {
     STREAMBP_E_CUDA = -6,            /* a CUDA runtime / driver call failed */
     STREAMBP_E_BAD_LABEL = -7,       /* device: label not in [0, vocab) and != ignore_index */
     STREAMBP_E_NO_VALID_LABELS = -8, /* device: every label ignored; loss and grads are 0 */
-    STREAMBP_E_DEVICE_TIMEOUT = -9   /* device: a bounded wait inside a kernel ran out */
+    STREAMBP_E_DEVICE_TIMEOUT = -9,  /* device: a bounded wait inside a kernel ran out */
+    STREAMBP_E_WORKSPACE_GUARD = -10 /* device, debug mode STREAMBP_WS_GUARD: a kernel wrote past a workspace sub-buffer */
 } streambp_status;
 
 typedef enum { STREAMBP_F32 = 0, STREAMBP_BF16 = 1 } streambp_dtype;
@@ -398,8 +403,14 @@ int streambp_product_kernel(void);
  * streambp_test_per_device_value: the library caches per-device facts (SM count, shared-memory opt-in, product
  * kernel choice) by device ordinal.  This runs that cache with `ordinal` in place of the current device and a
  * value to remember on first use: it returns the value cached for that ordinal.  Host-only.
+ *
+ * streambp_test_workspace_guard: plans three sub-buffers with guards in `workspace` (>= 4096 bytes, 256-byte
+ * aligned; guards are used here whether or not STREAMBP_WS_GUARD is set), fills the guards, has a kernel write
+ * `overrun` floats past the end of the second sub-buffer (0: none), checks the guards and records the outcome in the
+ * workspace header: afterwards streambp_last_device_status is STREAMBP_OK or STREAMBP_E_WORKSPACE_GUARD.
  */
 int streambp_test_expire_wait(uint64_t limit_ns, void *cuda_stream);
+int streambp_test_workspace_guard(void *workspace, size_t workspace_bytes, int32_t overrun, void *cuda_stream);
 int streambp_test_per_device_value(int ordinal, int value);
 
 #ifdef __cplusplus

@@ -19,7 +19,8 @@ LIB_PATH = os.path.join(_HERE, "libstreambp.so")
 
 STREAMBP_F32, STREAMBP_BF16 = 0, 1
 OK = 0
-E_NULL, E_SHAPE, E_ALIGN, E_WORKSPACE, E_DTYPE, E_CUDA, E_BAD_LABEL, E_NO_VALID_LABELS, E_DEVICE_TIMEOUT = range(-1, -10, -1)
+E_NULL, E_SHAPE, E_ALIGN, E_WORKSPACE, E_DTYPE, E_CUDA, E_BAD_LABEL, E_NO_VALID_LABELS, E_DEVICE_TIMEOUT, \
+    E_WORKSPACE_GUARD = range(-1, -11, -1)
 OP_NT, OP_NN, OP_TN = 0, 1, 2
 
 WEIGHT_FIELDS = ("g1", "wq", "bq", "wk", "bk", "wv", "bv", "wo", "g2", "w_gate", "w_up", "w_down")
@@ -35,7 +36,7 @@ EXPORTS = (
     "streambp_attention_forward", "streambp_attention_backward", "streambp_attention_backward_static",
     "streambp_lmhead_rl_backward", "streambp_layer_backward_packed",
     "streambp_test_expire_wait", "streambp_test_per_device_value",
-    "streambp_layer_workspace_bytes_grouped", "streambp_layer_backward_grouped",
+    "streambp_layer_workspace_bytes_grouped", "streambp_layer_backward_grouped", "streambp_test_workspace_guard",
 )
 
 
@@ -149,6 +150,8 @@ def lib() -> C.CDLL:
     L.streambp_profile_read.argtypes = [C.c_int, C.POINTER(C.c_double), C.POINTER(i64), C.POINTER(C.c_double)]
     L.streambp_test_expire_wait.restype = C.c_int
     L.streambp_test_expire_wait.argtypes = [C.c_uint64, vp]
+    L.streambp_test_workspace_guard.restype = C.c_int
+    L.streambp_test_workspace_guard.argtypes = [vp, sz, i32, vp]
     L.streambp_test_per_device_value.restype = C.c_int
     L.streambp_test_per_device_value.argtypes = [C.c_int, C.c_int]
     _lib = L

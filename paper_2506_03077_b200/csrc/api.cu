@@ -4,9 +4,21 @@
 #include <cstring>
 #include <vector>
 
+#include <cstdio>
+
+#include <nvtx3/nvToolsExt.h>
+
 #include "common.cuh"
 
 namespace sbp {
+
+NvtxRange::NvtxRange(const char *name) { nvtxRangePushA(name); }
+NvtxRange::NvtxRange(const char *name, long long index) {
+    char buf[64];
+    std::snprintf(buf, sizeof(buf), "%s %lld", name, index);
+    nvtxRangePushA(buf);
+}
+NvtxRange::~NvtxRange() { nvtxRangePop(); }
 
 CallState &call_state() {
     static thread_local CallState s;
@@ -50,6 +62,11 @@ int gemm_engine() {
         return 0;
     }();
     return engine;
+}
+
+bool ws_guard_enabled() {
+    static const bool on = std::getenv("STREAMBP_WS_GUARD") != nullptr;
+    return on;
 }
 
 int current_device_ordinal() {
@@ -516,6 +533,7 @@ const char *streambp_status_string(int s) {
         case STREAMBP_E_BAD_LABEL: return "label or token id out of range";
         case STREAMBP_E_NO_VALID_LABELS: return "no unmasked label";
         case STREAMBP_E_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+        case STREAMBP_E_WORKSPACE_GUARD: return "a kernel wrote past a workspace sub-buffer (guard overwritten)";
         default: return "unknown status";
     }
 }
@@ -582,6 +600,15 @@ int streambp_test_expire_wait(uint64_t limit_ns, void *cuda_stream) {
     call_state().cuda_error = 0;
     call_state().launches = 0;
     return wait_probe_launch(limit_ns, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int streambp_test_workspace_guard(void *workspace, size_t workspace_bytes, int32_t overrun, void *cuda_stream) {
+    if (!workspace) return STREAMBP_E_NULL;
+    if (!aligned(workspace, 256)) return STREAMBP_E_ALIGN;
+    if (overrun < 0 || overrun > 64) return STREAMBP_E_SHAPE;
+    call_state().cuda_error = 0;
+    call_state().launches = 0;
+    return ws_guard_selftest(workspace, workspace_bytes, overrun, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int streambp_test_per_device_value(int ordinal, int value) {

@@ -6,6 +6,7 @@
 #include <stdint.h>
 
 #include <mutex>
+#include <vector>
 
 #include "../../include/streambp.h"
 
@@ -75,6 +76,17 @@ public:
         int _st = (expr);                     \
         if (_st != STREAMBP_OK) return _st;   \
     } while (0)
+
+// ---- NVTX ranges -----------------------------------------------------------------------
+// Host-side ranges around every call, chunk and phase of the schedulers, visible in a timeline profiler
+// (header-only NVTX: without a profiler attached a range costs a null-pointer check).
+struct NvtxRange {
+    explicit NvtxRange(const char *name);
+    NvtxRange(const char *name, long long index);     // "name index"
+    ~NvtxRange();
+    NvtxRange(const NvtxRange &) = delete;
+    NvtxRange &operator=(const NvtxRange &) = delete;
+};
 
 // ---- optional per-class device timing (off by default) -----------------------------
 // When enabled through streambp_profile_enable(), every product and attention launch is bracketed
@@ -205,19 +217,36 @@ __device__ __forceinline__ void set_status(WsHeader *h, int st, int detail) {
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Bump allocator over the caller's workspace; also used (with base == nullptr) to plan sizes.
+// Debug mode (environment STREAMBP_WS_GUARD set, read once per process): every sub-buffer is followed by a
+// 256-byte guard that the schedulers fill with a pattern before the first launch of a call and check after the
+// last one; a kernel that wrote past the end of its sub-buffer shows up as STREAMBP_E_WORKSPACE_GUARD in
+// streambp_last_device_status (detail = index of the sub-buffer).  The stand-in for a memory checker on a pool
+// where none can be run.  Workspace sizes grow accordingly, consistently in the size queries and in the calls.
+bool ws_guard_enabled();
+constexpr size_t kGuardBytes = 256;
 struct Arena {
     char *base;
     size_t off;
-    explicit Arena(void *b) : base(static_cast<char *>(b)), off(0) {}
+    std::vector<size_t> guards;     // byte offsets of the guards (debug mode only)
+    bool guarded;
+    explicit Arena(void *b) : base(static_cast<char *>(b)), off(0), guarded(ws_guard_enabled()) {}
     template <typename T> T *take(size_t count) {
         off = align_up(off, 256);
         T *p = base ? reinterpret_cast<T *>(base + off) : nullptr;
         off += count * sizeof(T);
+        if (guarded) {      // the guard starts right behind the last element (rounded up to a word), not at the next boundary
+            off = align_up(off, 4);
+            guards.push_back(off);
+            off += kGuardBytes;
+        }
         return p;
     }
     void *take_bytes(size_t bytes) { return take<char>(bytes); }
     size_t size() const { return align_up(off, 256); }
 };
+// Fill / check the guards of a planned workspace (no-ops when the list is empty).
+int ws_guards_arm(void *base, const std::vector<size_t> &guards, cudaStream_t st);
+int ws_guards_check(void *base, const std::vector<size_t> &guards, WsHeader *hdr, cudaStream_t st);
 
 // ---- internal kernels (host launchers); T = storage dtype -----------------------
 enum GemmOp { OP_NT = 0, OP_NN = 1, OP_TN = 2 };
@@ -314,6 +343,7 @@ int cast_from_f32(const float *in, int64_t n, T *out, cudaStream_t st);
 template <typename T>
 int add_cast(const float *a, const float *b, int64_t n, T *out, cudaStream_t st);
 int fill_zero(void *p, size_t bytes, cudaStream_t st);
+int ws_guard_selftest(void *ws, size_t bytes, int overrun, cudaStream_t st);
 
 // Attention of one chunk of queries against the key/value prefix [0, q0 + n).
 // q,o,do: [n, Hq, dh]; k,v: [q0+n, Hkv, dh]; query row i sits at absolute row q0 + i and sees keys <= q0 + i.

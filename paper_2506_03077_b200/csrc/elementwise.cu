@@ -1,6 +1,8 @@
 // HBM-bound steps of the streamed backward: RMSNorm forward/backward, RoPE, SwiGLU,
 // column sums, casts, cross-entropy rows, embedding gather / scatter-add.
 // All kernels move 16 bytes per thread per access and reduce rows with warp shuffles.
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace sbp {
@@ -454,6 +456,66 @@ int add_cast(const float *a, const float *b, int64_t n, T *out, cudaStream_t st)
 }
 template int add_cast<float>(const float *, const float *, int64_t, float *, cudaStream_t);
 template int add_cast<bf16>(const float *, const float *, int64_t, bf16 *, cudaStream_t);
+
+// ---- workspace guards (debug mode) ---------------------------------------------------------------
+namespace {
+constexpr int kGuardsPerLaunch = 48;
+struct GuardList {
+    unsigned long long off[kGuardsPerLaunch];
+    int first, n;
+};
+__device__ __forceinline__ uint32_t guard_word(int guard, int word) { return 0xA5C3F00Du ^ ((uint32_t)guard * 2654435761u) ^ (uint32_t)word; }
+__global__ void guards_arm_kernel(char *base, GuardList g) {
+    uint32_t *p = reinterpret_cast<uint32_t *>(base + g.off[blockIdx.x]);
+    p[threadIdx.x] = guard_word(g.first + blockIdx.x, threadIdx.x);
+}
+__global__ void guards_check_kernel(const char *base, GuardList g, WsHeader *hdr) {
+    const uint32_t *p = reinterpret_cast<const uint32_t *>(base + g.off[blockIdx.x]);
+    if (p[threadIdx.x] != guard_word(g.first + blockIdx.x, threadIdx.x)) set_status(hdr, STREAMBP_E_WORKSPACE_GUARD, g.first + blockIdx.x);
+}
+template <typename F>
+int for_guard_batches(const std::vector<size_t> &guards, F launch) {
+    for (size_t i = 0; i < guards.size(); i += kGuardsPerLaunch) {
+        GuardList g;
+        g.first = (int)i;
+        g.n = (int)std::min<size_t>(kGuardsPerLaunch, guards.size() - i);
+        for (int k = 0; k < g.n; k++) g.off[k] = guards[i + k];
+        SBP_TRY(launch(g));
+    }
+    return STREAMBP_OK;
+}
+}  // namespace
+
+int ws_guards_arm(void *base, const std::vector<size_t> &guards, cudaStream_t st) {
+    return for_guard_batches(guards, [&](const GuardList &g) -> int {
+        SBP_LAUNCH(guards_arm_kernel, g.n, (int)(kGuardBytes / 4), 0, st, static_cast<char *>(base), g);
+        return (int)STREAMBP_OK;
+    });
+}
+int ws_guards_check(void *base, const std::vector<size_t> &guards, WsHeader *hdr, cudaStream_t st) {
+    return for_guard_batches(guards, [&](const GuardList &g) -> int {
+        SBP_LAUNCH(guards_check_kernel, g.n, (int)(kGuardBytes / 4), 0, st, static_cast<const char *>(base), g, hdr);
+        return (int)STREAMBP_OK;
+    });
+}
+
+// test hook: `overrun` floats written past the end of a buffer of `count` floats
+__global__ void overrun_kernel(float *buf, int count, int overrun) {
+    for (int i = threadIdx.x; i < count + overrun; i += blockDim.x) buf[i] = 1.f;
+}
+int ws_guard_selftest(void *ws, size_t bytes, int overrun, cudaStream_t st) {
+    if (bytes < 4096) return STREAMBP_E_WORKSPACE;
+    Arena a(ws);
+    a.guarded = true;
+    WsHeader *hdr = reinterpret_cast<WsHeader *>(a.take_bytes(kHeaderBytes));
+    float *b0 = a.take<float>(100), *b1 = a.take<float>(77), *b2 = a.take<float>(64);
+    (void)b0; (void)b2;
+    if (a.size() > bytes) return STREAMBP_E_WORKSPACE;
+    SBP_TRY(fill_zero(ws, kHeaderBytes, st));
+    SBP_TRY(ws_guards_arm(ws, a.guards, st));
+    SBP_LAUNCH(overrun_kernel, 1, 128, 0, st, b1, 77, overrun);
+    return ws_guards_check(ws, a.guards, hdr, st);
+}
 
 int fill_zero(void *p, size_t bytes, cudaStream_t st) {
     if (bytes == 0 || p == nullptr) return STREAMBP_OK;

@@ -44,6 +44,7 @@ struct LayerWs {
     float *fa, *r, *dr, *rstd1, *rstd2, *lse, *delta, *partials;
     size_t bytes;
     int slots;            // chunks per weight-gradient group
+    std::vector<size_t> guards;   // debug mode: offsets of the guards behind the sub-buffers
 };
 
 // `wg` >= 1 is the number of consecutive chunks whose weight-gradient products are summed in ONE pass over the
@@ -93,7 +94,8 @@ LayerWs<T> plan(const streambp_layer_cfg &c, int64_t T_, int64_t chunk, void *ba
         w.dr = a.take<float>(cn * d);
         // dm = dY Wd lives only from its product to the SwiGLU backward, while dr_s, dO, dk_s, dv_s, fa and dr are all
         // dead: it is laid over that span when it fits (it does for every LLM-shaped layer), else it gets its own block
-        if (a.off - dead_begin >= (size_t)(cn * I) * sizeof(T))
+        // (not in the guarded debug mode: the overlay would run over the guards of the buffers it covers)
+        if (!a.guarded && a.off - dead_begin >= (size_t)(cn * I) * sizeof(T))
             w.dm = a.base ? reinterpret_cast<T *>(a.base + dead_begin) : nullptr;
         else
             w.dm = a.take<T>(cn * I);
@@ -105,6 +107,7 @@ LayerWs<T> plan(const streambp_layer_cfg &c, int64_t T_, int64_t chunk, void *ba
     w.delta = a.take<float>(cn * c.n_q_heads);
     w.partials = a.take<float>(64 * wide);
     w.bytes = a.size();
+    w.guards = a.guards;
     return w;
 }
 
@@ -188,6 +191,7 @@ int layer_forward(const streambp_layer_cfg &c, const streambp_layer_weights &w, 
     const SchedScope sched(s.hdr);
     const int d = c.d_model;
     const int64_t I = c.d_ff;
+    SBP_TRY(ws_guards_arm(ws, s.guards, st));
     SBP_TRY(kv_prologue<T>(c, w, X, T_, cn, pos0, seg, s, st));
     for (int64_t r0 = 0; r0 < T_; r0 += cn) {
         const int64_t n = (T_ - r0 < cn) ? T_ - r0 : cn;
@@ -195,13 +199,14 @@ int layer_forward(const streambp_layer_cfg &c, const streambp_layer_weights &w, 
         SBP_TRY((mm<T, float>(OP_NT, n, d, I, s.m, I, (const T *)w.w_down, I, s.fa, d, nullptr, false, st)));
         SBP_TRY(add_cast<T>(s.r, s.fa, n * d, Y + r0 * d, st));
     }
-    return STREAMBP_OK;
+    return ws_guards_check(ws, s.guards, s.hdr, st);
 }
 
 template <typename T>
 int layer_backward(const streambp_layer_cfg &c, const streambp_layer_weights &w, const T *X, const T *dY, int64_t T_,
                    int64_t chunk, int64_t pos0, bool accumulate, const streambp_layer_grads &G, T *dX, void *ws,
                    cudaStream_t st, const int64_t *cu_seqlens, int n_seqs, int wgrad_group) {
+    const NvtxRange call_range("streambp layer backward");
     const Segments seg(cu_seqlens, n_seqs, T_);
     const int64_t cn = chunk < T_ ? chunk : T_;
     LayerWs<T> base = plan<T>(c, T_, chunk, ws, wgrad_group);
@@ -210,7 +215,11 @@ int layer_backward(const streambp_layer_cfg &c, const streambp_layer_weights &w,
     const int64_t dq = (int64_t)Hq * dh, dkv = (int64_t)Hkv * dh, I = c.d_ff;
     constexpr bool kF32 = sizeof(T) == 4;
 
-    SBP_TRY(kv_prologue<T>(c, w, X, T_, cn, pos0, seg, base, st));
+    SBP_TRY(ws_guards_arm(ws, base.guards, st));
+    {
+        const NvtxRange r("K/V prologue");
+        SBP_TRY(kv_prologue<T>(c, w, X, T_, cn, pos0, seg, base, st));
+    }
     SBP_TRY(fill_zero(base.dK, sizeof(float) * T_ * dkv, st));
     SBP_TRY(fill_zero(base.dV, sizeof(float) * T_ * dkv, st));
     if (!accumulate) {  // vectors are always added to; matrices are overwritten by the first group's product
@@ -228,6 +237,7 @@ int layer_backward(const streambp_layer_cfg &c, const streambp_layer_weights &w,
         // Chunks are grouped from the end: {D-1 .. D-k}, {D-k-1 .. D-2k}, ...  The weight-gradient products of a
         // group run once, when its first chunk (the last one processed) is done, over all the group's rows: the
         // operands of a group are contiguous in row order (X, dY in the caller's arrays, the rest in the slots).
+        const NvtxRange chunk_range("chunk", i);
         const int64_t g_hi = D - 1 - ((D - 1 - i) / k) * k, g_lo = g_hi - k + 1 > 0 ? g_hi - k + 1 : 0;
         const bool group_done = i == g_lo;
         const int64_t r0 = i * cn, gr0 = g_lo * cn;
@@ -236,7 +246,11 @@ int layer_backward(const streambp_layer_cfg &c, const streambp_layer_weights &w,
         const bool acc = accumulate || g_hi != D - 1;
         const T *Xi = X + r0 * d, *dYi = dY + r0 * d, *dYg = dY + gr0 * d;
         LayerWs<T> s = at_slot<T>(base, c, r0 - gr0);
-        SBP_TRY(chunk_forward<T>(c, w, X, r0, n, seg, s, st));
+        {
+            const NvtxRange r("re-forward");
+            SBP_TRY(chunk_forward<T>(c, w, X, r0, n, seg, s, st));
+        }
+        const NvtxRange bwd_range("backward");
 
         // ---- MLP backward ----
         SBP_TRY((mm<T, T>(OP_NN, n, I, d, dYi, d, (const T *)w.w_down, I, s.dm, I, nullptr, false, st)));  // dm = dY Wd
@@ -304,7 +318,7 @@ int layer_backward(const streambp_layer_cfg &c, const streambp_layer_weights &w,
         SBP_TRY(rmsnorm_bwd<T>(s.fa, Xi, nullptr, s.rstd1, (const T *)w.g1, nullptr, s.dr, n, d, nullptr, dX + r0 * d,
                                G.g1, s.partials, st));
     }
-    return STREAMBP_OK;
+    return ws_guards_check(ws, base.guards, base.hdr, st);
 }
 
 template size_t layer_workspace<float>(const streambp_layer_cfg &, int64_t, int64_t, int);

@@ -12,6 +12,7 @@ struct HeadWs {
     float *z, *dhn, *rstd, *row_loss, *partials;
     int *chunk_valid;     // [number of chunks] unmasked labels per chunk: the device-side gate of each chunk
     size_t bytes;
+    std::vector<size_t> guards;   // debug mode: offsets of the guards behind the sub-buffers
 };
 
 template <typename T>
@@ -31,6 +32,7 @@ HeadWs<T> plan(const streambp_head_cfg &c, int64_t T_, int64_t chunk, void *base
     w.partials = a.take<float>(64 * d);
     w.chunk_valid = a.take<int>((T_ + cn - 1) / cn);
     w.bytes = a.size();
+    w.guards = a.guards;
     return w;
 }
 }  // namespace
@@ -44,11 +46,13 @@ template <typename T>
 int lmhead_backward(const streambp_head_cfg &c, const T *g_final, const T *w_vocab, const T *H, const int64_t *labels,
                     int64_t T_, int64_t chunk, bool accumulate, float *loss, int64_t *n_valid, T *dH, float *d_w_vocab,
                     float *d_g_final, void *ws, cudaStream_t st, const RlRows *rl, float *ell) {
+    const NvtxRange call_range(rl ? "streambp lm-head RL backward" : "streambp lm-head CE backward");
     const int64_t cn = chunk < T_ ? chunk : T_;
     HeadWs<T> s = plan<T>(c, T_, chunk, ws);
     const SchedScope sched(s.hdr);
     const int d = c.d_model;
     const int64_t V = c.vocab;
+    SBP_TRY(ws_guards_arm(ws, s.guards, st));
     // N is global: it is counted before the chunk loop so that every chunk scales by the same 1/N
     SBP_TRY(count_valid_labels(labels, T_, V, c.ignore_index, s.hdr, st));
     SBP_TRY(count_valid_per_chunk(labels, T_, cn, c.ignore_index, s.chunk_valid, st));
@@ -66,6 +70,7 @@ int lmhead_backward(const streambp_head_cfg &c, const T *g_final, const T *w_voc
         ~GateScope() { call_state().gate = nullptr; }
     };
     for (int64_t i = 0; i < D; i++) {
+        const NvtxRange chunk_range("chunk", i);
         const int64_t r0 = i * cn;
         const int64_t n = (T_ - r0 < cn) ? T_ - r0 : cn;
         const bool acc = true;
@@ -88,7 +93,7 @@ int lmhead_backward(const streambp_head_cfg &c, const T *g_final, const T *w_voc
     }
     if (!rl) {
         SBP_TRY(loss_finalize(s.hdr, loss, n_valid, st));
-        return STREAMBP_OK;
+        return ws_guards_check(ws, s.guards, s.hdr, st);
     }
     SBP_TRY(rl_finalize(s.hdr, rl->objective, rl->beta, loss, ell, st));
     if (rl->objective == STREAMBP_OBJ_DPO) {
@@ -97,7 +102,7 @@ int lmhead_backward(const streambp_head_cfg &c, const T *g_final, const T *w_voc
         SBP_TRY(scale_by_factor<float>(d_g_final, d, s.hdr, st));
         SBP_TRY(scale_by_factor<T>(dH, T_ * d, s.hdr, st));
     }
-    return STREAMBP_OK;
+    return ws_guards_check(ws, s.guards, s.hdr, st);
 }
 
 template size_t lmhead_workspace<float>(const streambp_head_cfg &, int64_t, int64_t);

@@ -13,6 +13,7 @@ struct ModelWs {
     T *ga, *gb;   // [T, d] ping-pong buffers for the gradient travelling down the stack
     void *sub;    // workspace shared (in turn) by the layer forward, the head and the layer backward
     size_t sub_bytes, bytes;
+    std::vector<size_t> guards;   // debug mode: offsets of the guards behind the sub-buffers
 };
 
 template <typename T>
@@ -28,6 +29,7 @@ ModelWs<T> plan(const streambp_model_cfg &c, int64_t T_, int64_t chunk_layer, in
     w.sub_bytes = lb > hb ? lb : hb;
     w.sub = a.take_bytes(w.sub_bytes);
     w.bytes = a.size();
+    w.guards = a.guards;
     return w;
 }
 
@@ -54,10 +56,12 @@ int model_backward(const streambp_model_cfg &c, const T *embed, const streambp_l
                    int64_t chunk_layer, int64_t chunk_head, bool accumulate, float *loss, float *d_embed,
                    const streambp_layer_grads *layer_grads, float *d_g_final, float *d_w_vocab, T *dX0, void *ws,
                    cudaStream_t st) {
+    const NvtxRange call_range("streambp model backward");
     ModelWs<T> s = plan<T>(c, T_, chunk_layer, chunk_head, ws);
     const int d = c.layer.d_model;
     const int L = c.n_layers;
     const int64_t act = T_ * d;
+    SBP_TRY(ws_guards_arm(ws, s.guards, st));
     // layer 0 input
     if (ids) {
         SBP_TRY(embedding_gather<T>(embed, ids, T_, d, c.head.vocab, s.ckpt, s.hdr, st));
@@ -66,9 +70,11 @@ int model_backward(const streambp_model_cfg &c, const T *embed, const streambp_l
     }
     // forward, storing only layer inputs
     for (int l = 0; l < L; l++) {
+        const NvtxRange r("checkpointing forward, layer", l);
         SBP_TRY(fill_zero(s.sub, kHeaderBytes, st));
         SBP_TRY(layer_forward<T>(c.layer, layers[l], s.ckpt + (int64_t)l * act, T_, chunk_layer, 0,
                                  s.ckpt + (int64_t)(l + 1) * act, s.sub, st));
+        SBP_TRY(merge_status(s.hdr, s.sub, st));
     }
     // head
     SBP_TRY(fill_zero(s.sub, kHeaderBytes, st));
@@ -78,6 +84,7 @@ int model_backward(const streambp_model_cfg &c, const T *embed, const streambp_l
     // layers, last to first
     T *gin = s.ga, *gout = s.gb;
     for (int l = L - 1; l >= 0; l--) {
+        const NvtxRange r("layer", l);
         SBP_TRY(fill_zero(s.sub, kHeaderBytes, st));
         T *dst = (l == 0 && dX0 && !ids) ? dX0 : gout;
         SBP_TRY(layer_backward<T>(c.layer, layers[l], s.ckpt + (int64_t)l * act, gin, T_, chunk_layer, 0, accumulate,
@@ -94,7 +101,7 @@ int model_backward(const streambp_model_cfg &c, const T *embed, const streambp_l
     if (dX0 && gin != dX0) {
         if (!cuda_ok(cudaMemcpyAsync(dX0, gin, sizeof(T) * act, cudaMemcpyDeviceToDevice, st))) return STREAMBP_E_CUDA;
     }
-    return STREAMBP_OK;
+    return ws_guards_check(ws, s.guards, s.hdr, st);
 }
 
 template size_t model_workspace<float>(const streambp_model_cfg &, int64_t, int64_t, int64_t);

@@ -36,8 +36,8 @@ def test_every_declared_symbol_is_exported(lib):
 
 def test_status_strings(lib):
     assert B.status_string(0) == "ok"
-    seen = {B.status_string(s) for s in range(-9, 1)}
-    assert len(seen) == 10 and "unknown status" not in seen
+    seen = {B.status_string(s) for s in range(-10, 1)}
+    assert len(seen) == 11 and "unknown status" not in seen
     assert B.status_string(-77) == "unknown status"
 
 

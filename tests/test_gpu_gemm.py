@@ -262,3 +262,34 @@ def test_bounded_wait_runs_out_and_the_context_stays_usable():
     ref = A.double() @ Bm.double().T
     assert float((Cm.double() - ref).norm() / ref.norm()) < 1e-5
     assert B.last_device_status(ws) == B.OK
+
+
+def test_workspace_guards_catch_an_overrun():
+    """Debug mode STREAMBP_WS_GUARD puts a guard after every workspace sub-buffer, filled before and checked after each
+    call.  The hook runs that mechanism on three small sub-buffers: untouched guards -> OK; a kernel that writes one
+    float (or more) past the end of the second sub-buffer -> E_WORKSPACE_GUARD."""
+    ws = B.alloc_workspace(8192)
+    L = B.lib()
+    for overrun, want in ((0, B.OK), (1, B.E_WORKSPACE_GUARD), (40, B.E_WORKSPACE_GUARD), (0, B.OK)):
+        assert L.streambp_test_workspace_guard(ws.data_ptr(), ws.numel(), overrun, None) == B.OK
+        assert B.last_device_status(ws) == want, overrun
+    assert L.streambp_test_workspace_guard(ws.data_ptr(), 1024, 0, None) == B.E_WORKSPACE
+    assert L.streambp_test_workspace_guard(ws.data_ptr() + 4, ws.numel(), 0, None) == B.E_ALIGN
+
+
+def test_whole_path_is_clean_under_workspace_guards():
+    """Layer, packed, grouped, head (SFT / GRPO / DPO) and model calls in a fresh process with STREAMBP_WS_GUARD set:
+    every call's guards must be intact (device status OK) and the results must still match the oracle."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, STREAMBP_WS_GUARD="1")
+    sel = ["tests/test_gpu_layer.py::test_layer_bf16_matches_oracle", "tests/test_gpu_layer.py::test_layer_fp32_shapes",
+           "tests/test_gpu_layer.py::test_weight_gradients_summed_over_groups_of_chunks",
+           "tests/test_gpu_layer.py::test_grouped_packed_batch_matches_packed",
+           "tests/test_gpu_lmhead.py", "tests/test_gpu_rl_heads.py",
+           "tests/test_gpu_model.py::test_tiny_configuration_end_to_end_fp32", "tests/test_gpu_model.py::test_small_model_with_embedding"]
+    r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-m", "gpu", "-p", "no:cacheprovider"] + sel, cwd=root,
+                       env=env, capture_output=True, text=True, timeout=1500)
+    assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-2000:]
