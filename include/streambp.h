@@ -339,7 +339,12 @@ int streambp_gemm_swiglu(const void *A, int64_t lda, const void *w_gate, const v
  * delta: scratch [n_q_heads, n] fp32; dq: [n, n_q_heads, head_dim] fp32, overwritten;
  * dk, dv: [q0+n, n_kv_heads, head_dim] fp32, ADDED to (the key-prefix accumulators).
  * engine: 0 automatic, 1 CUDA cores, 2 tensor cores (bf16, head_dim 128 only); the forward also takes 3 / 4 =
- * tensor cores with one / two 128-query tiles per CTA (2 picks between them from the grid size).
+ * tensor cores with one / two 128-query tiles per CTA (2 picks between them from the grid size); the backward also
+ * takes 5 = the five-product tensor-core kernel: one CTA role, the key-tile owners also form dQ and add their
+ * shares into it in global memory (dq is cleared by the call), so S and dP are not recomputed by a second role.
+ * Its dQ is not bit-reproducible from run to run (the order of those adds is not fixed; dK and dV are), which is
+ * why the deterministic two-role kernel stays the default.  Environment STREAMBP_ATTN_BWD=five makes the
+ * five-product kernel the choice of the schedulers (layer / model entry points) in this process.
  */
 int streambp_attention_forward(const void *q, const void *k, const void *v, int64_t n, int64_t q0,
                                int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, int32_t dtype,

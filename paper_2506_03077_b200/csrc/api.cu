@@ -208,12 +208,17 @@ template <>
 int attn_bwd<bf16>(const bf16 *q, const bf16 *k, const bf16 *v, const bf16 *o, const bf16 *dout, const float *lse,
                    int64_t n, int64_t q0, int Hq, int Hkv, int dh, float *delta, float *dq, float *dk, float *dv,
                    cudaStream_t st, int engine) {
+    static const bool five_default = [] {
+        const char *v = std::getenv("STREAMBP_ATTN_BWD");
+        return v && !std::strcmp(v, "five");
+    }();
     const int e = engine < 0 ? gemm_engine() : engine;
     if (e != 1 && attention_tc_supported(n, q0, Hq, Hkv, dh, q, k, v)) {
         SBP_TRY(attention_delta<bf16>(o, dout, n, Hq, dh, delta, st));
-        return attention_bwd_tc(q, k, v, dout, lse, delta, n, q0, Hq, Hkv, dq, dk, dv, st);
+        return attention_bwd_tc(q, k, v, dout, lse, delta, n, q0, Hq, Hkv, dq, dk, dv, st,
+                                e == 5 || (engine < 0 && five_default));
     }
-    if (e == 2) return STREAMBP_E_SHAPE;
+    if (e == 2 || e == 5) return STREAMBP_E_SHAPE;
     return attention_bwd<bf16>(q, k, v, o, dout, lse, n, q0, Hq, Hkv, dh, delta, dq, dk, dv, st);
 }
 
@@ -582,13 +587,13 @@ int streambp_attention_backward(const void *q, const void *k, const void *v, con
     call_state().cuda_error = 0;
     call_state().launches = 0;
     if (dtype == STREAMBP_F32) {
-        if (engine == 2) return STREAMBP_E_DTYPE;
+        if (engine == 2 || engine == 5) return STREAMBP_E_DTYPE;
         return attention_bwd<float>((const float *)q, (const float *)k, (const float *)v, (const float *)o,
                                     (const float *)d_o, lse, n, q0, n_q_heads, n_kv_heads, head_dim, delta, dq, dk, dv,
                                     st);
     }
     if (dtype != STREAMBP_BF16) return STREAMBP_E_DTYPE;
-    if (engine < 0 || engine > 2) return STREAMBP_E_SHAPE;
+    if (engine < 0 || (engine > 2 && engine != 5)) return STREAMBP_E_SHAPE;
     return attn_bwd<bf16>((const bf16 *)q, (const bf16 *)k, (const bf16 *)v, (const bf16 *)o, (const bf16 *)d_o, lse, n,
                           q0, n_q_heads, n_kv_heads, head_dim, delta, dq, dk, dv, st, engine);
 }

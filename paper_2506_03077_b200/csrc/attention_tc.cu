@@ -1046,6 +1046,399 @@ __device__ __forceinline__ void attn_bwd_dq_body(const CUtensorMap &map_q, const
     }
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Five-product backward: the key-tile owners also form dQ.  One role only (the dK/dV role above plus one
+// product): per tile pair dQ^T_partial = K^T dS^T lands in the dP^T region once dV and dK have read P^T and dS^T
+// from it, four drain warps add it into the fp32 dQ in global memory (L2-resident: [chunk, Hq, 128] floats), and
+// the region then takes dP^T of the next iteration.  dS^T reaches that product through shared memory (the softmax
+// warps write their row segments in the swizzled tile layout), next to its packed copy in tensor memory for dK.
+// Five executed products per tile pair instead of seven.  The adds of different key tiles into one dQ tile arrive in
+// whatever order the CTAs run, so dQ is NOT bit-reproducible from run to run (dK and dV are): an opt-in variant,
+// not what the layer uses.  Measured (2048 queries, 16384-key prefix, back to back for seconds at the power limit):
+// 1.73 ms per call against 1.81 ms for the two-role kernel; 1.54 vs 1.57 ms in a burst.  An iteration takes ~5900
+// cycles here against ~3200 + ~2550 for the two roles; what bounds it is shared-memory traffic (~540 KB per
+// iteration: five products' operands, the incoming Q / dO tiles, dS^T and the drain's staging) and the rate at which
+// L2 takes the reduce-adds (64 KB per tile pair) while it also serves the K / V / Q / dO stream.
+// ---------------------------------------------------------------------------------------------
+constexpr int FUSED_QSTAGES = 2;
+constexpr int FUSED_DRAIN_WARP0 = 18;
+constexpr int FUSED_THREADS = (FUSED_DRAIN_WARP0 + 4) * 32;
+static_assert((5 + FUSED_QSTAGES) * TILE_BYTES + 4 * TILE * 4 + 256 + BWD_ALIGN_SLACK <= 232448, "fused role exceeds shared memory");
+
+__device__ __forceinline__ void attn_bwd_fused_body(const CUtensorMap &map_q, const CUtensorMap &map_k,
+                                                   const CUtensorMap &map_v, const CUtensorMap &map_do,
+                                                   const CUtensorMap &map_dq, const BwdParams &p, uint8_t *smem_raw, int block_x, int block_y) {
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    // K, V (resident), Q x 2, dO x 1 (its successor is fetched while dK, dQ and the drain run), dS^T, and 32 KiB of
+    // staging for the drain warps
+    const uint32_t sK = base, sV = sK + TILE_BYTES, sQ = sV + TILE_BYTES, sdO = sQ + FUSED_QSTAGES * TILE_BYTES,
+                   sdS = sdO + TILE_BYTES, sStage = sdS + TILE_BYTES;
+    uint8_t *tail = smem_raw + (base - raw) + (5 + FUSED_QSTAGES) * TILE_BYTES;
+    float *s_lse = reinterpret_cast<float *>(tail);           // [2][128], pre-multiplied by log2(e)
+    float *s_delta = s_lse + 2 * TILE;                        // [2][128], pre-multiplied by the score scale
+    uint8_t *aux = tail + 4 * TILE * 4;
+    const uint32_t bars = smem_u32(aux);
+    const uint32_t kv_full = bars, q_full = bars + 8, q_empty = bars + 32, do_full = bars + 56, do_empty = bars + 64,
+                   rows_full = bars + 72, rows_empty = bars + 88, s_full = bars + 104, dp_full = bars + 112, loaded = bars + 120,
+                   p1_full = bars + 128, p2_full = bars + 136, acc_full = bars + 144, dq_full = bars + 152,
+                   b_free = bars + 160, stage_free = bars + 168, p3_full = bars + 176;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux + 184);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(aux + 192);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = block_y, G = p.Hq / p.Hkv;
+    const long long k_abs0 = (long long)block_x * TILE;
+    const int nqt = (p.n + TILE - 1) / TILE;
+    const int first_qt = k_abs0 > p.q0 ? (int)((k_abs0 - p.q0) / TILE) : 0;
+    const int per_head = nqt - first_qt;
+    const int iters = G * per_head;
+    // CTAs that run at the same time (neighbouring key tiles) start their walk over the (head, query tile) pairs at
+    // different places, so that their adds into dQ do not all hit the same lines at once
+    const int rot = (int)(((long long)block_x * 37) % iters);
+
+    if (threadIdx.x == 0) {
+        mbar_init(kv_full, 1);
+        for (int s = 0; s < FUSED_QSTAGES; s++) {
+            mbar_init(q_full + 8 * s, 1);
+            mbar_init(q_empty + 8 * s, 1);
+        }
+        mbar_init(do_full, 1);
+        mbar_init(do_empty, 1);
+        for (int s = 0; s < 2; s++) {
+            mbar_init(rows_full + 8 * s, 1);
+            mbar_init(rows_empty + 8 * s, 1);
+        }
+        mbar_init(s_full, 1);
+        mbar_init(dp_full, 1);
+        mbar_init(loaded, 16);
+        mbar_init(p1_full, 16);
+        mbar_init(p2_full, 16);
+        mbar_init(acc_full, 1);
+        mbar_init(dq_full, 1);
+        mbar_init(b_free, 4);
+        mbar_init(p3_full, 16);
+        // the carve-out leaves at most 768 bytes for aligning the tiles to 1024: a base that needs more cannot be used
+        *abort_flag = (base - raw) > BWD_ALIGN_SLACK ? 1 : 0;
+        if (*abort_flag) atomicExch(&g_tc_fault, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    // columns: S^T at 0; dP^T at 128, later P^T (packed) in the first and dS^T (packed) in the second 16 columns of
+    // every 32-column group, and then this tile pair's dQ^T (head dims on the lanes); dV at 256, dK at 384
+    const uint32_t tST = tmem, tDPT = tmem + 128, tDV = tmem + 256, tDK = tmem + 384;
+    const bool usable = *abort_flag == 0;
+
+    if (!usable) {
+        // nothing was issued: fall through to the common exit
+    } else if (warp == 0) {
+        // ---- producer: K, V once; per iteration the dO tile with the lse / delta rows (two stages) and the Q tile
+        // (three stages: Q_i is read by S^T_i, which is issued a whole iteration ahead, and again by dK_i at the end)
+        if (lane == 0) {
+            mbar_expect_tx(kv_full, 2 * TILE_BYTES);
+            tma_load_2d(sK, &map_k, kv_full, g * TILE, (int)k_abs0);
+            tma_load_2d(sK + HALF_BYTES, &map_k, kv_full, g * TILE + 64, (int)k_abs0);
+            tma_load_2d(sV, &map_v, kv_full, g * TILE, (int)k_abs0);
+            tma_load_2d(sV + HALF_BYTES, &map_v, kv_full, g * TILE + 64, (int)k_abs0);
+        }
+        uint32_t sq = 0, qph = 0;
+        for (int it = 0; it < iters; it++) {
+            const int il = (it + rot) % iters, h = g * G + il / per_head, qt0 = (first_qt + il % per_head) * TILE;
+            const uint32_t sd = it & 1, dph = (it >> 1) & 1;
+            int ok = 1;
+            if (lane == 0) {
+                ok = mbar_wait(q_empty + 8 * sq, qph ^ 1u, abort_flag) ? 1 : 0;          // dK of the stage's last user
+                if (ok) {
+                    mbar_expect_tx(q_full + 8 * sq, TILE_BYTES);
+                    tma_load_2d(sQ + sq * TILE_BYTES, &map_q, q_full + 8 * sq, h * TILE, qt0);
+                    tma_load_2d(sQ + sq * TILE_BYTES + HALF_BYTES, &map_q, q_full + 8 * sq, h * TILE + 64, qt0);
+                    ok = mbar_wait(do_empty, (uint32_t)(it & 1) ^ 1u, abort_flag) ? 1 : 0;   // dV of the previous iteration
+                }
+                if (ok) {
+                    mbar_expect_tx(do_full, TILE_BYTES);
+                    tma_load_2d(sdO, &map_do, do_full, h * TILE, qt0);
+                    tma_load_2d(sdO + HALF_BYTES, &map_do, do_full, h * TILE + 64, qt0);
+                    ok = mbar_wait(rows_empty + 8 * sd, dph ^ 1u, abort_flag) ? 1 : 0;   // delta rows: read until dS^T is packed
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+#pragma unroll
+            for (int e = 0; e < 4; e++) {
+                const int col = lane * 4 + e, r = qt0 + col;
+                s_lse[sd * TILE + col] = r < p.n ? p.lse[(long long)h * p.n + r] * kLog2e : 0.f;
+                s_delta[sd * TILE + col] = r < p.n ? p.delta[(long long)h * p.n + r] * p.scale : 0.f;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(rows_full + 8 * sd);   // publishes the rows
+            if (++sq == FUSED_QSTAGES) { sq = 0; qph ^= 1u; }
+        }
+    }
+    else if (warp == 1) {
+        // the whole warp runs the issue loop; each MMA / commit executes in one elected lane
+        constexpr uint32_t idesc_kk = make_idesc(TILE, TILE, false, false);     // both operands K-major
+        constexpr uint32_t idesc_acc = make_idesc(TILE, TILE, false, true);     // B MN-major (N = head dims)
+        constexpr uint32_t idesc_tt = make_idesc(TILE, TILE, true, true);       // both MN-major (contraction along rows)
+        bool alive = mbar_wait_warp(kv_full, 0, abort_flag);
+        const uint32_t k_lo = klo(sK), v_lo = klo(sV), k_mn = mnlo(sK), ds_mn = mnlo(sdS);
+        uint32_t sq_s = 0, qph_s = 0;      // Q stage / phase of the next S^T
+        uint32_t sq_k = 0;                 // Q stage of the next dK
+        auto issue_st = [&]() -> bool {    // S^T = K Q^T for the next iteration
+            if (!mbar_wait_warp(q_full + 8 * sq_s, qph_s, abort_flag)) return false;
+            tc_fence_after();
+            const uint32_t q_lo = klo(sQ + sq_s * TILE_BYTES);
+#pragma unroll
+            for (int kk = 0; kk < 8; kk++) umma_ss_w(tST, k_lo + kstep(kk), q_lo + kstep(kk), idesc_kk, kk != 0);
+            umma_commit_w(s_full);
+            if (++sq_s == FUSED_QSTAGES) { sq_s = 0; qph_s ^= 1u; }
+            return true;
+        };
+        auto issue_dpt = [&](int it) -> bool {     // dP^T = V dO^T of iteration `it`
+            if (!mbar_wait_warp(do_full, it & 1, abort_flag)) return false;
+            tc_fence_after();
+            const uint32_t do_lo = klo(sdO);
+#pragma unroll
+            for (int kk = 0; kk < 8; kk++) umma_ss_w(tDPT, v_lo + kstep(kk), do_lo + kstep(kk), idesc_kk, kk != 0);
+            umma_commit_w(dp_full);
+            return true;
+        };
+        if (alive && iters > 0) alive = issue_st() && issue_dpt(0);
+        for (int it = 0; it < iters && alive; it++) {
+            const uint32_t sd = it & 1;
+            // the softmax warps hold S^T_it in registers: its columns take S^T of the next iteration at once
+            if (it + 1 < iters) {
+                if (!mbar_wait_warp(loaded, it & 1, abort_flag)) { alive = false; break; }
+                tc_fence_after();
+                if (!issue_st()) { alive = false; break; }
+            }
+            // dV += P^T dO as soon as P^T is packed (first 16 columns of each group of the dP^T region)
+            if (!mbar_wait_warp(p1_full, it & 1, abort_flag)) { alive = false; break; }
+            tc_fence_after();
+            const uint32_t do_mn = mnlo(sdO);
+#pragma unroll
+            for (int kk = 0; kk < 8; kk++)
+                umma_ts_w(tDV, tDPT + (kk >> 1) * 32 + (kk & 1) * 8, do_mn + mnstep(kk), idesc_acc, (it | kk) != 0);
+            umma_commit_w(do_empty);                     // dO is consumed (dP^T was issued earlier): fetch the next one
+            // dK += dS^T Q (second 16 columns of each group)
+            if (!mbar_wait_warp(p2_full, it & 1, abort_flag)) { alive = false; break; }
+            tc_fence_after();
+            const uint32_t q_mn = mnlo(sQ + sq_k * TILE_BYTES);
+#pragma unroll
+            for (int kk = 0; kk < 8; kk++)
+                umma_ts_w(tDK, tDPT + (kk >> 1) * 32 + 16 + (kk & 1) * 8, q_mn + mnstep(kk), idesc_acc, (it | kk) != 0);
+            umma_commit_w(q_empty + 8 * sq_k);           // Q of this stage is consumed
+            umma_commit_w(rows_empty + 8 * sd);          // and so are the lse / delta rows
+            if (++sq_k == FUSED_QSTAGES) sq_k = 0;
+            // this tile pair's share of dQ = dS K: both operands from shared memory with the contraction (the keys) along
+            // their rows; it overwrites the dP^T region, which dV and dK (queued before it) have read by then
+            if (!mbar_wait_warp(p3_full, it & 1, abort_flag)) { alive = false; break; }
+            tc_fence_after();
+#pragma unroll
+            for (int kk = 0; kk < 8; kk++)
+                umma_ss_w(tDPT, ds_mn + mnstep(kk), k_mn + mnstep(kk), idesc_tt, kk != 0);
+            umma_commit_w(dq_full);
+            // the drain warps have dQ^T in registers: the region takes dP^T of the next iteration
+            if (it + 1 < iters) {
+                if (!mbar_wait_warp(b_free, it & 1, abort_flag)) { alive = false; break; }
+                tc_fence_after();
+                if (!issue_dpt(it + 1)) { alive = false; break; }
+            }
+        }
+        if (alive) umma_commit_w(acc_full);
+    }
+    else if (warp >= FUSED_DRAIN_WARP0) {
+        // ---- drain warps: this tile pair's share of dQ from tensor memory into the fp32 dQ in global memory, added
+        // there by the copy engine (TMA reduce-add of 32 x 32 blocks staged in shared memory with the swizzle the
+        // tensor map expects).  A warp owns 32 query rows (its lane quarter) and walks the four 32-column blocks; the
+        // staging area is its own 8 KiB per warp: two rounds of two blocks, the second round's loads leave tensor memory
+        // free while the first round's blocks are still being read by the copy engine.
+        const int quarter = warp & 3;
+        const uint32_t tD = tDPT + ((uint32_t)(quarter * 32) << 16);
+        const uint32_t stage0 = sStage + (uint32_t)quarter * 8192u;     // two 4 KiB blocks per warp
+        bool alive = true;
+        for (int it = 0; it < iters && alive; it++) {
+            const int il = (it + rot) % iters, h = g * G + il / per_head, qt0 = (first_qt + il % per_head) * TILE;
+            if (!mbar_wait(dq_full, it & 1, abort_flag)) { alive = false; break; }
+            tc_fence_after();
+#pragma unroll 1
+            for (int half = 0; half < 2; half++) {
+                // 64 columns at a time: after the second load the whole block row is out of tensor memory
+                uint32_t r[64];
+                tmem_ld32_async(tD + half * 64, r);
+                tmem_ld32_async(tD + half * 64 + 32, r + 32);
+                tmem_wait_ld();
+                if (half == 1) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(b_free);
+                }
+                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // both staging blocks are free
+                __syncwarp();
+#pragma unroll
+                for (int c = 0; c < 2; c++) {
+                    const uint32_t buf_s = stage0 + c * 4096u;
+#pragma unroll
+                    for (int j = 0; j < 8; j++) {
+                        const uint32_t dst = buf_s + lane * 128 + ((j ^ (lane & 7)) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(r[32 * c + 4 * j]),
+                                     "r"(r[32 * c + 4 * j + 1]), "r"(r[32 * c + 4 * j + 2]), "r"(r[32 * c + 4 * j + 3]) : "memory");
+                    }
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) {
+                    tma_reduce_add_2d(&map_dq, stage0, h * TILE + half * 64, qt0 + quarter * 32);   // rows past the chunk are clipped
+                    tma_reduce_add_2d(&map_dq, stage0 + 4096u, h * TILE + half * 64 + 32, qt0 + quarter * 32);
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                }
+            }
+        }
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        __syncwarp();
+    } else {
+        const int quarter = warp & 3;
+        const int wg = (warp - 2) >> 2;                           // 0..3: 32-query group of the tile
+        const int col_base = wg * 32;
+        const int row = quarter * 32 + lane;                      // key row within the tile
+        const long long k_abs = k_abs0 + row;
+        const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+        // The group reads its 32 fp32 columns of S^T and of dP^T into registers, then writes the packed bf16 pairs
+        // of P^T over the first and of dS^T over the second 16 of ITS OWN dP^T columns; the MMA thread addresses
+        // each 16-query slice of those A operands separately.  S^T's columns are never written by these warps, so
+        // the product of the next iteration can refill them while this iteration's exponentials are computed.
+        const uint32_t tS_g = tST + col_base + lane_base, tP_g = tDPT + col_base + lane_base;
+        bool alive = true;
+        for (int it = 0; it < iters && alive; it++) {
+            const int qt0 = (first_qt + (it + rot) % iters % per_head) * TILE;
+            const uint32_t sd = it & 1;
+            if (!mbar_wait(s_full, it & 1, abort_flag)) { alive = false; break; }
+            tc_fence_after();
+            uint32_t rs[32];
+            tmem_ld32(tS_g, rs);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(loaded);
+            // the producer's lse / delta rows of this stage are published together with the dO tile
+            if (!mbar_wait(rows_full + 8 * sd, (it >> 1) & 1, abort_flag)) { alive = false; break; }
+            const long long q_abs0 = p.q0 + qt0;
+            const bool diag = k_abs0 + TILE - 1 > q_abs0;          // the tile pair holds masked (query, key) pairs
+            // query column c of the tile is visible to this key iff q_abs0 + c >= k_abs
+            const int first_col = (k_abs > q_abs0) ? (int)((k_abs - q_abs0) > TILE ? TILE : (k_abs - q_abs0)) : 0;
+            const float *lse2 = s_lse + sd * TILE + col_base, *dl = s_delta + sd * TILE + col_base;
+            // phase 1: P^T = exp2(S^T * scale - lse), all the dV product needs
+            float pv[32];
+#pragma unroll
+            for (int e = 0; e < 32; e += 4) {
+                const float4 l4 = *reinterpret_cast<const float4 *>(lse2 + e);
+                const float lv[4] = {l4.x, l4.y, l4.z, l4.w};
+#pragma unroll
+                for (int t = 0; t < 4; t++) {
+                    float x = fmaf(__uint_as_float(rs[e + t]), p.scale_log2, -lv[t]);
+                    if (diag && col_base + e + t < first_col) x = -INFINITY;
+                    pv[e + t] = fast_exp2(x);
+                }
+            }
+            // dP^T of this iteration was queued a whole iteration ago; its columns become P^T and dS^T
+            uint32_t pp[16];
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) pp[e / 2] = pack_bf16(pv[e], pv[e + 1]);
+            if (!mbar_wait(dp_full, it & 1, abort_flag)) { alive = false; break; }
+            tc_fence_after();
+            uint32_t rp[32];
+            tmem_ld32(tP_g, rp);
+            {
+                tmem_st16(tP_g, pp);
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(p1_full);
+            }
+            // phase 2: dS^T = P^T * (dP^T * scale - delta * scale)
+            {
+                uint32_t ds[16];
+#pragma unroll
+                for (int e = 0; e < 32; e += 4) {
+                    const float4 d4 = *reinterpret_cast<const float4 *>(dl + e);
+                    const float dv[4] = {d4.x, d4.y, d4.z, d4.w};
+                    float dsv[4];
+#pragma unroll
+                    for (int t = 0; t < 4; t++) dsv[t] = pv[e + t] * fmaf(__uint_as_float(rp[e + t]), p.scale, -dv[t]);
+                    ds[e / 2] = pack_bf16(dsv[0], dsv[1]);
+                    ds[e / 2 + 1] = pack_bf16(dsv[2], dsv[3]);
+                }
+                tmem_st16(tP_g + 16, ds);
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(p2_full);          // dK may start; the dQ product waits for the copy below
+                // the same dS^T row segment into shared memory for dQ = dS K: [128 keys][128 queries] bf16 as two
+                // 64-query sub-tiles of 128-byte rows, 16-byte chunks swizzled by the row (what a TMA tile load leaves);
+                // the buffer is free once the previous iteration's dQ product has read it
+                if (it > 0 && !mbar_wait(dq_full, (it - 1) & 1, abort_flag)) { alive = false; break; }
+                {
+                    const uint32_t row_base = sdS + (uint32_t)(wg >> 1) * HALF_BYTES + (uint32_t)row * 128u;
+#pragma unroll
+                    for (int j = 0; j < 4; j++) {
+                        const uint32_t chunk = (uint32_t)((wg & 1) * 4 + j) ^ (uint32_t)(row & 7);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row_base + (chunk << 4)), "r"(ds[4 * j]),
+                                     "r"(ds[4 * j + 1]), "r"(ds[4 * j + 2]), "r"(ds[4 * j + 3]) : "memory");
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(p3_full);
+            }
+        }
+        if (alive && mbar_wait(acc_full, 0, abort_flag)) {
+            tc_fence_after();
+            const bool in_range = k_abs < p.q0 + p.n;
+            // group wg writes head dims 32*wg .. 32*wg+31
+            uint32_t rv[32], rk[32];
+            tmem_ld32(tDV + lane_base + col_base, rv);
+            tmem_ld32(tDK + lane_base + col_base, rk);
+            if (in_range) {
+                float *pv = p.dv + (k_abs * p.Hkv + g) * TILE + col_base;
+                float *pk = p.dk + (k_abs * p.Hkv + g) * TILE + col_base;
+#pragma unroll
+                for (int e = 0; e < 32; e += 4) {
+                    float4 a = *reinterpret_cast<float4 *>(pv + e);
+                    a.x += __uint_as_float(rv[e]); a.y += __uint_as_float(rv[e + 1]);
+                    a.z += __uint_as_float(rv[e + 2]); a.w += __uint_as_float(rv[e + 3]);
+                    *reinterpret_cast<float4 *>(pv + e) = a;
+                    float4 b = *reinterpret_cast<float4 *>(pk + e);
+                    b.x += __uint_as_float(rk[e]); b.y += __uint_as_float(rk[e + 1]);
+                    b.z += __uint_as_float(rk[e + 2]); b.w += __uint_as_float(rk[e + 3]);
+                    *reinterpret_cast<float4 *>(pk + e) = b;
+                }
+            }
+        }
+    }
+
+    __syncwarp();
+    abort_drain(abort_flag);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem, 512);
+    }
+}
+
+
+__global__ void __launch_bounds__(FUSED_THREADS, 1)
+    attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                          const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
+                          const __grid_constant__ CUtensorMap map_dq, const BwdParams p, int kv_tiles) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const int b = (int)blockIdx.x;
+    attn_bwd_fused_body(map_q, map_k, map_v, map_do, map_dq, p, smem_raw, b % kv_tiles, b / kv_tiles);
+}
+
 // One launch for both backward kernels.  They are independent (both read Q, K, V, dO, lse, delta; one owns dK / dV
 // tiles, the other dQ tiles), and at short prefixes or small chunks neither fills the GPU on its own (e.g. 32 to
 // 256 key-tile CTAs and 224 query-tile CTAs per chunk of the 7B layer at chunk 1024): as one grid their CTAs pack
@@ -1109,7 +1502,7 @@ int attention_fwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, int64_t n, int
 
 int attention_bwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, const bf16 *dout, const float *lse,
                      const float *delta, int64_t n, int64_t q0, int Hq, int Hkv, float *dq, float *dk, float *dv,
-                     cudaStream_t st) {
+                     cudaStream_t st, bool five_products) {
     CUtensorMap mq, mk, mv, mdo;
     const int64_t kv_len = q0 + n;
     if (!make_tensor_map(&mq, q, n, (int64_t)Hq * TILE, (int64_t)Hq * TILE, 64, TILE, false) ||
@@ -1124,6 +1517,15 @@ int attention_bwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, const bf16 *do
     const int kv_tiles = (int)((kv_len + TILE - 1) / TILE), q_tiles = (int)((n + TILE - 1) / TILE);
     const int64_t n_dkdv = (int64_t)kv_tiles * Hkv, n_dq = (int64_t)q_tiles * Hq;
     if (n_dkdv + n_dq > 0x7fffffff) return STREAMBP_E_SHAPE;
+    if (five_products) {
+        static PerDevice configured_f;
+        if (!configured_f.get([] { return opt_in_smem(attn_bwd_fused_kernel, BWD_SMEM) ? 1 : 0; })) return STREAMBP_E_CUDA;
+        CUtensorMap mdq;
+        if (!make_tensor_map(&mdq, dq, n, (int64_t)Hq * TILE, (int64_t)Hq * TILE, 32, 32, true)) return STREAMBP_E_CUDA;
+        if (!cuda_ok(cudaMemsetAsync(dq, 0, sizeof(float) * (size_t)n * Hq * TILE, st))) return STREAMBP_E_CUDA;
+        SBP_LAUNCH(attn_bwd_fused_kernel, (unsigned)n_dkdv, FUSED_THREADS, BWD_SMEM, st, mq, mk, mv, mdo, mdq, p, kv_tiles);
+        return STREAMBP_OK;
+    }
     SBP_LAUNCH(attn_bwd_tc_kernel, (unsigned)(n_dkdv + n_dq), BWD_THREADS, BWD_FUSED_SMEM, st, mq, mk, mv, mdo, p,
                kv_tiles, (int)n_dkdv, q_tiles);
     return STREAMBP_OK;

@@ -363,10 +363,11 @@ bool attention_tc_supported(int64_t n, int64_t q0, int Hq, int Hkv, int dh, cons
 // tiles_per_cta: 0 = chosen from the grid size, 1 / 2 = one / two 128-query tiles per CTA (tests, profiling)
 int attention_fwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, int64_t n, int64_t q0, int Hq, int Hkv, bf16 *o,
                      float *lse, cudaStream_t st, int tiles_per_cta = 0);
-// delta [Hq, n] must already hold rowsum(dO * O) (attention_delta below).
+// delta [Hq, n] must already hold rowsum(dO * O) (attention_delta below).  five_products: the single-role kernel
+// whose key-tile owners also form dQ and add it into global memory (dq is cleared first; not bit-reproducible).
 int attention_bwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, const bf16 *dout, const float *lse,
                      const float *delta, int64_t n, int64_t q0, int Hq, int Hkv, float *dq, float *dk, float *dv,
-                     cudaStream_t st);
+                     cudaStream_t st, bool five_products = false);
 template <typename T>
 int attention_delta(const T *o, const T *dout, int64_t n, int Hq, int dh, float *delta, cudaStream_t st);
 int attention_tc_take_fault();
@@ -380,7 +381,8 @@ bool attention_bwd_aligned(const void *q, const void *k, const void *v, const vo
 template <typename T>
 int attn_fwd(const T *q, const T *k, const T *v, int64_t n, int64_t q0, int Hq, int Hkv, int dh, T *o, float *lse,
              cudaStream_t st);
-// engine: -1 = the process-wide choice (gemm_engine()), else 0 / 1 / 2 as above for this call only.
+// engine: -1 = the process-wide choice (gemm_engine()), else 0 / 1 / 2 as above for this call only; 5 = tensor cores,
+// five-product kernel (the process-wide default of that choice: STREAMBP_ATTN_BWD=five).
 template <typename T>
 int attn_bwd(const T *q, const T *k, const T *v, const T *o, const T *dout, const float *lse, int64_t n, int64_t q0,
              int Hq, int Hkv, int dh, float *delta, float *dq, float *dk, float *dv, cudaStream_t st, int engine = -1);

@@ -86,7 +86,7 @@ def test_attention_forward_bf16(engine, n, q0, Hq, Hkv):
     assert np.abs(lse.cpu().numpy() - lse_ref).max() < 2e-3
 
 
-@pytest.mark.parametrize("engine", [1, 2])
+@pytest.mark.parametrize("engine", [1, 2, 5])          # CUDA cores; tensor cores: two-role kernel, five-product kernel
 @pytest.mark.parametrize("n,q0,Hq,Hkv", CASES)
 def test_attention_backward_bf16(engine, n, q0, Hq, Hkv):
     dh, dt = 128, torch.bfloat16
@@ -130,14 +130,15 @@ def test_attention_full_prefix_bf16(n, q0):
         torch.cuda.synchronize()
         assert_close(f"o (engine {engine})", o, o_ref, 6e-3, heads=Hq)
         assert torch.isfinite(lse).all()
-    dq = torch.full((n, Hq, dh), float("nan"), device="cuda")
-    dk = torch.zeros((kv, Hkv, dh), device="cuda")
-    dv = torch.zeros((kv, Hkv, dh), device="cuda")
-    B.attention_backward(qd, kd, vd, o, dod, lse, q0, dq, dk, dv, engine=2)
-    torch.cuda.synchronize()
-    assert_close("dq", dq, dq_ref, 1.5e-2, heads=Hq)
-    assert_close("dk", dk, dk_ref, 1.5e-2, heads=Hkv)
-    assert_close("dv", dv, dv_ref, 1.5e-2, heads=Hkv)
+    for engine in (2, 5):                  # the two-role kernel and the five-product kernel
+        dq = torch.full((n, Hq, dh), float("nan"), device="cuda")
+        dk = torch.zeros((kv, Hkv, dh), device="cuda")
+        dv = torch.zeros((kv, Hkv, dh), device="cuda")
+        B.attention_backward(qd, kd, vd, o, dod, lse, q0, dq, dk, dv, engine=engine)
+        torch.cuda.synchronize()
+        assert_close(f"dq (engine {engine})", dq, dq_ref, 1.5e-2, heads=Hq)
+        assert_close(f"dk (engine {engine})", dk, dk_ref, 1.5e-2, heads=Hkv)
+        assert_close(f"dv (engine {engine})", dv, dv_ref, 1.5e-2, heads=Hkv)
 
 
 @pytest.mark.parametrize("dh,dtype", [(64, torch.float32), (128, torch.float32), (64, torch.bfloat16)])
