@@ -73,3 +73,41 @@ def test_output_check_rejects_skipped_work():
         bench.check_outputs({"a": torch.zeros(4)})                       # a step that never wrote its output
     with pytest.raises(AssertionError):
         bench.check_outputs({"a": torch.tensor([1.0, float("nan")])})
+
+
+def test_roofline_object_names_the_dominant_class_and_carries_the_others():
+    """The roofline entry is the kernel class with the largest share of the step that was run; every class keeps its own
+    achieved rate; traffic is looked up per (config, chunk, class) and never silently absent."""
+    import copy
+    peaks = dict(hbm=6484.6, burst=1648.7, sustained=1392.7, source="measured")
+    steps = 4
+    # (milliseconds over all steps, launches, algorithmic FLOPs): attention backward is the largest here
+    prof = {"gemm": (4 * 30.0, 4 * 128, 4 * 39.0e12), "attention_fwd": (4 * 10.0, 4 * 16, 4 * 8.8e12),
+            "attention_bwd": (4 * 32.0, 4 * 16, 4 * 22.0e12)}
+    cfg = copy.copy(synth.CONFIGS["llama8b_layer"])
+    dom, classes, roof = bench.roofline_object(prof, steps, peaks, cfg, cfg.chunk, 4 * 78.0)
+    assert dom == "attention_bwd" and roof["class"] == "attention_bwd" and roof["bound"] == "tensor"
+    assert roof["achieved"] == pytest.approx(22.0e12 / 32.0e-3 / 1e12) and roof["frac"] == pytest.approx(roof["achieved"] / 1392.7)
+    assert set(roof["classes"]) == {"gemm", "attention_fwd", "attention_bwd"}
+    assert classes["gemm"]["tflops"] == pytest.approx(1300.0) and classes["gemm"]["launches_per_step"] == 128
+    assert roof["launches"] == 64 and roof["ms_per_step"] == pytest.approx(32.0)
+    # traffic: the captured 16384-key launch scaled to the step's average launch by algorithmic bytes
+    s = cfg.layer
+    ends = [min(cfg.T, r0 + cfg.chunk) for r0 in range(0, cfg.T, cfg.chunk)]
+    avg = sum(bench.attn_bwd_bytes(s, e, cfg.chunk) for e in ends) / len(ends)
+    assert roof["traffic"] == pytest.approx(488.6e6 * avg / bench.attn_bwd_bytes(s, 16384, 2048))
+    assert "profiles/" in roof["traffic_note"]
+    # products dominate on the short-sequence layer: the entry switches class; an uncaptured chunk says why it has no figure
+    prof2 = dict(prof, gemm=(4 * 40.0, 4 * 64, 4 * 40e12))
+    q = copy.copy(synth.CONFIGS["qwen7b_layer"])
+    dom2, _, roof2 = bench.roofline_object(prof2, steps, peaks, q, 512, 4 * 90.0)
+    assert dom2 == "gemm" and roof2["traffic"] is None and "no ncu capture" in roof2["traffic_note"]
+    _, _, roof3 = bench.roofline_object(prof2, steps, peaks, q, 1024, 4 * 90.0)
+    assert roof3["traffic"] == pytest.approx(2142.5e6)
+
+
+def test_attention_byte_model():
+    s = synth.LLAMA8B_LAYER
+    # K, V read (bf16), dK, dV read + written (fp32), Q, dO read (bf16), dQ written (fp32), lse and delta read
+    assert bench.attn_bwd_bytes(s, 16384, 2048) == 16384 * 1024 * (4 + 16) + 2048 * 4096 * (4 + 4) + 8 * 2048 * 32
+    assert bench.attn_fwd_bytes(s, 16384, 2048) == 16384 * 1024 * 4 + 2048 * 4096 * 4 + 4 * 2048 * 32
