@@ -359,7 +359,7 @@ int streambp_attention_backward(const void *q, const void *k, const void *v, con
  * to offer for `delta` and cannot obtain one when they call: host code in a latency-critical loop
  * where cudaMalloc / cudaFree would stall the whole device, a plug-in whose host framework already owns
  * all device memory, a process whose memory budget is frozen after start-up.  Same arguments and results
- * as streambp_attention_backward minus `delta`: the row sums live in a fixed array inside the library
+ * as streambp_attention_backward minus `delta` (engine 0, 1 or 2 only): the row sums live in a fixed array inside the library
  * image, STREAMBP_STATIC_DELTA_MAX_FLOATS floats (4 MiB) that every GPU loading the library holds until
  * the process exits.  The call performs no device-memory allocation of any kind.
  *   - Limit: n * n_q_heads <= STREAMBP_STATIC_DELTA_MAX_FLOATS, else STREAMBP_E_WORKSPACE is returned

@@ -55,6 +55,7 @@ extern "C" int streambp_attention_backward_static(const void *q, const void *k, 
     // the fixed scratch holds n_q_heads * n row sums: larger problems are refused, never truncated
     if (n > kMaxDeltaFloats / n_q_heads) return STREAMBP_E_WORKSPACE;
     if (dtype != STREAMBP_F32 && dtype != STREAMBP_BF16) return STREAMBP_E_DTYPE;
+    if (engine < 0 || engine > 2) return STREAMBP_E_SHAPE;      // 0 automatic, 1 CUDA cores, 2 tensor cores (two-role kernel)
     if (dtype == STREAMBP_F32 && engine == 2) return STREAMBP_E_DTYPE;
     // misaligned tensors are refused on the host: on the device they would fault and poison the context
     if (!attention_bwd_aligned(q, k, v, o, d_o, lse, nullptr, dq, dk, dv)) return STREAMBP_E_ALIGN;
