@@ -1083,7 +1083,7 @@ __device__ __forceinline__ void attn_bwd_fused_body(const CUtensorMap &map_q, co
     const uint32_t kv_full = bars, q_full = bars + 8, q_empty = bars + 32, do_full = bars + 56, do_empty = bars + 64,
                    rows_full = bars + 72, rows_empty = bars + 88, s_full = bars + 104, dp_full = bars + 112, loaded = bars + 120,
                    p1_full = bars + 128, p2_full = bars + 136, acc_full = bars + 144, dq_full = bars + 152,
-                   b_free = bars + 160, stage_free = bars + 168, p3_full = bars + 176;
+                   b_free = bars + 160, p3_full = bars + 176;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux + 184);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(aux + 192);
 
@@ -1095,7 +1095,8 @@ __device__ __forceinline__ void attn_bwd_fused_body(const CUtensorMap &map_q, co
     const int per_head = nqt - first_qt;
     const int iters = G * per_head;
     // CTAs that run at the same time (neighbouring key tiles) start their walk over the (head, query tile) pairs at
-    // different places, so that their adds into dQ do not all hit the same lines at once
+    // different places, so that their adds into dQ do not all go to the same tile at once (no measurable effect on
+    // the time; kept because it costs nothing)
     const int rot = (int)(((long long)block_x * 37) % iters);
 
     if (threadIdx.x == 0) {
@@ -1130,15 +1131,15 @@ __device__ __forceinline__ void attn_bwd_fused_body(const CUtensorMap &map_q, co
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
     // columns: S^T at 0; dP^T at 128, later P^T (packed) in the first and dS^T (packed) in the second 16 columns of
-    // every 32-column group, and then this tile pair's dQ^T (head dims on the lanes); dV at 256, dK at 384
+    // every 32-column group, and then this tile pair's share of dQ (queries on the lanes); dV at 256, dK at 384
     const uint32_t tST = tmem, tDPT = tmem + 128, tDV = tmem + 256, tDK = tmem + 384;
     const bool usable = *abort_flag == 0;
 
     if (!usable) {
         // nothing was issued: fall through to the common exit
     } else if (warp == 0) {
-        // ---- producer: K, V once; per iteration the dO tile with the lse / delta rows (two stages) and the Q tile
-        // (three stages: Q_i is read by S^T_i, which is issued a whole iteration ahead, and again by dK_i at the end)
+        // ---- producer: K, V once; per iteration the Q tile (two stages), the dO tile (one: its successor is fetched
+        // as soon as dV has read it) and the lse / delta rows (two stages)
         if (lane == 0) {
             mbar_expect_tx(kv_full, 2 * TILE_BYTES);
             tma_load_2d(sK, &map_k, kv_full, g * TILE, (int)k_abs0);
@@ -1242,7 +1243,7 @@ __device__ __forceinline__ void attn_bwd_fused_body(const CUtensorMap &map_q, co
             for (int kk = 0; kk < 8; kk++)
                 umma_ss_w(tDPT, ds_mn + mnstep(kk), k_mn + mnstep(kk), idesc_tt, kk != 0);
             umma_commit_w(dq_full);
-            // the drain warps have dQ^T in registers: the region takes dP^T of the next iteration
+            // the drain warps have the dQ share in registers: the region takes dP^T of the next iteration
             if (it + 1 < iters) {
                 if (!mbar_wait_warp(b_free, it & 1, abort_flag)) { alive = false; break; }
                 tc_fence_after();
