@@ -105,7 +105,10 @@ LayerWs<T> plan(const streambp_layer_cfg &c, int64_t T_, int64_t chunk, void *ba
     w.rstd2 = a.take<float>(cn);
     w.lse = a.take<float>(cn * c.n_q_heads);
     w.delta = a.take<float>(cn * c.n_q_heads);
-    w.partials = a.take<float>(64 * wide);
+    // reduction partials: up to 64 row splits of the widest row reduced -- a gain gradient (d) or, with biases, the
+    // three bias column sums of a chunk or group side by side (dq + 2 dkv)
+    const int64_t bias_cols = c.qkv_bias ? dq + 2 * dkv : 0;
+    w.partials = a.take<float>(64 * (bias_cols > wide ? bias_cols : wide));
     w.bytes = a.size();
     w.guards = a.guards;
     return w;

@@ -288,6 +288,7 @@ def test_whole_path_is_clean_under_workspace_guards():
     sel = ["tests/test_gpu_layer.py::test_layer_bf16_matches_oracle", "tests/test_gpu_layer.py::test_layer_fp32_shapes",
            "tests/test_gpu_layer.py::test_weight_gradients_summed_over_groups_of_chunks",
            "tests/test_gpu_layer.py::test_grouped_packed_batch_matches_packed",
+           "tests/test_gpu_layer.py::test_bias_column_sums_with_many_row_splits",
            "tests/test_gpu_lmhead.py", "tests/test_gpu_rl_heads.py",
            "tests/test_gpu_model.py::test_tiny_configuration_end_to_end_fp32", "tests/test_gpu_model.py::test_small_model_with_embedding"]
     r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-m", "gpu", "-p", "no:cacheprovider"] + sel, cwd=root,

@@ -72,6 +72,17 @@ def test_weight_gradients_summed_over_groups_of_chunks(dtype, T, chunk, group):
         assert w3 - w2 <= w2 - w1 + 4096 and w3 > w2
 
 
+def test_bias_column_sums_with_many_row_splits():
+    """Biases with dq + 2 dkv wider than the model width and a chunk long enough for the column sums to be split over
+    many row blocks: the reduction partials are (row splits) x (dq + 2 dkv) floats.  (The workspace plan once sized them
+    by the model width; the guarded debug mode found the overrun.  tests/test_gpu_gemm.py runs this case under guards.)"""
+    shape = synth.LayerShape(256, 2, 2, 128, 512, True, 1e6)
+    ocfg, bcfg, W, X, dY = layer_case(shape, 13, 1100, torch.bfloat16)
+    for chunk, group in ((1024, 1), (512, 2)):
+        dX, grads = run_layer(bcfg, W, X, dY, chunk, wgrad_group=group)
+        compare_layer(ocfg, W, X, dY, dX, grads, TOL[torch.bfloat16])
+
+
 def test_grouped_packed_batch_matches_packed():
     shape = synth.LayerShape(256, 4, 2, 128, 512, False, 1e6)
     ocfg, bcfg, W, X, dY = layer_case(shape, 12, 300, torch.bfloat16)
