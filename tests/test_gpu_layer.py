@@ -242,3 +242,67 @@ def test_data_parallel_runner_single_rank_matches_direct_call():
         assert torch.equal(full[k], g_ref[k])
     assert r.shard.numel() == r.bucket.total
 
+
+
+class _Fenced:
+    """A device tensor with sentinel-filled fences of `pad` elements before and after it in the same allocation."""
+
+    def __init__(self, shape, dtype, pad=512, fill=float("nan")):
+        n = int(np.prod(shape))
+        self.pad, self.n = pad, n
+        self.sentinel = 12345.0 if dtype != torch.int64 else 12345
+        self.buf = torch.full((n + 2 * pad,), self.sentinel, dtype=dtype, device="cuda")
+        self.t = self.buf[pad:pad + n].view(*shape)
+        self.t.fill_(fill)
+        assert self.t.data_ptr() % 16 == 0
+
+    def intact(self):
+        return bool((self.buf[:self.pad] == self.sentinel).all()) and bool((self.buf[self.pad + self.n:] == self.sentinel).all())
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_no_write_outside_the_outputs(dtype):
+    """Every output of the layer, the head and the attention building blocks sits between sentinel fences; ragged
+    sizes (rows, chunk and vocabulary not multiples of any tile).  Nothing outside the outputs may change."""
+    shape = synth.LayerShape(256, 4, 2, 128, 520, True, 1e6) if dtype == torch.bfloat16 else \
+        synth.LayerShape(128, 4, 2, 64, 168, True, 1e4)
+    T, chunk = 333, 100
+    ocfg, bcfg, W, X, dY = layer_case(shape, 21, T, dtype)
+    Wd = {k: to_dev(v, dtype) for k, v in W.items()}
+    dX = _Fenced((T, shape.d_model), dtype)
+    G = {k: _Fenced(shp, torch.float32) for k, shp in B.layer_grad_shapes(bcfg).items()}
+    for group in (1, 2):
+        ws = B.alloc_workspace(B.layer_workspace_bytes(bcfg, T, chunk, group))
+        B.layer_backward(bcfg, Wd, to_dev(X, dtype), to_dev(dY, dtype), chunk, {k: g.t for k, g in G.items()}, dX.t, ws,
+                         wgrad_group=group)
+        assert B.last_device_status(ws) == B.OK
+        assert dX.intact() and all(g.intact() for g in G.values()), [k for k, g in G.items() if not g.intact()]
+        assert torch.isfinite(dX.t.float()).all() and all(torch.isfinite(g.t).all() for g in G.values())
+    # head: vocabulary and rows ragged
+    hs = synth.HeadShape(shape.d_model, 1003)
+    g, Wv, H, labels = synth.make_head_inputs(hs, 22, 211, dtype == torch.bfloat16, 40)
+    hc = B.HeadConfig(hs.d_model, hs.vocab, hs.rms_eps, hs.ignore_index, dtype)
+    dH, dWv, dg = _Fenced((211, hs.d_model), dtype), _Fenced((hs.vocab, hs.d_model), torch.float32), _Fenced((hs.d_model,), torch.float32)
+    loss, nv = _Fenced((1,), torch.float32), _Fenced((1,), torch.int64, fill=0)
+    ws = B.alloc_workspace(B.lmhead_workspace_bytes(hc, 211, 64))
+    B.lmhead_ce_backward(hc, to_dev(g, dtype), to_dev(Wv, dtype), to_dev(H, dtype), torch.from_numpy(labels).cuda(), 64,
+                         loss.t, nv.t, dH.t, dWv.t, dg.t, ws)
+    assert B.last_device_status(ws) == B.OK
+    assert all(f.intact() for f in (dH, dWv, dg, loss, nv))
+    assert torch.isfinite(dWv.t).all() and torch.isfinite(dH.t.float()).all()
+    # attention building blocks (both tensor-core backward kernels in bf16)
+    n, q0, Hq, Hkv, dh = 150, 139, shape.n_q_heads, shape.n_kv_heads, shape.head_dim
+    mk = lambda *s: torch.randn(*s, device="cuda").to(dtype)
+    q, do, k, v = mk(n, Hq, dh), mk(n, Hq, dh), mk(q0 + n, Hkv, dh), mk(q0 + n, Hkv, dh)
+    o, lse = _Fenced((n, Hq, dh), dtype), _Fenced((Hq, n), torch.float32)
+    for engine in ((1, 3, 4) if dtype == torch.bfloat16 else (1,)):
+        B.attention_forward(q, k, v, q0, o.t, lse.t, engine=engine)
+        torch.cuda.synchronize()
+        assert o.intact() and lse.intact(), engine
+    for engine in ((1, 2, 5) if dtype == torch.bfloat16 else (1,)):
+        dq, dk, dv = _Fenced((n, Hq, dh), torch.float32), _Fenced((q0 + n, Hkv, dh), torch.float32, fill=0.0), \
+            _Fenced((q0 + n, Hkv, dh), torch.float32, fill=0.0)
+        B.attention_backward(q, k, v, o.t, do, lse.t, q0, dq.t, dk.t, dv.t, engine=engine)
+        torch.cuda.synchronize()
+        assert dq.intact() and dk.intact() and dv.intact(), engine
+        assert torch.isfinite(dq.t).all() and torch.isfinite(dk.t).all()
