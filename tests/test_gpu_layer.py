@@ -271,11 +271,13 @@ def test_no_write_outside_the_outputs(dtype):
     Wd = {k: to_dev(v, dtype) for k, v in W.items()}
     dX = _Fenced((T, shape.d_model), dtype)
     G = {k: _Fenced(shp, torch.float32) for k, shp in B.layer_grad_shapes(bcfg).items()}
+    Xd, dYd = to_dev(X, dtype), to_dev(dY, dtype)
+    before = {k: v.clone() for k, v in dict(Wd, X=Xd, dY=dYd).items()}
     for group in (1, 2):
         ws = B.alloc_workspace(B.layer_workspace_bytes(bcfg, T, chunk, group))
-        B.layer_backward(bcfg, Wd, to_dev(X, dtype), to_dev(dY, dtype), chunk, {k: g.t for k, g in G.items()}, dX.t, ws,
-                         wgrad_group=group)
+        B.layer_backward(bcfg, Wd, Xd, dYd, chunk, {k: g.t for k, g in G.items()}, dX.t, ws, wgrad_group=group)
         assert B.last_device_status(ws) == B.OK
+        assert all(torch.equal(v, dict(Wd, X=Xd, dY=dYd)[k]) for k, v in before.items())      # inputs are read only
         assert dX.intact() and all(g.intact() for g in G.values()), [k for k, g in G.items() if not g.intact()]
         assert torch.isfinite(dX.t.float()).all() and all(torch.isfinite(g.t).all() for g in G.values())
     # head: vocabulary and rows ragged
