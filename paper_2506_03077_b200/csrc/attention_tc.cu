@@ -1443,18 +1443,24 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1)
 // One launch for both backward kernels.  They are independent (both read Q, K, V, dO, lse, delta; one owns dK / dV
 // tiles, the other dQ tiles), and at short prefixes or small chunks neither fills the GPU on its own (e.g. 32 to
 // 256 key-tile CTAs and 224 query-tile CTAs per chunk of the 7B layer at chunk 1024): as one grid their CTAs pack
-// onto the SMs together.  The dK / dV CTAs come first (they run longest), lowest key tiles (most query tiles) first.
+// onto the SMs together.  The role whose CTAs run longest comes first (longest jobs first keeps the tail of the launch
+// short): a dK / dV CTA walks G x (query tiles) tile pairs, a dQ CTA as many as its prefix has key tiles -- so the dQ
+// CTAs lead at long prefixes and the dK / dV CTAs at short ones; within a role the longest CTAs come first too
+// (lowest key tiles, highest query tiles).
 constexpr int BWD_FUSED_SMEM = BWD_SMEM > DQ_SMEM ? BWD_SMEM : DQ_SMEM;
 __global__ void __launch_bounds__(BWD_THREADS, 1)
     attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                        const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
-                       const BwdParams p, int kv_tiles, int n_dkdv, int q_tiles) {
+                       const BwdParams p, int kv_tiles, int n_dkdv, int q_tiles, int n_dq_first) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    const int b = (int)blockIdx.x;
-    if (b < n_dkdv) {
+    // block order = dispatch order: n_dq_first dQ CTAs (all of them or none), then the dK/dV CTAs, then the rest
+    int b = (int)blockIdx.x;
+    const bool dq_role = b < n_dq_first || b >= n_dq_first + n_dkdv;
+    if (!dq_role) {
+        b -= n_dq_first;
         attn_bwd_dkdv_body(map_q, map_k, map_v, map_do, p, smem_raw, b % kv_tiles, b / kv_tiles);
     } else {
-        const int c = b - n_dkdv;
+        const int c = b < n_dq_first ? b : b - n_dkdv;
         attn_bwd_dq_body(map_q, map_k, map_v, map_do, p, smem_raw, q_tiles - 1 - c % q_tiles, c / q_tiles);
     }
 }
@@ -1527,8 +1533,11 @@ int attention_bwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, const bf16 *do
         SBP_LAUNCH(attn_bwd_fused_kernel, (unsigned)n_dkdv, FUSED_THREADS, BWD_SMEM, st, mq, mk, mv, mdo, mdq, p, kv_tiles);
         return STREAMBP_OK;
     }
+    // cost of the longest CTA of each role in tile pairs (a dK/dV pair takes ~1.25x a dQ pair: four products against three)
+    const int64_t dq_longest = 4 * (int64_t)kv_tiles, dkdv_longest = 5 * (int64_t)(Hq / Hkv) * q_tiles;
+    const int n_dq_first = dq_longest > dkdv_longest ? (int)n_dq : 0;
     SBP_LAUNCH(attn_bwd_tc_kernel, (unsigned)(n_dkdv + n_dq), BWD_THREADS, BWD_FUSED_SMEM, st, mq, mk, mv, mdo, p,
-               kv_tiles, (int)n_dkdv, q_tiles);
+               kv_tiles, (int)n_dkdv, q_tiles, n_dq_first);
     return STREAMBP_OK;
 }
 
