@@ -1458,7 +1458,10 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
     const bool dq_role = b < n_dq_first || b >= n_dq_first + n_dkdv;
     if (!dq_role) {
         b -= n_dq_first;
-        attn_bwd_dkdv_body(map_q, map_k, map_v, map_do, p, smem_raw, b % kv_tiles, b / kv_tiles);
+        // key tiles in ascending order, the KV heads of a key tile side by side: the cost of a CTA (the number of
+        // query tiles that see its key tile) never increases along the list
+        const int n_kv_heads = n_dkdv / kv_tiles;
+        attn_bwd_dkdv_body(map_q, map_k, map_v, map_do, p, smem_raw, b / n_kv_heads, b % n_kv_heads);
     } else {
         const int c = b < n_dq_first ? b : b - n_dkdv;
         attn_bwd_dq_body(map_q, map_k, map_v, map_do, p, smem_raw, q_tiles - 1 - c % q_tiles, c / q_tiles);
