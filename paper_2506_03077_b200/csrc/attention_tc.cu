@@ -82,8 +82,9 @@ __global__ void __launch_bounds__(FWD16_THREADS, 1)
     volatile int *abort_flag = reinterpret_cast<volatile int *>(aux + 152);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int h = blockIdx.y, g = h / (p.Hq / p.Hkv);
-    const int qt0 = blockIdx.x * TILE;
+    // grid (heads, query tiles): the tiles with the longest key prefix are dispatched first
+    const int h = blockIdx.x, g = h / (p.Hq / p.Hkv);
+    const int qt0 = (int)(gridDim.y - 1 - blockIdx.y) * TILE;
     const long long q_abs0 = p.q0 + qt0;
     const int rows_here = (p.n - qt0) < TILE ? (p.n - qt0) : TILE;
     const long long kv_end = q_abs0 + rows_here;
@@ -311,8 +312,9 @@ __global__ void __launch_bounds__(FWD2Q_THREADS, 1)
     volatile int *abort_flag = reinterpret_cast<volatile int *>(aux + 128);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int h = blockIdx.y, g = h / (p.Hq / p.Hkv);
-    const int qt0 = blockIdx.x * 2 * TILE;
+    // grid (heads, query tile pairs): the pairs with the longest key prefix are dispatched first
+    const int h = blockIdx.x, g = h / (p.Hq / p.Hkv);
+    const int qt0 = (int)(gridDim.y - 1 - blockIdx.y) * 2 * TILE;
     // team X: query rows qt0 + X * TILE .. ; its key tiles 0 .. nkv[X] - 1 (0 tiles: team absent)
     int nkv[2];
 #pragma unroll
@@ -1501,11 +1503,11 @@ int attention_fwd_tc(const bf16 *q, const bf16 *k, const bf16 *v, int64_t n, int
     const int64_t sms = sm_count();
     const bool two = tiles_per_cta == 2 || (tiles_per_cta == 0 && n > TILE && 3 * ((ctas2 + sms - 1) / sms) <= 2 * ((ctas1 + sms - 1) / sms));
     if (two) {
-        dim3 grid((unsigned)((n + 2 * TILE - 1) / (2 * TILE)), Hq);
+        dim3 grid(Hq, (unsigned)((n + 2 * TILE - 1) / (2 * TILE)));
         SBP_LAUNCH(attn_fwd_2q_kernel, grid, FWD2Q_THREADS, FWD2Q_SMEM, st, mq, mk, mv, p);
         return STREAMBP_OK;
     }
-    dim3 grid((unsigned)((n + TILE - 1) / TILE), Hq);
+    dim3 grid(Hq, (unsigned)((n + TILE - 1) / TILE));
     SBP_LAUNCH(attn_fwd_tc16_kernel, grid, FWD16_THREADS, FWD16_SMEM, st, mq, mk, mv, p);
     return STREAMBP_OK;
 }
