@@ -135,6 +135,23 @@ def test_attention_entry_points_refuse_misaligned_pointers(lib):
     assert bwd(False, delta=a + 2) == B.E_ALIGN
 
 
+def test_grouped_entry_point_validates_on_the_host(lib):
+    import torch
+    c = cfg().c()
+    w = B.LayerPtrsC(**{f: 4096 for f in B.WEIGHT_FIELDS})
+    call = lambda group, wsb=16, cu=None, n=0: lib.streambp_layer_backward_grouped(
+        C.byref(c), C.byref(w), 4096, 8192, 512, 128, group, cu, n, 0, 0, C.byref(w), 12288, 1 << 20, wsb, None)
+    assert call(0) == B.E_SHAPE and call(-3) == B.E_SHAPE
+    assert call(2) == B.E_WORKSPACE                      # 16 bytes of workspace are never enough
+    # the size query grows with the group and saturates at the number of chunks (512 / 128 = 4)
+    sizes = [lib.streambp_layer_workspace_bytes_grouped(C.byref(c), 512, 128, g) for g in (1, 2, 4, 9)]
+    assert sizes[0] == B.layer_workspace_bytes(cfg(), 512, 128) and sizes[0] < sizes[1] < sizes[2] == sizes[3]
+    assert lib.streambp_layer_workspace_bytes_grouped(C.byref(c), 512, 128, 0) == 0
+    # malformed sequence boundaries are refused before anything else happens
+    bad = (C.c_int64 * 3)(0, 300, 400)
+    assert call(2, wsb=1 << 30, cu=bad, n=2) == B.E_SHAPE
+
+
 def test_per_device_facts_are_keyed_by_device_ordinal(lib):
     """SM count, shared-memory opt-in and product-kernel choice are cached per device: a second device must not get
     the first one's answer.  The hook runs that cache with a stand-in ordinal."""
