@@ -265,10 +265,11 @@ def run_head_or_model(args, cfg):
         ld = torch.from_numpy(labels).cuda()
         nv = torch.zeros(1, dtype=torch.int64, device="cuda")
         dH, dW, dg = torch.empty_like(Hd), torch.empty(h.vocab, h.d_model, device="cuda"), torch.empty(h.d_model, device="cuda")
-        ws_bytes = B.lmhead_workspace_bytes(hc, T, cfg.chunk)
+        ws_bytes = B.lmhead_workspace_bytes(hc, T, cfg.chunk, args.wgrad_group)
         ws_full = B.lmhead_workspace_bytes(hc, T, T)
         ws = B.alloc_workspace(ws_bytes)
-        step = lambda: B.lmhead_ce_backward(hc, gd, Wd, Hd, ld, cfg.chunk, loss, nv, dH, dW, dg, ws)
+        step = lambda: B.lmhead_ce_backward(hc, gd, Wd, Hd, ld, cfg.chunk, loss, nv, dH, dW, dg, ws,
+                                            wgrad_group=args.wgrad_group)
         flops, name = head_flops(h, T), "streamed_lmhead_ce_backward_tokens_per_s"
         if args.objective != "sft":
             # synthetic per-token inputs of the RL objectives: behaviour / reference log-probabilities around the
@@ -286,14 +287,17 @@ def run_head_or_model(args, cfg):
                 wt = torch.where(torch.arange(T, device="cuda") < half, 1.0, -1.0).float()
                 obj, beta, eps = B.OBJ_DPO, 0.1, 0.0
             step = lambda: B.lmhead_rl_backward(hc, obj, beta, eps, gd, Wd, Hd, ld, old, ref, adv, wt, cfg.chunk, loss,
-                                                dH, dW, dg, ws)
+                                                dH, dW, dg, ws, wgrad_group=args.wgrad_group)
             name = f"streamed_lmhead_{args.objective}_backward_tokens_per_s"
         H_host, l_host = torch.from_numpy(H).to(dt).pin_memory(), torch.from_numpy(labels).pin_memory()
         dH_host, loss_host = torch.empty_like(H_host).pin_memory(), torch.zeros(1).pin_memory()
         e2e_io = lambda: ([(Hd, H_host), (ld, l_host)], [(dH_host, dH), (loss_host, loss)])
-        # chunks whose labels are all ignored are skipped on the device (their gradient is exactly zero)
-        live_chunks = sum(1 for r0 in range(0, T, cfg.chunk) if (labels[r0:r0 + cfg.chunk] != h.ignore_index).any())
-        executed_flops = head_flops(h, min(T, live_chunks * cfg.chunk))
+        # chunks (with --wgrad-group, groups of chunks) whose labels are all ignored are skipped on the device (their
+        # gradient is exactly zero)
+        gate_rows = cfg.chunk * max(1, args.wgrad_group)
+        live = sum(min(gate_rows, T - r0) for r0 in range(0, T, gate_rows)
+                   if (labels[r0:r0 + gate_rows] != h.ignore_index).any())
+        executed_flops = head_flops(h, live)
     else:
         s, L = cfg.layer, cfg.n_layers
         lc = B.LayerConfig(s.d_model, s.n_q_heads, s.n_kv_heads, s.head_dim, s.d_ff, s.qkv_bias, s.rope_theta, s.rms_eps, dt)
@@ -354,7 +358,8 @@ def run_head_or_model(args, cfg):
         "metric": name, "value": T / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic", "loss": loss.item(),
-        "config": {"workload": cfg.name, "T": T, "chunk": cfg.chunk, "n_layers": cfg.n_layers, "vocab": h.vocab,
+        "config": {"workload": cfg.name, "T": T, "chunk": cfg.chunk,
+                   "wgrad_group": args.wgrad_group if cfg.n_layers == 0 else 1, "n_layers": cfg.n_layers, "vocab": h.vocab,
                    "l2": "inputs larger than L2", "product_kernel": B.product_kernel()},
         "algorithmic_tflop_per_step": flops / 1e12, "tflops": flops / (ms * 1e-3) / 1e12,
         "frac_of_measured_sustained_bf16": flops / (ms * 1e-3) / 1e12 / peaks["sustained"],
@@ -431,7 +436,7 @@ def main():
                     help="objective of the qwen7b_head workload (Sec. 3.2.1)")
     ap.add_argument("--chunk", type=int, default=0)
     ap.add_argument("--wgrad-group", type=int, default=1,
-                    help="layer workloads: chunks per weight-gradient pass (the second partition size, Sec. 4.3)")
+                    help="layer and head workloads: chunks per weight-gradient pass (the second partition size, Sec. 4.3)")
     ap.add_argument("--T", type=int, default=0, help="override the sequence length (profiling on small cases)")
     ap.add_argument("--ref-tokens", type=int, default=512)
     ap.add_argument("--cpu-baseline-tokens", type=int, default=1024)

@@ -224,6 +224,33 @@ int streambp_lmhead_rl_backward(const streambp_head_cfg *cfg, const streambp_rl_
                                 float *d_w_vocab, float *d_g_final, void *workspace, size_t workspace_bytes,
                                 void *cuda_stream);
 
+/*
+ * The streamed LM-head backward with a SECOND partition size for the vocabulary weight gradient (Sec. 4.3, effect of
+ * the partition size; Sec. 3.2.1 for the step itself).  Logits, loss rows and dL/dH still run per `chunk` rows, but
+ * d_w_vocab += dlogits^T hn is formed once per `wgrad_group` consecutive chunks, as one product over
+ * wgrad_group * chunk rows: the [vocab, d_model] fp32 accumulator is read and written D / wgrad_group times instead of
+ * D times.  The price is memory: the normalised hidden rows and the dlogits are kept for every chunk of a group (the
+ * fp32 logits still exist for one chunk only when storage is bf16).  A group whose labels are all ignored is skipped
+ * on the device; a masked chunk inside a live group is processed (its dlogits are zero).  wgrad_group = 1 is the plain
+ * entry point; values above the number of chunks act like that number.  Same sums in a different association.
+ * All other arguments, outputs and errors as in streambp_lmhead_ce_backward / streambp_lmhead_rl_backward;
+ * STREAMBP_E_SHAPE also for wgrad_group < 1.  Workspace: streambp_lmhead_workspace_bytes_grouped().
+ */
+size_t streambp_lmhead_workspace_bytes_grouped(const streambp_head_cfg *cfg, int64_t T, int64_t chunk,
+                                               int32_t wgrad_group);
+int streambp_lmhead_ce_backward_grouped(const streambp_head_cfg *cfg, const void *g_final, const void *w_vocab,
+                                        const void *H, const int64_t *labels, int64_t T, int64_t chunk,
+                                        int32_t wgrad_group, int accumulate, float *loss, int64_t *n_valid, void *dH,
+                                        float *d_w_vocab, float *d_g_final, void *workspace, size_t workspace_bytes,
+                                        void *cuda_stream);
+int streambp_lmhead_rl_backward_grouped(const streambp_head_cfg *cfg, const streambp_rl_cfg *rl, const void *g_final,
+                                        const void *w_vocab, const void *H, const int64_t *tokens,
+                                        const float *logp_old, const float *logp_ref, const float *advantage,
+                                        const float *weight, int64_t T, int64_t chunk, int32_t wgrad_group,
+                                        int accumulate, float *loss, float *logp, float *ell, void *dH,
+                                        float *d_w_vocab, float *d_g_final, void *workspace, size_t workspace_bytes,
+                                        void *cuda_stream);
+
 typedef struct {
     int32_t n_layers;
     streambp_layer_cfg layer;

@@ -37,6 +37,8 @@ EXPORTS = (
     "streambp_lmhead_rl_backward", "streambp_layer_backward_packed",
     "streambp_test_expire_wait", "streambp_test_per_device_value",
     "streambp_layer_workspace_bytes_grouped", "streambp_layer_backward_grouped", "streambp_test_workspace_guard",
+    "streambp_lmhead_workspace_bytes_grouped", "streambp_lmhead_ce_backward_grouped",
+    "streambp_lmhead_rl_backward_grouped",
 )
 
 
@@ -111,6 +113,15 @@ def lib() -> C.CDLL:
     L.streambp_lmhead_rl_backward.restype = C.c_int
     L.streambp_lmhead_rl_backward.argtypes = [C.POINTER(HeadCfgC), C.POINTER(RlCfgC), vp, vp, vp, vp, vp, vp, vp, vp,
                                               i64, i64, C.c_int, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    L.streambp_lmhead_workspace_bytes_grouped.restype = sz
+    L.streambp_lmhead_workspace_bytes_grouped.argtypes = [C.POINTER(HeadCfgC), i64, i64, i32]
+    L.streambp_lmhead_ce_backward_grouped.restype = C.c_int
+    L.streambp_lmhead_ce_backward_grouped.argtypes = [C.POINTER(HeadCfgC), vp, vp, vp, vp, i64, i64, i32, C.c_int, vp,
+                                                      vp, vp, vp, vp, vp, sz, vp]
+    L.streambp_lmhead_rl_backward_grouped.restype = C.c_int
+    L.streambp_lmhead_rl_backward_grouped.argtypes = [C.POINTER(HeadCfgC), C.POINTER(RlCfgC), vp, vp, vp, vp, vp, vp,
+                                                      vp, vp, i64, i64, i32, C.c_int, vp, vp, vp, vp, vp, vp, vp, sz,
+                                                      vp]
     L.streambp_model_workspace_bytes.restype = sz
     L.streambp_model_workspace_bytes.argtypes = [C.POINTER(ModelCfgC), i64, i64, i64]
     L.streambp_model_backward.restype = C.c_int
@@ -353,20 +364,28 @@ def layer_backward_packed(cfg: LayerConfig, weights, X, dY, chunk: int, cu_seqle
     return st
 
 
-def lmhead_workspace_bytes(cfg: HeadConfig, T: int, chunk: int) -> int:
+def lmhead_workspace_bytes(cfg: HeadConfig, T: int, chunk: int, wgrad_group: int = 1) -> int:
     c = cfg.c()
-    return int(lib().streambp_lmhead_workspace_bytes(C.byref(c), T, chunk))
+    if wgrad_group == 1:
+        return int(lib().streambp_lmhead_workspace_bytes(C.byref(c), T, chunk))
+    return int(lib().streambp_lmhead_workspace_bytes_grouped(C.byref(c), T, chunk, wgrad_group))
 
 
 def lmhead_ce_backward(cfg: HeadConfig, g_final, w_vocab, H, labels, chunk: int, loss, n_valid, dH, d_w_vocab,
-                       d_g_final, workspace, accumulate: bool = False, stream=None, check: bool = True) -> int:
+                       d_g_final, workspace, accumulate: bool = False, stream=None, check: bool = True,
+                       wgrad_group: int = 1) -> int:
+    """streambp_lmhead_ce_backward; wgrad_group != 1 goes through streambp_lmhead_ce_backward_grouped."""
     c = cfg.c()
-    st = lib().streambp_lmhead_ce_backward(C.byref(c), _ptr(g_final), _ptr(w_vocab), _ptr(H), _ptr(labels),
-                                           H.shape[0], chunk, 1 if accumulate else 0, _ptr(loss), _ptr(n_valid),
-                                           _ptr(dH), _ptr(d_w_vocab), _ptr(d_g_final), _ptr(workspace),
-                                           workspace.numel(), _stream_ptr(stream))
+    head = (C.byref(c), _ptr(g_final), _ptr(w_vocab), _ptr(H), _ptr(labels), H.shape[0], chunk)
+    tail = (1 if accumulate else 0, _ptr(loss), _ptr(n_valid), _ptr(dH), _ptr(d_w_vocab), _ptr(d_g_final),
+            _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+    if wgrad_group == 1:
+        name, st = "streambp_lmhead_ce_backward", lib().streambp_lmhead_ce_backward(*head, *tail)
+    else:
+        name = "streambp_lmhead_ce_backward_grouped"
+        st = lib().streambp_lmhead_ce_backward_grouped(*head, wgrad_group, *tail)
     if check:
-        _check(st, "streambp_lmhead_ce_backward")
+        _check(st, name)
     return st
 
 
@@ -540,15 +559,21 @@ OBJ_GRPO, OBJ_DPO = 1, 2
 
 def lmhead_rl_backward(cfg: HeadConfig, objective: int, beta: float, clip_eps: float, g_final, w_vocab, H, tokens,
                        logp_old, logp_ref, advantage, weight, chunk: int, loss, dH, d_w_vocab, d_g_final, workspace,
-                       logp=None, ell=None, accumulate: bool = False, stream=None, check: bool = True) -> int:
-    """streambp_lmhead_rl_backward (GRPO / DPO objectives of the streamed LM head)."""
+                       logp=None, ell=None, accumulate: bool = False, stream=None, check: bool = True,
+                       wgrad_group: int = 1) -> int:
+    """streambp_lmhead_rl_backward (GRPO / DPO objectives of the streamed LM head); wgrad_group != 1 goes through
+    streambp_lmhead_rl_backward_grouped."""
     c = cfg.c()
     rl = RlCfgC(objective, beta, clip_eps)
-    st = lib().streambp_lmhead_rl_backward(C.byref(c), C.byref(rl), _ptr(g_final), _ptr(w_vocab), _ptr(H),
-                                           _ptr(tokens), _ptr(logp_old), _ptr(logp_ref), _ptr(advantage),
-                                           _ptr(weight), H.shape[0], chunk, 1 if accumulate else 0, _ptr(loss),
-                                           _ptr(logp), _ptr(ell), _ptr(dH), _ptr(d_w_vocab), _ptr(d_g_final),
-                                           _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+    head = (C.byref(c), C.byref(rl), _ptr(g_final), _ptr(w_vocab), _ptr(H), _ptr(tokens), _ptr(logp_old),
+            _ptr(logp_ref), _ptr(advantage), _ptr(weight), H.shape[0], chunk)
+    tail = (1 if accumulate else 0, _ptr(loss), _ptr(logp), _ptr(ell), _ptr(dH), _ptr(d_w_vocab), _ptr(d_g_final),
+            _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+    if wgrad_group == 1:
+        name, st = "streambp_lmhead_rl_backward", lib().streambp_lmhead_rl_backward(*head, *tail)
+    else:
+        name = "streambp_lmhead_rl_backward_grouped"
+        st = lib().streambp_lmhead_rl_backward_grouped(*head, wgrad_group, *tail)
     if check:
-        _check(st, "streambp_lmhead_rl_backward")
+        _check(st, name)
     return st

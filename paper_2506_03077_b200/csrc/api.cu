@@ -395,43 +395,61 @@ int streambp_layer_backward_packed(const streambp_layer_cfg *cfg, const streambp
                                   workspace_bytes, cuda_stream);
 }
 
+size_t streambp_lmhead_workspace_bytes_grouped(const streambp_head_cfg *cfg, int64_t T, int64_t chunk,
+                                               int32_t wgrad_group) {
+    if (check_head_cfg(cfg) != STREAMBP_OK || T < 1 || chunk < 1 || wgrad_group < 1) return 0;
+    return cfg->dtype == STREAMBP_F32 ? lmhead_workspace<float>(*cfg, T, chunk, wgrad_group)
+                                      : lmhead_workspace<bf16>(*cfg, T, chunk, wgrad_group);
+}
+
 size_t streambp_lmhead_workspace_bytes(const streambp_head_cfg *cfg, int64_t T, int64_t chunk) {
-    if (check_head_cfg(cfg) != STREAMBP_OK || T < 1 || chunk < 1) return 0;
-    return cfg->dtype == STREAMBP_F32 ? lmhead_workspace<float>(*cfg, T, chunk) : lmhead_workspace<bf16>(*cfg, T, chunk);
+    return streambp_lmhead_workspace_bytes_grouped(cfg, T, chunk, 1);
+}
+
+int streambp_lmhead_ce_backward_grouped(const streambp_head_cfg *cfg, const void *g_final, const void *w_vocab,
+                                        const void *H, const int64_t *labels, int64_t T, int64_t chunk,
+                                        int32_t wgrad_group, int accumulate, float *loss, int64_t *n_valid, void *dH,
+                                        float *d_w_vocab, float *d_g_final, void *workspace, size_t workspace_bytes,
+                                        void *cuda_stream) {
+    SBP_TRY(check_head_cfg(cfg));
+    if (T < 1 || chunk < 1 || wgrad_group < 1) return STREAMBP_E_SHAPE;
+    if (!g_final || !w_vocab || !H || !labels || !loss || !dH || !d_w_vocab || !d_g_final || !workspace)
+        return STREAMBP_E_NULL;
+    if (!aligned(g_final, 16) || !aligned(w_vocab, 16) || !aligned(H, 16) || !aligned(dH, 16) ||
+        !aligned(d_w_vocab, 16) || !aligned(d_g_final, 16) || !aligned(labels, 8) || !aligned(workspace, 256))
+        return STREAMBP_E_ALIGN;
+    if (workspace_bytes < streambp_lmhead_workspace_bytes_grouped(cfg, T, chunk, wgrad_group))
+        return STREAMBP_E_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    SBP_TRY(begin_call(workspace, st));
+    if (cfg->dtype == STREAMBP_F32)
+        return lmhead_backward<float>(*cfg, (const float *)g_final, (const float *)w_vocab, (const float *)H, labels, T,
+                                      chunk, accumulate != 0, loss, n_valid, (float *)dH, d_w_vocab, d_g_final,
+                                      workspace, st, nullptr, nullptr, wgrad_group);
+    return lmhead_backward<bf16>(*cfg, (const bf16 *)g_final, (const bf16 *)w_vocab, (const bf16 *)H, labels, T, chunk,
+                                 accumulate != 0, loss, n_valid, (bf16 *)dH, d_w_vocab, d_g_final, workspace, st,
+                                 nullptr, nullptr, wgrad_group);
 }
 
 int streambp_lmhead_ce_backward(const streambp_head_cfg *cfg, const void *g_final, const void *w_vocab, const void *H,
                                 const int64_t *labels, int64_t T, int64_t chunk, int accumulate, float *loss,
                                 int64_t *n_valid, void *dH, float *d_w_vocab, float *d_g_final, void *workspace,
                                 size_t workspace_bytes, void *cuda_stream) {
-    SBP_TRY(check_head_cfg(cfg));
-    if (T < 1 || chunk < 1) return STREAMBP_E_SHAPE;
-    if (!g_final || !w_vocab || !H || !labels || !loss || !dH || !d_w_vocab || !d_g_final || !workspace)
-        return STREAMBP_E_NULL;
-    if (!aligned(g_final, 16) || !aligned(w_vocab, 16) || !aligned(H, 16) || !aligned(dH, 16) ||
-        !aligned(d_w_vocab, 16) || !aligned(d_g_final, 16) || !aligned(labels, 8) || !aligned(workspace, 256))
-        return STREAMBP_E_ALIGN;
-    if (workspace_bytes < streambp_lmhead_workspace_bytes(cfg, T, chunk)) return STREAMBP_E_WORKSPACE;
-    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    SBP_TRY(begin_call(workspace, st));
-    if (cfg->dtype == STREAMBP_F32)
-        return lmhead_backward<float>(*cfg, (const float *)g_final, (const float *)w_vocab, (const float *)H, labels, T,
-                                      chunk, accumulate != 0, loss, n_valid, (float *)dH, d_w_vocab, d_g_final,
-                                      workspace, st);
-    return lmhead_backward<bf16>(*cfg, (const bf16 *)g_final, (const bf16 *)w_vocab, (const bf16 *)H, labels, T, chunk,
-                                 accumulate != 0, loss, n_valid, (bf16 *)dH, d_w_vocab, d_g_final, workspace, st);
+    return streambp_lmhead_ce_backward_grouped(cfg, g_final, w_vocab, H, labels, T, chunk, 1, accumulate, loss, n_valid,
+                                               dH, d_w_vocab, d_g_final, workspace, workspace_bytes, cuda_stream);
 }
 
-int streambp_lmhead_rl_backward(const streambp_head_cfg *cfg, const streambp_rl_cfg *rl, const void *g_final,
-                                const void *w_vocab, const void *H, const int64_t *tokens, const float *logp_old,
-                                const float *logp_ref, const float *advantage, const float *weight, int64_t T,
-                                int64_t chunk, int accumulate, float *loss, float *logp, float *ell, void *dH,
-                                float *d_w_vocab, float *d_g_final, void *workspace, size_t workspace_bytes,
-                                void *cuda_stream) {
+int streambp_lmhead_rl_backward_grouped(const streambp_head_cfg *cfg, const streambp_rl_cfg *rl, const void *g_final,
+                                        const void *w_vocab, const void *H, const int64_t *tokens,
+                                        const float *logp_old, const float *logp_ref, const float *advantage,
+                                        const float *weight, int64_t T, int64_t chunk, int32_t wgrad_group,
+                                        int accumulate, float *loss, float *logp, float *ell, void *dH,
+                                        float *d_w_vocab, float *d_g_final, void *workspace, size_t workspace_bytes,
+                                        void *cuda_stream) {
     SBP_TRY(check_head_cfg(cfg));
     if (!rl) return STREAMBP_E_NULL;
     if (rl->objective != STREAMBP_OBJ_GRPO && rl->objective != STREAMBP_OBJ_DPO) return STREAMBP_E_SHAPE;
-    if (T < 1 || chunk < 1 || !(rl->beta >= 0.f)) return STREAMBP_E_SHAPE;
+    if (T < 1 || chunk < 1 || wgrad_group < 1 || !(rl->beta >= 0.f)) return STREAMBP_E_SHAPE;
     if (rl->objective == STREAMBP_OBJ_GRPO && !(rl->clip_eps >= 0.f && rl->clip_eps < 1.f)) return STREAMBP_E_SHAPE;
     if (rl->objective == STREAMBP_OBJ_DPO && accumulate) return STREAMBP_E_SHAPE;   // in-place correction at the end
     if (!g_final || !w_vocab || !H || !tokens || !logp_ref || !weight || !loss || !dH || !d_w_vocab || !d_g_final ||
@@ -441,17 +459,29 @@ int streambp_lmhead_rl_backward(const streambp_head_cfg *cfg, const streambp_rl_
     if (!aligned(g_final, 16) || !aligned(w_vocab, 16) || !aligned(H, 16) || !aligned(dH, 16) ||
         !aligned(d_w_vocab, 16) || !aligned(d_g_final, 16) || !aligned(tokens, 8) || !aligned(workspace, 256))
         return STREAMBP_E_ALIGN;
-    if (workspace_bytes < streambp_lmhead_workspace_bytes(cfg, T, chunk)) return STREAMBP_E_WORKSPACE;
+    if (workspace_bytes < streambp_lmhead_workspace_bytes_grouped(cfg, T, chunk, wgrad_group))
+        return STREAMBP_E_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     SBP_TRY(begin_call(workspace, st));
     const RlRows rows{rl->objective, rl->beta, rl->clip_eps, logp_old, logp_ref, advantage, weight, logp};
     if (cfg->dtype == STREAMBP_F32)
         return lmhead_backward<float>(*cfg, (const float *)g_final, (const float *)w_vocab, (const float *)H, tokens, T,
                                       chunk, accumulate != 0, loss, nullptr, (float *)dH, d_w_vocab, d_g_final,
-                                      workspace, st, &rows, ell);
+                                      workspace, st, &rows, ell, wgrad_group);
     return lmhead_backward<bf16>(*cfg, (const bf16 *)g_final, (const bf16 *)w_vocab, (const bf16 *)H, tokens, T, chunk,
                                  accumulate != 0, loss, nullptr, (bf16 *)dH, d_w_vocab, d_g_final, workspace, st, &rows,
-                                 ell);
+                                 ell, wgrad_group);
+}
+
+int streambp_lmhead_rl_backward(const streambp_head_cfg *cfg, const streambp_rl_cfg *rl, const void *g_final,
+                                const void *w_vocab, const void *H, const int64_t *tokens, const float *logp_old,
+                                const float *logp_ref, const float *advantage, const float *weight, int64_t T,
+                                int64_t chunk, int accumulate, float *loss, float *logp, float *ell, void *dH,
+                                float *d_w_vocab, float *d_g_final, void *workspace, size_t workspace_bytes,
+                                void *cuda_stream) {
+    return streambp_lmhead_rl_backward_grouped(cfg, rl, g_final, w_vocab, H, tokens, logp_old, logp_ref, advantage,
+                                               weight, T, chunk, 1, accumulate, loss, logp, ell, dH, d_w_vocab,
+                                               d_g_final, workspace, workspace_bytes, cuda_stream);
 }
 
 static int check_model_cfg(const streambp_model_cfg *cfg) {

@@ -485,13 +485,15 @@ int layer_forward(const streambp_layer_cfg &c, const streambp_layer_weights &w, 
                   int64_t pos0, T *Y, void *ws, cudaStream_t st, const int64_t *cu_seqlens = nullptr, int n_seqs = 0);
 
 template <typename T>
-size_t lmhead_workspace(const streambp_head_cfg &c, int64_t T_, int64_t chunk);
+size_t lmhead_workspace(const streambp_head_cfg &c, int64_t T_, int64_t chunk, int wgrad_group = 1);
 // rl == nullptr: SFT cross-entropy (labels = targets); else the RL objective described by *rl (labels = the
-// sampled tokens, rl->logp_* etc. indexed by absolute row), `ell` optional (DPO).
+// sampled tokens, rl->logp_* etc. indexed by absolute row), `ell` optional (DPO).  wgrad_group >= 1: the vocabulary
+// weight gradient is formed once per group of that many chunks.
 template <typename T>
 int lmhead_backward(const streambp_head_cfg &c, const T *g_final, const T *w_vocab, const T *H, const int64_t *labels,
                     int64_t T_, int64_t chunk, bool accumulate, float *loss, int64_t *n_valid, T *dH, float *d_w_vocab,
-                    float *d_g_final, void *ws, cudaStream_t st, const RlRows *rl = nullptr, float *ell = nullptr);
+                    float *d_g_final, void *ws, cudaStream_t st, const RlRows *rl = nullptr, float *ell = nullptr,
+                    int wgrad_group = 1);
 
 template <typename T>
 size_t model_workspace(const streambp_model_cfg &c, int64_t T_, int64_t chunk_layer, int64_t chunk_head);

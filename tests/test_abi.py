@@ -152,6 +152,29 @@ def test_grouped_entry_point_validates_on_the_host(lib):
     assert call(2, wsb=1 << 30, cu=bad, n=2) == B.E_SHAPE
 
 
+def test_grouped_head_entry_points_validate_on_the_host(lib):
+    import torch
+    hc = B.HeadConfig(256, 4096, 1e-6, -100, torch.bfloat16)
+    c = hc.c()
+    rl = B.RlCfgC(B.OBJ_GRPO, 0.04, 0.2)
+    ce = lambda group, wsb=16: lib.streambp_lmhead_ce_backward_grouped(
+        C.byref(c), 4096, 8192, 12288, 16384, 512, 128, group, 0, 4096, 4096, 4096, 4096, 4096, 1 << 20, wsb, None)
+    rlc = lambda group, wsb=16: lib.streambp_lmhead_rl_backward_grouped(
+        C.byref(c), C.byref(rl), 4096, 8192, 12288, 16384, 4096, 4096, 4096, 4096, 512, 128, group, 0, 4096, None,
+        None, 4096, 4096, 4096, 1 << 20, wsb, None)
+    for call in (ce, rlc):
+        assert call(0) == B.E_SHAPE and call(-1) == B.E_SHAPE
+        assert call(2) == B.E_WORKSPACE
+    # one more chunk of normalised rows and dlogits per slot; saturates at the number of chunks (512 / 128 = 4)
+    sizes = [lib.streambp_lmhead_workspace_bytes_grouped(C.byref(c), 512, 128, g) for g in (1, 2, 4, 9)]
+    assert sizes[0] == B.lmhead_workspace_bytes(hc, 512, 128) and sizes[0] < sizes[1] < sizes[2] == sizes[3]
+    per_slot = 128 * (256 + 4096) * 2
+    assert per_slot <= sizes[1] - sizes[0] <= per_slot + 2048
+    assert lib.streambp_lmhead_workspace_bytes_grouped(C.byref(c), 512, 128, 0) == 0
+    # a workspace sized for the plain call is too small for a grouped one
+    assert ce(2, wsb=sizes[0]) == B.E_WORKSPACE
+
+
 def test_per_device_facts_are_keyed_by_device_ordinal(lib):
     """SM count, shared-memory opt-in and product-kernel choice are cached per device: a second device must not get
     the first one's answer.  The hook runs that cache with a stand-in ordinal."""

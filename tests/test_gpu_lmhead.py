@@ -11,7 +11,7 @@ from helpers import TOL, assert_close, to_dev
 pytestmark = pytest.mark.gpu
 
 
-def run_head(hs: synth.HeadShape, g, W, H, labels, chunk, dtype, accumulate=False, prior=None):
+def run_head(hs: synth.HeadShape, g, W, H, labels, chunk, dtype, accumulate=False, prior=None, wgrad_group=1):
     cfg = B.HeadConfig(hs.d_model, hs.vocab, hs.rms_eps, hs.ignore_index, dtype)
     gd, Wd, Hd = to_dev(g, dtype), to_dev(W, dtype), to_dev(H, dtype)
     ld = torch.from_numpy(labels).cuda()
@@ -24,8 +24,9 @@ def run_head(hs: synth.HeadShape, g, W, H, labels, chunk, dtype, accumulate=Fals
         dg = torch.full((hs.d_model,), float("nan"), device="cuda")
     else:
         dW, dg = prior
-    ws = B.alloc_workspace(B.lmhead_workspace_bytes(cfg, T, chunk))
-    B.lmhead_ce_backward(cfg, gd, Wd, Hd, ld, chunk, loss, nv, dH, dW, dg, ws, accumulate=accumulate)
+    ws = B.alloc_workspace(B.lmhead_workspace_bytes(cfg, T, chunk, wgrad_group))
+    B.lmhead_ce_backward(cfg, gd, Wd, Hd, ld, chunk, loss, nv, dH, dW, dg, ws, accumulate=accumulate,
+                         wgrad_group=wgrad_group)
     return loss, nv, dH, dW, dg, B.last_device_status(ws)
 
 
@@ -126,4 +127,47 @@ def test_fully_masked_chunks_are_skipped_exactly(dtype):
     assert_close("dW", dW, ref[3], TOL[dtype])
     assert_close("dg", dg, ref[4], TOL[dtype])
     for rows in (slice(0, 64), slice(128, 192), slice(200, 201)):
+        assert torch.count_nonzero(dH[rows]) == 0
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("group", [2, 3, 100])
+def test_vocab_gradient_summed_over_groups_of_chunks(dtype, group):
+    """The second partition size: dW_vocab formed once per `group` chunks (ragged last chunk, ragged last group,
+    a group larger than the number of chunks) equals the oracle and changes nothing but dW's summation order."""
+    hs = synth.HeadShape(128, 1003)
+    T, chunk = 330, 48                       # 7 chunks, the last of 42 rows
+    g, W, H, labels = synth.make_head_inputs(hs, 31, T, dtype == torch.bfloat16, 20)
+    labels[100] = -100
+    ref = O.lmhead_ce_backward(O.HeadCfg(128, 1003), g, W, H, labels)
+    base = run_head(hs, g, W, H, labels, chunk, dtype)
+    loss, nv, dH, dW, dg, st = run_head(hs, g, W, H, labels, chunk, dtype, wgrad_group=group)
+    assert st == B.OK and int(nv.item()) == ref[1]
+    assert abs(loss.item() - ref[0]) <= (1e-5 if dtype == torch.float32 else 2e-3) * abs(ref[0])
+    assert_close("dH", dH, ref[2], TOL[dtype])
+    assert_close("dW", dW, ref[3], TOL[dtype])
+    assert_close("dg", dg, ref[4], TOL[dtype])
+    # everything but dW is computed by the same launches on the same operands
+    assert torch.equal(dH, base[2]) and torch.equal(dg, base[4]) and loss.item() == base[0].item()
+    assert O.rel_frobenius(dW.cpu().numpy(), base[3].cpu().numpy().astype(np.float64)) < 1e-5
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_grouped_head_with_masked_chunks_and_groups(dtype):
+    """Groups of 2 chunks: group 0 fully masked (skipped on the device), group 1 half masked (its masked chunk is
+    processed and contributes exact zeros), accumulate on top of a prior value."""
+    hs = synth.HeadShape(128, 1536)
+    T, chunk = 384, 64
+    g, W, H, labels = synth.make_head_inputs(hs, 23, T, dtype == torch.bfloat16, 0)
+    labels[0:128] = -100       # chunks 0, 1 = group 0
+    labels[192:256] = -100     # chunk 3, second half of group 1
+    ref = O.lmhead_ce_backward(O.HeadCfg(128, 1536), g, W, H, labels)
+    prior = (torch.full((1536, 128), 0.5, device="cuda"), torch.full((128,), -0.25, device="cuda"))
+    loss, nv, dH, dW, dg, st = run_head(hs, g, W, H, labels, chunk, dtype, accumulate=True, prior=prior,
+                                        wgrad_group=2)
+    assert st == B.OK and int(nv.item()) == ref[1] == 192
+    assert_close("dH", dH, ref[2], TOL[dtype])
+    assert_close("dW", dW - 0.5, ref[3], TOL[dtype])
+    assert_close("dg", dg + 0.25, ref[4], TOL[dtype])
+    for rows in (slice(0, 128), slice(192, 256)):
         assert torch.count_nonzero(dH[rows]) == 0

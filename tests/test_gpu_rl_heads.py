@@ -38,7 +38,8 @@ def make_case(seed, T, d, V, dtype, masked):
     return hs, cfg, g, W, H, tok, old, ref, adv
 
 
-def run_rl(hs, objective, beta, eps, g, W, H, tok, old, ref, adv, wt, chunk, dtype, accumulate=False, check=True):
+def run_rl(hs, objective, beta, eps, g, W, H, tok, old, ref, adv, wt, chunk, dtype, accumulate=False, check=True,
+           wgrad_group=1):
     cfg = B.HeadConfig(hs.d_model, hs.vocab, hs.rms_eps, hs.ignore_index, dtype)
     T = H.shape[0]
     f32 = lambda a: None if a is None else torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).cuda()
@@ -48,10 +49,11 @@ def run_rl(hs, objective, beta, eps, g, W, H, tok, old, ref, adv, wt, chunk, dty
     dH = torch.full((T, hs.d_model), float("nan"), device="cuda", dtype=dtype)
     dW = torch.full((hs.vocab, hs.d_model), float("nan"), device="cuda")
     dg = torch.full((hs.d_model,), float("nan"), device="cuda")
-    ws = B.alloc_workspace(B.lmhead_workspace_bytes(cfg, T, chunk))
+    ws = B.alloc_workspace(B.lmhead_workspace_bytes(cfg, T, chunk, wgrad_group))
     st = B.lmhead_rl_backward(cfg, objective, beta, eps, to_dev(g, dtype), to_dev(W, dtype), to_dev(H, dtype),
                               torch.from_numpy(tok).cuda(), f32(old), f32(ref), f32(adv), f32(wt), chunk, loss, dH, dW,
-                              dg, ws, logp=logp, ell=ell, accumulate=accumulate, check=check)
+                              dg, ws, logp=logp, ell=ell, accumulate=accumulate, check=check,
+                              wgrad_group=wgrad_group)
     if st != B.OK:
         return st
     assert B.last_device_status(ws) == B.OK
@@ -74,8 +76,9 @@ def test_grpo_matches_oracle(dtype, T, V, chunk):
     r = np.exp(ref_out[1] - old)[part]
     assert (r > 1 + eps).any() and (r < 1 - eps).any() and ((r > 1 - eps) & (r < 1 + eps)).any()
     assert np.abs(adv[part]).min() > 0.0
-    for ch in (chunk, 23):                         # chunk invariance, ragged
-        loss, _, logp, dH, dW, dg = run_rl(hs, B.OBJ_GRPO, beta, eps, g, W, H, tok, old, ref, adv, wt, ch, dtype)
+    for ch, grp in ((chunk, 1), (23, 1), (23, 3)):     # chunk invariance, ragged; vocabulary gradient per 3 chunks
+        loss, _, logp, dH, dW, dg = run_rl(hs, B.OBJ_GRPO, beta, eps, g, W, H, tok, old, ref, adv, wt, ch, dtype,
+                                           wgrad_group=grp)
         assert np.abs(logp.cpu().numpy()[part] - ref_out[1][part]).max() < LOGP_TOL[dtype]
         assert torch.count_nonzero(logp[torch.from_numpy(~part).cuda()]) == 0
         assert abs(loss - ref_out[0]) <= (2e-5 if dtype == torch.float32 else 2e-2) * max(1.0, abs(ref_out[0]))
@@ -94,8 +97,10 @@ def test_dpo_matches_oracle(dtype):
     sign = np.where(np.arange(T) < 128, 1.0, -1.0).astype(np.float32)
     beta = 0.25
     ref_out = O.lmhead_dpo_backward(cfg, g, W, H, tok, ref, sign, beta)
-    for ch in (chunk, T, 50):
-        loss, ell, logp, dH, dW, dg = run_rl(hs, B.OBJ_DPO, beta, 0.0, g, W, H, tok, None, ref, None, sign, ch, dtype)
+    for ch, grp in ((chunk, 1), (T, 1), (50, 1), (32, 2)):
+        # the last case forms the vocabulary gradient per 2 chunks; rows 64..127 are then one whole skipped group
+        loss, ell, logp, dH, dW, dg = run_rl(hs, B.OBJ_DPO, beta, 0.0, g, W, H, tok, None, ref, None, sign, ch, dtype,
+                                             wgrad_group=grp)
         # bf16: ell sums 152 log-probabilities whose errors (up to 6e-3 each, from the bf16 operands of the logits
         # product) add up to 0.04; the correction factor sigmoid(beta ell) - 1 moves by beta * 0.04 / 2 < 1e-2
         assert abs(ell - ref_out[1]) <= (1e-4 if dtype == torch.float32 else 0.1)
