@@ -103,7 +103,36 @@ int mm<bf16, bf16>(GemmOp op, int64_t M, int64_t N, int64_t K, const bf16 *A, in
     return gemm<bf16, bf16>(op, M, N, K, A, lda, B, ldb, C, ldc, bias, accumulate, st);
 }
 template <>
+int mm_group<float>(const MmProb<float> *probs, int n, cudaStream_t st);
+template <>
+int mm_group<bf16>(const MmProb<bf16> *probs, int n, cudaStream_t st);
+// Products whose output is to be rotated, without the fused epilogue: the product goes to the fp32 scratch the
+// caller named, a row kernel rotates it into C.
+template <typename T>
+static int mm_group_rope_unfused(const MmProb<T> *probs, int n, cudaStream_t st) {
+    if (n > 4) return STREAMBP_E_SHAPE;
+    MmProb<T> plain[4];
+    for (int i = 0; i < n; i++) {
+        plain[i] = probs[i];
+        if (!probs[i].rope) continue;
+        if (!probs[i].rope_tmp || probs[i].ldc != probs[i].N || probs[i].accumulate ||
+            probs[i].N != (int64_t)probs[i].rope_heads * probs[i].rope_dh)
+            return STREAMBP_E_SHAPE;
+        plain[i].rope = nullptr;
+        plain[i].C = probs[i].rope_tmp;
+        plain[i].c_is_f32 = true;
+    }
+    SBP_TRY(mm_group<T>(plain, n, st));
+    for (int i = 0; i < n; i++)
+        if (probs[i].rope)
+            SBP_TRY(rope_apply<T>(probs[i].rope_tmp, probs[i].rope, probs[i].M, probs[i].rope_heads, probs[i].rope_dh,
+                                  false, (T *)probs[i].C, st));
+    return STREAMBP_OK;
+}
+template <>
 int mm_group<float>(const MmProb<float> *probs, int n, cudaStream_t st) {
+    for (int i = 0; i < n; i++)
+        if (probs[i].rope) return mm_group_rope_unfused<float>(probs, n, st);
     for (int i = 0; i < n; i++) {
         const MmProb<float> &g = probs[i];
         for (int s = 0; s < g.nseg; s++)
@@ -116,9 +145,18 @@ template <>
 int mm_group<bf16>(const MmProb<bf16> *probs, int n, cudaStream_t st) {
     GemmProb gp[4];
     bool grouped = gemm_engine() != 1 && n <= 4;
+    bool any_rope = false;
+    for (int i = 0; i < n; i++) {
+        any_rope = any_rope || probs[i].rope != nullptr;
+        // the fused rotation handles heads of 128 columns written as bf16
+        if (probs[i].rope && (probs[i].rope_dh != 128 || probs[i].c_is_f32 ||
+                              probs[i].N != (int64_t)probs[i].rope_heads * probs[i].rope_dh))
+            grouped = false;
+    }
     if (grouped) {
         for (int i = 0; i < n; i++) {
             const MmProb<bf16> &g = probs[i];
+            gp[i].rope = g.rope;
             gp[i].op = g.op; gp[i].M = g.M; gp[i].N = g.N; gp[i].nseg = g.nseg;
             for (int s = 0; s < g.nseg; s++) gp[i].seg[s] = GemmSeg{g.seg[s].A, g.seg[s].lda, g.seg[s].B, g.seg[s].ldb, g.seg[s].K};
             gp[i].C = g.C; gp[i].ldc = g.ldc; gp[i].c_is_f32 = g.c_is_f32; gp[i].bias = g.bias; gp[i].accumulate = g.accumulate;
@@ -134,6 +172,7 @@ int mm_group<bf16>(const MmProb<bf16> *probs, int n, cudaStream_t st) {
         int *sched = cs.sched ? cs.sched + 2 * (cs.sched_slot++ % kSchedSlots) : nullptr;
         return gemm_tc_group(gp, n, sched, st);
     }
+    if (any_rope) return mm_group_rope_unfused<bf16>(probs, n, st);
     for (int i = 0; i < n; i++) {
         const MmProb<bf16> &g = probs[i];
         // a bf16 output cannot be accumulated into: several segments need an fp32 C

@@ -285,6 +285,9 @@ struct GemmProb {
     // outputs C = g = A W_gate^T, C_up = u = A W_up^T and C_act = silu(g) * u share ldc.  N counts the columns of each.
     bool swiglu = false;
     void *C_up = nullptr, *C_act = nullptr;
+    // Rotary embedding in the epilogue (bf16 output, heads of 128 columns, N a multiple of 128): row r of `rope` holds
+    // (cos, sin) of the 64 frequencies at the position of row r of C; C = rotate(A B^T + bias), rounded once.
+    const float *rope = nullptr;
 };
 bool gemm_tc_group_supported(const GemmProb *probs, int n);
 // sched: two ints of device memory that are zero when the launch starts (the kernel leaves them zero),
@@ -446,6 +449,10 @@ struct MmProb {
     bool c_is_f32;
     const T *bias;
     bool accumulate;
+    // optional rotary embedding of the output (set by mm_set_rope): C (type T) = rotate(A B^T + bias)
+    const float *rope = nullptr;
+    float *rope_tmp = nullptr;
+    int rope_heads = 0, rope_dh = 0;
 };
 template <typename T>
 MmProb<T> mm_prob(GemmOp op, int64_t M, int64_t N, int64_t K, const T *A, int64_t lda, const T *B, int64_t ldb, void *C,
@@ -455,6 +462,13 @@ MmProb<T> mm_prob(GemmOp op, int64_t M, int64_t N, int64_t K, const T *A, int64_
     g.seg[0] = MmSeg<T>{A, lda, B, ldb, K};
     g.C = C; g.ldc = ldc; g.c_is_f32 = c_is_f32; g.bias = bias; g.accumulate = accumulate;
     return g;
+}
+// The output of g (type T, c_is_f32 must be false unless T is float) becomes the rotary embedding of the product:
+// `cs` holds, per row of C, (cos, sin) of dh / 2 frequencies (rope_table's layout).  The tensor-core kernel rotates
+// in its epilogue when dh = 128; otherwise the product goes to `tmp` (fp32 [M, N], dense) and a row kernel rotates.
+template <typename T>
+void mm_set_rope(MmProb<T> &g, const float *cs, int heads, int dh, float *tmp) {
+    g.rope = cs; g.rope_heads = heads; g.rope_dh = dh; g.rope_tmp = tmp;
 }
 template <typename T>
 void mm_add_seg(MmProb<T> &g, int64_t K, const T *A, int64_t lda, const T *B, int64_t ldb) {

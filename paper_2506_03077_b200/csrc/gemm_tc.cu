@@ -120,7 +120,7 @@ namespace {
 // Operand layouts, output type and accumulation are per-problem run-time flags.
 // ---------------------------------------------------------------------------------------------
 constexpr int MAX_PROBS = 4, MAX_SEGS = 8, RING = 4;
-constexpr uint32_t F_A_MN = 1u, F_B_MN = 2u, F_OUT_F32 = 4u, F_ACC = 8u, F_SWIGLU = 16u;
+constexpr uint32_t F_A_MN = 1u, F_B_MN = 2u, F_OUT_F32 = 4u, F_ACC = 8u, F_SWIGLU = 16u, F_ROPE = 32u;
 
 struct GroupParams {
     CUtensorMap map_a[MAX_SEGS];
@@ -135,6 +135,7 @@ struct GroupParams {
     void *C_up[MAX_PROBS], *C_act[MAX_PROBS];   // SwiGLU pairs: u and silu(g) * u beside g in C
     long long ldc[MAX_PROBS];
     const bf16 *bias[MAX_PROBS];
+    const float2 *rope[MAX_PROBS];     // F_ROPE: (cos, sin) of 64 frequencies per row of the problem
     uint32_t flags[MAX_PROBS];
     int nprob;
     int *sched;                        // {next tile, CTAs finished}, both zero at launch; or nullptr: static schedule
@@ -290,6 +291,51 @@ __device__ __forceinline__ void epilogue_rows(const GroupParams &p, const TileRe
         return;
     }
     bf16 *out_row = reinterpret_cast<bf16 *>(pick(p.C, t.q)) + (long long)row * pick(p.ldc, t.q);
+    if (fl & F_ROPE) {
+        // rotary embedding of 128-wide heads (a tile holds two): the accumulator columns of a head are [x1 | x2],
+        // 64 each; out1 = x1 cos - x2 sin, out2 = x2 cos + x1 sin with the row's (cos, sin) of frequency j, in fp32
+        // from the accumulator (+ bias), rounded to bf16 once.  N is a multiple of 128 (checked on the host).
+        const float2 *cs = pick(p.rope, t.q) + (long long)(row < Mq ? row : 0) * 64;
+#pragma unroll 1
+        for (int f0 = 0; f0 < 64; f0 += 32) {
+            // the row's (cos, sin) of 32 frequencies, fetched once for both heads of the tile
+            float4 q[16];
+#pragma unroll
+            for (int e = 0; e < 16; e++) q[e] = *reinterpret_cast<const float4 *>(cs + f0 + 2 * e);
+#pragma unroll 1
+            for (int head = 0; head < BN / 128; head++) {
+                const int col0 = t.n0 + head * 128;
+                if (col0 >= Nq) break;               // uniform across the warp
+                uint32_t ra[32], rb[32];
+                tmem_ld32(taddr + head * 128 + f0, ra);
+                tmem_ld32(taddr + head * 128 + 64 + f0, rb);
+                if (row >= Mq) continue;
+#pragma unroll
+                for (int j = 0; j < 32; j += 8) {
+                    uint32_t w1[4], w2[4];
+#pragma unroll
+                    for (int e = 0; e < 4; e++) {
+                        float a0 = __uint_as_float(ra[j + 2 * e]), a1 = __uint_as_float(ra[j + 2 * e + 1]);
+                        float b0 = __uint_as_float(rb[j + 2 * e]), b1 = __uint_as_float(rb[j + 2 * e + 1]);
+                        if (bias) {
+                            const __nv_bfloat162 ba = *reinterpret_cast<const __nv_bfloat162 *>(bias + col0 + f0 + j + 2 * e);
+                            const __nv_bfloat162 bb = *reinterpret_cast<const __nv_bfloat162 *>(bias + col0 + 64 + f0 + j + 2 * e);
+                            a0 += __low2float(ba); a1 += __high2float(ba);
+                            b0 += __low2float(bb); b1 += __high2float(bb);
+                        }
+                        const float4 k = q[(j >> 1) + e];       // (cos, sin) of frequencies f0 + j + 2e, + 1
+                        const __nv_bfloat162 h1 = __floats2bfloat162_rn(a0 * k.x - b0 * k.y, a1 * k.z - b1 * k.w);
+                        const __nv_bfloat162 h2 = __floats2bfloat162_rn(b0 * k.x + a0 * k.y, b1 * k.z + a1 * k.w);
+                        w1[e] = *reinterpret_cast<const uint32_t *>(&h1);
+                        w2[e] = *reinterpret_cast<const uint32_t *>(&h2);
+                    }
+                    *reinterpret_cast<uint4 *>(out_row + col0 + f0 + j) = make_uint4(w1[0], w1[1], w1[2], w1[3]);
+                    *reinterpret_cast<uint4 *>(out_row + col0 + 64 + f0 + j) = make_uint4(w2[0], w2[1], w2[2], w2[3]);
+                }
+            }
+        }
+        return;
+    }
 #pragma unroll 1
     for (int c = 0; c < BN / 32; c++) {
         const int col0 = t.n0 + c * 32;
@@ -788,6 +834,9 @@ bool gemm_tc_group_supported(const GemmProb *probs, int n) {
                 !al16(g.C_up) || !al16(g.C_act) || !pair_kernel_available())
                 return false;
         }
+        if (g.rope && (g.c_is_f32 || g.accumulate || g.swiglu || (g.N % 128) ||
+                       (reinterpret_cast<uintptr_t>(g.rope) & 15u)))
+            return false;
         segs += g.nseg;
         for (int s = 0; s < g.nseg; s++)
             if (!gemm_tc_supported(g.op, g.M, g.N, g.seg[s].K, g.seg[s].lda, g.seg[s].ldb, g.ldc, g.seg[s].A,
@@ -846,10 +895,11 @@ int gemm_tc_group(const GemmProb *probs, int n, int *sched, cudaStream_t st) {
         p.C[i] = g.C;
         p.ldc[i] = g.ldc;
         p.bias[i] = g.bias;
+        p.rope[i] = reinterpret_cast<const float2 *>(g.rope);
         p.C_up[i] = g.C_up;
         p.C_act[i] = g.C_act;
         p.flags[i] = (a_mn ? F_A_MN : 0u) | (b_mn ? F_B_MN : 0u) | (g.c_is_f32 ? F_OUT_F32 : 0u) |
-                     (g.accumulate ? F_ACC : 0u) | (g.swiglu ? F_SWIGLU : 0u);
+                     (g.accumulate ? F_ACC : 0u) | (g.swiglu ? F_SWIGLU : 0u) | (g.rope ? F_ROPE : 0u);
         // a SwiGLU tile covers BN / 2 output columns (g and u of the same columns side by side in the accumulator)
         const int64_t tile_n = g.swiglu ? BN / 2 : BN;
         tiles += (int64_t)p.tiles_m[i] * ((g.N + tile_n - 1) / tile_n);

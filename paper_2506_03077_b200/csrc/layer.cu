@@ -142,12 +142,14 @@ int kv_prologue(const streambp_layer_cfg &c, const streambp_layer_weights &w, co
     for (int64_t r0 = 0; r0 < T_; r0 += cn) {
         const int64_t n = (T_ - r0 < cn) ? T_ - r0 : cn;
         SBP_TRY(rmsnorm_fwd<T>(X + r0 * d, nullptr, (const T *)w.g1, c.rms_eps, n, d, s.h1, s.rstd1, nullptr, st));
-        const MmProb<T> kv[2] = {
-            mm_prob<T>(OP_NT, n, dkv, d, s.h1, d, (const T *)w.wk, d, s.fa, dkv, true, (const T *)w.bk, false),
+        // K = rotate(h1 Wk^T + bk) (the rotation in the product's epilogue where the kernel has it), V = h1 Wv^T + bv
+        MmProb<T> kv[2] = {
+            mm_prob<T>(OP_NT, n, dkv, d, s.h1, d, (const T *)w.wk, d, s.K + r0 * dkv, dkv, sizeof(T) == 4,
+                       (const T *)w.bk, false),
             mm_prob<T>(OP_NT, n, dkv, d, s.h1, d, (const T *)w.wv, d, s.V + r0 * dkv, dkv, sizeof(T) == 4,
                        (const T *)w.bv, false)};
+        mm_set_rope<T>(kv[0], s.cs + r0 * dh, Hkv, dh, s.fa);
         SBP_TRY(mm_group<T>(kv, 2, st));
-        SBP_TRY(rope_apply<T>(s.fa, s.cs + r0 * dh, n, Hkv, dh, false, s.K + r0 * dkv, st));
     }
     return STREAMBP_OK;
 }
@@ -160,8 +162,12 @@ int chunk_forward(const streambp_layer_cfg &c, const streambp_layer_weights &w, 
     const int64_t dq = (int64_t)Hq * dh, I = c.d_ff;
     const T *Xi = X + r0 * d;
     SBP_TRY(rmsnorm_fwd<T>(Xi, nullptr, (const T *)w.g1, c.rms_eps, n, d, s.h1, s.rstd1, nullptr, st));
-    SBP_TRY((mm<T, float>(OP_NT, n, dq, d, s.h1, d, (const T *)w.wq, d, s.fa, dq, (const T *)w.bq, false, st)));
-    SBP_TRY(rope_apply<T>(s.fa, s.cs + r0 * dh, n, Hq, dh, false, s.Q, st));
+    {   // Q = rotate(h1 Wq^T + bq)
+        MmProb<T> qp = mm_prob<T>(OP_NT, n, dq, d, s.h1, d, (const T *)w.wq, d, s.Q, dq, sizeof(T) == 4,
+                                  (const T *)w.bq, false);
+        mm_set_rope<T>(qp, s.cs + r0 * dh, Hq, dh, s.fa);
+        SBP_TRY(mm_group<T>(&qp, 1, st));
+    }
     // the chunk's queries against the key / value prefix of their own sequence, one call per sequence the
     // chunk touches (a = first row, e = end row, q_seq = start of that sequence)
     SBP_TRY(seg.for_each(r0, r0 + n, [&](int64_t a, int64_t e, int64_t q_seq) {
