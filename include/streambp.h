@@ -43,8 +43,11 @@
  *     that puts a 256-byte guard after every sub-buffer of the workspaces (the size
  *     queries grow accordingly), fills the guards before and checks them after each
  *     call, and reports an overwritten guard as STREAMBP_E_WORKSPACE_GUARD through
- *     streambp_last_device_status.  None of them changes a result beyond floating-point
- *     summation order.
+ *     streambp_last_device_status; STREAMBP_PDL=0 launches every kernel with plain
+ *     stream ordering instead of programmatic dependent launch (by default a kernel's
+ *     blocks may become resident while the kernel before it in the stream is finishing;
+ *     every kernel waits for that kernel's completion before it touches memory).  None of
+ *     them changes a result beyond floating-point summation order.
  */
 #ifndef STREAMBP_H_
 #define STREAMBP_H_

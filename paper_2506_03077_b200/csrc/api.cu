@@ -54,6 +54,14 @@ ProfScope::~ProfScope() {
     if (idx >= 0) cudaEventRecord(g_prof[idx].b, st);
 }
 
+bool pdl_enabled() {
+    static const bool on = [] {
+        const char *e = getenv("STREAMBP_PDL");      // on unless set to 0
+        return !e || atoi(e) != 0;
+    }();
+    return on;
+}
+
 int gemm_engine() {
     static const int engine = [] {
         const char *e = std::getenv("STREAMBP_GEMM_ENGINE");

@@ -52,6 +52,7 @@ template <typename T, int DH>
 __global__ void __launch_bounds__(256)
     attn_fwd_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ v, int64_t n, int64_t q0,
                     int Hq, int Hkv, T *__restrict__ o, float *__restrict__ lse) {
+    pdl_enter();
     constexpr int LD = DH + 4, DPL = DH / 32;  // dims per lane
     extern __shared__ __align__(16) float smem[];
     float *Qs = smem, *Ks = Qs + 32 * LD, *Vs = Ks + 32 * LD;
@@ -114,6 +115,7 @@ template <typename T>
 __global__ void __launch_bounds__(256)
     attn_delta_kernel(const T *__restrict__ o, const T *__restrict__ dout, int64_t n, int Hq, int dh,
                       float *__restrict__ delta) {
+    pdl_enter();
     const int64_t wid = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (wid >= n * Hq) return;
@@ -152,6 +154,7 @@ __global__ void __launch_bounds__(256)
     attn_bwd_dkdv_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ v,
                          const T *__restrict__ dout, const float *__restrict__ lse, const float *__restrict__ delta,
                          int64_t n, int64_t q0, int Hq, int Hkv, float *__restrict__ dk, float *__restrict__ dv) {
+    pdl_enter();
     constexpr int LD = DH + 4, NE = DH / 32;
     extern __shared__ __align__(16) float smem[];
     float *Ks = smem, *Vs = Ks + 32 * LD, *Qs = Vs + 32 * LD, *dOs = Qs + 32 * LD;
@@ -225,6 +228,7 @@ __global__ void __launch_bounds__(256)
     attn_bwd_dq_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ v,
                        const T *__restrict__ dout, const float *__restrict__ lse, const float *__restrict__ delta,
                        int64_t n, int64_t q0, int Hq, int Hkv, float *__restrict__ dq) {
+    pdl_enter();
     constexpr int LD = DH + 4, NE = DH / 32;
     extern __shared__ __align__(16) float smem[];
     float *Ks = smem, *Vs = Ks + 32 * LD, *Qs = Vs + 32 * LD, *dOs = Qs + 32 * LD;

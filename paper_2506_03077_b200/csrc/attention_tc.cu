@@ -66,6 +66,7 @@ constexpr int FWD16_SMEM = 5 * TILE_BYTES + 3 * 4 * TILE * 4 /* row max x2, row 
 __global__ void __launch_bounds__(FWD16_THREADS, 1)
     attn_fwd_tc16_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                          const __grid_constant__ CUtensorMap map_v, const FwdParams p) {
+    pdl_enter();
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -300,6 +301,7 @@ constexpr int FWD2Q_SMEM = 6 * TILE_BYTES + 1024 + 256;
 __global__ void __launch_bounds__(FWD2Q_THREADS, 1)
     attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                        const __grid_constant__ CUtensorMap map_v, const FwdParams p) {
+    pdl_enter();
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -1437,6 +1439,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1)
     attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                           const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
                           const __grid_constant__ CUtensorMap map_dq, const BwdParams p, int kv_tiles) {
+    pdl_enter();
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const int b = (int)blockIdx.x;
     attn_bwd_fused_body(map_q, map_k, map_v, map_do, map_dq, p, smem_raw, b % kv_tiles, b / kv_tiles);
@@ -1454,6 +1457,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
     attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                        const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
                        const BwdParams p, int kv_tiles, int n_dkdv, int q_tiles, int n_dq_first) {
+    pdl_enter();
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     // block order = dispatch order: n_dq_first dQ CTAs (all of them or none), then the dK/dV CTAs, then the rest
     int b = (int)blockIdx.x;

@@ -64,11 +64,34 @@ public:
 
 // Every kernel launch goes through this so launches are counted and launch errors
 // are caught without synchronising.
-#define SBP_LAUNCH(kernel, grid, block, smem, stream, ...)                         \
+// Every kernel of the library starts with pdl_enter(): it waits until the grids before it in the stream have
+// completed and their writes are visible, then lets the grid after it be scheduled early (programmatic dependent
+// launch: that grid's blocks become resident as this grid's blocks retire and sit in their own pdl_enter() until this
+// grid is done).  At most one grid is launched ahead, and no kernel touches memory before the wait.
+__device__ __forceinline__ void pdl_enter() {
+#ifdef __CUDA_ARCH__
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+#endif
+}
+bool pdl_enabled();   // STREAMBP_PDL (read once per process)
+
+#define SBP_LAUNCH(kernel, grid_, block_, smem_, stream_, ...)                     \
     do {                                                                           \
-        kernel<<<(grid), (block), (smem), (stream)>>>(__VA_ARGS__);                \
+        cudaLaunchConfig_t _cfg;                                                   \
+        memset(&_cfg, 0, sizeof(_cfg));                                            \
+        _cfg.gridDim = dim3(grid_);                                                \
+        _cfg.blockDim = dim3(block_);                                              \
+        _cfg.dynamicSmemBytes = (smem_);                                           \
+        _cfg.stream = (stream_);                                                   \
+        cudaLaunchAttribute _attr[1];                                              \
+        _attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;          \
+        _attr[0].val.programmaticStreamSerializationAllowed = 1;                   \
+        _cfg.attrs = _attr;                                                        \
+        _cfg.numAttrs = ::sbp::pdl_enabled() ? 1 : 0;                              \
+        cudaError_t _le = cudaLaunchKernelEx(&_cfg, kernel, __VA_ARGS__);          \
         ::sbp::call_state().launches++;                                            \
-        if (!::sbp::cuda_ok(cudaGetLastError())) return STREAMBP_E_CUDA;           \
+        if (!::sbp::cuda_ok(_le) || !::sbp::cuda_ok(cudaGetLastError())) return STREAMBP_E_CUDA; \
     } while (0)
 
 #define SBP_TRY(expr)                         \

@@ -15,6 +15,7 @@ __global__ void __launch_bounds__(256) rmsnorm_fwd_kernel(const T *__restrict__ 
                                                           const T *__restrict__ gain, float eps, int d,
                                                           T *__restrict__ h, float *__restrict__ rstd_out,
                                                           float *__restrict__ r_out, const int *gate) {
+    pdl_enter();
     __shared__ float red[33];
     if (gated_off(gate)) return;
     const int64_t row = blockIdx.x;
@@ -98,6 +99,7 @@ __global__ void __launch_bounds__(256)
                             const float *__restrict__ rstd_in, const T *__restrict__ gain,
                             const T *__restrict__ addT, const float *__restrict__ addF, int d,
                             float *__restrict__ outF, T *__restrict__ outT, const int *gate) {
+    pdl_enter();
     __shared__ float red[33];
     const int64_t row = blockIdx.x;
     if (gated_off(gate)) {   // the upstream gradient of this block of rows is exactly zero
@@ -151,6 +153,7 @@ __global__ void __launch_bounds__(256)
     rmsnorm_dgain_partial_kernel(const float *__restrict__ dh, const T *__restrict__ xT, const float *__restrict__ xF,
                                  const float *__restrict__ rstd, int64_t rows, int d, int rows_per_split,
                                  float *__restrict__ partial, const int *gate) {
+    pdl_enter();
     const int col = blockIdx.x * 256 + threadIdx.x;
     if (col >= d || gated_off(gate)) return;
     const int64_t r0 = (int64_t)blockIdx.y * rows_per_split;
@@ -166,6 +169,7 @@ __global__ void __launch_bounds__(256)
 __global__ void __launch_bounds__(256)
     partial_reduce_kernel(const float *__restrict__ partial, int nsplit, int cols, float *__restrict__ out,
                           int accumulate, const int *gate) {
+    pdl_enter();
     const int col = blockIdx.x * 256 + threadIdx.x;
     if (col >= cols || gated_off(gate)) return;
     float acc = 0.f;
@@ -210,6 +214,7 @@ template <typename T>
 __global__ void __launch_bounds__(256)
     colsum_partial_kernel(const T *__restrict__ a, int64_t rows, int cols, int rows_per_split,
                           float *__restrict__ partial) {
+    pdl_enter();
     const int col = blockIdx.x * 256 + threadIdx.x;
     if (col >= cols) return;
     const int64_t r0 = (int64_t)blockIdx.y * rows_per_split;
@@ -241,6 +246,7 @@ struct Colsum3 {
 template <typename T>
 __global__ void __launch_bounds__(256)
     colsum3_partial_kernel(const Colsum3<T> q, int64_t rows, int rows_per_split, float *__restrict__ partial) {
+    pdl_enter();
     const int total = q.cols[0] + q.cols[1] + q.cols[2];
     int col = blockIdx.x * 256 + threadIdx.x;
     if (col >= total) return;
@@ -259,6 +265,7 @@ __global__ void __launch_bounds__(256)
 template <typename T>
 __global__ void __launch_bounds__(256)
     colsum3_reduce_kernel(const Colsum3<T> q, const float *__restrict__ partial, int nsplit) {
+    pdl_enter();
     const int total = q.cols[0] + q.cols[1] + q.cols[2];
     int col = blockIdx.x * 256 + threadIdx.x;
     if (col >= total) return;
@@ -295,6 +302,7 @@ template int colsum<bf16>(const bf16 *, int64_t, int, float *, bool, float *, cu
 // RoPE: table of (cos, sin) built in double precision, applied in fp32.
 // ---------------------------------------------------------------------------------
 __global__ void rope_table_kernel(float2 *__restrict__ cs, int64_t pos0, int64_t rows, int half, double theta) {
+    pdl_enter();
     const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= rows * half) return;
     const int64_t t = idx / half;
@@ -319,6 +327,7 @@ template <typename TO>
 __global__ void __launch_bounds__(256)
     rope_apply_kernel(const float *__restrict__ in, const float2 *__restrict__ cs, int64_t rows, int heads, int dh,
                       int transpose, TO *__restrict__ out) {
+    pdl_enter();
     const int half = dh / 2, q4 = half / 4;
     const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= rows * heads * q4) return;
@@ -363,6 +372,7 @@ template int rope_apply<bf16>(const float *, const float *, int64_t, int, int, b
 template <typename T>
 __global__ void __launch_bounds__(256) swiglu_fwd_kernel(const T *__restrict__ g, const T *__restrict__ u, int64_t n,
                                                          T *__restrict__ m) {
+    pdl_enter();
     constexpr int N = Vec<T>::N;
     const int64_t i0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * N;
     if (i0 >= n) return;
@@ -379,6 +389,7 @@ __global__ void __launch_bounds__(256) swiglu_fwd_kernel(const T *__restrict__ g
 template <typename T>
 __global__ void __launch_bounds__(256) swiglu_bwd_kernel(const T *__restrict__ dm, T *__restrict__ g, T *__restrict__ u,
                                                          int64_t n) {
+    pdl_enter();
     constexpr int N = Vec<T>::N;
     const int64_t i0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * N;
     if (i0 >= n) return;
@@ -419,6 +430,7 @@ template int swiglu_bwd<bf16>(const bf16 *, bf16 *, bf16 *, int64_t, cudaStream_
 // ---------------------------------------------------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(256) cast_kernel(const float *__restrict__ in, int64_t n, T *__restrict__ out) {
+    pdl_enter();
     const int64_t i0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
     if (i0 >= n) return;
     const float4 a = *reinterpret_cast<const float4 *>(in + i0);
@@ -439,6 +451,7 @@ template int cast_from_f32<bf16>(const float *, int64_t, bf16 *, cudaStream_t);
 template <typename T>
 __global__ void __launch_bounds__(256) add_cast_kernel(const float *__restrict__ a, const float *__restrict__ b,
                                                        int64_t n, T *__restrict__ out) {
+    pdl_enter();
     const int64_t i0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
     if (i0 >= n) return;
     const float4 x = *reinterpret_cast<const float4 *>(a + i0);
@@ -466,10 +479,12 @@ struct GuardList {
 };
 __device__ __forceinline__ uint32_t guard_word(int guard, int word) { return 0xA5C3F00Du ^ ((uint32_t)guard * 2654435761u) ^ (uint32_t)word; }
 __global__ void guards_arm_kernel(char *base, GuardList g) {
+    pdl_enter();
     uint32_t *p = reinterpret_cast<uint32_t *>(base + g.off[blockIdx.x]);
     p[threadIdx.x] = guard_word(g.first + blockIdx.x, threadIdx.x);
 }
 __global__ void guards_check_kernel(const char *base, GuardList g, WsHeader *hdr) {
+    pdl_enter();
     const uint32_t *p = reinterpret_cast<const uint32_t *>(base + g.off[blockIdx.x]);
     if (p[threadIdx.x] != guard_word(g.first + blockIdx.x, threadIdx.x)) set_status(hdr, STREAMBP_E_WORKSPACE_GUARD, g.first + blockIdx.x);
 }
@@ -501,6 +516,7 @@ int ws_guards_check(void *base, const std::vector<size_t> &guards, WsHeader *hdr
 
 // test hook: `overrun` floats written past the end of a buffer of `count` floats
 __global__ void overrun_kernel(float *buf, int count, int overrun) {
+    pdl_enter();
     for (int i = threadIdx.x; i < count + overrun; i += blockDim.x) buf[i] = 1.f;
 }
 int ws_guard_selftest(void *ws, size_t bytes, int overrun, cudaStream_t st) {
@@ -527,6 +543,7 @@ int fill_zero(void *p, size_t bytes, cudaStream_t st) {
 // ---------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
     count_labels_kernel(const int64_t *__restrict__ labels, int64_t T_, int64_t vocab, int64_t ignore, WsHeader *hdr) {
+    pdl_enter();
     __shared__ unsigned int cnt;
     if (threadIdx.x == 0) cnt = 0;
     __syncthreads();
@@ -557,6 +574,7 @@ int count_valid_labels(const int64_t *labels, int64_t T_, int64_t vocab, int64_t
 __global__ void __launch_bounds__(256)
     count_chunk_labels_kernel(const int64_t *__restrict__ labels, int64_t T_, int64_t chunk, int64_t ignore,
                               int *__restrict__ counts) {
+    pdl_enter();
     __shared__ int cnt;
     if (threadIdx.x == 0) cnt = 0;
     __syncthreads();
@@ -579,6 +597,7 @@ template <typename T>
 __global__ void __launch_bounds__(1024)
     ce_rows_kernel(const float *z, const int64_t *__restrict__ labels, int64_t V, int64_t ignore,
                    const WsHeader *__restrict__ hdr, T *dz, float *__restrict__ row_loss, const int *gate) {
+    pdl_enter();
     __shared__ float red[33];
     __shared__ float zy_s;
     if (gated_off(gate)) return;
@@ -664,6 +683,7 @@ template <typename T>
 __global__ void __launch_bounds__(1024)
     rl_rows_kernel(const float *z, const int64_t *__restrict__ tokens, int64_t V, int64_t ignore, RlRows rl, int64_t row0,
                    T *dz, float *__restrict__ row_val, const int *gate) {
+    pdl_enter();
     __shared__ float red[33];
     __shared__ float zy_s;
     if (gated_off(gate)) return;
@@ -762,6 +782,7 @@ template int rl_rows<bf16>(const float *, const int64_t *, int64_t, int64_t, int
                            float *, cudaStream_t);
 
 __global__ void rl_finalize_kernel(WsHeader *hdr, int objective, float beta, float *loss, float *ell) {
+    pdl_enter();
     if (hdr->n_valid == 0) set_status(hdr, STREAMBP_E_NO_VALID_LABELS, 0);
     const double acc = hdr->loss_sum;
     if (objective == STREAMBP_OBJ_GRPO) {
@@ -784,6 +805,7 @@ int rl_finalize(WsHeader *hdr, int objective, float beta, float *loss, float *el
 
 template <typename T>
 __global__ void __launch_bounds__(256) scale_by_factor_kernel(T *p, int64_t n, const WsHeader *hdr) {
+    pdl_enter();
     const float f = hdr->factor;
     constexpr int N = Vec<T>::N;
     for (int64_t i0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * N; i0 < n; i0 += (int64_t)gridDim.x * blockDim.x * N) {
@@ -812,6 +834,7 @@ template int scale_by_factor<bf16>(bf16 *, int64_t, const WsHeader *, cudaStream
 
 __global__ void __launch_bounds__(1024) loss_accumulate_kernel(const float *__restrict__ row_loss, int64_t rows,
                                                                WsHeader *hdr, const int *gate) {
+    pdl_enter();
     __shared__ double red[32];
     if (gated_off(gate)) return;
     double acc = 0.0;
@@ -833,6 +856,7 @@ int loss_accumulate(const float *row_loss, int64_t rows, WsHeader *hdr, cudaStre
 }
 
 __global__ void loss_finalize_kernel(WsHeader *hdr, float *loss, int64_t *n_valid) {
+    pdl_enter();
     const unsigned long long N = hdr->n_valid;
     if (N == 0) {
         set_status(hdr, STREAMBP_E_NO_VALID_LABELS, 0);
@@ -854,6 +878,7 @@ template <typename T>
 __global__ void __launch_bounds__(256)
     embedding_gather_kernel(const T *__restrict__ embed, const int64_t *__restrict__ ids, int d, int64_t vocab,
                             T *__restrict__ out, WsHeader *hdr) {
+    pdl_enter();
     constexpr int N = Vec<T>::N;
     const int64_t row = blockIdx.x;
     const int64_t id = ids[row];
@@ -889,6 +914,7 @@ template <typename T>
 __global__ void __launch_bounds__(256)
     embedding_scatter_kernel(const T *__restrict__ dx, const int64_t *__restrict__ ids, int64_t rows, int d,
                              int64_t vocab, float *__restrict__ d_embed) {
+    pdl_enter();
     const int col = blockIdx.x * 256 + threadIdx.x;
     const int cls = blockIdx.y;
     for (int64_t t = 0; t < rows; t++) {

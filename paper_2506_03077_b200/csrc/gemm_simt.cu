@@ -15,6 +15,7 @@ __global__ void __launch_bounds__(256)
     gemm_simt_kernel(int64_t M, int64_t N, int64_t K, const TI *__restrict__ A, int64_t sam, int64_t sak,
                      const TI *__restrict__ B, int64_t sbk, int64_t sbn, TC *C, int64_t ldc,
                      const TI *__restrict__ bias, int accumulate, const int *gate) {
+    pdl_enter();
     __shared__ __align__(16) float As[BK][LDS];
     if (gated_off(gate)) return;
     __shared__ __align__(16) float Bs[BK][LDS];

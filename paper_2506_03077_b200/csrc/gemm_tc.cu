@@ -396,6 +396,7 @@ __device__ __forceinline__ void epilogue_rows(const GroupParams &p, const TileRe
 }
 
 __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_group_kernel(const __grid_constant__ GroupParams p) {
+    pdl_enter();
     extern __shared__ uint8_t smem_raw[];
     if (gated_off(p.gate)) return;
     const uint32_t raw = smem_u32(smem_raw);
@@ -613,6 +614,7 @@ __device__ __forceinline__ bool mma_tile_pair(const GroupParams &p, const TileRe
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
     gemm_pair_kernel(const __grid_constant__ GroupParams p) {
+    pdl_enter();
     extern __shared__ uint8_t smem_raw[];
     if (gated_off(p.gate)) return;
     const uint32_t raw = smem_u32(smem_raw);

@@ -34,6 +34,7 @@ ModelWs<T> plan(const streambp_model_cfg &c, int64_t T_, int64_t chunk_layer, in
 }
 
 __global__ void merge_status_kernel(WsHeader *top, const WsHeader *sub) {
+    pdl_enter();
     if (sub->status != 0 && top->status == 0) {
         top->status = sub->status;
         top->detail = sub->detail;

@@ -13,6 +13,7 @@ namespace sbp {
 namespace {
 
 __global__ void __launch_bounds__(64, 1) wait_probe_kernel(unsigned long long limit_ns) {
+    pdl_enter();
     __shared__ __align__(8) unsigned long long bar_storage;
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_storage;
