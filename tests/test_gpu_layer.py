@@ -126,6 +126,9 @@ def test_causality_zero_upstream_tail():
 @pytest.mark.parametrize("shape,T,chunk", [
     (synth.LayerShape(512, 8, 2, 64, 1376, True, 1e6), 640, 256),
     (synth.LayerShape(1024, 8, 2, 128, 2816, False, 5e5), 1100, 512),     # several tiles, ragged tail
+    # three query heads of 128: the second 256-column tile of the Q product holds one head only (rotation in the
+    # product's epilogue), one KV head, biases, ragged chunks
+    (synth.LayerShape(384, 3, 1, 128, 688, True, 1e6), 300, 128),
 ])
 def test_layer_bf16_matches_oracle(shape, T, chunk):
     ocfg, bcfg, W, X, dY = layer_case(shape, 8, T, torch.bfloat16)
@@ -138,8 +141,8 @@ def test_layer_bf16_matches_oracle(shape, T, chunk):
 
 
 def test_layer_bf16_long_prefix_small_width():
-    """Few query tiles against a long prefix: the attention kernels split their key range into pieces
-    (merged in a fixed order) to fill the SMs; results must match the oracle and stay bit-reproducible."""
+    """Few query tiles and heads against a long prefix (long key loops in few CTAs, many key-tile owners in the
+    backward): results must match the oracle and stay bit-reproducible from run to run."""
     shape = synth.LayerShape(256, 2, 1, 128, 688, True, 1e6)
     T, chunk = 4096 + 200, 512
     ocfg, bcfg, W, X, dY = layer_case(shape, 12, T, torch.bfloat16)
